@@ -1,0 +1,146 @@
+"""ctypes front end of oracle/moe_oracle.c (fp64 plain-loop CPU oracle).
+
+TEST INFRASTRUCTURE ONLY.  Inputs may be torch tensors or numpy arrays of any float
+dtype (bf16 included); they are widened exactly to float64 before the C code sees them.
+Each wrapper names the passage of the paper its C function follows.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "moe_oracle.c")
+_LIB = os.path.join(_HERE, "libmoe_oracle.so")
+_lib = None
+
+
+def build_oracle(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, OpenMP, strict IEEE: no fast-math)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build_oracle())
+        i32p, f32p, f64p, ci = (ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float),
+                                ctypes.POINTER(ctypes.c_double), ctypes.c_int)
+        lib.moe_oracle_threads.restype = ci
+        lib.moe_oracle_route.argtypes = [f32p, ci, ci, ci, ci, i32p, f64p]
+        lib.moe_oracle_layout.argtypes = [i32p, ci, ci, ci, ci, i32p, i32p, i32p, i32p]
+        lib.moe_oracle_fwd.argtypes = [f64p, i32p, f64p, f64p, f64p, ci, ci, ci, ci, ci, ci, f64p, f64p, f64p, f64p]
+        lib.moe_oracle_bwd.argtypes = [f64p, f64p, i32p, f64p, f64p, f64p, ci, ci, ci, ci, ci, ci,
+                                       f64p, f64p, f64p, f64p]
+        _lib = lib
+    return _lib
+
+
+def _np(a, dtype):
+    """torch tensor / array -> contiguous numpy array of `dtype` (exact widening for floats)."""
+    if hasattr(a, "detach"):
+        import torch
+        a = a.detach().to("cpu")
+        if a.dtype == torch.bfloat16:
+            a = a.to(torch.float32)
+        a = a.numpy()
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _p(a, ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def threads() -> int:
+    return int(_load().moe_oracle_threads())
+
+
+def route(logits, k: int, renorm: bool):
+    """Top-k routing scores (Section 2.2, router description).  -> ids int32 [T,k], w float64 [T,k]."""
+    l = _np(logits, np.float32)
+    T, E = l.shape
+    ids = np.empty((T, k), np.int32)
+    w = np.empty((T, k), np.float64)
+    rc = _load().moe_oracle_route(_p(l, ctypes.c_float), T, E, k, int(bool(renorm)),
+                                  _p(ids, ctypes.c_int32), _p(w, ctypes.c_double))
+    if rc:
+        raise ValueError(f"moe_oracle_route failed ({rc})")
+    return ids, w
+
+
+def layout(ids, E: int, S: int = 0):
+    """Dispatch layout (Section 2.2, Dispatch).  -> counts [E+S], offsets [E+S+1], row_of, src_of [T*(k+S)]."""
+    ids = _np(ids, np.int32)
+    T, k = ids.shape
+    n = T * (k + S)
+    counts = np.empty(E + S, np.int32)
+    offsets = np.empty(E + S + 1, np.int32)
+    row_of = np.empty(n, np.int32)
+    src_of = np.empty(n, np.int32)
+    rc = _load().moe_oracle_layout(_p(ids, ctypes.c_int32), T, E, k, S, _p(counts, ctypes.c_int32),
+                                   _p(offsets, ctypes.c_int32), _p(row_of, ctypes.c_int32),
+                                   _p(src_of, ctypes.c_int32))
+    if rc:
+        raise ValueError(f"moe_oracle_layout failed ({rc}): expert id out of range")
+    return counts, offsets, row_of, src_of
+
+
+def fwd(x, ids, w, W_gate_up, W_down, S: int = 0, save: bool = False):
+    """Forward MoE-FFN (Section 2.2, five forward operators).  -> out float64 [T,d]
+    (and, with save=True, per-slot H [T*(k+S),2F], A [.,F], Y [.,d])."""
+    x = _np(x, np.float64)
+    ids = _np(ids, np.int32)
+    w = _np(w, np.float64)
+    Wgu = _np(W_gate_up, np.float64)
+    Wd = _np(W_down, np.float64)
+    T, d = x.shape
+    k = ids.shape[1]
+    Ep, F2, d2 = Wgu.shape
+    F = F2 // 2
+    E = Ep - S
+    assert d2 == d and Wd.shape == (Ep, d, F) and w.shape == ids.shape and ids.shape[0] == T
+    out = np.empty((T, d), np.float64)
+    n = T * (k + S)
+    H = np.empty((n, 2 * F), np.float64) if save else None
+    A = np.empty((n, F), np.float64) if save else None
+    Y = np.empty((n, d), np.float64) if save else None
+    dp = ctypes.c_double
+    rc = _load().moe_oracle_fwd(_p(x, dp), _p(ids, ctypes.c_int32), _p(w, dp), _p(Wgu, dp), _p(Wd, dp),
+                                T, d, E, k, S, F, _p(out, dp), _p(H, dp), _p(A, dp), _p(Y, dp))
+    if rc:
+        raise ValueError(f"moe_oracle_fwd failed ({rc})")
+    return (out, H, A, Y) if save else out
+
+
+def bwd(dout, x, ids, w, W_gate_up, W_down, S: int = 0):
+    """Backward MoE-FFN (Section 2.2, seven backward operators).
+    -> dx [T,d], dW_gate_up [E+S,2F,d], dW_down [E+S,d,F], d_w [T,k] (all float64)."""
+    dout = _np(dout, np.float64)
+    x = _np(x, np.float64)
+    ids = _np(ids, np.int32)
+    w = _np(w, np.float64)
+    Wgu = _np(W_gate_up, np.float64)
+    Wd = _np(W_down, np.float64)
+    T, d = x.shape
+    k = ids.shape[1]
+    Ep, F2, _ = Wgu.shape
+    F = F2 // 2
+    E = Ep - S
+    assert dout.shape == x.shape and Wd.shape == (Ep, d, F)
+    dx = np.empty((T, d), np.float64)
+    dWgu = np.empty_like(Wgu)
+    dWd = np.empty_like(Wd)
+    dw = np.empty((T, k), np.float64)
+    dp = ctypes.c_double
+    rc = _load().moe_oracle_bwd(_p(dout, dp), _p(x, dp), _p(ids, ctypes.c_int32), _p(w, dp), _p(Wgu, dp),
+                                _p(Wd, dp), T, d, E, k, S, F, _p(dx, dp), _p(dWgu, dp), _p(dWd, dp), _p(dw, dp))
+    if rc:
+        raise ValueError(f"moe_oracle_bwd failed ({rc})")
+    return dx, dWgu, dWd, dw
