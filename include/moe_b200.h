@@ -1,0 +1,170 @@
+/*
+ * moe_b200 -- Dispatch->Combine MoE-FFN layer for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The layer is the one the paper schedules as a tile-level taskflow (Section 2.2):
+ * forward  = Dispatch, GroupedGEMM (gate+up), SwiGLU, GroupedGEMM (down), Combine;
+ * backward = backward Dispatch, GMM act_grad, GMM w2_grad, SwiGLU_grad, GMM gate_grad,
+ *            GMM w1_grad, backward Combine.
+ * On one GPU Dispatch and Combine are local permutes.  Every step runs in hand-written
+ * CUDA kernels of this library; there is no CPU fallback.
+ *
+ * Conventions
+ *   - Unless a parameter says "host", every tensor pointer is a DEVICE pointer owned by the
+ *     caller, row-major, 16-byte aligned.  The library neither frees nor keeps it after the
+ *     call's work has finished on `stream`.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     only enqueue work; they do not synchronise unless stated.
+ *   - bf16 tensors are passed as uint16_t (raw bits).
+ *   - Shapes: T tokens, d hidden, E routed experts, k routed experts per token, S shared
+ *     experts (taken by every token with weight 1), F expert intermediate size.
+ *     Requirements: d % 8 == 0, F % 8 == 0, 1 <= k <= E <= 1024, T <= T_max.
+ *   - Weights: W_gate_up[E+S][2F][d] (rows 0..F-1 = gate projection, F..2F-1 = up projection,
+ *     d contiguous) and W_down[E+S][d][F] (F contiguous); shared experts are the last S slabs.
+ *   - Return value: 0 on success; a negative MOE_ERR_* when an argument is rejected (nothing
+ *     was enqueued).  Conditions found by kernels (an expert id out of range, a bounded wait
+ *     that ran out) are recorded in the context and read with moe_get_status(); kernels always
+ *     terminate.
+ *   - A context serialises nothing: use one context per stream, and do not overlap two calls
+ *     on the same context.
+ */
+#ifndef MOE_B200_H
+#define MOE_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct moe_ctx moe_ctx; /* opaque: shape, workspace carving, tensor maps, status word */
+
+typedef struct {
+  int32_t T_max;    /* largest token count any call will pass */
+  int32_t d;        /* hidden size */
+  int32_t E;        /* routed experts */
+  int32_t k;        /* routed experts per token */
+  int32_t n_shared; /* S */
+  int32_t F;        /* expert intermediate size */
+  uint32_t flags;   /* MOE_FLAG_* */
+} moe_shape;
+
+enum {
+  MOE_FLAG_RENORM_TOPK = 1u,   /* moe_route: divide the k scores by their sum */
+  MOE_FLAG_SAVE_FOR_BWD = 2u,  /* moe_ffn_fwd keeps layout, gathered x, pre-activations and
+                                  activations in the workspace for the next moe_ffn_bwd */
+  MOE_FLAG_SERIAL_LAUNCH = 4u, /* run the layer as one kernel launch per operator (the paper's
+                                  operator-by-operator baseline, Section 5.2) instead of the
+                                  single persistent dependency-driven launch */
+};
+
+enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = -1,   /* NULL pointer, bad shape, T > T_max, misaligned pointer */
+  MOE_ERR_WORKSPACE = -2,     /* caller's workspace too small or misaligned */
+  MOE_ERR_CUDA = -3,          /* a CUDA runtime/driver call failed (see moe_last_cuda_error) */
+  MOE_ERR_NO_DEVICE = -4,     /* no sm_100 device is current */
+  MOE_ERR_STATE = -5,         /* moe_ffn_bwd without a saved forward of the same T */
+  MOE_ERR_TOO_LARGE = -6,     /* size beyond a documented fixed limit */
+  /* asynchronous, reported by moe_get_status(): */
+  MOE_ERR_BAD_EXPERT_ID = 1,  /* detail = flat slot index of one offending entry */
+  MOE_ERR_TIMEOUT = 2,        /* a bounded device-side wait expired; detail = where */
+};
+
+/* Bytes of device workspace a context of this shape needs (layout arrays, expert-ordered
+ * activations, tile table, dependency counters).  0 if the shape is invalid. */
+size_t moe_workspace_bytes(const moe_shape* shape);
+
+/* Create a context.  `workspace` is device memory of at least moe_workspace_bytes() bytes,
+ * 256-byte aligned, owned by the caller and kept alive until moe_destroy(); pass NULL to let the
+ * library cudaMalloc (and later free) it on the current device.  Host-side planning done here
+ * (workspace carving, tensor maps of workspace tensors) is outside the timed Dispatch->Combine
+ * interval, like the paper's schedule compilation (Section 5.1). */
+int moe_create(moe_ctx** out, const moe_shape* shape, void* workspace, size_t workspace_bytes);
+int moe_destroy(moe_ctx* ctx);
+
+/* Router scores -> top-k (Section 2.2, first paragraph).  logits[T][E] fp32.
+ * topk_ids[T][k]: the k largest raw logits, ties to the lower expert id, slots in descending
+ * logit order.  topk_w[T][k]: softmax over all E of the selected experts, renormalised over
+ * the k when MOE_FLAG_RENORM_TOPK is set.  counts[E] (may be NULL): tokens per routed expert. */
+int moe_route(moe_ctx* ctx, const float* logits, int32_t T, int32_t* topk_ids, float* topk_w,
+              int32_t* counts, void* stream);
+
+/* Dispatch layout only (Section 2.2, Dispatch: "permutes ... tokens according to the routing
+ * decisions").  Flat slot i = t*(k+S)+j; slots j >= k are the shared experts E..E+S-1.
+ * counts[E+S]; offsets[E+S+1] = exclusive scan; row_of[T*(k+S)] = expert-ordered row of each slot
+ * (rows of one expert keep slot order; -1 for a slot whose expert id is out of range);
+ * src_of[row] = slot.  Any output may be NULL.  moe_ffn_fwd computes the same layout internally. */
+int moe_layout(moe_ctx* ctx, const int32_t* topk_ids, int32_t T, int32_t* counts, int32_t* offsets,
+               int32_t* row_of, int32_t* src_of, void* stream);
+
+/* Forward layer (Section 2.2, second paragraph): for every token t
+ *   out[t] = sum_j w(t,j) * ( silu(x_t Wg_e^T) * (x_t Wu_e^T) ) Wd_e^T ,  e = expert of slot j,
+ * j over the k routed slots (weight topk_w) and the S shared experts (weight 1).
+ * x, out: bf16 [T][d]; topk_ids int32 [T][k]; topk_w fp32 [T][k].  bf16 inputs, fp32
+ * accumulation, bf16 output. */
+int moe_ffn_fwd(moe_ctx* ctx, const uint16_t* x, const int32_t* topk_ids, const float* topk_w,
+                const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* out, int32_t T,
+                void* stream);
+
+/* Backward layer (Section 2.2, third paragraph).  Needs the preceding moe_ffn_fwd on this context
+ * with MOE_FLAG_SAVE_FOR_BWD and the same x, topk_ids, topk_w, weights and T.
+ * dout bf16 [T][d] -> dx bf16 [T][d], dW_gate_up bf16 [E+S][2F][d], dW_down bf16 [E+S][d][F]
+ * (both overwritten; an expert that received no token gets exact zeros), d_topk_w fp32 [T][k]
+ * (gradient of the routing weights; may be NULL). */
+int moe_ffn_bwd(moe_ctx* ctx, const uint16_t* dout, const uint16_t* x, const int32_t* topk_ids,
+                const float* topk_w, const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* dx,
+                uint16_t* dW_gate_up, uint16_t* dW_down, float* d_topk_w, int32_t T, void* stream);
+
+/* The same two calls for callers whose activations live in HOST memory (pinned memory gives
+ * asynchronous copies).  x/topk_ids/topk_w/dout are host pointers copied to the device inside the
+ * call; out/dx/d_topk_w are host pointers filled from the device; weights and weight gradients
+ * stay device pointers (model state is resident).  The call returns after enqueueing; the host
+ * buffers are valid once `stream` has been synchronised. */
+int moe_ffn_fwd_host(moe_ctx* ctx, const uint16_t* x_host, const int32_t* topk_ids_host,
+                     const float* topk_w_host, const uint16_t* W_gate_up, const uint16_t* W_down,
+                     uint16_t* out_host, int32_t T, void* stream);
+int moe_ffn_bwd_host(moe_ctx* ctx, const uint16_t* dout_host, const uint16_t* W_gate_up,
+                     const uint16_t* W_down, uint16_t* dx_host, uint16_t* dW_gate_up,
+                     uint16_t* dW_down, float* d_topk_w_host, int32_t T, void* stream);
+
+/* Synchronises the stream of the context's last call, then reports what kernels recorded:
+ * *code = 0 or MOE_ERR_BAD_EXPERT_ID / MOE_ERR_TIMEOUT, *detail = where.  Clears the record. */
+int moe_get_status(moe_ctx* ctx, int32_t* code, int32_t* detail);
+
+/* Number of kernels the context's last call launched (for launch accounting). */
+int moe_last_launch_count(const moe_ctx* ctx);
+
+/* Budget, in milliseconds, of every bounded device-side wait (default 2000). */
+int moe_set_wait_budget_ms(moe_ctx* ctx, int32_t ms);
+
+/* Test/diagnostic access to workspace tensors of the last forward/backward.  `which` is a
+ * MOE_BUF_* id; *ptr receives a device pointer into the workspace (valid until the next call on
+ * the context), *elems its element count.  Rows of expert-ordered tensors live in a padded row
+ * space: expert e starts at row pad_off[e] (a multiple of 128) and holds counts[e] rows. */
+enum {
+  MOE_BUF_COUNTS = 0,    /* int32 [E+S] */
+  MOE_BUF_OFFSETS = 1,   /* int32 [E+S+1] */
+  MOE_BUF_ROW_OF = 2,    /* int32 [T*(k+S)] unpadded rows */
+  MOE_BUF_SRC_OF = 3,    /* int32 [T*(k+S)] */
+  MOE_BUF_PROW_OF = 4,   /* int32 [T*(k+S)] padded rows */
+  MOE_BUF_PAD_OFF = 5,   /* int32 [E+S+1] */
+  MOE_BUF_XP = 6,        /* bf16 [R_pad][d]   gathered x */
+  MOE_BUF_H = 7,         /* bf16 [R_pad][2F]  gate|up pre-activations */
+  MOE_BUF_A = 8,         /* bf16 [R_pad][F]   w * silu(g) * u */
+  MOE_BUF_Y = 9,         /* bf16 [R_pad][d]   expert outputs (already weighted) */
+  MOE_BUF_DOUTP = 10,    /* bf16 [R_pad][d]   gathered dout */
+  MOE_BUF_DH = 11,       /* bf16 [R_pad][2F]  gradient of the pre-activations */
+  MOE_BUF_DXP = 12,      /* bf16 [R_pad][d]   per-row input gradient */
+  MOE_BUF_META = 13,     /* int32 [8]: {num_mblocks, R_pad, rows, ...} */
+};
+int moe_debug_buffer(moe_ctx* ctx, int which, void** ptr, size_t* elems);
+
+const char* moe_strerror(int code);
+/* Text of the last CUDA error a call on this thread ran into ("" if none). */
+const char* moe_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_B200_H */

@@ -1,0 +1,274 @@
+"""ctypes binding of libmoe_b200.so: argument marshalling only.
+
+Every function has the name and argument order of its C counterpart in include/moe_b200.h and
+takes torch tensors where the C call takes pointers (CUDA tensors for device pointers, pinned
+CPU tensors for the *_host calls).  The current torch stream is passed as the stream argument.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+MOE_FLAG_RENORM_TOPK, MOE_FLAG_SAVE_FOR_BWD, MOE_FLAG_SERIAL_LAUNCH = 1, 2, 4
+MOE_BUF = {"counts": 0, "offsets": 1, "row_of": 2, "src_of": 3, "prow_of": 4, "pad_off": 5, "Xp": 6, "H": 7,
+           "A": 8, "Y": 9, "dOutp": 10, "dH": 11, "dXp": 12, "meta": 13}
+_BUF_DTYPE = {k: (torch.bfloat16 if k in ("Xp", "H", "A", "Y", "dOutp", "dH", "dXp") else torch.int32)
+              for k in MOE_BUF}
+
+EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe_layout", "moe_ffn_fwd",
+           "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
+           "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error"]
+
+
+class MoeShape(ctypes.Structure):
+    _fields_ = [("T_max", ctypes.c_int32), ("d", ctypes.c_int32), ("E", ctypes.c_int32), ("k", ctypes.c_int32),
+                ("n_shared", ctypes.c_int32), ("F", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class MoeError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmoe_b200.so")
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the C-ABI library; raises if it has not been built (there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = lib_path()
+    if not os.path.exists(path):
+        raise MoeError(f"{path} is missing: build it with `python -m paper_2605_23764_b200.build`")
+    lib = ctypes.CDLL(path)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+    lib.moe_workspace_bytes.restype = sz
+    lib.moe_workspace_bytes.argtypes = [ctypes.POINTER(MoeShape)]
+    lib.moe_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(MoeShape), vp, sz]
+    lib.moe_destroy.argtypes = [vp]
+    lib.moe_route.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.moe_layout.argtypes = [vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.moe_ffn_fwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.moe_ffn_bwd.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.moe_ffn_fwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.moe_ffn_bwd_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, vp]
+    lib.moe_get_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.moe_last_launch_count.argtypes = [vp]
+    lib.moe_set_wait_budget_ms.argtypes = [vp, i32]
+    lib.moe_debug_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(sz)]
+    lib.moe_strerror.restype = ctypes.c_char_p
+    lib.moe_strerror.argtypes = [ctypes.c_int]
+    lib.moe_last_cuda_error.restype = ctypes.c_char_p
+    _lib = lib
+    return lib
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        lib = load_library()
+        msg = lib.moe_strerror(rc).decode()
+        extra = lib.moe_last_cuda_error().decode()
+        raise MoeError(f"{what}: {msg} ({rc})" + (f" [{extra}]" if extra and rc == -3 else ""))
+
+
+def _dev(t, dtype, name):
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise MoeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _host(t, dtype, name):
+    if t is None:
+        return None
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise MoeError(f"{name}: expected a contiguous CPU tensor of {dtype}")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _shape(T_max, d, E, k, n_shared, F, flags):
+    return MoeShape(int(T_max), int(d), int(E), int(k), int(n_shared), int(F), int(flags))
+
+
+def moe_strerror(code: int) -> str:
+    return load_library().moe_strerror(code).decode()
+
+
+def moe_workspace_bytes(T_max, d, E, k, n_shared, F, flags=0) -> int:
+    s = _shape(T_max, d, E, k, n_shared, F, flags)
+    return int(load_library().moe_workspace_bytes(ctypes.byref(s)))
+
+
+def moe_create(T_max, d, E, k, n_shared, F, flags=0, workspace: torch.Tensor | None = None):
+    """-> opaque context handle.  `workspace`: CUDA uint8 tensor (kept alive by the caller) or None."""
+    s = _shape(T_max, d, E, k, n_shared, F, flags)
+    h = ctypes.c_void_p()
+    ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+    ws_bytes = workspace.numel() if workspace is not None else 0
+    _check(load_library().moe_create(ctypes.byref(h), ctypes.byref(s), ws_ptr, ws_bytes), "moe_create")
+    return h
+
+
+def moe_destroy(ctx):
+    _check(load_library().moe_destroy(ctx), "moe_destroy")
+
+
+def moe_route(ctx, logits, T, topk_ids, topk_w, counts=None):
+    _check(load_library().moe_route(ctx, _dev(logits, torch.float32, "logits"), T,
+                                    _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_w, torch.float32, "topk_w"),
+                                    _dev(counts, torch.int32, "counts"), _stream()), "moe_route")
+
+
+def moe_layout(ctx, topk_ids, T, counts=None, offsets=None, row_of=None, src_of=None):
+    _check(load_library().moe_layout(ctx, _dev(topk_ids, torch.int32, "topk_ids"), T,
+                                     _dev(counts, torch.int32, "counts"), _dev(offsets, torch.int32, "offsets"),
+                                     _dev(row_of, torch.int32, "row_of"), _dev(src_of, torch.int32, "src_of"),
+                                     _stream()), "moe_layout")
+
+
+def moe_ffn_fwd(ctx, x, topk_ids, topk_w, W_gate_up, W_down, out, T):
+    bf = torch.bfloat16
+    _check(load_library().moe_ffn_fwd(ctx, _dev(x, bf, "x"), _dev(topk_ids, torch.int32, "topk_ids"),
+                                      _dev(topk_w, torch.float32, "topk_w"), _dev(W_gate_up, bf, "W_gate_up"),
+                                      _dev(W_down, bf, "W_down"), _dev(out, bf, "out"), T, _stream()), "moe_ffn_fwd")
+
+
+def moe_ffn_bwd(ctx, dout, x, topk_ids, topk_w, W_gate_up, W_down, dx, dW_gate_up, dW_down, d_topk_w, T):
+    bf = torch.bfloat16
+    _check(load_library().moe_ffn_bwd(ctx, _dev(dout, bf, "dout"), _dev(x, bf, "x"),
+                                      _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_w, torch.float32, "topk_w"),
+                                      _dev(W_gate_up, bf, "W_gate_up"), _dev(W_down, bf, "W_down"),
+                                      _dev(dx, bf, "dx"), _dev(dW_gate_up, bf, "dW_gate_up"),
+                                      _dev(dW_down, bf, "dW_down"), _dev(d_topk_w, torch.float32, "d_topk_w"),
+                                      T, _stream()), "moe_ffn_bwd")
+
+
+def moe_ffn_fwd_host(ctx, x_host, topk_ids_host, topk_w_host, W_gate_up, W_down, out_host, T):
+    bf = torch.bfloat16
+    _check(load_library().moe_ffn_fwd_host(ctx, _host(x_host, bf, "x_host"),
+                                           _host(topk_ids_host, torch.int32, "topk_ids_host"),
+                                           _host(topk_w_host, torch.float32, "topk_w_host"),
+                                           _dev(W_gate_up, bf, "W_gate_up"), _dev(W_down, bf, "W_down"),
+                                           _host(out_host, bf, "out_host"), T, _stream()), "moe_ffn_fwd_host")
+
+
+def moe_ffn_bwd_host(ctx, dout_host, W_gate_up, W_down, dx_host, dW_gate_up, dW_down, d_topk_w_host, T):
+    bf = torch.bfloat16
+    _check(load_library().moe_ffn_bwd_host(ctx, _host(dout_host, bf, "dout_host"), _dev(W_gate_up, bf, "W_gate_up"),
+                                           _dev(W_down, bf, "W_down"), _host(dx_host, bf, "dx_host"),
+                                           _dev(dW_gate_up, bf, "dW_gate_up"), _dev(dW_down, bf, "dW_down"),
+                                           _host(d_topk_w_host, torch.float32, "d_topk_w_host"), T, _stream()),
+           "moe_ffn_bwd_host")
+
+
+def moe_get_status(ctx):
+    code, detail = ctypes.c_int32(), ctypes.c_int32()
+    _check(load_library().moe_get_status(ctx, ctypes.byref(code), ctypes.byref(detail)), "moe_get_status")
+    return code.value, detail.value
+
+
+def moe_last_launch_count(ctx) -> int:
+    return int(load_library().moe_last_launch_count(ctx))
+
+
+def moe_set_wait_budget_ms(ctx, ms: int):
+    _check(load_library().moe_set_wait_budget_ms(ctx, ms), "moe_set_wait_budget_ms")
+
+
+class _DevView:
+    """Minimal __cuda_array_interface__ holder so torch can view library-owned device memory."""
+
+    def __init__(self, ptr, n, typestr):
+        self.__cuda_array_interface__ = {"shape": (n,), "typestr": typestr, "data": (ptr, False), "version": 2}
+
+
+def moe_debug_buffer(ctx, which: str) -> torch.Tensor:
+    """Copy of a workspace tensor of the last call (see MOE_BUF_* in the header)."""
+    ptr, n = ctypes.c_void_p(), ctypes.c_size_t()
+    _check(load_library().moe_debug_buffer(ctx, MOE_BUF[which], ctypes.byref(ptr), ctypes.byref(n)),
+           "moe_debug_buffer")
+    if _BUF_DTYPE[which] == torch.int32:
+        return torch.as_tensor(_DevView(ptr.value, n.value, "<i4"), device="cuda").clone()
+    raw = torch.as_tensor(_DevView(ptr.value, n.value, "<i2"), device="cuda")
+    return raw.view(torch.bfloat16).clone()
+
+
+class MoeLayer:
+    """Owns a context and its workspace (a torch allocation); allocates outputs; same calls as the C ABI."""
+
+    def __init__(self, T_max, d, E, k, n_shared, F, renorm=False, save_for_bwd=False, serial=False):
+        self.T_max, self.d, self.E, self.k, self.S, self.F = T_max, d, E, k, n_shared, F
+        self.flags = ((MOE_FLAG_RENORM_TOPK if renorm else 0) | (MOE_FLAG_SAVE_FOR_BWD if save_for_bwd else 0) |
+                      (MOE_FLAG_SERIAL_LAUNCH if serial else 0))
+        nbytes = moe_workspace_bytes(T_max, d, E, k, n_shared, F, self.flags)
+        if nbytes == 0:
+            raise MoeError("invalid shape")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        self.ctx = moe_create(T_max, d, E, k, n_shared, F, self.flags, self.workspace)
+
+    def close(self):
+        if self.ctx is not None:
+            torch.cuda.synchronize()
+            moe_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def route(self, logits, with_counts=False):
+        T = logits.shape[0]
+        ids = torch.empty(T, self.k, dtype=torch.int32, device="cuda")
+        w = torch.empty(T, self.k, dtype=torch.float32, device="cuda")
+        counts = torch.empty(self.E, dtype=torch.int32, device="cuda") if with_counts else None
+        moe_route(self.ctx, logits, T, ids, w, counts)
+        return (ids, w, counts) if with_counts else (ids, w)
+
+    def layout(self, topk_ids):
+        T = topk_ids.shape[0]
+        n, Ep = T * (self.k + self.S), self.E + self.S
+        i32 = dict(dtype=torch.int32, device="cuda")
+        counts, offsets = torch.empty(Ep, **i32), torch.empty(Ep + 1, **i32)
+        row_of, src_of = torch.empty(n, **i32), torch.empty(n, **i32)
+        moe_layout(self.ctx, topk_ids, T, counts, offsets, row_of, src_of)
+        return counts, offsets, row_of, src_of
+
+    def ffn_fwd(self, x, topk_ids, topk_w, W_gate_up, W_down, out=None):
+        T = x.shape[0]
+        if out is None:
+            out = torch.empty(T, self.d, dtype=torch.bfloat16, device="cuda")
+        moe_ffn_fwd(self.ctx, x, topk_ids, topk_w, W_gate_up, W_down, out, T)
+        return out
+
+    def ffn_bwd(self, dout, x, topk_ids, topk_w, W_gate_up, W_down, dx=None, dW_gate_up=None, dW_down=None,
+                d_topk_w=None, want_d_topk_w=True):
+        T = x.shape[0]
+        dx = torch.empty_like(x) if dx is None else dx
+        dW_gate_up = torch.empty_like(W_gate_up) if dW_gate_up is None else dW_gate_up
+        dW_down = torch.empty_like(W_down) if dW_down is None else dW_down
+        if d_topk_w is None and want_d_topk_w:
+            d_topk_w = torch.empty(T, self.k, dtype=torch.float32, device="cuda")
+        moe_ffn_bwd(self.ctx, dout, x, topk_ids, topk_w, W_gate_up, W_down, dx, dW_gate_up, dW_down, d_topk_w, T)
+        return dx, dW_gate_up, dW_down, d_topk_w
+
+    def status(self):
+        return moe_get_status(self.ctx)
+
+    def launches(self):
+        return moe_last_launch_count(self.ctx)
+
+    def debug(self, which):
+        return moe_debug_buffer(self.ctx, which)

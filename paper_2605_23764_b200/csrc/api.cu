@@ -1,0 +1,567 @@
+// C ABI of libmoe_b200: context, workspace carving, tensor-map encoding and the launch
+// sequences of the forward and backward layer.  Argument marshalling and planning only; every
+// step of the layer runs in the kernels of route_layout.cu, permute.cu and gemm_tc.cu.
+#include <stdio.h>
+#include <string.h>
+
+#include <string>
+
+#include "../../include/moe_b200.h"
+#include "moe_internal.h"
+
+using namespace moe;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int cuda_fail(cudaError_t e, const char* what) {
+  g_cuda_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return MOE_ERR_CUDA;
+}
+#define MOE_CUDA(call)                                   \
+  do {                                                   \
+    cudaError_t _e = (call);                             \
+    if (_e != cudaSuccess) return cuda_fail(_e, #call);  \
+  } while (0)
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 row-major [rows][cols] tensor, box [box_rows][box_cols], 128-byte swizzle, zero fill outside.
+int encode_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+              uint32_t box_cols) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) {
+    g_cuda_error = "cuTensorMapEncodeTiled entry point not available";
+    return MOE_ERR_CUDA;
+  }
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstr[1] = {cols * 2};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    char buf[160];
+    snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed (%d) rows=%llu cols=%llu box=%ux%u", (int)r,
+             (unsigned long long)rows, (unsigned long long)cols, box_rows, box_cols);
+    g_cuda_error = buf;
+    return MOE_ERR_CUDA;
+  }
+  return MOE_OK;
+}
+
+bool shape_ok(const moe_shape* s) {
+  return s && s->T_max >= 0 && s->d >= 8 && s->d % 8 == 0 && s->F >= 8 && s->F % 8 == 0 && s->E >= 1 &&
+         s->E <= 1024 && s->k >= 1 && s->k <= s->E && s->k <= 32 && s->n_shared >= 0 && s->n_shared <= 64 &&
+         (long)s->T_max * (s->k + s->n_shared) < (1l << 30);
+}
+
+struct Carve {
+  size_t off = 0;
+  size_t take(size_t bytes) {
+    size_t o = off;
+    off += (bytes + 255) & ~size_t(255);
+    return o;
+  }
+};
+
+// Byte offsets of every workspace tensor.
+struct WsPlan {
+  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, total;
+  int cap_rows, nblk_max, ntn_act;
+};
+
+WsPlan plan_workspace(const moe_shape& s) {
+  WsPlan p;
+  Carve c;
+  const int Ep = s.E + s.n_shared, kp = s.k + s.n_shared;
+  const size_t slots = (size_t)s.T_max * kp;
+  p.cap_rows = padded_rows_max(s.T_max, kp, Ep);
+  p.nblk_max = (int)((slots + LAYOUT_CHUNK - 1) / LAYOUT_CHUNK);
+  if (p.nblk_max < 1) p.nblk_max = 1;
+  p.ntn_act = (s.F + 255) / 256;
+  const bool train = (s.flags & MOE_FLAG_SAVE_FOR_BWD) != 0;
+  const size_t cap = (size_t)p.cap_rows;
+  p.status = c.take(sizeof(DevStatus));
+  p.meta = c.take(sizeof(int) * 8);
+  p.counts = c.take(sizeof(int) * Ep);
+  p.offsets = c.take(sizeof(int) * (Ep + 1));
+  p.pad_off = c.take(sizeof(int) * (Ep + 1));
+  p.mb_start = c.take(sizeof(int) * (Ep + 1));
+  p.mblk_expert = c.take(sizeof(int) * (cap / BLOCK_M + 1));
+  p.blk_hist = c.take(sizeof(int) * (size_t)p.nblk_max * Ep);
+  p.row_of = c.take(sizeof(int) * (slots + 1));
+  p.src_of = c.take(sizeof(int) * (slots + 1));
+  p.prow_of = c.take(sizeof(int) * (slots + 1));
+  p.prow_w = c.take(sizeof(float) * cap);
+  p.dw_partial = c.take(train ? sizeof(float) * cap * p.ntn_act : 0);
+  p.Xp = c.take(2 * cap * s.d);
+  p.H = c.take(train ? 2 * cap * 2 * s.F : 0);
+  p.A = c.take(2 * cap * s.F);
+  p.Y = c.take(2 * cap * s.d);
+  p.dOutp = c.take(train ? 2 * cap * s.d : 0);
+  p.dH = c.take(train ? 2 * cap * 2 * s.F : 0);
+  p.st_x = c.take(2 * (size_t)s.T_max * s.d);
+  p.st_ids = c.take(sizeof(int) * (size_t)s.T_max * s.k);
+  p.st_w = c.take(sizeof(float) * (size_t)s.T_max * s.k);
+  p.st_out = c.take(2 * (size_t)s.T_max * s.d);
+  p.st_dw = c.take(sizeof(float) * (size_t)s.T_max * s.k);
+  p.total = c.off;
+  return p;
+}
+
+}  // namespace
+
+struct moe_ctx {
+  moe_shape shape;
+  WsPlan plan;
+  uint8_t* ws = nullptr;
+  bool owns_ws = false;
+  int device = 0;
+  int num_sms = 0;
+  int launches = 0;
+  int saved_T = -1;  // T of the forward whose tensors are in the workspace (-1: none)
+  uint64_t budget_ns = 2000ull * 1000 * 1000;
+  cudaStream_t last_stream = nullptr;
+  // tensor maps of workspace tensors (fixed for the context's lifetime)
+  CUtensorMap tm_Xp_k, tm_A_k, tm_dOutp_k, tm_dH_k;      // K-major A operands, box 128 x 64
+  CUtensorMap tm_dOutp_mn, tm_A_mn, tm_dH_mn, tm_Xp_mn;  // MN-major operands of the weight gradients, box 64 x 64
+  // tensor maps of the caller's weights, re-encoded when the pointers change
+  const void* w1_ptr = nullptr;
+  const void* w2_ptr = nullptr;
+  CUtensorMap tm_W1_k, tm_W2_k, tm_W1_mn, tm_W2_mn;
+
+  template <class T>
+  T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  DevStatus* status() const { return at<DevStatus>(plan.status); }
+  LayoutView layout() const {
+    LayoutView lv;
+    lv.counts = at<int>(plan.counts);
+    lv.offsets = at<int>(plan.offsets);
+    lv.row_of = at<int>(plan.row_of);
+    lv.src_of = at<int>(plan.src_of);
+    lv.prow_of = at<int>(plan.prow_of);
+    lv.pad_off = at<int>(plan.pad_off);
+    lv.mb_start = at<int>(plan.mb_start);
+    lv.mblk_expert = at<int>(plan.mblk_expert);
+    lv.meta = at<int>(plan.meta);
+    lv.blk_hist = at<int>(plan.blk_hist);
+    return lv;
+  }
+  Dims dims(int T) const { return Dims{T, shape.d, shape.E, shape.k, shape.n_shared, shape.F}; }
+  bool train() const { return (shape.flags & MOE_FLAG_SAVE_FOR_BWD) != 0; }
+};
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+int encode_weight_maps(moe_ctx* c, const uint16_t* W1, const uint16_t* W2) {
+  const moe_shape& s = c->shape;
+  const uint64_t Ep = s.E + s.n_shared;
+  int rc;
+  if (W1 != c->w1_ptr) {
+    if ((rc = encode_2d(&c->tm_W1_k, W1, Ep * 2 * s.F, s.d, 128, 64))) return rc;
+    if ((rc = encode_2d(&c->tm_W1_mn, W1, Ep * 2 * s.F, s.d, 64, 64))) return rc;
+    c->w1_ptr = W1;
+  }
+  if (W2 != c->w2_ptr) {
+    if ((rc = encode_2d(&c->tm_W2_k, W2, Ep * s.d, s.F, 256, 64))) return rc;
+    if ((rc = encode_2d(&c->tm_W2_mn, W2, Ep * s.d, s.F, 64, 64))) return rc;
+    c->w2_ptr = W2;
+  }
+  return MOE_OK;
+}
+
+GemmArgs base_args(const moe_ctx* c) {
+  GemmArgs g;
+  memset(&g, 0, sizeof g);
+  LayoutView lv = c->layout();
+  g.mblk_expert = lv.mblk_expert;
+  g.mb_start = lv.mb_start;
+  g.counts = lv.counts;
+  g.meta = lv.meta;
+  g.Ep = c->shape.E + c->shape.n_shared;
+  g.F = c->shape.F;
+  g.status = c->status();
+  g.budget_ns = c->budget_ns;
+  return g;
+}
+
+int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, const uint16_t* W1,
+            const uint16_t* W2, uint16_t* out, int T, cudaStream_t st) {
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  const Dims dm = c->dims(T);
+  const LayoutView lv = c->layout();
+  int rc = encode_weight_maps(c, W1, W2);
+  if (rc) return rc;
+  c->saved_T = -1;
+  MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
+  MOE_CUDA(launch_gather(x, w, dm, lv, c->at<uint16_t>(p.Xp), c->at<float>(p.prow_w), p.cap_rows, st,
+                         &c->launches));
+  {  // GMM1 + SwiGLU (+ routing weight)
+    GemmArgs g = base_args(c);
+    g.tmA = c->tm_Xp_k;
+    g.tmB = c->tm_W1_k;
+    g.n_tiles_n = (s.F + 127) / 128;
+    g.K = s.d;
+    g.N = s.F;
+    g.b_rows_per_expert = 2 * s.F;
+    g.out0 = c->at<uint16_t>(p.A);
+    g.ld_out0 = s.F;
+    g.out1 = c->train() ? c->at<uint16_t>(p.H) : nullptr;
+    g.ld_out1 = 2 * s.F;
+    g.prow_w = c->at<float>(p.prow_w);
+    MOE_CUDA(launch_gemm(GEMM_GATE_UP, g, c->num_sms, st, &c->launches));
+  }
+  {  // GMM2
+    GemmArgs g = base_args(c);
+    g.tmA = c->tm_A_k;
+    g.tmB = c->tm_W2_k;
+    g.n_tiles_n = (s.d + 255) / 256;
+    g.K = s.F;
+    g.N = s.d;
+    g.b_rows_per_expert = s.d;
+    g.out0 = c->at<uint16_t>(p.Y);
+    g.ld_out0 = s.d;
+    MOE_CUDA(launch_gemm(GEMM_DOWN, g, c->num_sms, st, &c->launches));
+  }
+  MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+  if (c->train()) c->saved_T = T;
+  return MOE_OK;
+}
+
+int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t* W2, uint16_t* dx, uint16_t* dW1,
+            uint16_t* dW2, float* d_w, int T, cudaStream_t st) {
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  const Dims dm = c->dims(T);
+  const LayoutView lv = c->layout();
+  int rc = encode_weight_maps(c, W1, W2);
+  if (rc) return rc;
+  // backward Dispatch: expert-ordered gather of the upstream gradient
+  MOE_CUDA(launch_gather(dout, nullptr, dm, lv, c->at<uint16_t>(p.dOutp), nullptr, p.cap_rows, st, &c->launches));
+  {  // act_grad + SwiGLU_grad (+ routing-weight gradient partials)
+    GemmArgs g = base_args(c);
+    g.tmA = c->tm_dOutp_k;
+    g.tmB = c->tm_W2_mn;
+    g.n_tiles_n = p.ntn_act;
+    g.K = s.d;
+    g.N = s.F;
+    g.b_rows_per_expert = s.d;
+    g.out0 = c->at<uint16_t>(p.dH);
+    g.ld_out0 = 2 * s.F;
+    g.in0 = c->at<uint16_t>(p.H);
+    g.ld_in0 = 2 * s.F;
+    g.prow_w = c->at<float>(p.prow_w);
+    g.dw_partial = d_w ? c->at<float>(p.dw_partial) : nullptr;
+    MOE_CUDA(launch_gemm(GEMM_ACT_GRAD, g, c->num_sms, st, &c->launches));
+  }
+  if (d_w) MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), p.ntn_act, dm, lv, d_w, st, &c->launches));
+  {  // w2_grad: dW_down[e][c][f] = sum_rows dOutp[r][c] * A[r][f]   (shares dOutp with act_grad)
+    GemmArgs g = base_args(c);
+    g.tmA = c->tm_dOutp_mn;
+    g.tmB = c->tm_A_mn;
+    g.M = s.d;
+    g.N = s.F;
+    g.n_tiles_m = (s.d + 127) / 128;
+    g.n_tiles_n = (s.F + 255) / 256;
+    g.out0 = dW2;
+    g.ld_out0 = s.F;
+    MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
+  }
+  {  // gate_grad: dXp = dH . W_gate_up[e]
+    GemmArgs g = base_args(c);
+    g.tmA = c->tm_dH_k;
+    g.tmB = c->tm_W1_mn;
+    g.n_tiles_n = (s.d + 255) / 256;
+    g.K = 2 * s.F;
+    g.N = s.d;
+    g.b_rows_per_expert = 2 * s.F;
+    g.out0 = c->at<uint16_t>(p.Y);  // the forward's Y is dead by now: reuse it for dXp
+    g.ld_out0 = s.d;
+    MOE_CUDA(launch_gemm(GEMM_GATE_GRAD, g, c->num_sms, st, &c->launches));
+  }
+  {  // w1_grad: dW_gate_up[e][n][c] = sum_rows dH[r][n] * Xp[r][c]   (shares dH with gate_grad)
+    GemmArgs g = base_args(c);
+    g.tmA = c->tm_dH_mn;
+    g.tmB = c->tm_Xp_mn;
+    g.M = 2 * s.F;
+    g.N = s.d;
+    g.n_tiles_m = (2 * s.F + 127) / 128;
+    g.n_tiles_n = (s.d + 255) / 256;
+    g.out0 = dW1;
+    g.ld_out0 = s.d;
+    MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
+  }
+  // backward Combine
+  MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
+  return MOE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t moe_workspace_bytes(const moe_shape* shape) {
+  if (!shape_ok(shape)) return 0;
+  return plan_workspace(*shape).total;
+}
+
+int moe_create(moe_ctx** out, const moe_shape* shape, void* workspace, size_t workspace_bytes) {
+  if (!out || !shape_ok(shape)) return MOE_ERR_INVALID_ARG;
+  *out = nullptr;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return MOE_ERR_NO_DEVICE;
+  }
+  int major = 0, sms = 0;
+  MOE_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+  MOE_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (major != 10) return MOE_ERR_NO_DEVICE;
+  moe_ctx* c = new moe_ctx();
+  c->shape = *shape;
+  c->plan = plan_workspace(*shape);
+  c->device = dev;
+  c->num_sms = sms;
+  if (workspace) {
+    if (workspace_bytes < c->plan.total || (reinterpret_cast<uintptr_t>(workspace) & 255)) {
+      delete c;
+      return MOE_ERR_WORKSPACE;
+    }
+    c->ws = static_cast<uint8_t*>(workspace);
+  } else {
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&c->ws), c->plan.total);
+    if (e != cudaSuccess) {
+      delete c;
+      return cuda_fail(e, "cudaMalloc(workspace)");
+    }
+    c->owns_ws = true;
+  }
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  const uint64_t cap = p.cap_rows;
+  const bool train = c->train();
+  int rc = MOE_OK;
+  cudaError_t e = cudaMemset(c->ws, 0, p.Xp);  // status, tables and small arrays start at zero
+  if (e != cudaSuccess) rc = cuda_fail(e, "cudaMemset(workspace)");
+  if (!rc) rc = encode_2d(&c->tm_Xp_k, c->ws + p.Xp, cap, s.d, 128, 64);
+  if (!rc) rc = encode_2d(&c->tm_A_k, c->ws + p.A, cap, s.F, 128, 64);
+  if (!rc && train) rc = encode_2d(&c->tm_dOutp_k, c->ws + p.dOutp, cap, s.d, 128, 64);
+  if (!rc && train) rc = encode_2d(&c->tm_dH_k, c->ws + p.dH, cap, 2 * s.F, 128, 64);
+  if (!rc && train) rc = encode_2d(&c->tm_dOutp_mn, c->ws + p.dOutp, cap, s.d, 64, 64);
+  if (!rc && train) rc = encode_2d(&c->tm_A_mn, c->ws + p.A, cap, s.F, 64, 64);
+  if (!rc && train) rc = encode_2d(&c->tm_dH_mn, c->ws + p.dH, cap, 2 * s.F, 64, 64);
+  if (!rc && train) rc = encode_2d(&c->tm_Xp_mn, c->ws + p.Xp, cap, s.d, 64, 64);
+  if (rc) {
+    if (c->owns_ws) cudaFree(c->ws);
+    delete c;
+    return rc;
+  }
+  *out = c;
+  return MOE_OK;
+}
+
+int moe_destroy(moe_ctx* c) {
+  if (!c) return MOE_OK;
+  if (c->owns_ws) cudaFree(c->ws);
+  delete c;
+  return MOE_OK;
+}
+
+int moe_route(moe_ctx* c, const float* logits, int32_t T, int32_t* topk_ids, float* topk_w, int32_t* counts,
+              void* stream) {
+  if (!c || !logits || !topk_ids || !topk_w || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
+  c->launches = 0;
+  c->last_stream = static_cast<cudaStream_t>(stream);
+  MOE_CUDA(launch_route(logits, T, c->shape.E, c->shape.k, (c->shape.flags & MOE_FLAG_RENORM_TOPK) != 0, topk_ids,
+                        topk_w, counts, c->last_stream, &c->launches));
+  return MOE_OK;
+}
+
+int moe_layout(moe_ctx* c, const int32_t* topk_ids, int32_t T, int32_t* counts, int32_t* offsets, int32_t* row_of,
+               int32_t* src_of, void* stream) {
+  if (!c || !topk_ids || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  c->launches = 0;
+  c->last_stream = st;
+  c->saved_T = -1;
+  const Dims dm = c->dims(T);
+  const LayoutView lv = c->layout();
+  MOE_CUDA(launch_layout(topk_ids, dm, lv, c->status(), st, &c->launches));
+  const size_t n = (size_t)dm.slots(), Ep = dm.Ep();
+  if (counts) MOE_CUDA(cudaMemcpyAsync(counts, lv.counts, sizeof(int) * Ep, cudaMemcpyDeviceToDevice, st));
+  if (offsets) MOE_CUDA(cudaMemcpyAsync(offsets, lv.offsets, sizeof(int) * (Ep + 1), cudaMemcpyDeviceToDevice, st));
+  if (row_of && n) MOE_CUDA(cudaMemcpyAsync(row_of, lv.row_of, sizeof(int) * n, cudaMemcpyDeviceToDevice, st));
+  if (src_of && n) MOE_CUDA(cudaMemcpyAsync(src_of, lv.src_of, sizeof(int) * n, cudaMemcpyDeviceToDevice, st));
+  return MOE_OK;
+}
+
+int moe_ffn_fwd(moe_ctx* c, const uint16_t* x, const int32_t* topk_ids, const float* topk_w,
+                const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* out, int32_t T, void* stream) {
+  if (!c || !x || !topk_ids || !topk_w || !W_gate_up || !W_down || !out || T < 0 || T > c->shape.T_max)
+    return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_gate_up) || !aligned16(W_down) || !aligned16(out)) return MOE_ERR_INVALID_ARG;
+  c->launches = 0;
+  c->last_stream = static_cast<cudaStream_t>(stream);
+  if (T == 0) return MOE_OK;
+  return run_fwd(c, x, topk_ids, topk_w, W_gate_up, W_down, out, T, c->last_stream);
+}
+
+int moe_ffn_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* x, const int32_t* topk_ids, const float* topk_w,
+                const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* dx, uint16_t* dW_gate_up,
+                uint16_t* dW_down, float* d_topk_w, int32_t T, void* stream) {
+  if (!c || !dout || !x || !topk_ids || !topk_w || !W_gate_up || !W_down || !dx || !dW_gate_up || !dW_down ||
+      T < 0 || T > c->shape.T_max)
+    return MOE_ERR_INVALID_ARG;
+  if (!aligned16(dout) || !aligned16(W_gate_up) || !aligned16(W_down) || !aligned16(dx) ||
+      !aligned16(dW_gate_up) || !aligned16(dW_down))
+    return MOE_ERR_INVALID_ARG;
+  if (!c->train()) return MOE_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  c->launches = 0;
+  c->last_stream = st;
+  if (T == 0) {
+    const moe_shape& s = c->shape;
+    const size_t Ep = s.E + s.n_shared;
+    MOE_CUDA(cudaMemsetAsync(dW_gate_up, 0, 2 * Ep * 2 * s.F * s.d, st));
+    MOE_CUDA(cudaMemsetAsync(dW_down, 0, 2 * Ep * s.d * s.F, st));
+    return MOE_OK;
+  }
+  if (c->saved_T != T) return MOE_ERR_STATE;
+  return run_bwd(c, dout, W_gate_up, W_down, dx, dW_gate_up, dW_down, d_topk_w, T, st);
+}
+
+int moe_ffn_fwd_host(moe_ctx* c, const uint16_t* x_host, const int32_t* topk_ids_host, const float* topk_w_host,
+                     const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* out_host, int32_t T,
+                     void* stream) {
+  if (!c || !x_host || !topk_ids_host || !topk_w_host || !W_gate_up || !W_down || !out_host || T < 0 ||
+      T > c->shape.T_max)
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  c->launches = 0;
+  c->last_stream = st;
+  if (T == 0) return MOE_OK;
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_x, x_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, st));
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_ids, topk_ids_host, sizeof(int) * (size_t)T * s.k, cudaMemcpyHostToDevice,
+                           st));
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_w, topk_w_host, sizeof(float) * (size_t)T * s.k, cudaMemcpyHostToDevice,
+                           st));
+  int rc = run_fwd(c, c->at<uint16_t>(p.st_x), c->at<int32_t>(p.st_ids), c->at<float>(p.st_w), W_gate_up, W_down,
+                   c->at<uint16_t>(p.st_out), T, st);
+  if (rc) return rc;
+  MOE_CUDA(cudaMemcpyAsync(out_host, c->ws + p.st_out, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
+  return MOE_OK;
+}
+
+int moe_ffn_bwd_host(moe_ctx* c, const uint16_t* dout_host, const uint16_t* W_gate_up, const uint16_t* W_down,
+                     uint16_t* dx_host, uint16_t* dW_gate_up, uint16_t* dW_down, float* d_topk_w_host, int32_t T,
+                     void* stream) {
+  if (!c || !dout_host || !W_gate_up || !W_down || !dx_host || !dW_gate_up || !dW_down || T <= 0 ||
+      T > c->shape.T_max)
+    return MOE_ERR_INVALID_ARG;
+  if (!c->train() || c->saved_T != T) return MOE_ERR_STATE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  c->launches = 0;
+  c->last_stream = st;
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  // the staged x is dead after the forward's gather: its buffer receives dout
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_x, dout_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, st));
+  int rc = run_bwd(c, c->at<uint16_t>(p.st_x), W_gate_up, W_down, c->at<uint16_t>(p.st_out), dW_gate_up, dW_down,
+                   d_topk_w_host ? c->at<float>(p.st_dw) : nullptr, T, st);
+  if (rc) return rc;
+  MOE_CUDA(cudaMemcpyAsync(dx_host, c->ws + p.st_out, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
+  if (d_topk_w_host)
+    MOE_CUDA(cudaMemcpyAsync(d_topk_w_host, c->ws + p.st_dw, sizeof(float) * (size_t)T * s.k,
+                             cudaMemcpyDeviceToHost, st));
+  return MOE_OK;
+}
+
+int moe_get_status(moe_ctx* c, int32_t* code, int32_t* detail) {
+  if (!c) return MOE_ERR_INVALID_ARG;
+  MOE_CUDA(cudaStreamSynchronize(c->last_stream));
+  DevStatus h;
+  MOE_CUDA(cudaMemcpy(&h, c->status(), sizeof h, cudaMemcpyDeviceToHost));
+  if (code) *code = h.code;
+  if (detail) *detail = h.detail;
+  if (h.code || h.abort) MOE_CUDA(cudaMemset(c->status(), 0, sizeof h));
+  return MOE_OK;
+}
+
+int moe_last_launch_count(const moe_ctx* c) { return c ? c->launches : 0; }
+
+int moe_set_wait_budget_ms(moe_ctx* c, int32_t ms) {
+  if (!c || ms < 1) return MOE_ERR_INVALID_ARG;
+  c->budget_ns = (uint64_t)ms * 1000 * 1000;
+  return MOE_OK;
+}
+
+int moe_debug_buffer(moe_ctx* c, int which, void** ptr, size_t* elems) {
+  if (!c || !ptr || !elems) return MOE_ERR_INVALID_ARG;
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  const size_t Ep = s.E + s.n_shared, slots = (size_t)s.T_max * (s.k + s.n_shared), cap = p.cap_rows;
+  const bool train = c->train();
+  size_t off = 0, n = 0;
+  switch (which) {
+    case MOE_BUF_COUNTS: off = p.counts; n = Ep; break;
+    case MOE_BUF_OFFSETS: off = p.offsets; n = Ep + 1; break;
+    case MOE_BUF_ROW_OF: off = p.row_of; n = slots; break;
+    case MOE_BUF_SRC_OF: off = p.src_of; n = slots; break;
+    case MOE_BUF_PROW_OF: off = p.prow_of; n = slots; break;
+    case MOE_BUF_PAD_OFF: off = p.pad_off; n = Ep + 1; break;
+    case MOE_BUF_XP: off = p.Xp; n = cap * s.d; break;
+    case MOE_BUF_H: if (!train) return MOE_ERR_STATE; off = p.H; n = cap * 2 * s.F; break;
+    case MOE_BUF_A: off = p.A; n = cap * s.F; break;
+    case MOE_BUF_Y: off = p.Y; n = cap * s.d; break;
+    case MOE_BUF_DOUTP: if (!train) return MOE_ERR_STATE; off = p.dOutp; n = cap * s.d; break;
+    case MOE_BUF_DH: if (!train) return MOE_ERR_STATE; off = p.dH; n = cap * 2 * s.F; break;
+    case MOE_BUF_DXP: off = p.Y; n = cap * s.d; break;
+    case MOE_BUF_META: off = p.meta; n = 8; break;
+    default: return MOE_ERR_INVALID_ARG;
+  }
+  *ptr = c->ws + off;
+  *elems = n;
+  return MOE_OK;
+}
+
+const char* moe_strerror(int code) {
+  switch (code) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case MOE_ERR_CUDA: return "CUDA call failed";
+    case MOE_ERR_NO_DEVICE: return "no sm_100 CUDA device is current";
+    case MOE_ERR_STATE: return "no matching saved forward (or context created without MOE_FLAG_SAVE_FOR_BWD)";
+    case MOE_ERR_TOO_LARGE: return "size beyond a fixed limit";
+    case MOE_ERR_BAD_EXPERT_ID: return "expert id out of range (slot dropped)";
+    case MOE_ERR_TIMEOUT: return "bounded device-side wait expired";
+    default: return "unknown code";
+  }
+}
+
+const char* moe_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,377 @@
+// Grouped GEMMs of the MoE-FFN layer on the sm_100a tensor cores.
+//
+// One persistent, warp-specialised kernel body serves the five GEMM-shaped operators of the layer
+// (forward GMM1+SwiGLU, GMM2; backward act_grad+SwiGLU_grad, gate_grad, and the two weight
+// gradients).  Per CTA: warp 0 = TMA producer (one elected lane), warp 1 = tcgen05.mma issuer (one
+// elected lane; the warp also owns the TMEM allocation), warps 2..5 = epilogue (TMEM -> registers
+// -> fused element-wise math -> global).  Operands travel global -> shared through TMA into a
+// 4-stage ring of 128-byte-swizzled tiles; accumulators live in TMEM, double-buffered (2 x 256
+// columns) so the epilogue of tile i overlaps the main loop of tile i+1.
+//
+// Tiles never straddle experts: rows live in a padded row space where every expert segment starts
+// on a multiple of 128 (the paper's rule that vector tiles align with GMM row partitions and that
+// the reduction dimension stays intact, Section 4.2).
+#include "moe_internal.h"
+
+namespace moe {
+
+constexpr int BN = 256;                       // accumulator columns per tile
+constexpr int BK = 64;                        // reduction elements per stage (one 128-byte swizzle row)
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BLOCK_M * BK * 2;  // 16 KB
+constexpr int B_STAGE_BYTES = BN * BK * 2;       // 32 KB
+constexpr int MN_BOX_BYTES = 64 * BK * 2;        // one [64 k][64 mn] box of an MN-major operand
+constexpr int GEMM_THREADS = 192;
+constexpr int TMEM_COLS = 512;
+
+struct __align__(8) GemmBarriers {
+  uint64_t full[STAGES];
+  uint64_t empty[STAGES];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  uint32_t pad;
+};
+
+constexpr size_t GEMM_SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
+                                   sizeof(GemmBarriers);
+size_t gemm_smem_bytes() { return GEMM_SMEM_BYTES; }
+
+struct Tile {
+  int e;      // expert
+  int row0;   // row-space modes: first padded row of the M-block; WGRAD: first padded row of the expert
+  int n0;     // first output column of the tile
+  int m0;     // WGRAD: first output row (within the expert's slab)
+  int nkb;    // k-blocks of the main loop (may be 0 for an expert without rows in WGRAD)
+  int nb;     // column-tile index (ACT_GRAD partials)
+};
+
+template <int MODE>
+__device__ __forceinline__ int total_tiles(const GemmArgs& a) {
+  if (MODE == GEMM_WGRAD) return a.Ep * a.n_tiles_m * a.n_tiles_n;
+  return a.meta[0] * a.n_tiles_n;
+}
+
+// Tile order.  Row-space modes: expert-major; inside an expert the column tile is the slow index
+// and the M-block the fast one, so CTAs running at the same time share one slab of weights (read
+// from HBM once, then from L2) while the expert's rows stay L2-resident.
+template <int MODE>
+__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int t) {
+  Tile tl;
+  if (MODE == GEMM_WGRAD) {
+    const int per_e = a.n_tiles_m * a.n_tiles_n;
+    tl.e = t / per_e;
+    const int r = t - tl.e * per_e;
+    const int mb = r / a.n_tiles_n;
+    tl.nb = r - mb * a.n_tiles_n;
+    tl.m0 = mb * BLOCK_M;
+    tl.n0 = tl.nb * BN;
+    tl.row0 = a.mb_start[tl.e] * BLOCK_M;
+    tl.nkb = (a.counts[tl.e] + BK - 1) / BK;
+  } else {
+    const int e = a.mblk_expert[t / a.n_tiles_n];
+    const int ms = a.mb_start[e];
+    const int mcount = a.mb_start[e + 1] - ms;
+    const int local = t - ms * a.n_tiles_n;
+    tl.nb = local / mcount;
+    const int mbl = local - tl.nb * mcount;
+    tl.e = e;
+    tl.row0 = (ms + mbl) * BLOCK_M;
+    tl.n0 = tl.nb * (MODE == GEMM_GATE_UP ? BN / 2 : BN);
+    tl.m0 = 0;
+    tl.nkb = (a.K + BK - 1) / BK;
+  }
+  return tl;
+}
+
+// ---------------------------------------------------------------- producer: TMA loads of one k-block
+template <int MODE>
+__device__ __forceinline__ void load_stage(const GemmArgs& a, const Tile& tl, int kb, uint8_t* sA, uint8_t* sB,
+                                           uint64_t* bar) {
+  const int k0 = kb * BK;
+  if (MODE == GEMM_WGRAD) {
+    // both operands MN-major: boxes of [64 rows of the expert][64 columns]
+    mbar_expect_tx(bar, 2 * MN_BOX_BYTES + 4 * MN_BOX_BYTES);
+#pragma unroll
+    for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * MN_BOX_BYTES, &a.tmA, tl.m0 + j * 64, tl.row0 + k0, bar);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + j * 64, tl.row0 + k0, bar);
+    return;
+  }
+  mbar_expect_tx(bar, A_STAGE_BYTES + B_STAGE_BYTES);
+  tma_load_2d(sA, &a.tmA, k0, tl.row0, bar);  // A: [128 rows][64 k], K-major
+  const int brow = tl.e * a.b_rows_per_expert;
+  if (MODE == GEMM_GATE_UP) {
+    tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);                          // gate rows -> columns 0..127
+    tma_load_2d(sB + B_STAGE_BYTES / 2, &a.tmB, k0, brow + a.F + tl.n0, bar);  // up rows   -> columns 128..255
+  } else if (MODE == GEMM_DOWN) {
+    tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);  // [256 rows of W_down][64 k], K-major
+  } else {
+    // ACT_GRAD / GATE_GRAD: B = forward weight read along its rows (reduction) -> MN-major boxes
+#pragma unroll
+    for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + j * 64, brow + k0, bar);
+  }
+}
+
+// ---------------------------------------------------------------- epilogues (one thread = one tile row)
+__device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
+}
+__device__ __forceinline__ void store8_bf16(uint16_t* p, const float* v) {
+  st_v4(p, pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+}
+__device__ __forceinline__ void load8_bf16(const uint16_t* p, float* v) {
+  uint4 r = *reinterpret_cast<const uint4*>(p);
+  v[0] = bf16lo(r.x); v[1] = bf16hi(r.x); v[2] = bf16lo(r.y); v[3] = bf16hi(r.y);
+  v[4] = bf16lo(r.z); v[5] = bf16hi(r.z); v[6] = bf16lo(r.w); v[7] = bf16hi(r.w);
+}
+__device__ __forceinline__ float sigmoidf_fast(float g) { return 1.0f / (1.0f + __expf(-g)); }
+
+template <int MODE>
+__device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl, uint32_t tmem_acc, int quad,
+                                              int lane) {
+  const int r = quad * 32 + lane;                   // row of the tile held by this thread
+  const uint32_t trow = tmem_acc + (static_cast<uint32_t>(quad * 32) << 16);
+  if (MODE == GEMM_GATE_UP) {
+    const size_t p = (size_t)tl.row0 + r;
+    const float w = a.prow_w[p];
+    uint16_t* arow = a.out0 + p * a.ld_out0;
+    uint16_t* hrow = a.out1 ? a.out1 + p * a.ld_out1 : nullptr;
+    for (int c = 0; c < BN / 2; c += 16) {
+      float g[16], u[16], act[16];
+      tmem_ld16(trow + c, g);
+      tmem_ld16(trow + BN / 2 + c, u);
+      tmem_ld_wait();
+#pragma unroll
+      for (int i = 0; i < 16; ++i) act[i] = w * (g[i] * sigmoidf_fast(g[i]) * u[i]);
+#pragma unroll
+      for (int h = 0; h < 16; h += 8) {
+        const int col = tl.n0 + c + h;
+        if (col < a.F) {
+          store8_bf16(arow + col, act + h);
+          if (hrow) {
+            store8_bf16(hrow + col, g + h);
+            store8_bf16(hrow + a.F + col, u + h);
+          }
+        }
+      }
+    }
+  } else if (MODE == GEMM_ACT_GRAD) {
+    const size_t p = (size_t)tl.row0 + r;
+    const float w = a.prow_w[p];
+    const uint16_t* hrow = a.in0 + p * a.ld_in0;
+    uint16_t* drow = a.out0 + p * a.ld_out0;
+    float part = 0.f;
+    for (int c = 0; c < BN; c += 16) {
+      float da[16];
+      tmem_ld16(trow + c, da);
+      tmem_ld_wait();
+#pragma unroll
+      for (int h = 0; h < 16; h += 8) {
+        const int col = tl.n0 + c + h;
+        if (col < a.F) {
+          float g[8], u[8], dg[8], du[8];
+          load8_bf16(hrow + col, g);
+          load8_bf16(hrow + a.F + col, u);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const float s = sigmoidf_fast(g[i]);
+            const float gs = g[i] * s;
+            part += da[h + i] * (gs * u[i]);          // <dA_unweighted, a>: gradient of the routing weight
+            const float dav = w * da[h + i];          // backward Dispatch's weight, applied here
+            dg[i] = dav * u[i] * (s * (1.0f + g[i] * (1.0f - s)));
+            du[i] = dav * gs;
+          }
+          store8_bf16(drow + col, dg);
+          store8_bf16(drow + a.F + col, du);
+        }
+      }
+    }
+    if (a.dw_partial) a.dw_partial[p * a.n_tiles_n + tl.nb] = part;
+  } else {
+    // plain bf16 store of the accumulator: DOWN (Y), GATE_GRAD (dXp), WGRAD (dW)
+    size_t row;
+    bool row_ok = true;
+    if (MODE == GEMM_WGRAD) {
+      row = (size_t)tl.e * a.M + tl.m0 + r;
+      row_ok = tl.m0 + r < a.M;
+    } else {
+      row = (size_t)tl.row0 + r;
+    }
+    uint16_t* orow = a.out0 + row * a.ld_out0;
+    for (int c = 0; c < BN; c += 16) {
+      float v[16];
+      if (MODE == GEMM_WGRAD && tl.nkb == 0) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) v[i] = 0.f;
+      } else {
+        tmem_ld16(trow + c, v);
+        tmem_ld_wait();
+      }
+      if (row_ok) {
+#pragma unroll
+        for (int h = 0; h < 16; h += 8) {
+          const int col = tl.n0 + c + h;
+          if (col < a.N) store8_bf16(orow + col, v + h);
+        }
+      }
+    }
+  }
+}
+
+// ---------------------------------------------------------------- the kernel
+template <int MODE>
+__global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __grid_constant__ GemmArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + STAGES * A_STAGE_BYTES;
+  GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WaitCtl wc{a.status, a.budget_ns};
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bars->tmem_full[s], 1);
+      mbar_init(&bars->tmem_empty[s], 4);
+    }
+    mbar_init(&bars->drain, 1);
+    mbar_fence_init();
+    fence_proxy_async();
+    tma_prefetch_desc(&a.tmA);
+    tma_prefetch_desc(&a.tmB);
+  }
+  if (warp == 1) {
+    tmem_alloc(&bars->tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+  const int total = total_tiles<MODE>(a);
+  constexpr bool A_MN = (MODE == GEMM_WGRAD);
+  constexpr bool B_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD || MODE == GEMM_WGRAD);
+
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const Tile tl = decode_tile<MODE>(a, t);
+        for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(&bars->empty[s], ph ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
+          load_stage<MODE>(a, tl, kb, sA + s * A_STAGE_BYTES, sB + s * B_STAGE_BYTES, &bars->full[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_bf16(BLOCK_M, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
+      uint32_t it = 0, acc_it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const Tile tl = decode_tile<MODE>(a, t);
+        if (tl.nkb == 0) continue;
+        const int as = acc_it & 1;
+        const uint32_t aph = (acc_it >> 1) & 1;
+        if (!mbar_wait(&bars->tmem_empty[as], aph ^ 1, wc, SITE_TMEM_EMPTY, t)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + as * BN;
+        for (int kb = 0; kb < tl.nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait(&bars->full[s], ph, wc, SITE_FULL, t)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES);
+          const uint32_t b_addr = smem_u32(sB + s * B_STAGE_BYTES);
+#pragma unroll
+          for (int k16 = 0; k16 < BK / 16; ++k16) {
+            // K-major: 16 k-elements = 32 bytes inside the swizzled row; MN-major: 16 k-rows of 128 bytes
+            const uint64_t da = A_MN ? make_smem_desc(a_addr + k16 * 2048, MN_BOX_BYTES, 1024)
+                                     : make_smem_desc(a_addr + k16 * 32, 16, 1024);
+            const uint64_t db = B_MN ? make_smem_desc(b_addr + k16 * 2048, MN_BOX_BYTES, 1024)
+                                     : make_smem_desc(b_addr + k16 * 32, 16, 1024);
+            tc_mma_bf16(d_tmem, da, db, idesc, (kb | k16) != 0);
+          }
+          tc_commit(&bars->empty[s]);  // frees the smem stage once these MMAs have read it
+        }
+        if (!ok) break;
+        tc_commit(&bars->tmem_full[as]);  // accumulator complete
+        ++acc_it;
+      }
+      if (!ok || *reinterpret_cast<volatile int*>(&a.status->abort)) {
+        // leave only after the tensor core has stopped touching shared memory and TMEM
+        tc_commit(&bars->drain);
+        const WaitCtl shortwc{a.status, 20ull * 1000 * 1000};
+        mbar_wait(&bars->drain, 0, shortwc, SITE_DRAIN, 0);
+      }
+    }
+  } else {
+    // ------------------------------------------------ epilogue warps
+    const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+    uint32_t acc_it = 0;
+    for (int t = blockIdx.x; t < total; t += gridDim.x) {
+      const Tile tl = decode_tile<MODE>(a, t);
+      if (tl.nkb == 0) {
+        epilogue_tile<MODE>(a, tl, 0, quad, lane);  // WGRAD of an expert without rows: zeros
+        continue;
+      }
+      const int as = acc_it & 1;
+      const uint32_t aph = (acc_it >> 1) & 1;
+      if (!mbar_wait(&bars->tmem_full[as], aph, wc, SITE_TMEM_FULL, t)) break;
+      tc_fence_after_sync();
+      epilogue_tile<MODE>(a, tl, tmem_base + as * BN, quad, lane);
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars->tmem_empty[as]);
+      ++acc_it;
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  if (*reinterpret_cast<volatile int*>(&a.status->abort)) __nanosleep(200000);  // let in-flight copies land
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int MODE>
+static cudaError_t launch_mode(const GemmArgs& a, int num_sms, cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(grouped_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)GEMM_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  grouped_gemm_kernel<MODE><<<num_sms, GEMM_THREADS, GEMM_SMEM_BYTES, s>>>(a);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_gemm(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches) {
+  ++*launches;
+  switch (mode) {
+    case GEMM_GATE_UP: return launch_mode<GEMM_GATE_UP>(a, num_sms, s);
+    case GEMM_DOWN: return launch_mode<GEMM_DOWN>(a, num_sms, s);
+    case GEMM_ACT_GRAD: return launch_mode<GEMM_ACT_GRAD>(a, num_sms, s);
+    case GEMM_GATE_GRAD: return launch_mode<GEMM_GATE_GRAD>(a, num_sms, s);
+    case GEMM_WGRAD: return launch_mode<GEMM_WGRAD>(a, num_sms, s);
+  }
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace moe

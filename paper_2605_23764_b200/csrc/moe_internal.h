@@ -1,0 +1,100 @@
+// Host-side declarations shared by the translation units of libmoe_b200: problem dimensions,
+// workspace views and the launch functions of each kernel family.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace moe {
+
+struct Dims {
+  int T, d, E, k, S, F;
+  int Ep() const { return E + S; }
+  int kp() const { return k + S; }
+  int slots() const { return T * (k + S); }
+};
+
+// Row capacity of the padded expert-ordered row space: every expert segment starts on a
+// multiple of BLOCK_M, so at most BLOCK_M-1 padding rows per expert.
+inline int padded_rows_max(int T_max, int kp, int Ep) {
+  long r = (long)T_max * kp + (long)Ep * (BLOCK_M - 1);
+  return (int)(((r + BLOCK_M - 1) / BLOCK_M) * BLOCK_M);
+}
+
+constexpr int LAYOUT_CHUNK = 2048;  // flat slots per block of the layout kernels (8 warps x 256)
+
+// Device arrays describing one dispatch layout.
+struct LayoutView {
+  int* counts;       // [Ep]
+  int* offsets;      // [Ep+1]  exclusive scan of counts (unpadded rows)
+  int* row_of;       // [slots] unpadded row of each slot, -1 if the slot's expert id is invalid
+  int* src_of;       // [slots] slot of each unpadded row
+  int* prow_of;      // [slots] padded row of each slot (-1 if invalid)
+  int* pad_off;      // [Ep+1]  first padded row of each expert (multiple of BLOCK_M)
+  int* mb_start;     // [Ep+1]  first M-block of each expert
+  int* mblk_expert;  // [R_pad_max / BLOCK_M] expert of each M-block
+  int* meta;         // [8]     {num_mblocks, R_pad, rows, 0...}
+  int* blk_hist;     // [nblk][Ep] per-block histograms, then per-block exclusive prefixes
+};
+
+// ---- route_layout.cu
+cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, int* topk_ids, float* topk_w,
+                         int* counts, cudaStream_t s, int* launches);
+cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView& lv, DevStatus* status,
+                          cudaStream_t s, int* launches);
+
+// ---- permute.cu
+// Xp[p] = src[token of padded row p] (zeros on padding rows); optionally prow_w[p] = routing weight
+// of the row (1 for shared experts, 0 on padding rows).
+cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& dm, const LayoutView& lv,
+                          uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches);
+// out[t] = sum_j rows[prow_of[t*kp+j]] in slot order, fp32 accumulate, bf16 result.
+cudaError_t launch_combine(const uint16_t* rows, const Dims& dm, const LayoutView& lv, uint16_t* out,
+                           cudaStream_t s, int* launches);
+// d_topk_w[t][j] = sum_nb partial[prow_of[t*kp+j]][nb]
+cudaError_t launch_dw_reduce(const float* partial, int nparts, const Dims& dm, const LayoutView& lv,
+                             float* d_topk_w, cudaStream_t s, int* launches);
+
+// ---- gemm_tc.cu (tcgen05 grouped GEMMs)
+enum GemmMode : int {
+  GEMM_GATE_UP = 0,    // H = Xp . W_gate_up[e]^T, epilogue A = w * silu(g) * u     (fwd GMM1 + SwiGLU)
+  GEMM_DOWN = 1,       // Y = A . W_down[e]^T                                        (fwd GMM2)
+  GEMM_ACT_GRAD = 2,   // dA = dOutp . W_down[e], epilogue SwiGLU_grad -> dH, d_w    (bwd act_grad + SwiGLU_grad)
+  GEMM_GATE_GRAD = 3,  // dXp = dH . W_gate_up[e]                                    (bwd gate_grad)
+  GEMM_WGRAD = 4,      // dW[e] = P_e^T . Q_e over the expert's rows                 (bwd w1_grad / w2_grad)
+};
+
+struct GemmArgs {
+  CUtensorMap tmA;     // A operand
+  CUtensorMap tmB;     // B operand
+  // tile table
+  const int* mblk_expert;
+  const int* mb_start;
+  const int* counts;
+  const int* meta;
+  int Ep;
+  int n_tiles_n;       // tiles along N per M-block (row-space modes) / per expert (WGRAD)
+  int n_tiles_m;       // WGRAD only: tiles along M per expert
+  int K;               // reduction length (row-space modes)
+  int N;               // output columns (for masking); WGRAD: columns of dW
+  int M;               // WGRAD: rows of dW per expert
+  int b_rows_per_expert;  // rows of the B tensor map per expert slab
+  int F;               // intermediate size (GATE_UP / ACT_GRAD epilogues)
+  // epilogue tensors
+  uint16_t* out0;      // GATE_UP: A; DOWN: Y; ACT_GRAD: dH; GATE_GRAD: dXp; WGRAD: dW
+  uint16_t* out1;      // GATE_UP: H (may be NULL)
+  const uint16_t* in0; // ACT_GRAD: H
+  const float* prow_w; // GATE_UP, ACT_GRAD: routing weight per padded row
+  float* dw_partial;   // ACT_GRAD: [R_pad][n_tiles_n] partial <dA_unweighted, a> (may be NULL)
+  long ld_out0, ld_out1, ld_in0;
+  DevStatus* status;
+  uint64_t budget_ns;
+};
+
+cudaError_t launch_gemm(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
+size_t gemm_smem_bytes();
+
+}  // namespace moe

@@ -1,0 +1,116 @@
+// Permute-gather (Dispatch / backward Dispatch on one GPU), combine (Combine / backward Combine)
+// and the small reduction that finishes the routing-weight gradient.  All three are pure
+// HBM-bandwidth work: 16-byte vector accesses, one row handled by one block at a time.
+#include "moe_internal.h"
+
+namespace moe {
+
+constexpr int PERM_THREADS = 128;
+
+__device__ __forceinline__ uint4 ld_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+// dst[p][:] = src[token(p)][:] for every padded row p < R_pad; padding rows are zero-filled so
+// that reductions over an expert's rows (weight gradients) may run over whole M-blocks.
+__global__ void __launch_bounds__(PERM_THREADS) gather_rows_kernel(const uint16_t* __restrict__ src,
+                                                                    const float* __restrict__ topk_w, int d, int k,
+                                                                    int kp, LayoutView lv,
+                                                                    uint16_t* __restrict__ dst,
+                                                                    float* __restrict__ prow_w) {
+  const int r_pad = lv.meta[1];
+  const int nvec = d >> 3;
+  for (int p = blockIdx.x; p < r_pad; p += gridDim.x) {
+    const int e = lv.mblk_expert[p / BLOCK_M];
+    const int local = p - lv.pad_off[e];
+    const bool valid = local < lv.counts[e];
+    uint4* out = reinterpret_cast<uint4*>(dst + (size_t)p * d);
+    if (valid) {
+      const int slot = lv.src_of[lv.offsets[e] + local];
+      const int t = slot / kp, j = slot - t * kp;
+      const uint4* in = reinterpret_cast<const uint4*>(src + (size_t)t * d);
+      for (int v = threadIdx.x; v < nvec; v += PERM_THREADS) out[v] = ld_nc_v4(in + v);
+      if (prow_w && threadIdx.x == 0) prow_w[p] = j < k ? topk_w[(size_t)t * k + j] : 1.0f;
+    } else {
+      for (int v = threadIdx.x; v < nvec; v += PERM_THREADS) out[v] = make_uint4(0, 0, 0, 0);
+      if (prow_w && threadIdx.x == 0) prow_w[p] = 0.0f;
+    }
+  }
+}
+
+cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& dm, const LayoutView& lv,
+                          uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches) {
+  int grid = rows_cap < 148 * 16 ? rows_cap : 148 * 16;
+  if (grid < 1) grid = 1;
+  gather_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// out[t][:] = sum_j rows[prow_of[t*kp+j]][:], j ascending, fp32 accumulation, one bf16 rounding.
+// Rows already carry their routing weight (it is applied where the activations are produced).
+__global__ void __launch_bounds__(PERM_THREADS) combine_rows_kernel(const uint16_t* __restrict__ rows, int T, int d,
+                                                                     int kp, const int* __restrict__ prow_of,
+                                                                     uint16_t* __restrict__ out) {
+  const int nvec = d >> 3;
+  for (int t = blockIdx.x; t < T; t += gridDim.x) {
+    for (int v = threadIdx.x; v < nvec; v += PERM_THREADS) {
+      float acc[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+      for (int j = 0; j < kp; ++j) {
+        int p = prow_of[(size_t)t * kp + j];
+        if (p < 0) continue;
+        uint4 r = ld_nc_v4(reinterpret_cast<const uint4*>(rows + (size_t)p * d) + v);
+        acc[0] += bf16lo(r.x); acc[1] += bf16hi(r.x);
+        acc[2] += bf16lo(r.y); acc[3] += bf16hi(r.y);
+        acc[4] += bf16lo(r.z); acc[5] += bf16hi(r.z);
+        acc[6] += bf16lo(r.w); acc[7] += bf16hi(r.w);
+      }
+      uint4 o;
+      o.x = pack_bf16x2(acc[0], acc[1]);
+      o.y = pack_bf16x2(acc[2], acc[3]);
+      o.z = pack_bf16x2(acc[4], acc[5]);
+      o.w = pack_bf16x2(acc[6], acc[7]);
+      reinterpret_cast<uint4*>(out + (size_t)t * d)[v] = o;
+    }
+  }
+}
+
+cudaError_t launch_combine(const uint16_t* rows, const Dims& dm, const LayoutView& lv, uint16_t* out,
+                           cudaStream_t s, int* launches) {
+  int grid = dm.T < 148 * 16 ? dm.T : 148 * 16;
+  if (grid < 1) grid = 1;
+  combine_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(rows, dm.T, dm.d, dm.kp(), lv.prow_of, out);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// d_topk_w[t][j] = sum over the act_grad column tiles of their per-row partial dot products,
+// in tile order (deterministic).
+__global__ void dw_reduce_kernel(const float* __restrict__ partial, int nparts, int T, int k, int kp,
+                                 const int* __restrict__ prow_of, float* __restrict__ d_topk_w) {
+  int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= T * k) return;
+  int t = i / k, j = i - t * k;
+  int p = prow_of[(size_t)t * kp + j];
+  float s = 0.f;
+  if (p >= 0)
+    for (int q = 0; q < nparts; ++q) s += partial[(size_t)p * nparts + q];
+  d_topk_w[i] = s;
+}
+
+cudaError_t launch_dw_reduce(const float* partial, int nparts, const Dims& dm, const LayoutView& lv,
+                             float* d_topk_w, cudaStream_t s, int* launches) {
+  int n = dm.T * dm.k;
+  if (n == 0) return cudaSuccess;
+  dw_reduce_kernel<<<(n + 255) / 256, 256, 0, s>>>(partial, nparts, dm.T, dm.k, dm.kp(), lv.prow_of, d_topk_w);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+}  // namespace moe

@@ -1,0 +1,264 @@
+// Routing (softmax top-k) and the dispatch layout (per-expert histogram, prefix scan, stable
+// permutation, M-block table).  Integer results are bit-exact by construction: every count and
+// rank is an integer sum whose value does not depend on evaluation order.
+#include <limits.h>
+
+#include "moe_internal.h"
+
+namespace moe {
+
+// ------------------------------------------------------------------------------------------
+// Router: one warp per token.  Expert e is held by lane e%32 in register e/32.
+// Selection compares raw logits (softmax is monotone), ties go to the lower expert id, slots
+// come out in descending logit order.  Scores: fp32 softmax over all E, max-subtracted.
+// ------------------------------------------------------------------------------------------
+template <int NPL>
+__global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ logits, int T, int E, int k,
+                                                     int renorm, int* __restrict__ topk_ids,
+                                                     float* __restrict__ topk_w, int* __restrict__ counts) {
+  const int lane = threadIdx.x & 31;
+  const int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (t >= T) return;
+  const float* row = logits + (size_t)t * E;
+  float v[NPL];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < NPL; ++i) {
+    int e = i * 32 + lane;
+    v[i] = e < E ? row[e] : -INFINITY;
+    mx = fmaxf(mx, v[i]);
+  }
+#pragma unroll
+  for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  float den = 0.f;
+#pragma unroll
+  for (int i = 0; i < NPL; ++i)
+    if (i * 32 + lane < E) den += expf(v[i] - mx);
+#pragma unroll
+  for (int off = 16; off; off >>= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
+
+  uint32_t taken = 0;
+  int my_id = 0;
+  float my_p = 0.f, wsum = 0.f;
+  for (int j = 0; j < k; ++j) {
+    float bv = 0.f;
+    int bi = INT_MAX;
+#pragma unroll
+    for (int i = 0; i < NPL; ++i) {
+      int e = i * 32 + lane;
+      if (e < E && !((taken >> i) & 1u) && (bi == INT_MAX || v[i] > bv)) { bv = v[i]; bi = e; }
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) {
+      float ov = __shfl_xor_sync(0xffffffffu, bv, off);
+      int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+      if (oi != INT_MAX && (bi == INT_MAX || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
+    }
+    if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
+    float p = expf(bv - mx) / den;
+    if (lane == j) { my_id = bi; my_p = p; }
+    wsum += p;
+  }
+  if (lane < k) {
+    if (renorm) my_p /= wsum;
+    topk_ids[(size_t)t * k + lane] = my_id;
+    topk_w[(size_t)t * k + lane] = my_p;
+    if (counts) atomicAdd(&counts[my_id], 1);
+  }
+}
+
+cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, int* topk_ids, float* topk_w,
+                         int* counts, cudaStream_t s, int* launches) {
+  if (T == 0) return cudaSuccess;
+  if (counts) {
+    cudaError_t e = cudaMemsetAsync(counts, 0, sizeof(int) * (size_t)E, s);
+    if (e != cudaSuccess) return e;
+  }
+  const int threads = 256, tokens_per_block = threads / 32;
+  dim3 grid((T + tokens_per_block - 1) / tokens_per_block);
+  const int npl = (E + 31) / 32;
+#define MOE_ROUTE_CASE(N) \
+  route_kernel<N><<<grid, threads, 0, s>>>(logits, T, E, k, renorm ? 1 : 0, topk_ids, topk_w, counts)
+  if (npl <= 1) MOE_ROUTE_CASE(1);
+  else if (npl <= 2) MOE_ROUTE_CASE(2);
+  else if (npl <= 4) MOE_ROUTE_CASE(4);
+  else if (npl <= 8) MOE_ROUTE_CASE(8);
+  else if (npl <= 16) MOE_ROUTE_CASE(16);
+  else MOE_ROUTE_CASE(32);
+#undef MOE_ROUTE_CASE
+  ++*launches;
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Dispatch layout.  Flat slot i = t*kp + j; block b owns slots [b*CHUNK, (b+1)*CHUNK), warp w of
+// the block owns 256 consecutive slots of it, processed 32 at a time in slot order.
+// ------------------------------------------------------------------------------------------
+constexpr int LAYOUT_THREADS = 256;
+constexpr int LAYOUT_WARPS = LAYOUT_THREADS / 32;
+constexpr int SLOTS_PER_WARP = LAYOUT_CHUNK / LAYOUT_WARPS;
+
+__device__ __forceinline__ int slot_expert(const int* __restrict__ ids, int i, int k, int kp, int E) {
+  int t = i / kp, j = i - t * kp;
+  if (j >= k) return E + (j - k);
+  int e = ids[(size_t)t * k + j];
+  return (e >= 0 && e < E) ? e : -1;
+}
+
+// Per-warp histograms of this block's chunk into shared memory whist[LAYOUT_WARPS][Ep].
+__device__ __forceinline__ void chunk_histogram(const int* __restrict__ ids, int n, int k, int kp, int E, int Ep,
+                                                int* whist) {
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int q = threadIdx.x; q < LAYOUT_WARPS * Ep; q += LAYOUT_THREADS) whist[q] = 0;
+  __syncthreads();
+  int* mine = whist + warp * Ep;
+  const int base = blockIdx.x * LAYOUT_CHUNK + warp * SLOTS_PER_WARP;
+  for (int g = 0; g < SLOTS_PER_WARP; g += 32) {
+    int i = base + g + lane;
+    int e = i < n ? slot_expert(ids, i, k, kp, E) : -1;
+    uint32_t peers = __match_any_sync(0xffffffffu, e);
+    if (e >= 0 && lane == __ffs(peers) - 1) mine[e] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(LAYOUT_THREADS) layout_hist_kernel(const int* __restrict__ ids, int n, int k,
+                                                                      int kp, int E, int Ep,
+                                                                      int* __restrict__ blk_hist) {
+  extern __shared__ int whist[];
+  chunk_histogram(ids, n, k, kp, E, Ep, whist);
+  for (int e = threadIdx.x; e < Ep; e += LAYOUT_THREADS) {
+    int tot = 0;
+#pragma unroll
+    for (int w = 0; w < LAYOUT_WARPS; ++w) tot += whist[w * Ep + e];
+    blk_hist[(size_t)blockIdx.x * Ep + e] = tot;
+  }
+}
+
+// One block.  (1) per expert, exclusive scan of the block histograms over blocks (warp per expert);
+// (2) exclusive scans over experts for row offsets and M-block starts; (3) M-block -> expert table.
+__global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, LayoutView lv) {
+  extern __shared__ int sm[];
+  int* s_counts = sm;            // [Ep]
+  int* s_mbstart = sm + Ep;      // [Ep+1]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int e = warp; e < Ep; e += 32) {
+    int carry = 0;
+    for (int b0 = 0; b0 < nblk; b0 += 32) {
+      int b = b0 + lane;
+      int v = b < nblk ? lv.blk_hist[(size_t)b * Ep + e] : 0;
+      int incl = v;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        int o = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += o;
+      }
+      if (b < nblk) lv.blk_hist[(size_t)b * Ep + e] = carry + incl - v;
+      carry += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) s_counts[e] = carry;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    int carry_rows = 0, carry_mb = 0;
+    for (int e0 = 0; e0 < Ep; e0 += 32) {
+      int e = e0 + lane;
+      int c = e < Ep ? s_counts[e] : 0;
+      int m = (c + BLOCK_M - 1) / BLOCK_M;
+      int ic = c, im = m;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        int oc = __shfl_up_sync(0xffffffffu, ic, off);
+        int om = __shfl_up_sync(0xffffffffu, im, off);
+        if (lane >= off) { ic += oc; im += om; }
+      }
+      if (e < Ep) {
+        lv.counts[e] = c;
+        lv.offsets[e] = carry_rows + ic - c;
+        int ms = carry_mb + im - m;
+        s_mbstart[e] = ms;
+        lv.mb_start[e] = ms;
+        lv.pad_off[e] = ms * BLOCK_M;
+      }
+      carry_rows += __shfl_sync(0xffffffffu, ic, 31);
+      carry_mb += __shfl_sync(0xffffffffu, im, 31);
+    }
+    if (lane == 0) {
+      lv.offsets[Ep] = carry_rows;
+      s_mbstart[Ep] = carry_mb;
+      lv.mb_start[Ep] = carry_mb;
+      lv.pad_off[Ep] = carry_mb * BLOCK_M;
+      lv.meta[0] = carry_mb;
+      lv.meta[1] = carry_mb * BLOCK_M;
+      lv.meta[2] = carry_rows;
+    }
+  }
+  __syncthreads();
+  const int num_mb = s_mbstart[Ep];
+  for (int mb = threadIdx.x; mb < num_mb; mb += blockDim.x) {
+    int lo = 0, hi = Ep - 1;  // last expert whose mb_start <= mb
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (s_mbstart[mid] <= mb) lo = mid; else hi = mid - 1;
+    }
+    lv.mblk_expert[mb] = lo;
+  }
+}
+
+__global__ void __launch_bounds__(LAYOUT_THREADS) layout_rank_kernel(const int* __restrict__ ids, int n, int k,
+                                                                      int kp, int E, int Ep, LayoutView lv,
+                                                                      DevStatus* status) {
+  extern __shared__ int whist[];
+  chunk_histogram(ids, n, k, kp, E, Ep, whist);
+  // per expert: running base of each warp inside the block = block prefix + earlier warps
+  for (int e = threadIdx.x; e < Ep; e += LAYOUT_THREADS) {
+    int run = lv.blk_hist[(size_t)blockIdx.x * Ep + e];
+#pragma unroll
+    for (int w = 0; w < LAYOUT_WARPS; ++w) {
+      int c = whist[w * Ep + e];
+      whist[w * Ep + e] = run;
+      run += c;
+    }
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  int* mine = whist + warp * Ep;
+  const int base = blockIdx.x * LAYOUT_CHUNK + warp * SLOTS_PER_WARP;
+  for (int g = 0; g < SLOTS_PER_WARP; g += 32) {
+    int i = base + g + lane;
+    int e = i < n ? slot_expert(ids, i, k, kp, E) : -1;
+    uint32_t peers = __match_any_sync(0xffffffffu, e);
+    int r = 0;
+    if (e >= 0) r = mine[e] + __popc(peers & ((1u << lane) - 1u));
+    __syncwarp();
+    if (e >= 0 && lane == __ffs(peers) - 1) mine[e] += __popc(peers);
+    __syncwarp();
+    if (i < n) {
+      if (e >= 0) {
+        int row = lv.offsets[e] + r;
+        lv.row_of[i] = row;
+        lv.prow_of[i] = lv.pad_off[e] + r;
+        lv.src_of[row] = i;
+      } else {
+        lv.row_of[i] = -1;
+        lv.prow_of[i] = -1;
+        note(status, /*MOE_ERR_BAD_EXPERT_ID*/ 1, i);  // the slot is dropped, the layer carries on
+      }
+    }
+  }
+}
+
+cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView& lv, DevStatus* status,
+                          cudaStream_t s, int* launches) {
+  const int n = dm.slots(), Ep = dm.Ep();
+  const int nblk = n > 0 ? (n + LAYOUT_CHUNK - 1) / LAYOUT_CHUNK : 1;
+  const size_t sm_hist = sizeof(int) * (size_t)LAYOUT_WARPS * Ep;
+  layout_hist_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv.blk_hist);
+  layout_scan_kernel<<<1, 1024, sizeof(int) * (size_t)(2 * Ep + 1), s>>>(nblk, Ep, lv);
+  layout_rank_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv, status);
+  *launches += 3;
+  return cudaGetLastError();
+}
+
+}  // namespace moe
