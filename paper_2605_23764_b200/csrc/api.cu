@@ -418,12 +418,12 @@ int moe_layout(moe_ctx* c, const int32_t* topk_ids, int32_t T, int32_t* counts, 
 
 int moe_ffn_fwd(moe_ctx* c, const uint16_t* x, const int32_t* topk_ids, const float* topk_w,
                 const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* out, int32_t T, void* stream) {
-  if (!c || !x || !topk_ids || !topk_w || !W_gate_up || !W_down || !out || T < 0 || T > c->shape.T_max)
-    return MOE_ERR_INVALID_ARG;
-  if (!aligned16(x) || !aligned16(W_gate_up) || !aligned16(W_down) || !aligned16(out)) return MOE_ERR_INVALID_ARG;
+  if (!c || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
   c->launches = 0;
   c->last_stream = static_cast<cudaStream_t>(stream);
-  if (T == 0) return MOE_OK;
+  if (T == 0) return MOE_OK;  // nothing to compute; tensor pointers of an empty batch may be NULL
+  if (!x || !topk_ids || !topk_w || !W_gate_up || !W_down || !out) return MOE_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(W_gate_up) || !aligned16(W_down) || !aligned16(out)) return MOE_ERR_INVALID_ARG;
   return run_fwd(c, x, topk_ids, topk_w, W_gate_up, W_down, out, T, c->last_stream);
 }
 
