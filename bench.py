@@ -1,0 +1,457 @@
+#!/usr/bin/env python
+"""Benchmark of the Dispatch->Combine MoE-FFN layer on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--serial] [--impl reference]
+
+One step = one pass of the whole hot path on one batch of seeded synthetic input: routing,
+forward (dispatch layout, permute-gather, grouped GEMM gate+up with SwiGLU, grouped GEMM down,
+combine) and, for the training workloads, backward (the seven backward operators).  Rank 0
+prints ONE JSON line.  Throughput counts 6*R*d*F FLOP per forward and 12*R*d*F per backward
+(R = tokens x experts per token).  With N > 1 every rank runs an independent replica on its
+own GPU (the layer is not sharded; there is no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import configs  # noqa: E402
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+# ----------------------------------------------------------------------------------------------
+# algorithmic work per operator (what the method must compute / move: inputs read once, outputs
+# written once; padding rows and re-reads are not credited)
+# ----------------------------------------------------------------------------------------------
+def phase_work(cfg, train):
+    R, d, F, Ep, T = cfg.R, cfg.d, cfg.F, cfg.Ep, cfg.T
+    bf = 2
+    W1, W2 = Ep * 2 * F * d * bf, Ep * d * F * bf
+    work = {
+        "gather": (0.0, T * d * bf + R * d * bf),
+        "gemm_gate_up": (2.0 * R * d * 2 * F, R * d * bf + W1 + R * F * bf + (R * 2 * F * bf if train else 0)),
+        "gemm_down": (2.0 * R * F * d, R * F * bf + W2 + R * d * bf),
+        "combine": (0.0, R * d * bf + T * d * bf),
+    }
+    if train:
+        work.update({
+            "bwd_gather": (0.0, T * d * bf + R * d * bf),
+            "act_grad": (2.0 * R * d * F, R * d * bf + W2 + R * 2 * F * bf * 2),
+            "wgrad_down": (2.0 * R * d * F, R * d * bf + R * F * bf + W2),
+            "gate_grad": (2.0 * R * 2 * F * d, R * 2 * F * bf + W1 + R * d * bf),
+            "wgrad_gate_up": (2.0 * R * 2 * F * d, R * 2 * F * bf + R * d * bf + W1),
+            "bwd_combine": (0.0, R * d * bf + T * d * bf),
+        })
+    return work
+
+
+def step_flops(cfg, train):
+    return cfg.flops_fwd() * (3.0 if train else 1.0)
+
+
+def step_min_bytes(cfg, train):
+    """Minimum HBM traffic of a step: weights, activations in and out, weight gradients."""
+    bf = 2
+    W = cfg.weight_bytes()
+    io = 2 * cfg.T * cfg.d * bf
+    if not train:
+        return W + io
+    saved = 2 * cfg.R * 2 * cfg.F * bf  # pre-activations written by forward, read by backward
+    return 3 * W + 2 * io + cfg.T * cfg.d * bf + saved
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def max_over_ranks(v, world):
+    if world == 1:
+        return v
+    import torch.distributed as dist
+    t = torch.tensor([v], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle legs (rank 0 only): a bounded sample of the same workload
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(cfg, train, n_experts, inputs=None, max_rows=None):
+    """Times the oracle on the rows of `n_experts` experts (forward, and backward if `train`).
+
+    Returns (seconds, flops, description).  A weight gradient and an expert's rows need only that
+    expert's slabs, so the sample is an exact sub-problem of the workload."""
+    import oracle
+    dev = "cpu"
+    x = inputs["x"].cpu() if inputs else configs.make_x(cfg, dev)
+    logits = inputs["logits"].cpu() if inputs else configs.make_logits(cfg, x)
+    ids, w = oracle.route(logits, cfg.k, cfg.renorm)
+    ids_t = torch.from_numpy(ids)
+    dout = (inputs["dout"].cpu() if inputs else configs.make_dout(cfg, dev)) if train else None
+    counts = torch.bincount(ids_t.flatten().long(), minlength=cfg.E)
+    order = torch.argsort(counts, descending=True)
+    picked = [int(e) for e in order[len(order) // 2: len(order) // 2 + n_experts]]  # median-loaded experts
+    secs, flops, rows = 0.0, 0.0, 0
+    for e in picked:
+        tok, slot = torch.nonzero(ids_t == e, as_tuple=True)
+        if max_rows is not None:
+            tok, slot = tok[:max_rows], slot[:max_rows]
+        n = tok.numel()
+        if n == 0:
+            continue
+        W1 = configs.w_gate_up_slab(cfg, e)[None]
+        W2 = configs.w_down_slab(cfg, e)[None]
+        sub_ids = torch.zeros(n, 1, dtype=torch.int32)
+        sub_w = torch.from_numpy(w)[tok, slot][:, None]
+        xs = x[tok]
+        t0 = time.perf_counter()
+        oracle.fwd(xs, sub_ids, sub_w, W1, W2)
+        if train:
+            oracle.bwd(dout[tok], xs, sub_ids, sub_w, W1, W2)
+        secs += time.perf_counter() - t0
+        flops += 6.0 * n * cfg.d * cfg.F * (3.0 if train else 1.0)
+        rows += n
+    desc = (f"{'fwd+bwd' if train else 'fwd'} of {rows} rows of {len(picked)} median-loaded experts "
+            f"(of {cfg.R} rows, {cfg.Ep} experts)")
+    return secs, flops, desc
+
+
+def calibrate_sample(cfg, train, target_s=15.0):
+    """(experts, rows per expert) giving roughly `target_s` seconds of oracle work.  The rate is a
+    fixed estimate of the plain-loop fp64 oracle (its weight-gradient loop of a one-expert
+    sub-problem runs on one thread), not a measurement."""
+    rows_per_expert = max(1, int(cfg.T * cfg.k / cfg.E))
+    flop_per_row = 6.0 * cfg.d * cfg.F * (3.0 if train else 1.0)
+    est_rate = 3.0e9 if train else 1.0e10
+    rows = max(1, int(target_s * est_rate / flop_per_row))
+    if rows <= rows_per_expert:
+        return 1, rows
+    return int(min(cfg.E, max(1, round(rows / rows_per_expert)))), None
+
+
+def run_reference(args, cfg, train):
+    import oracle
+    n_exp, max_rows = calibrate_sample(cfg, train, target_s=4.0)
+    times, flops, desc = [], 0.0, ""
+    for i in range(args.warmup + args.steps):
+        secs, flops, desc = oracle_sample(cfg, train, n_exp, max_rows=max_rows)
+        if i >= args.warmup:
+            times.append(secs)
+    ms = 1e3 * sum(times) / len(times)
+    val = flops / (ms * 1e-3) / 1e12
+    cfg_desc = workload_desc(cfg, train, args)
+    cfg_desc["launch"] = "none (CPU oracle on host cores)"
+    line = {
+        "impl": "reference", "metric": "moe_ffn_dispatch_to_combine_tflops", "value": val, "unit": "TFLOP/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": cfg_desc, "gpu_launches": 0,
+        "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_desc(cfg, train, args):
+    return {"workload": cfg.name, "T": cfg.T, "d": cfg.d, "E": cfg.E, "top_k": cfg.k, "shared": cfg.S, "F": cfg.F,
+            "pass": "route+fwd+bwd" if train else "route+fwd",
+            "launch": "serial kernels" if args.serial else "fused persistent",
+            "l2": "weights and expert-ordered activations exceed the 126 MB L2 (no flush needed)"
+            if cfg.weight_bytes() > 4e8 else "L2 flushed between timed steps"}
+
+
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, help="index into BASELINE.json configs (default: the training step)")
+    ap.add_argument("--serial", action="store_true", help="one kernel launch per operator instead of the fused launch")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--fwd-only", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    cfg = configs.CONFIGS[args.config]
+    if args.small:
+        v = [int(q) for q in args.small.split(",")]
+        cfg = configs.small_variant(cfg, v[0], v[1], v[2], v[3] if len(v) > 3 else None)
+    train = cfg.bwd and not args.fwd_only
+
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, cfg, train)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the layer has no CPU path)")
+    from paper_2605_23764_b200 import MoeLayer, binding as B
+
+    world, rank, local = dist_setup(args.gpus)
+    torch.cuda.set_device(local)
+    peaks = load_peaks()
+
+    inp = configs.make_inputs(cfg, "cuda")
+    x, W1, W2, logits = inp["x"], inp["W_gate_up"], inp["W_down"], inp["logits"]
+    dout = inp.get("dout")
+    layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=train,
+                     serial=args.serial)
+    T = cfg.T
+    ids = torch.empty(T, cfg.k, dtype=torch.int32, device="cuda")
+    w = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
+    out = torch.empty_like(x)
+    if train:
+        dx, dW1, dW2 = torch.empty_like(x), torch.empty_like(W1), torch.empty_like(W2)
+        dw = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
+    flush = None
+    if cfg.weight_bytes() <= 4e8:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    launches = 0
+
+    def step():
+        nonlocal launches
+        B.moe_route(layer.ctx, logits, T, ids, w)
+        launches += layer.launches()
+        B.moe_ffn_fwd(layer.ctx, x, ids, w, W1, W2, out, T)
+        launches += layer.launches()
+        if train:
+            B.moe_ffn_bwd(layer.ctx, dout, x, ids, w, W1, W2, dx, dW1, dW2, dw, T)
+            launches += layer.launches()
+
+    # ---- device-resident timing --------------------------------------------------------------
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert layer.status() == (0, 0), "device-side error during warm-up"
+    B.moe_set_profiling(layer.ctx, True)
+    phase_sum, launches = {}, 0
+    sampler = ClockSampler(local)
+    sampler.start()
+    barrier(world)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush_ms = 0.0
+    ev0.record()
+    for _ in range(args.steps):
+        if flush is not None:
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(); flush.zero_(); f1.record()
+        B.moe_route(layer.ctx, logits, T, ids, w)
+        launches += layer.launches()
+        ph = B.moe_get_phase_ms(layer.ctx)
+        B.moe_ffn_fwd(layer.ctx, x, ids, w, W1, W2, out, T)
+        launches += layer.launches()
+        ph.update(B.moe_get_phase_ms(layer.ctx))
+        if train:
+            B.moe_ffn_bwd(layer.ctx, dout, x, ids, w, W1, W2, dx, dW1, dW2, dw, T)
+            launches += layer.launches()
+            ph.update(B.moe_get_phase_ms(layer.ctx))
+        for kname, v in ph.items():
+            phase_sum[kname] = phase_sum.get(kname, 0.0) + v
+        if flush is not None:
+            f1.synchronize()
+            flush_ms += f0.elapsed_time(f1)
+    ev1.record()
+    barrier(world)
+    clocks = sampler.stop()
+    elapsed_ms = ev0.elapsed_time(ev1) - flush_ms
+    elapsed_ms = max_over_ranks(elapsed_ms, world)
+    B.moe_set_profiling(layer.ctx, False)
+    code, detail = layer.status()
+    assert code == 0, f"device-side error {code} detail {detail:#x}"
+    ms_per_step = elapsed_ms / args.steps
+    flops = step_flops(cfg, train)
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # ---- roofline of the dominant kernel --------------------------------------------------------
+    work = phase_work(cfg, train)
+    phases_ms = {k: v / args.steps for k, v in phase_sum.items()}
+    peak_tf = peaks["bf16_tflops_sustained"] if ms_per_step * args.steps > 500 else peaks["bf16_tflops"]
+    peak_gb = peaks["hbm_gbs"]
+    dom = max((k for k in phases_ms if k in work), key=lambda k: phases_ms[k], default=None)
+    roofline = None
+    if dom:
+        fl, by = work[dom]
+        t_s = phases_ms[dom] * 1e-3
+        tensor_bound = fl / (peak_tf * 1e12) >= by / (peak_gb * 1e9)
+        if tensor_bound:
+            roofline = {"kernel": dom, "bound": "tensor", "achieved": fl / t_s / 1e12, "peak": peak_tf,
+                        "unit": "TFLOP/s"}
+        else:
+            roofline = {"kernel": dom, "bound": "hbm", "achieved": by / t_s / 1e9, "peak": peak_gb, "unit": "GB/s"}
+        roofline["frac"] = roofline["achieved"] / roofline["peak"]
+        roofline["peak_source"] = peaks["source"] + (" sustained" if peak_tf == peaks.get("bf16_tflops_sustained")
+                                                     and tensor_bound else "")
+        roofline["traffic"] = ncu_traffic(dom, cfg)
+        roofline["launch_ms"] = phases_ms[dom]
+    t_roof = max(flops / (peak_tf * 1e12), step_min_bytes(cfg, train) / (peak_gb * 1e9))
+    step_roofline = {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step,
+                     "flop_ms": flops / (peak_tf * 1e12) * 1e3,
+                     "hbm_ms": step_min_bytes(cfg, train) / (peak_gb * 1e9) * 1e3}
+
+    # ---- end to end through the host-buffer entry points ------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        pin = dict(pin_memory=True)
+        xh, lh = x.cpu().pin_memory(), logits.cpu().pin_memory()
+        idh = torch.empty(T, cfg.k, dtype=torch.int32, **pin)
+        wh = torch.empty(T, cfg.k, dtype=torch.float32, **pin)
+        oh = torch.empty(T, cfg.d, dtype=torch.bfloat16, **pin)
+        h2d = lh.numel() * 4 + xh.numel() * 2 + idh.numel() * 4 + wh.numel() * 4
+        d2h = idh.numel() * 4 + wh.numel() * 4 + oh.numel() * 2
+        if train:
+            doh = dout.cpu().pin_memory()
+            dxh = torch.empty(T, cfg.d, dtype=torch.bfloat16, **pin)
+            dwh = torch.empty(T, cfg.k, dtype=torch.float32, **pin)
+            h2d += doh.numel() * 2
+            d2h += dxh.numel() * 2 + dwh.numel() * 4
+
+        def e2e_step():
+            B.moe_route_host(layer.ctx, lh, T, idh, wh)
+            B.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, W1, W2, oh, T)
+            if train:
+                B.moe_ffn_bwd_host(layer.ctx, doh, W1, W2, dxh, dW1, dW2, dwh, T)
+
+        for _ in range(2):
+            e2e_step()
+        barrier(world)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            e2e_step()
+        e1.record()
+        barrier(world)
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / args.steps
+        assert layer.status()[0] == 0
+        assert torch.equal(oh.cuda(), out), "host-buffer path disagrees with the device-buffer path"
+        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # ---- CPU oracle baseline (rank 0, single-GPU run only) ----------------------------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n_exp, max_rows = calibrate_sample(cfg, train)
+        secs, fl, desc = oracle_sample(cfg, train, n_exp, inputs=inp, max_rows=max_rows)
+        cpu_baseline = {"value": fl / secs / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                        "sample": desc, "seconds": secs}
+
+    if rank == 0:
+        line = {
+            "metric": "moe_ffn_dispatch_to_combine_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": workload_desc(cfg, train, args), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "step_roofline": step_roofline, "phases_ms": phases_ms,
+            "cpu_baseline": cpu_baseline,
+        }
+        per_step = launches / max(1, args.steps)
+        line["config"]["launch"] = ("fused persistent" if per_step <= (4 if train else 3)
+                                    else "serial kernels (one launch per operator)")
+        line["config"]["launches_per_step"] = per_step
+        print(json.dumps(line), flush=True)
+    layer.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def ncu_traffic(phase, cfg):
+    """DRAM bytes per launch of `phase` on this workload from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+    if not os.path.exists(path):
+        return None
+    for ln in open(path):
+        parts = ln.split()
+        if len(parts) >= 3 and not ln.startswith("#") and parts[0] == phase and parts[1] == cfg.name:
+            return float(parts[2])
+    return None
+
+
+if __name__ == "__main__":
+    main()

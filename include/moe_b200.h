@@ -138,6 +138,36 @@ int moe_last_launch_count(const moe_ctx* ctx);
 /* Budget, in milliseconds, of every bounded device-side wait (default 2000). */
 int moe_set_wait_budget_ms(moe_ctx* ctx, int32_t ms);
 
+/* Per-operator device times.  With profiling on, every later call records CUDA events on its
+ * stream between the operators it launches (the operators of Section 2.2; a single persistent
+ * launch reports one entry).  moe_get_phase_ms synchronises on the last event of the context's
+ * last call and fills ms[MOE_NUM_PHASES] with that call's times (0 for operators it did not run). */
+enum {
+  MOE_PHASE_ROUTE = 0,
+  MOE_PHASE_LAYOUT = 1,        /* histogram + scan + permutation (Dispatch, index part) */
+  MOE_PHASE_GATHER = 2,        /* Dispatch, data part */
+  MOE_PHASE_GEMM_GATE_UP = 3,  /* GMM1 + SwiGLU */
+  MOE_PHASE_GEMM_DOWN = 4,     /* GMM2 */
+  MOE_PHASE_COMBINE = 5,
+  MOE_PHASE_BWD_GATHER = 6,    /* backward Dispatch */
+  MOE_PHASE_ACT_GRAD = 7,      /* GMM act_grad + SwiGLU_grad */
+  MOE_PHASE_DW_REDUCE = 8,     /* routing-weight gradient */
+  MOE_PHASE_WGRAD_DOWN = 9,    /* GMM w2_grad */
+  MOE_PHASE_GATE_GRAD = 10,    /* GMM gate_grad */
+  MOE_PHASE_WGRAD_GATE_UP = 11,/* GMM w1_grad */
+  MOE_PHASE_BWD_COMBINE = 12,
+  MOE_PHASE_FUSED_FWD = 13,    /* the single persistent forward launch */
+  MOE_PHASE_FUSED_BWD = 14,    /* the single persistent backward launch */
+  MOE_NUM_PHASES = 15,
+};
+int moe_set_profiling(moe_ctx* ctx, int32_t on);
+int moe_get_phase_ms(moe_ctx* ctx, float* ms);
+
+/* moe_route for host buffers: logits_host[T][E] is copied in, topk_ids_host / topk_w_host are
+ * filled from the device (valid once `stream` has been synchronised). */
+int moe_route_host(moe_ctx* ctx, const float* logits_host, int32_t T, int32_t* topk_ids_host,
+                   float* topk_w_host, void* stream);
+
 /* Test/diagnostic access to workspace tensors of the last forward/backward.  `which` is a
  * MOE_BUF_* id; *ptr receives a device pointer into the workspace (valid until the next call on
  * the context), *elems its element count.  Rows of expert-ordered tensors live in a padded row

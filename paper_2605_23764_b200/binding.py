@@ -19,7 +19,10 @@ _BUF_DTYPE = {k: (torch.bfloat16 if k in ("Xp", "H", "A", "Y", "dOutp", "dH", "d
 
 EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe_layout", "moe_ffn_fwd",
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
-           "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error"]
+           "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
+           "moe_set_profiling", "moe_get_phase_ms", "moe_route_host"]
+PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
+          "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
 
 class MoeShape(ctypes.Structure):
@@ -62,6 +65,9 @@ def load_library() -> ctypes.CDLL:
     lib.moe_last_launch_count.argtypes = [vp]
     lib.moe_set_wait_budget_ms.argtypes = [vp, i32]
     lib.moe_debug_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp), ctypes.POINTER(sz)]
+    lib.moe_set_profiling.argtypes = [vp, i32]
+    lib.moe_get_phase_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.moe_route_host.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -184,6 +190,24 @@ def moe_last_launch_count(ctx) -> int:
 
 def moe_set_wait_budget_ms(ctx, ms: int):
     _check(load_library().moe_set_wait_budget_ms(ctx, ms), "moe_set_wait_budget_ms")
+
+
+def moe_set_profiling(ctx, on: bool):
+    _check(load_library().moe_set_profiling(ctx, 1 if on else 0), "moe_set_profiling")
+
+
+def moe_get_phase_ms(ctx) -> dict:
+    """Device milliseconds of each operator of the context's last call (operators it ran only)."""
+    buf = (ctypes.c_float * len(PHASES))()
+    _check(load_library().moe_get_phase_ms(ctx, buf), "moe_get_phase_ms")
+    return {name: float(buf[i]) for i, name in enumerate(PHASES) if buf[i] > 0.0}
+
+
+def moe_route_host(ctx, logits_host, T, topk_ids_host, topk_w_host):
+    _check(load_library().moe_route_host(ctx, _host(logits_host, torch.float32, "logits_host"), T,
+                                         _host(topk_ids_host, torch.int32, "topk_ids_host"),
+                                         _host(topk_w_host, torch.float32, "topk_w_host"), _stream()),
+           "moe_route_host")
 
 
 class _DevView:

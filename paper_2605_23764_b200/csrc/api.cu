@@ -84,7 +84,7 @@ struct Carve {
 // Byte offsets of every workspace tensor.
 struct WsPlan {
   size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
-      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, total;
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, total;
   int cap_rows, nblk_max, ntn_act;
 };
 
@@ -123,6 +123,7 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.st_w = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_out = c.take(2 * (size_t)s.T_max * s.d);
   p.st_dw = c.take(sizeof(float) * (size_t)s.T_max * s.k);
+  p.st_logits = c.take(sizeof(float) * (size_t)s.T_max * s.E);
   p.total = c.off;
   return p;
 }
@@ -140,6 +141,16 @@ struct moe_ctx {
   int saved_T = -1;  // T of the forward whose tensors are in the workspace (-1: none)
   uint64_t budget_ns = 2000ull * 1000 * 1000;
   cudaStream_t last_stream = nullptr;
+  // optional per-operator timing
+  bool profiling = false;
+  bool events_made = false;
+  cudaEvent_t ev_start[MOE_NUM_PHASES], ev_stop[MOE_NUM_PHASES];
+  bool phase_used[MOE_NUM_PHASES] = {};
+  void begin_call(cudaStream_t st) {
+    launches = 0;
+    last_stream = st;
+    for (bool& u : phase_used) u = false;
+  }
   // tensor maps of workspace tensors (fixed for the context's lifetime)
   CUtensorMap tm_Xp_k, tm_A_k, tm_dOutp_k, tm_dH_k;      // K-major A operands, box 128 x 64
   CUtensorMap tm_dOutp_mn, tm_A_mn, tm_dH_mn, tm_Xp_mn;  // MN-major operands of the weight gradients, box 64 x 64
@@ -170,6 +181,22 @@ struct moe_ctx {
 };
 
 namespace {
+
+// Brackets one operator's launches with events when profiling is on.
+struct Phase {
+  moe_ctx* c;
+  int id;
+  cudaStream_t st;
+  Phase(moe_ctx* c_, int id_, cudaStream_t st_) : c(c_), id(id_), st(st_) {
+    if (c->profiling) cudaEventRecord(c->ev_start[id], st);
+  }
+  ~Phase() {
+    if (c->profiling) {
+      cudaEventRecord(c->ev_stop[id], st);
+      c->phase_used[id] = true;
+    }
+  }
+};
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -214,9 +241,15 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
   int rc = encode_weight_maps(c, W1, W2);
   if (rc) return rc;
   c->saved_T = -1;
-  MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
-  MOE_CUDA(launch_gather(x, w, dm, lv, c->at<uint16_t>(p.Xp), c->at<float>(p.prow_w), p.cap_rows, st,
-                         &c->launches));
+  {
+    Phase ph(c, MOE_PHASE_LAYOUT, st);
+    MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
+  }
+  {
+    Phase ph(c, MOE_PHASE_GATHER, st);
+    MOE_CUDA(launch_gather(x, w, dm, lv, c->at<uint16_t>(p.Xp), c->at<float>(p.prow_w), p.cap_rows, st,
+                           &c->launches));
+  }
   {  // GMM1 + SwiGLU (+ routing weight)
     GemmArgs g = base_args(c);
     g.tmA = c->tm_Xp_k;
@@ -230,6 +263,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     g.out1 = c->train() ? c->at<uint16_t>(p.H) : nullptr;
     g.ld_out1 = 2 * s.F;
     g.prow_w = c->at<float>(p.prow_w);
+    Phase ph(c, MOE_PHASE_GEMM_GATE_UP, st);
     MOE_CUDA(launch_gemm(GEMM_GATE_UP, g, c->num_sms, st, &c->launches));
   }
   {  // GMM2
@@ -242,9 +276,13 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     g.b_rows_per_expert = s.d;
     g.out0 = c->at<uint16_t>(p.Y);
     g.ld_out0 = s.d;
+    Phase ph(c, MOE_PHASE_GEMM_DOWN, st);
     MOE_CUDA(launch_gemm(GEMM_DOWN, g, c->num_sms, st, &c->launches));
   }
-  MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+  {
+    Phase ph(c, MOE_PHASE_COMBINE, st);
+    MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+  }
   if (c->train()) c->saved_T = T;
   return MOE_OK;
 }
@@ -258,7 +296,10 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
   int rc = encode_weight_maps(c, W1, W2);
   if (rc) return rc;
   // backward Dispatch: expert-ordered gather of the upstream gradient
-  MOE_CUDA(launch_gather(dout, nullptr, dm, lv, c->at<uint16_t>(p.dOutp), nullptr, p.cap_rows, st, &c->launches));
+  {
+    Phase ph(c, MOE_PHASE_BWD_GATHER, st);
+    MOE_CUDA(launch_gather(dout, nullptr, dm, lv, c->at<uint16_t>(p.dOutp), nullptr, p.cap_rows, st, &c->launches));
+  }
   {  // act_grad + SwiGLU_grad (+ routing-weight gradient partials)
     GemmArgs g = base_args(c);
     g.tmA = c->tm_dOutp_k;
@@ -273,9 +314,13 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.ld_in0 = 2 * s.F;
     g.prow_w = c->at<float>(p.prow_w);
     g.dw_partial = d_w ? c->at<float>(p.dw_partial) : nullptr;
+    Phase ph(c, MOE_PHASE_ACT_GRAD, st);
     MOE_CUDA(launch_gemm(GEMM_ACT_GRAD, g, c->num_sms, st, &c->launches));
   }
-  if (d_w) MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), p.ntn_act, dm, lv, d_w, st, &c->launches));
+  if (d_w) {
+    Phase ph(c, MOE_PHASE_DW_REDUCE, st);
+    MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), p.ntn_act, dm, lv, d_w, st, &c->launches));
+  }
   {  // w2_grad: dW_down[e][c][f] = sum_rows dOutp[r][c] * A[r][f]   (shares dOutp with act_grad)
     GemmArgs g = base_args(c);
     g.tmA = c->tm_dOutp_mn;
@@ -286,6 +331,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.n_tiles_n = (s.F + 255) / 256;
     g.out0 = dW2;
     g.ld_out0 = s.F;
+    Phase ph(c, MOE_PHASE_WGRAD_DOWN, st);
     MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
   }
   {  // gate_grad: dXp = dH . W_gate_up[e]
@@ -298,6 +344,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.b_rows_per_expert = 2 * s.F;
     g.out0 = c->at<uint16_t>(p.Y);  // the forward's Y is dead by now: reuse it for dXp
     g.ld_out0 = s.d;
+    Phase ph(c, MOE_PHASE_GATE_GRAD, st);
     MOE_CUDA(launch_gemm(GEMM_GATE_GRAD, g, c->num_sms, st, &c->launches));
   }
   {  // w1_grad: dW_gate_up[e][n][c] = sum_rows dH[r][n] * Xp[r][c]   (shares dH with gate_grad)
@@ -310,10 +357,13 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.n_tiles_n = (s.d + 255) / 256;
     g.out0 = dW1;
     g.ld_out0 = s.d;
+    Phase ph(c, MOE_PHASE_WGRAD_GATE_UP, st);
     MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
   }
-  // backward Combine
-  MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
+  {  // backward Combine
+    Phase ph(c, MOE_PHASE_BWD_COMBINE, st);
+    MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
+  }
   return MOE_OK;
 }
 
@@ -383,6 +433,11 @@ int moe_create(moe_ctx** out, const moe_shape* shape, void* workspace, size_t wo
 
 int moe_destroy(moe_ctx* c) {
   if (!c) return MOE_OK;
+  if (c->events_made)
+    for (int i = 0; i < MOE_NUM_PHASES; ++i) {
+      cudaEventDestroy(c->ev_start[i]);
+      cudaEventDestroy(c->ev_stop[i]);
+    }
   if (c->owns_ws) cudaFree(c->ws);
   delete c;
   return MOE_OK;
@@ -391,10 +446,33 @@ int moe_destroy(moe_ctx* c) {
 int moe_route(moe_ctx* c, const float* logits, int32_t T, int32_t* topk_ids, float* topk_w, int32_t* counts,
               void* stream) {
   if (!c || !logits || !topk_ids || !topk_w || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
-  c->launches = 0;
-  c->last_stream = static_cast<cudaStream_t>(stream);
+  c->begin_call(static_cast<cudaStream_t>(stream));
+  Phase ph(c, MOE_PHASE_ROUTE, c->last_stream);
   MOE_CUDA(launch_route(logits, T, c->shape.E, c->shape.k, (c->shape.flags & MOE_FLAG_RENORM_TOPK) != 0, topk_ids,
                         topk_w, counts, c->last_stream, &c->launches));
+  return MOE_OK;
+}
+
+int moe_route_host(moe_ctx* c, const float* logits_host, int32_t T, int32_t* topk_ids_host, float* topk_w_host,
+                   void* stream) {
+  if (!c || !logits_host || !topk_ids_host || !topk_w_host || T < 0 || T > c->shape.T_max)
+    return MOE_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  c->begin_call(st);
+  if (T == 0) return MOE_OK;
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_logits, logits_host, sizeof(float) * (size_t)T * s.E,
+                           cudaMemcpyHostToDevice, st));
+  {
+    Phase ph(c, MOE_PHASE_ROUTE, st);
+    MOE_CUDA(launch_route(c->at<float>(p.st_logits), T, s.E, s.k, (s.flags & MOE_FLAG_RENORM_TOPK) != 0,
+                          c->at<int32_t>(p.st_ids), c->at<float>(p.st_w), nullptr, st, &c->launches));
+  }
+  MOE_CUDA(cudaMemcpyAsync(topk_ids_host, c->ws + p.st_ids, sizeof(int) * (size_t)T * s.k, cudaMemcpyDeviceToHost,
+                           st));
+  MOE_CUDA(cudaMemcpyAsync(topk_w_host, c->ws + p.st_w, sizeof(float) * (size_t)T * s.k, cudaMemcpyDeviceToHost,
+                           st));
   return MOE_OK;
 }
 
@@ -402,8 +480,7 @@ int moe_layout(moe_ctx* c, const int32_t* topk_ids, int32_t T, int32_t* counts, 
                int32_t* src_of, void* stream) {
   if (!c || !topk_ids || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  c->launches = 0;
-  c->last_stream = st;
+  c->begin_call(st);
   c->saved_T = -1;
   const Dims dm = c->dims(T);
   const LayoutView lv = c->layout();
@@ -419,8 +496,7 @@ int moe_layout(moe_ctx* c, const int32_t* topk_ids, int32_t T, int32_t* counts, 
 int moe_ffn_fwd(moe_ctx* c, const uint16_t* x, const int32_t* topk_ids, const float* topk_w,
                 const uint16_t* W_gate_up, const uint16_t* W_down, uint16_t* out, int32_t T, void* stream) {
   if (!c || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
-  c->launches = 0;
-  c->last_stream = static_cast<cudaStream_t>(stream);
+  c->begin_call(static_cast<cudaStream_t>(stream));
   if (T == 0) return MOE_OK;  // nothing to compute; tensor pointers of an empty batch may be NULL
   if (!x || !topk_ids || !topk_w || !W_gate_up || !W_down || !out) return MOE_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(W_gate_up) || !aligned16(W_down) || !aligned16(out)) return MOE_ERR_INVALID_ARG;
@@ -438,8 +514,7 @@ int moe_ffn_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* x, const int32
     return MOE_ERR_INVALID_ARG;
   if (!c->train()) return MOE_ERR_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  c->launches = 0;
-  c->last_stream = st;
+  c->begin_call(st);
   if (T == 0) {
     const moe_shape& s = c->shape;
     const size_t Ep = s.E + s.n_shared;
@@ -458,8 +533,7 @@ int moe_ffn_fwd_host(moe_ctx* c, const uint16_t* x_host, const int32_t* topk_ids
       T > c->shape.T_max)
     return MOE_ERR_INVALID_ARG;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  c->launches = 0;
-  c->last_stream = st;
+  c->begin_call(st);
   if (T == 0) return MOE_OK;
   const moe_shape& s = c->shape;
   const WsPlan& p = c->plan;
@@ -483,8 +557,7 @@ int moe_ffn_bwd_host(moe_ctx* c, const uint16_t* dout_host, const uint16_t* W_ga
     return MOE_ERR_INVALID_ARG;
   if (!c->train() || c->saved_T != T) return MOE_ERR_STATE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  c->launches = 0;
-  c->last_stream = st;
+  c->begin_call(st);
   const moe_shape& s = c->shape;
   const WsPlan& p = c->plan;
   // the staged x is dead after the forward's gather: its buffer receives dout
@@ -515,6 +588,31 @@ int moe_last_launch_count(const moe_ctx* c) { return c ? c->launches : 0; }
 int moe_set_wait_budget_ms(moe_ctx* c, int32_t ms) {
   if (!c || ms < 1) return MOE_ERR_INVALID_ARG;
   c->budget_ns = (uint64_t)ms * 1000 * 1000;
+  return MOE_OK;
+}
+
+int moe_set_profiling(moe_ctx* c, int32_t on) {
+  if (!c) return MOE_ERR_INVALID_ARG;
+  if (on && !c->events_made) {
+    for (int i = 0; i < MOE_NUM_PHASES; ++i) {
+      MOE_CUDA(cudaEventCreate(&c->ev_start[i]));
+      MOE_CUDA(cudaEventCreate(&c->ev_stop[i]));
+    }
+    c->events_made = true;
+  }
+  c->profiling = on != 0;
+  return MOE_OK;
+}
+
+int moe_get_phase_ms(moe_ctx* c, float* ms) {
+  if (!c || !ms) return MOE_ERR_INVALID_ARG;
+  for (int i = 0; i < MOE_NUM_PHASES; ++i) {
+    ms[i] = 0.f;
+    if (c->events_made && c->phase_used[i]) {
+      MOE_CUDA(cudaEventSynchronize(c->ev_stop[i]));
+      MOE_CUDA(cudaEventElapsedTime(&ms[i], c->ev_start[i], c->ev_stop[i]));
+    }
+  }
   return MOE_OK;
 }
 
