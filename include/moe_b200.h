@@ -190,6 +190,29 @@ enum {
 };
 int moe_debug_buffer(moe_ctx* ctx, int which, void** ptr, size_t* elems);
 
+/* Dispatch layout for callers that cannot allocate device memory (no counterpart in the paper:
+ * this is a convenience of this library).  Who needs it: code that runs where cudaMalloc is not
+ * allowed or not wanted -- inside a framework's pre-planned memory region, a latency-critical
+ * serving loop (cudaMalloc synchronises the device), a plugin that only receives its input and
+ * output buffers -- and callers without a moe_ctx.  It computes exactly what moe_layout computes
+ * and needs no context: the scratch memory of the layout kernels is a fixed array inside the
+ * library (about 1.6 MB held on every GPU that loads the library, until the process exits), and
+ * the call performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *   topk_ids[T][k] -> counts[E+S], offsets[E+S+1], row_of[T*(k+S)], src_of[T*(k+S)] (all device
+ *   pointers, all required); status2 (device int32[2], may be NULL) receives {code, detail}:
+ *   {0,0} or {MOE_ERR_BAD_EXPERT_ID, slot}.
+ * Limits: T*(k+S) <= MOE_NOALLOC_MAX_SLOTS, E+S <= MOE_NOALLOC_MAX_EXPERTS, and
+ * ceil(T*(k+S)/2048)*(E+S) <= 131072; larger problems return MOE_ERR_TOO_LARGE (use moe_layout).
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls share the one array, which keeps the
+ * previous call's contents (the call clears what must start at zero): two calls whose work overlaps
+ * on the GPU -- different streams, or different threads -- race; serialise them. */
+#define MOE_NOALLOC_MAX_SLOTS 262144
+#define MOE_NOALLOC_MAX_EXPERTS 1088
+int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E, int32_t k, int32_t n_shared,
+                       int32_t* counts, int32_t* offsets, int32_t* row_of, int32_t* src_of,
+                       int32_t* status2, void* stream);
+
 const char* moe_strerror(int code);
 /* Text of the last CUDA error a call on this thread ran into ("" if none). */
 const char* moe_last_cuda_error(void);

@@ -20,7 +20,7 @@ _BUF_DTYPE = {k: (torch.bfloat16 if k in ("Xp", "H", "A", "Y", "dOutp", "dH", "d
 EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe_layout", "moe_ffn_fwd",
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
-           "moe_set_profiling", "moe_get_phase_ms", "moe_route_host"]
+           "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -68,6 +68,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_set_profiling.argtypes = [vp, i32]
     lib.moe_get_phase_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.moe_route_host.argtypes = [vp, vp, i32, vp, vp, vp]
+    lib.moe_layout_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -208,6 +209,16 @@ def moe_route_host(ctx, logits_host, T, topk_ids_host, topk_w_host):
                                          _host(topk_ids_host, torch.int32, "topk_ids_host"),
                                          _host(topk_w_host, torch.float32, "topk_w_host"), _stream()),
            "moe_route_host")
+
+
+def moe_layout_noalloc(topk_ids, T, E, k, n_shared, counts, offsets, row_of, src_of, status2=None):
+    """Dispatch layout through the entry point that allocates nothing and needs no context (for
+    callers that may not cudaMalloc).  All tensors are caller-owned CUDA int32 tensors."""
+    i32 = torch.int32
+    _check(load_library().moe_layout_noalloc(_dev(topk_ids, i32, "topk_ids"), T, E, k, n_shared,
+                                             _dev(counts, i32, "counts"), _dev(offsets, i32, "offsets"),
+                                             _dev(row_of, i32, "row_of"), _dev(src_of, i32, "src_of"),
+                                             _dev(status2, i32, "status2"), _stream()), "moe_layout_noalloc")
 
 
 class _DevView:

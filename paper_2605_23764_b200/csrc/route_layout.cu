@@ -262,3 +262,94 @@ cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView&
 }
 
 }  // namespace moe
+
+// ------------------------------------------------------------------------------------------
+// Dispatch layout without any allocation.
+//
+// Some callers may not allocate device memory at the point where they need the layout: code
+// running inside a framework's memory-planned region or a real-time serving loop where cudaMalloc
+// (which synchronises the device and may fail under fragmentation) is forbidden, plugins that are
+// handed only their input and output buffers, and callers that never created a moe_ctx.  For them
+// the scratch of the layout kernels (per-block histograms, M-block table, padded-row indices,
+// status word) lives in the fixed-size array below, which every GPU that loads this library holds
+// until the process exits (about 1.6 MB).  All calls share it.
+// ------------------------------------------------------------------------------------------
+#include <mutex>
+
+#include "../../include/moe_b200.h"
+
+namespace {
+
+constexpr int NA_MAX_SLOTS = MOE_NOALLOC_MAX_SLOTS;             // T * (k + S)
+constexpr int NA_MAX_EP = MOE_NOALLOC_MAX_EXPERTS;              // E + S
+constexpr int NA_MAX_BLOCKS = NA_MAX_SLOTS / moe::LAYOUT_CHUNK; // blocks of the layout kernels
+constexpr int NA_MAX_HIST = 1 << 17;                            // ints of per-block histograms (nblk * (E+S))
+constexpr int NA_MAX_MBLK = (NA_MAX_SLOTS + NA_MAX_EP * (moe::BLOCK_M - 1)) / moe::BLOCK_M + 2;
+
+struct NoAllocScratch {
+  moe::DevStatus status;
+  int meta[8];
+  int pad_off[NA_MAX_EP + 1];
+  int mb_start[NA_MAX_EP + 1];
+  int mblk_expert[NA_MAX_MBLK];
+  int blk_hist[NA_MAX_HIST];
+  int prow_of[NA_MAX_SLOTS];
+};
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+constexpr int NA_MAX_DEVICES = 64;
+std::mutex g_na_mutex;
+NoAllocScratch* g_na_ptr[NA_MAX_DEVICES] = {};
+
+}  // namespace
+
+extern "C" int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E, int32_t k, int32_t n_shared,
+                                  int32_t* counts, int32_t* offsets, int32_t* row_of, int32_t* src_of,
+                                  int32_t* status2, void* stream) {
+  if (!topk_ids || !counts || !offsets || !row_of || !src_of) return MOE_ERR_INVALID_ARG;
+  if (T < 1 || E < 1 || E > 1024 || k < 1 || k > E || n_shared < 0) return MOE_ERR_INVALID_ARG;
+  const long slots = (long)T * (k + n_shared);
+  const int Ep = E + n_shared;
+  const long nblk = (slots + moe::LAYOUT_CHUNK - 1) / moe::LAYOUT_CHUNK;
+  if (slots > NA_MAX_SLOTS || Ep > NA_MAX_EP || nblk > NA_MAX_BLOCKS || nblk * Ep > NA_MAX_HIST)
+    return MOE_ERR_TOO_LARGE;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NA_MAX_DEVICES) return MOE_ERR_NO_DEVICE;
+  NoAllocScratch* sc = nullptr;
+  {
+    // first call on this device: resolve the device address of the static array (device `dev` is current)
+    std::lock_guard<std::mutex> lock(g_na_mutex);
+    if (!g_na_ptr[dev]) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) {
+        cudaGetLastError();
+        return MOE_ERR_CUDA;
+      }
+      g_na_ptr[dev] = static_cast<NoAllocScratch*>(p);
+    }
+    sc = g_na_ptr[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the array keeps the previous call's contents: the status word must start at zero
+  if (cudaMemsetAsync(&sc->status, 0, sizeof(moe::DevStatus), st) != cudaSuccess) return MOE_ERR_CUDA;
+  moe::Dims dm{T, 8, E, k, n_shared, 8};
+  moe::LayoutView lv;
+  lv.counts = counts;
+  lv.offsets = offsets;
+  lv.row_of = row_of;
+  lv.src_of = src_of;
+  lv.prow_of = sc->prow_of;
+  lv.pad_off = sc->pad_off;
+  lv.mb_start = sc->mb_start;
+  lv.mblk_expert = sc->mblk_expert;
+  lv.meta = sc->meta;
+  lv.blk_hist = sc->blk_hist;
+  int launches = 0;
+  if (moe::launch_layout(topk_ids, dm, lv, &sc->status, st, &launches) != cudaSuccess) return MOE_ERR_CUDA;
+  if (status2 &&
+      cudaMemcpyAsync(status2, &sc->status, 2 * sizeof(int), cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  return MOE_OK;
+}
