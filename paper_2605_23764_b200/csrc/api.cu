@@ -41,29 +41,53 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// bf16 row-major [rows][cols] tensor, box [box_rows][box_cols], 128-byte swizzle, zero fill outside.
-int encode_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
-              uint32_t box_cols) {
+// bf16 tensor of `rank` dimensions (dims[0] innermost, strides in bytes for dims 1..), 128-byte
+// swizzle, zero fill outside the tensor on loads, clipping on stores.
+int encode_tiled(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+                 const uint32_t* box) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) {
     g_cuda_error = "cuTensorMapEncodeTiled entry point not available";
     return MOE_ERR_CUDA;
   }
-  cuuint64_t gdim[2] = {cols, rows};
-  cuuint64_t gstr[1] = {cols * 2};
-  cuuint32_t box[2] = {box_cols, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), gdim, gstr, box, estr,
+  cuuint64_t gdim[3], gstr[2];
+  cuuint32_t bx[3], estr[3] = {1, 1, 1};
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides[i];
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), gdim, gstr, bx, estr,
                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
-    char buf[160];
-    snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed (%d) rows=%llu cols=%llu box=%ux%u", (int)r,
-             (unsigned long long)rows, (unsigned long long)cols, box_rows, box_cols);
+    char buf[200];
+    snprintf(buf, sizeof buf, "cuTensorMapEncodeTiled failed (%d) rank=%d dims=%llu,%llu box=%u,%u", (int)r, rank,
+             (unsigned long long)dims[0], (unsigned long long)dims[1], box[0], box[1]);
     g_cuda_error = buf;
     return MOE_ERR_CUDA;
   }
   return MOE_OK;
+}
+
+// Row-major [rows][cols] matrix, box [box_rows][box_cols].
+int encode_2d(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows,
+              uint32_t box_cols) {
+  const uint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
+  const uint32_t box[2] = {box_cols, box_rows};
+  return encode_tiled(tm, base, 2, dims, strides, box);
+}
+
+// Store map of a [rows][2][F] view of a [rows][2F] matrix (gate half, up half): box 32 rows x 64 columns
+// of one half, so a column tile that ends past F is clipped instead of spilling into the other half.
+int encode_halves(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t F) {
+  const uint64_t dims[3] = {F, 2, rows}, strides[2] = {F * 2, 2 * F * 2};
+  const uint32_t box[3] = {64, 1, 32};
+  return encode_tiled(tm, base, 3, dims, strides, box);
+}
+
+// Store map of a weight-gradient tensor [Ep][M][N]: box 32 rows x 64 columns inside one expert slab.
+int encode_slabs(CUtensorMap* tm, const void* base, uint64_t Ep, uint64_t M, uint64_t N) {
+  const uint64_t dims[3] = {N, M, Ep}, strides[2] = {N * 2, M * N * 2};
+  const uint32_t box[3] = {64, 32, 1};
+  return encode_tiled(tm, base, 3, dims, strides, box);
 }
 
 bool shape_ok(const moe_shape* s) {
@@ -158,6 +182,11 @@ struct moe_ctx {
   const void* w1_ptr = nullptr;
   const void* w2_ptr = nullptr;
   CUtensorMap tm_W1_k, tm_W2_k, tm_W1_mn, tm_W2_mn;
+  // store maps: workspace tensors (fixed) and the caller's weight gradients (re-encoded on change)
+  CUtensorMap ts_A, ts_H, ts_Y, ts_dH;
+  const void* dw1_ptr = nullptr;
+  const void* dw2_ptr = nullptr;
+  CUtensorMap ts_dW1, ts_dW2;
 
   template <class T>
   T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
@@ -258,10 +287,9 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     g.K = s.d;
     g.N = s.F;
     g.b_rows_per_expert = 2 * s.F;
-    g.out0 = c->at<uint16_t>(p.A);
-    g.ld_out0 = s.F;
-    g.out1 = c->train() ? c->at<uint16_t>(p.H) : nullptr;
-    g.ld_out1 = 2 * s.F;
+    g.tmOut0 = c->ts_A;
+    g.tmOut1 = c->ts_H;
+    g.save_h = c->train() ? 1 : 0;
     g.prow_w = c->at<float>(p.prow_w);
     Phase ph(c, MOE_PHASE_GEMM_GATE_UP, st);
     MOE_CUDA(launch_gemm(GEMM_GATE_UP, g, c->num_sms, st, &c->launches));
@@ -274,8 +302,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     g.K = s.F;
     g.N = s.d;
     g.b_rows_per_expert = s.d;
-    g.out0 = c->at<uint16_t>(p.Y);
-    g.ld_out0 = s.d;
+    g.tmOut0 = c->ts_Y;
     Phase ph(c, MOE_PHASE_GEMM_DOWN, st);
     MOE_CUDA(launch_gemm(GEMM_DOWN, g, c->num_sms, st, &c->launches));
   }
@@ -295,6 +322,15 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
   const LayoutView lv = c->layout();
   int rc = encode_weight_maps(c, W1, W2);
   if (rc) return rc;
+  const uint64_t Ep = s.E + s.n_shared;
+  if (dW1 != c->dw1_ptr) {
+    if ((rc = encode_slabs(&c->ts_dW1, dW1, Ep, 2 * s.F, s.d))) return rc;
+    c->dw1_ptr = dW1;
+  }
+  if (dW2 != c->dw2_ptr) {
+    if ((rc = encode_slabs(&c->ts_dW2, dW2, Ep, s.d, s.F))) return rc;
+    c->dw2_ptr = dW2;
+  }
   // backward Dispatch: expert-ordered gather of the upstream gradient
   {
     Phase ph(c, MOE_PHASE_BWD_GATHER, st);
@@ -308,8 +344,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.K = s.d;
     g.N = s.F;
     g.b_rows_per_expert = s.d;
-    g.out0 = c->at<uint16_t>(p.dH);
-    g.ld_out0 = 2 * s.F;
+    g.tmOut0 = c->ts_dH;
     g.in0 = c->at<uint16_t>(p.H);
     g.ld_in0 = 2 * s.F;
     g.prow_w = c->at<float>(p.prow_w);
@@ -329,8 +364,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.N = s.F;
     g.n_tiles_m = (s.d + 127) / 128;
     g.n_tiles_n = (s.F + 255) / 256;
-    g.out0 = dW2;
-    g.ld_out0 = s.F;
+    g.tmOut0 = c->ts_dW2;
     Phase ph(c, MOE_PHASE_WGRAD_DOWN, st);
     MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
   }
@@ -342,8 +376,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.K = 2 * s.F;
     g.N = s.d;
     g.b_rows_per_expert = 2 * s.F;
-    g.out0 = c->at<uint16_t>(p.Y);  // the forward's Y is dead by now: reuse it for dXp
-    g.ld_out0 = s.d;
+    g.tmOut0 = c->ts_Y;  // the forward's Y is dead by now: its buffer receives dXp
     Phase ph(c, MOE_PHASE_GATE_GRAD, st);
     MOE_CUDA(launch_gemm(GEMM_GATE_GRAD, g, c->num_sms, st, &c->launches));
   }
@@ -355,8 +388,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     g.N = s.d;
     g.n_tiles_m = (2 * s.F + 127) / 128;
     g.n_tiles_n = (s.d + 255) / 256;
-    g.out0 = dW1;
-    g.ld_out0 = s.d;
+    g.tmOut0 = c->ts_dW1;
     Phase ph(c, MOE_PHASE_WGRAD_GATE_UP, st);
     MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
   }
@@ -416,6 +448,10 @@ int moe_create(moe_ctx** out, const moe_shape* shape, void* workspace, size_t wo
   if (e != cudaSuccess) rc = cuda_fail(e, "cudaMemset(workspace)");
   if (!rc) rc = encode_2d(&c->tm_Xp_k, c->ws + p.Xp, cap, s.d, 128, 64);
   if (!rc) rc = encode_2d(&c->tm_A_k, c->ws + p.A, cap, s.F, 128, 64);
+  if (!rc) rc = encode_2d(&c->ts_A, c->ws + p.A, cap, s.F, 32, 64);
+  if (!rc) rc = encode_2d(&c->ts_Y, c->ws + p.Y, cap, s.d, 32, 64);
+  if (!rc && train) rc = encode_halves(&c->ts_H, c->ws + p.H, cap, s.F);
+  if (!rc && train) rc = encode_halves(&c->ts_dH, c->ws + p.dH, cap, s.F);
   if (!rc && train) rc = encode_2d(&c->tm_dOutp_k, c->ws + p.dOutp, cap, s.d, 128, 64);
   if (!rc && train) rc = encode_2d(&c->tm_dH_k, c->ws + p.dH, cap, 2 * s.F, 128, 64);
   if (!rc && train) rc = encode_2d(&c->tm_dOutp_mn, c->ws + p.dOutp, cap, s.d, 64, 64);

@@ -4,9 +4,9 @@
 // (forward GMM1+SwiGLU, GMM2; backward act_grad+SwiGLU_grad, gate_grad, and the two weight
 // gradients).  Per CTA: warp 0 = TMA producer (one elected lane), warp 1 = tcgen05.mma issuer (one
 // elected lane; the warp also owns the TMEM allocation), warps 2..5 = epilogue (TMEM -> registers
-// -> fused element-wise math -> global).  Operands travel global -> shared through TMA into a
-// 4-stage ring of 128-byte-swizzled tiles; accumulators live in TMEM, double-buffered (2 x 256
-// columns) so the epilogue of tile i overlaps the main loop of tile i+1.
+// -> fused element-wise math -> swizzled shared staging -> TMA store).  Operands travel global ->
+// shared through TMA into a 4-stage ring of 128-byte-swizzled tiles; accumulators live in TMEM,
+// double-buffered (2 x 256 columns) so the epilogue of tile i overlaps the main loop of tile i+1.
 //
 // Tiles never straddle experts: rows live in a padded row space where every expert segment starts
 // on a multiple of 128 (the paper's rule that vector tiles align with GMM row partitions and that
@@ -23,6 +23,8 @@ constexpr int B_STAGE_BYTES = BN * BK * 2;       // 32 KB
 constexpr int MN_BOX_BYTES = 64 * BK * 2;        // one [64 k][64 mn] box of an MN-major operand
 constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
+constexpr int OUT_BOX_BYTES = 32 * 64 * 2;       // epilogue staging box: 32 rows x 64 bf16 columns
+constexpr int OUT_STAGE_BYTES = 2 * OUT_BOX_BYTES;  // per epilogue warp: two boxes
 
 struct __align__(8) GemmBarriers {
   uint64_t full[STAGES];
@@ -35,7 +37,8 @@ struct __align__(8) GemmBarriers {
 };
 
 constexpr size_t GEMM_SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
-                                   sizeof(GemmBarriers);
+                                   4 * OUT_STAGE_BYTES + sizeof(GemmBarriers);
+static_assert(GEMM_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 size_t gemm_smem_bytes() { return GEMM_SMEM_BYTES; }
 
 struct Tile {
@@ -114,30 +117,45 @@ __device__ __forceinline__ void load_stage(const GemmArgs& a, const Tile& tl, in
   }
 }
 
-// ---------------------------------------------------------------- epilogues (one thread = one tile row)
-__device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
-}
-__device__ __forceinline__ void store8_bf16(uint16_t* p, const float* v) {
-  st_v4(p, pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]), pack_bf16x2(v[6], v[7]));
+// ---------------------------------------------------------------- epilogues
+// Each epilogue warp owns 32 rows of the tile (its TMEM lane quadrant) and a private staging area of
+// two [32 rows][64 columns] bf16 boxes in the 128-byte-swizzled layout the store tensor maps expect.
+// A thread (= one row) writes 16-byte chunks at chunk index (j ^ (row & 7)): conflict-free.
+__device__ __forceinline__ void stage8(uint8_t* box, int lane, int j, const float* v) {
+  uint4 q = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
+                       pack_bf16x2(v[6], v[7]));
+  *reinterpret_cast<uint4*>(box + lane * 128 + ((j ^ (lane & 7)) << 4)) = q;
 }
 __device__ __forceinline__ void load8_bf16(const uint16_t* p, float* v) {
-  uint4 r = *reinterpret_cast<const uint4*>(p);
+  uint4 r;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
   v[0] = bf16lo(r.x); v[1] = bf16hi(r.x); v[2] = bf16lo(r.y); v[3] = bf16hi(r.y);
   v[4] = bf16lo(r.z); v[5] = bf16hi(r.z); v[6] = bf16lo(r.w); v[7] = bf16hi(r.w);
 }
 __device__ __forceinline__ float sigmoidf_fast(float g) { return 1.0f / (1.0f + __expf(-g)); }
 
+// Before refilling the staging area: the previous stores must have finished reading it.
+__device__ __forceinline__ void staging_acquire(int lane) {
+  if (lane == 0) tma_store_wait_read();
+  __syncwarp();
+}
+// After filling: publish the writes to the async proxy; lane 0 then issues the stores.
+__device__ __forceinline__ void staging_release() {
+  fence_proxy_async_smem();
+  __syncwarp();
+}
+
 template <int MODE>
 __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl, uint32_t tmem_acc, int quad,
-                                              int lane) {
-  const int r = quad * 32 + lane;                   // row of the tile held by this thread
+                                              int lane, uint8_t* stg) {
   const uint32_t trow = tmem_acc + (static_cast<uint32_t>(quad * 32) << 16);
+  uint8_t* box0 = stg;
+  uint8_t* box1 = stg + OUT_BOX_BYTES;
   if (MODE == GEMM_GATE_UP) {
-    const size_t p = (size_t)tl.row0 + r;
-    const float w = a.prow_w[p];
-    uint16_t* arow = a.out0 + p * a.ld_out0;
-    uint16_t* hrow = a.out1 ? a.out1 + p * a.ld_out1 : nullptr;
+    const int prow0 = tl.row0 + quad * 32;             // first padded row of this warp's slab
+    const float w = a.prow_w[prow0 + lane];
+    // round 1: A = w * silu(g) * u, 128 columns
+    staging_acquire(lane);
     for (int c = 0; c < BN / 2; c += 16) {
       float g[16], u[16], act[16];
       tmem_ld16(trow + c, g);
@@ -145,76 +163,118 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
       tmem_ld_wait();
 #pragma unroll
       for (int i = 0; i < 16; ++i) act[i] = w * (g[i] * sigmoidf_fast(g[i]) * u[i]);
-#pragma unroll
-      for (int h = 0; h < 16; h += 8) {
-        const int col = tl.n0 + c + h;
-        if (col < a.F) {
-          store8_bf16(arow + col, act + h);
-          if (hrow) {
-            store8_bf16(hrow + col, g + h);
-            store8_bf16(hrow + a.F + col, u + h);
-          }
+      uint8_t* box = (c < 64) ? box0 : box1;
+      stage8(box, lane, (c & 63) >> 3, act);
+      stage8(box, lane, ((c & 63) >> 3) + 1, act + 8);
+    }
+    staging_release();
+    if (lane == 0) {
+      tma_store_2d(&a.tmOut0, tl.n0, prow0, box0);
+      if (tl.n0 + 64 < a.F) tma_store_2d(&a.tmOut0, tl.n0 + 64, prow0, box1);
+      tma_store_commit();
+    }
+    if (a.save_h) {
+      // rounds 2, 3: the pre-activations, kept for the backward pass (H viewed as [row][gate|up][F])
+#pragma unroll 1
+      for (int half = 0; half < 2; ++half) {
+        staging_acquire(lane);
+        for (int c = 0; c < BN / 2; c += 16) {
+          float v[16];
+          tmem_ld16(trow + half * (BN / 2) + c, v);
+          tmem_ld_wait();
+          uint8_t* box = (c < 64) ? box0 : box1;
+          stage8(box, lane, (c & 63) >> 3, v);
+          stage8(box, lane, ((c & 63) >> 3) + 1, v + 8);
+        }
+        staging_release();
+        if (lane == 0) {
+          tma_store_3d(&a.tmOut1, tl.n0, half, prow0, box0);
+          if (tl.n0 + 64 < a.F) tma_store_3d(&a.tmOut1, tl.n0 + 64, half, prow0, box1);
+          tma_store_commit();
         }
       }
     }
   } else if (MODE == GEMM_ACT_GRAD) {
-    const size_t p = (size_t)tl.row0 + r;
+    const int prow0 = tl.row0 + quad * 32;
+    const size_t p = (size_t)prow0 + lane;
     const float w = a.prow_w[p];
     const uint16_t* hrow = a.in0 + p * a.ld_in0;
-    uint16_t* drow = a.out0 + p * a.ld_out0;
     float part = 0.f;
-    for (int c = 0; c < BN; c += 16) {
-      float da[16];
-      tmem_ld16(trow + c, da);
-      tmem_ld_wait();
+    // 64 columns of F per round: box0 <- d(gate), box1 <- d(up)
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 64) {
+      if (tl.n0 + c0 >= a.F) break;  // uniform: whole round outside the tensor
+      staging_acquire(lane);
 #pragma unroll
-      for (int h = 0; h < 16; h += 8) {
-        const int col = tl.n0 + c + h;
-        if (col < a.F) {
+      for (int c = 0; c < 64; c += 16) {
+        float da[16];
+        tmem_ld16(trow + c0 + c, da);
+        tmem_ld_wait();
+#pragma unroll
+        for (int h = 0; h < 16; h += 8) {
+          const int col = tl.n0 + c0 + c + h;
           float g[8], u[8], dg[8], du[8];
-          load8_bf16(hrow + col, g);
-          load8_bf16(hrow + a.F + col, u);
+          if (col < a.F) {
+            load8_bf16(hrow + col, g);
+            load8_bf16(hrow + a.F + col, u);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) g[i] = u[i] = 0.f;
+          }
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             const float s = sigmoidf_fast(g[i]);
             const float gs = g[i] * s;
-            part += da[h + i] * (gs * u[i]);          // <dA_unweighted, a>: gradient of the routing weight
-            const float dav = w * da[h + i];          // backward Dispatch's weight, applied here
+            part += da[h + i] * (gs * u[i]);        // <dA_unweighted, a>: gradient of the routing weight
+            const float dav = w * da[h + i];        // backward Dispatch's weight, applied here
             dg[i] = dav * u[i] * (s * (1.0f + g[i] * (1.0f - s)));
             du[i] = dav * gs;
           }
-          store8_bf16(drow + col, dg);
-          store8_bf16(drow + a.F + col, du);
+          stage8(box0, lane, (c + h) >> 3, dg);
+          stage8(box1, lane, (c + h) >> 3, du);
         }
+      }
+      staging_release();
+      if (lane == 0) {
+        tma_store_3d(&a.tmOut0, tl.n0 + c0, 0, prow0, box0);
+        tma_store_3d(&a.tmOut0, tl.n0 + c0, 1, prow0, box1);
+        tma_store_commit();
       }
     }
     if (a.dw_partial) a.dw_partial[p * a.n_tiles_n + tl.nb] = part;
   } else {
     // plain bf16 store of the accumulator: DOWN (Y), GATE_GRAD (dXp), WGRAD (dW)
-    size_t row;
-    bool row_ok = true;
-    if (MODE == GEMM_WGRAD) {
-      row = (size_t)tl.e * a.M + tl.m0 + r;
-      row_ok = tl.m0 + r < a.M;
-    } else {
-      row = (size_t)tl.row0 + r;
-    }
-    uint16_t* orow = a.out0 + row * a.ld_out0;
-    for (int c = 0; c < BN; c += 16) {
-      float v[16];
-      if (MODE == GEMM_WGRAD && tl.nkb == 0) {
+    const int y0 = (MODE == GEMM_WGRAD ? tl.m0 : tl.row0) + quad * 32;
+#pragma unroll 1
+    for (int c0 = 0; c0 < BN; c0 += 128) {
+      if (tl.n0 + c0 >= a.N) break;
+      if (MODE == GEMM_WGRAD && y0 >= a.M) break;
+      staging_acquire(lane);
 #pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = 0.f;
-      } else {
-        tmem_ld16(trow + c, v);
-        tmem_ld_wait();
-      }
-      if (row_ok) {
+      for (int c = 0; c < 128; c += 32) {
+        float v[32];
+        if (MODE == GEMM_WGRAD && tl.nkb == 0) {
 #pragma unroll
-        for (int h = 0; h < 16; h += 8) {
-          const int col = tl.n0 + c + h;
-          if (col < a.N) store8_bf16(orow + col, v + h);
+          for (int i = 0; i < 32; ++i) v[i] = 0.f;
+        } else {
+          tmem_ld16(trow + c0 + c, v);
+          tmem_ld16(trow + c0 + c + 16, v + 16);
+          tmem_ld_wait();
         }
+        uint8_t* box = (c < 64) ? box0 : box1;
+#pragma unroll
+        for (int h = 0; h < 32; h += 8) stage8(box, lane, ((c & 63) + h) >> 3, v + h);
+      }
+      staging_release();
+      if (lane == 0) {
+        if (MODE == GEMM_WGRAD) {
+          tma_store_3d(&a.tmOut0, tl.n0 + c0, y0, tl.e, box0);
+          if (tl.n0 + c0 + 64 < a.N) tma_store_3d(&a.tmOut0, tl.n0 + c0 + 64, y0, tl.e, box1);
+        } else {
+          tma_store_2d(&a.tmOut0, tl.n0 + c0, y0, box0);
+          if (tl.n0 + c0 + 64 < a.N) tma_store_2d(&a.tmOut0, tl.n0 + c0 + 64, y0, box1);
+        }
+        tma_store_commit();
       }
     }
   }
@@ -227,7 +287,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;
   uint8_t* sB = smem + STAGES * A_STAGE_BYTES;
-  GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  uint8_t* sOut = smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+  GemmBarriers* bars = reinterpret_cast<GemmBarriers*>(sOut + 4 * OUT_STAGE_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const WaitCtl wc{a.status, a.budget_ns};
@@ -246,6 +307,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
     fence_proxy_async();
     tma_prefetch_desc(&a.tmA);
     tma_prefetch_desc(&a.tmB);
+    tma_prefetch_desc(&a.tmOut0);
   }
   if (warp == 1) {
     tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -320,23 +382,25 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   } else {
     // ------------------------------------------------ epilogue warps
     const int quad = warp & 3;  // TMEM lane quadrant this warp may access
+    uint8_t* stg = sOut + quad * OUT_STAGE_BYTES;
     uint32_t acc_it = 0;
     for (int t = blockIdx.x; t < total; t += gridDim.x) {
       const Tile tl = decode_tile<MODE>(a, t);
       if (tl.nkb == 0) {
-        epilogue_tile<MODE>(a, tl, 0, quad, lane);  // WGRAD of an expert without rows: zeros
+        epilogue_tile<MODE>(a, tl, 0, quad, lane, stg);  // WGRAD of an expert without rows: zeros
         continue;
       }
       const int as = acc_it & 1;
       const uint32_t aph = (acc_it >> 1) & 1;
       if (!mbar_wait(&bars->tmem_full[as], aph, wc, SITE_TMEM_FULL, t)) break;
       tc_fence_after_sync();
-      epilogue_tile<MODE>(a, tl, tmem_base + as * BN, quad, lane);
+      epilogue_tile<MODE>(a, tl, tmem_base + as * BN, quad, lane, stg);
       tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars->tmem_empty[as]);
       ++acc_it;
     }
+    if (lane == 0) tma_store_wait_all();  // this warp's stores are complete before the CTA exits
   }
 
   // ---------------------------------------------------------------- teardown

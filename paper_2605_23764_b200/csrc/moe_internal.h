@@ -70,6 +70,8 @@ enum GemmMode : int {
 struct GemmArgs {
   CUtensorMap tmA;     // A operand
   CUtensorMap tmB;     // B operand
+  CUtensorMap tmOut0;  // store map of out0: [rows][N] (2-D), [rows][2][F] (dH), or [Ep][M][N] (WGRAD)
+  CUtensorMap tmOut1;  // GATE_UP: store map of H as [rows][2][F]
   // tile table
   const int* mblk_expert;
   const int* mb_start;
@@ -84,12 +86,11 @@ struct GemmArgs {
   int b_rows_per_expert;  // rows of the B tensor map per expert slab
   int F;               // intermediate size (GATE_UP / ACT_GRAD epilogues)
   // epilogue tensors
-  uint16_t* out0;      // GATE_UP: A; DOWN: Y; ACT_GRAD: dH; GATE_GRAD: dXp; WGRAD: dW
-  uint16_t* out1;      // GATE_UP: H (may be NULL)
+  int save_h;          // GATE_UP: also store the pre-activations H
   const uint16_t* in0; // ACT_GRAD: H
   const float* prow_w; // GATE_UP, ACT_GRAD: routing weight per padded row
   float* dw_partial;   // ACT_GRAD: [R_pad][n_tiles_n] partial <dA_unweighted, a> (may be NULL)
-  long ld_out0, ld_out1, ld_in0;
+  long ld_in0;
   DevStatus* status;
   uint64_t budget_ns;
 };
