@@ -20,7 +20,8 @@ _BUF_DTYPE = {k: (torch.bfloat16 if k in ("Xp", "H", "A", "Y", "dOutp", "dH", "d
 EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe_layout", "moe_ffn_fwd",
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
-           "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc"]
+           "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
+           "moe_debug_simulate_schedule"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -69,6 +70,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_get_phase_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.moe_route_host.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.moe_layout_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+    lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, i32, vp]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -219,6 +221,16 @@ def moe_layout_noalloc(topk_ids, T, E, k, n_shared, counts, offsets, row_of, src
                                              _dev(counts, i32, "counts"), _dev(offsets, i32, "offsets"),
                                              _dev(row_of, i32, "row_of"), _dev(src_of, i32, "src_of"),
                                              _dev(status2, i32, "status2"), _stream()), "moe_layout_noalloc")
+
+
+def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_workers, vec_workers):
+    """Host-only schedule check; returns (code, stats) with code 0 = schedule is sound."""
+    c = (ctypes.c_int32 * len(counts))(*[int(v) for v in counts])
+    seg = (ctypes.c_int32 * 4)(*[int(v) for v in seg_tiles])
+    stats = (ctypes.c_int64 * 4)()
+    rc = load_library().moe_debug_simulate_schedule(c, len(counts), T, k, int(is_bwd), seg, lag, mat_workers,
+                                                    vec_workers, stats)
+    return rc, list(stats)
 
 
 class _DevView:

@@ -5,6 +5,7 @@
 #include <string.h>
 
 #include <string>
+#include <vector>
 
 #include "../../include/moe_b200.h"
 #include "moe_internal.h"
@@ -96,6 +97,8 @@ bool shape_ok(const moe_shape* s) {
          (long)s->T_max * (s->k + s->n_shared) < (1l << 30);
 }
 
+constexpr int SCHED_LAG_MAX = 64;
+
 struct Carve {
   size_t off = 0;
   size_t take(size_t bytes) {
@@ -108,8 +111,8 @@ struct Carve {
 // Byte offsets of every workspace tensor.
 struct WsPlan {
   size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
-      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, total;
-  int cap_rows, nblk_max, ntn_act;
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, total;
+  int cap_rows, nblk_max, ntn_act, ctr_count;
 };
 
 WsPlan plan_workspace(const moe_shape& s) {
@@ -148,6 +151,9 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.st_out = c.take(2 * (size_t)s.T_max * s.d);
   p.st_dw = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_logits = c.take(sizeof(float) * (size_t)s.T_max * s.E);
+  p.ctr_count = ctr_ints((int)(cap / BLOCK_M) + 1);
+  p.step_start = c.take(sizeof(int) * (cap / BLOCK_M + SCHED_LAG_MAX + 4));
+  p.ctr = c.take(sizeof(int) * (size_t)p.ctr_count);
   p.total = c.off;
   return p;
 }
@@ -164,6 +170,7 @@ struct moe_ctx {
   int launches = 0;
   int saved_T = -1;  // T of the forward whose tensors are in the workspace (-1: none)
   uint64_t budget_ns = 2000ull * 1000 * 1000;
+  int sched_lag = 8;  // M-blocks between a producer step and its consumer step in the matrix queue
   cudaStream_t last_stream = nullptr;
   // optional per-operator timing
   bool profiling = false;
@@ -261,9 +268,136 @@ GemmArgs base_args(const moe_ctx* c) {
   return g;
 }
 
+// GMM1 + SwiGLU (+ routing weight): A = w * silu(Xp.Wg^T) * (Xp.Wu^T)
+GemmArgs args_gate_up(const moe_ctx* c) {
+  const moe_shape& s = c->shape;
+  GemmArgs g = base_args(c);
+  g.tmA = c->tm_Xp_k;
+  g.tmB = c->tm_W1_k;
+  g.n_tiles_n = (s.F + 127) / 128;
+  g.K = s.d;
+  g.N = s.F;
+  g.b_rows_per_expert = 2 * s.F;
+  g.tmOut0 = c->ts_A;
+  g.tmOut1 = c->ts_H;
+  g.save_h = c->train() ? 1 : 0;
+  g.prow_w = c->at<float>(c->plan.prow_w);
+  return g;
+}
+// GMM2: Y = A . W_down^T
+GemmArgs args_down(const moe_ctx* c) {
+  const moe_shape& s = c->shape;
+  GemmArgs g = base_args(c);
+  g.tmA = c->tm_A_k;
+  g.tmB = c->tm_W2_k;
+  g.n_tiles_n = (s.d + 255) / 256;
+  g.K = s.F;
+  g.N = s.d;
+  g.b_rows_per_expert = s.d;
+  g.tmOut0 = c->ts_Y;
+  return g;
+}
+// act_grad + SwiGLU_grad (+ routing-weight gradient partials)
+GemmArgs args_act_grad(const moe_ctx* c, bool want_dw) {
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  GemmArgs g = base_args(c);
+  g.tmA = c->tm_dOutp_k;
+  g.tmB = c->tm_W2_mn;
+  g.n_tiles_n = p.ntn_act;
+  g.K = s.d;
+  g.N = s.F;
+  g.b_rows_per_expert = s.d;
+  g.tmOut0 = c->ts_dH;
+  g.in0 = c->at<uint16_t>(p.H);
+  g.ld_in0 = 2 * s.F;
+  g.prow_w = c->at<float>(p.prow_w);
+  g.dw_partial = want_dw ? c->at<float>(p.dw_partial) : nullptr;
+  return g;
+}
+// w2_grad: dW_down[e][c][f] = sum_rows dOutp[r][c] * A[r][f]   (shares dOutp with act_grad)
+GemmArgs args_wgrad_down(const moe_ctx* c) {
+  const moe_shape& s = c->shape;
+  GemmArgs g = base_args(c);
+  g.tmA = c->tm_dOutp_mn;
+  g.tmB = c->tm_A_mn;
+  g.M = s.d;
+  g.N = s.F;
+  g.n_tiles_m = (s.d + 127) / 128;
+  g.n_tiles_n = (s.F + 255) / 256;
+  g.tmOut0 = c->ts_dW2;
+  return g;
+}
+// gate_grad: dXp = dH . W_gate_up[e]   (the forward's Y is dead by now: its buffer receives dXp)
+GemmArgs args_gate_grad(const moe_ctx* c) {
+  const moe_shape& s = c->shape;
+  GemmArgs g = base_args(c);
+  g.tmA = c->tm_dH_k;
+  g.tmB = c->tm_W1_mn;
+  g.n_tiles_n = (s.d + 255) / 256;
+  g.K = 2 * s.F;
+  g.N = s.d;
+  g.b_rows_per_expert = 2 * s.F;
+  g.tmOut0 = c->ts_Y;
+  return g;
+}
+// w1_grad: dW_gate_up[e][n][c] = sum_rows dH[r][n] * Xp[r][c]   (shares dH with gate_grad)
+GemmArgs args_wgrad_gate_up(const moe_ctx* c) {
+  const moe_shape& s = c->shape;
+  GemmArgs g = base_args(c);
+  g.tmA = c->tm_dH_mn;
+  g.tmB = c->tm_Xp_mn;
+  g.M = 2 * s.F;
+  g.N = s.d;
+  g.n_tiles_m = (2 * s.F + 127) / 128;
+  g.n_tiles_n = (s.d + 255) / 256;
+  g.tmOut0 = c->ts_dW1;
+  return g;
+}
+
+bool serial_mode(const moe_ctx* c) { return (c->shape.flags & MOE_FLAG_SERIAL_LAUNCH) != 0; }
+
+SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
+  const moe_shape& s = c->shape;
+  SchedParams sp;
+  memset(&sp, 0, sizeof sp);
+  sp.is_bwd = bwd ? 1 : 0;
+  sp.lag = c->sched_lag;
+  sp.Ep = s.E + s.n_shared;
+  sp.T = T;
+  sp.k = s.k;
+  if (!bwd) {
+    sp.seg_tiles[0] = (s.F + 127) / 128;
+    sp.seg_tiles[1] = (s.d + 255) / 256;
+  } else {
+    sp.seg_tiles[0] = c->plan.ntn_act;
+    sp.wgrad_tn[0] = (s.F + 255) / 256;
+    sp.seg_tiles[1] = ((s.d + 127) / 128) * sp.wgrad_tn[0];
+    sp.seg_tiles[2] = (s.d + 255) / 256;
+    sp.wgrad_tn[1] = (s.d + 255) / 256;
+    sp.seg_tiles[3] = ((2 * s.F + 127) / 128) * sp.wgrad_tn[1];
+  }
+  return sp;
+}
+
+FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
+  const moe_shape& s = c->shape;
+  const WsPlan& p = c->plan;
+  FusedArgs fa;
+  memset(&fa, 0, sizeof fa);
+  fa.sp = sched_params(c, bwd, T);
+  fa.lv = c->layout();
+  fa.step_start = c->at<int>(p.step_start);
+  fa.ctr = c->at<int>(p.ctr);
+  fa.d = s.d;
+  fa.kp = s.k + s.n_shared;
+  fa.status = c->status();
+  fa.budget_ns = c->budget_ns;
+  return fa;
+}
+
 int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, const uint16_t* W1,
             const uint16_t* W2, uint16_t* out, int T, cudaStream_t st) {
-  const moe_shape& s = c->shape;
   const WsPlan& p = c->plan;
   const Dims dm = c->dims(T);
   const LayoutView lv = c->layout();
@@ -274,41 +408,39 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     Phase ph(c, MOE_PHASE_LAYOUT, st);
     MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
   }
-  {
-    Phase ph(c, MOE_PHASE_GATHER, st);
-    MOE_CUDA(launch_gather(x, w, dm, lv, c->at<uint16_t>(p.Xp), c->at<float>(p.prow_w), p.cap_rows, st,
-                           &c->launches));
-  }
-  {  // GMM1 + SwiGLU (+ routing weight)
-    GemmArgs g = base_args(c);
-    g.tmA = c->tm_Xp_k;
-    g.tmB = c->tm_W1_k;
-    g.n_tiles_n = (s.F + 127) / 128;
-    g.K = s.d;
-    g.N = s.F;
-    g.b_rows_per_expert = 2 * s.F;
-    g.tmOut0 = c->ts_A;
-    g.tmOut1 = c->ts_H;
-    g.save_h = c->train() ? 1 : 0;
-    g.prow_w = c->at<float>(p.prow_w);
-    Phase ph(c, MOE_PHASE_GEMM_GATE_UP, st);
-    MOE_CUDA(launch_gemm(GEMM_GATE_UP, g, c->num_sms, st, &c->launches));
-  }
-  {  // GMM2
-    GemmArgs g = base_args(c);
-    g.tmA = c->tm_A_k;
-    g.tmB = c->tm_W2_k;
-    g.n_tiles_n = (s.d + 255) / 256;
-    g.K = s.F;
-    g.N = s.d;
-    g.b_rows_per_expert = s.d;
-    g.tmOut0 = c->ts_Y;
-    Phase ph(c, MOE_PHASE_GEMM_DOWN, st);
-    MOE_CUDA(launch_gemm(GEMM_DOWN, g, c->num_sms, st, &c->launches));
-  }
-  {
-    Phase ph(c, MOE_PHASE_COMBINE, st);
-    MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+  if (serial_mode(c)) {
+    {
+      Phase ph(c, MOE_PHASE_GATHER, st);
+      MOE_CUDA(launch_gather(x, w, dm, lv, c->at<uint16_t>(p.Xp), c->at<float>(p.prow_w), p.cap_rows, st,
+                             &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_GEMM_GATE_UP, st);
+      MOE_CUDA(launch_gemm(GEMM_GATE_UP, args_gate_up(c), c->num_sms, st, &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_GEMM_DOWN, st);
+      MOE_CUDA(launch_gemm(GEMM_DOWN, args_down(c), c->num_sms, st, &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_COMBINE, st);
+      MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+    }
+  } else {
+    // one persistent launch: gather, GMM1+SwiGLU, GMM2 and combine tiles ordered by event counters
+    FusedArgs fa = fused_base(c, false, T);
+    fa.op[0] = args_gate_up(c);
+    fa.op[1] = args_down(c);
+    fa.gather_src = x;
+    fa.gather_dst = c->at<uint16_t>(p.Xp);
+    fa.topk_w = w;
+    fa.prow_w = c->at<float>(p.prow_w);
+    fa.combine_rows = c->at<uint16_t>(p.Y);
+    fa.combine_out = out;
+    Phase ph(c, MOE_PHASE_FUSED_FWD, st);
+    MOE_CUDA(launch_build_schedule(fa.sp, lv, c->at<int>(p.step_start), c->at<int>(p.ctr), p.ctr_count, st,
+                                   &c->launches));
+    MOE_CUDA(launch_fused(false, fa, c->num_sms, st, &c->launches));
   }
   if (c->train()) c->saved_T = T;
   return MOE_OK;
@@ -331,70 +463,57 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     if ((rc = encode_slabs(&c->ts_dW2, dW2, Ep, s.d, s.F))) return rc;
     c->dw2_ptr = dW2;
   }
-  // backward Dispatch: expert-ordered gather of the upstream gradient
-  {
-    Phase ph(c, MOE_PHASE_BWD_GATHER, st);
-    MOE_CUDA(launch_gather(dout, nullptr, dm, lv, c->at<uint16_t>(p.dOutp), nullptr, p.cap_rows, st, &c->launches));
-  }
-  {  // act_grad + SwiGLU_grad (+ routing-weight gradient partials)
-    GemmArgs g = base_args(c);
-    g.tmA = c->tm_dOutp_k;
-    g.tmB = c->tm_W2_mn;
-    g.n_tiles_n = p.ntn_act;
-    g.K = s.d;
-    g.N = s.F;
-    g.b_rows_per_expert = s.d;
-    g.tmOut0 = c->ts_dH;
-    g.in0 = c->at<uint16_t>(p.H);
-    g.ld_in0 = 2 * s.F;
-    g.prow_w = c->at<float>(p.prow_w);
-    g.dw_partial = d_w ? c->at<float>(p.dw_partial) : nullptr;
-    Phase ph(c, MOE_PHASE_ACT_GRAD, st);
-    MOE_CUDA(launch_gemm(GEMM_ACT_GRAD, g, c->num_sms, st, &c->launches));
-  }
-  if (d_w) {
-    Phase ph(c, MOE_PHASE_DW_REDUCE, st);
-    MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), p.ntn_act, dm, lv, d_w, st, &c->launches));
-  }
-  {  // w2_grad: dW_down[e][c][f] = sum_rows dOutp[r][c] * A[r][f]   (shares dOutp with act_grad)
-    GemmArgs g = base_args(c);
-    g.tmA = c->tm_dOutp_mn;
-    g.tmB = c->tm_A_mn;
-    g.M = s.d;
-    g.N = s.F;
-    g.n_tiles_m = (s.d + 127) / 128;
-    g.n_tiles_n = (s.F + 255) / 256;
-    g.tmOut0 = c->ts_dW2;
-    Phase ph(c, MOE_PHASE_WGRAD_DOWN, st);
-    MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
-  }
-  {  // gate_grad: dXp = dH . W_gate_up[e]
-    GemmArgs g = base_args(c);
-    g.tmA = c->tm_dH_k;
-    g.tmB = c->tm_W1_mn;
-    g.n_tiles_n = (s.d + 255) / 256;
-    g.K = 2 * s.F;
-    g.N = s.d;
-    g.b_rows_per_expert = 2 * s.F;
-    g.tmOut0 = c->ts_Y;  // the forward's Y is dead by now: its buffer receives dXp
-    Phase ph(c, MOE_PHASE_GATE_GRAD, st);
-    MOE_CUDA(launch_gemm(GEMM_GATE_GRAD, g, c->num_sms, st, &c->launches));
-  }
-  {  // w1_grad: dW_gate_up[e][n][c] = sum_rows dH[r][n] * Xp[r][c]   (shares dH with gate_grad)
-    GemmArgs g = base_args(c);
-    g.tmA = c->tm_dH_mn;
-    g.tmB = c->tm_Xp_mn;
-    g.M = 2 * s.F;
-    g.N = s.d;
-    g.n_tiles_m = (2 * s.F + 127) / 128;
-    g.n_tiles_n = (s.d + 255) / 256;
-    g.tmOut0 = c->ts_dW1;
-    Phase ph(c, MOE_PHASE_WGRAD_GATE_UP, st);
-    MOE_CUDA(launch_gemm(GEMM_WGRAD, g, c->num_sms, st, &c->launches));
-  }
-  {  // backward Combine
-    Phase ph(c, MOE_PHASE_BWD_COMBINE, st);
-    MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
+  if (serial_mode(c)) {
+    {  // backward Dispatch: expert-ordered gather of the upstream gradient
+      Phase ph(c, MOE_PHASE_BWD_GATHER, st);
+      MOE_CUDA(launch_gather(dout, nullptr, dm, lv, c->at<uint16_t>(p.dOutp), nullptr, p.cap_rows, st,
+                             &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_ACT_GRAD, st);
+      MOE_CUDA(launch_gemm(GEMM_ACT_GRAD, args_act_grad(c, d_w != nullptr), c->num_sms, st, &c->launches));
+    }
+    if (d_w) {
+      Phase ph(c, MOE_PHASE_DW_REDUCE, st);
+      MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), p.ntn_act, dm, lv, d_w, st, &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_WGRAD_DOWN, st);
+      MOE_CUDA(launch_gemm(GEMM_WGRAD, args_wgrad_down(c), c->num_sms, st, &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_GATE_GRAD, st);
+      MOE_CUDA(launch_gemm(GEMM_GATE_GRAD, args_gate_grad(c), c->num_sms, st, &c->launches));
+    }
+    {
+      Phase ph(c, MOE_PHASE_WGRAD_GATE_UP, st);
+      MOE_CUDA(launch_gemm(GEMM_WGRAD, args_wgrad_gate_up(c), c->num_sms, st, &c->launches));
+    }
+    {  // backward Combine
+      Phase ph(c, MOE_PHASE_BWD_COMBINE, st);
+      MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
+    }
+  } else {
+    FusedArgs fa = fused_base(c, true, T);
+    fa.op[0] = args_act_grad(c, d_w != nullptr);
+    fa.op[1] = args_wgrad_down(c);
+    fa.op[2] = args_gate_grad(c);
+    fa.op[3] = args_wgrad_gate_up(c);
+    fa.gather_src = dout;
+    fa.gather_dst = c->at<uint16_t>(p.dOutp);
+    fa.combine_rows = c->at<uint16_t>(p.Y);
+    fa.combine_out = dx;
+    fa.dw_partial = c->at<float>(p.dw_partial);
+    fa.dw_nparts = p.ntn_act;
+    fa.d_topk_w = d_w;
+    fa.dW1 = dW1;
+    fa.dW2 = dW2;
+    fa.dW1_slab_vec = (size_t)2 * s.F * s.d * 2 / 16;
+    fa.dW2_slab_vec = (size_t)s.d * s.F * 2 / 16;
+    Phase ph(c, MOE_PHASE_FUSED_BWD, st);
+    MOE_CUDA(launch_build_schedule(fa.sp, lv, c->at<int>(p.step_start), c->at<int>(p.ctr), p.ctr_count, st,
+                                   &c->launches));
+    MOE_CUDA(launch_fused(true, fa, c->num_sms, st, &c->launches));
   }
   return MOE_OK;
 }
@@ -678,6 +797,104 @@ int moe_debug_buffer(moe_ctx* c, int which, void** ptr, size_t* elems) {
   }
   *ptr = c->ws + off;
   *elems = n;
+  return MOE_OK;
+}
+
+// Host-only check of the static schedule (no GPU needed): builds the tile queues for the given
+// per-expert row counts and lets `mat_workers` matrix workers and `vec_workers` vector workers
+// consume them in ticket order, each blocking on its tile's dependent counters.
+int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t is_bwd,
+                                const int32_t* seg_tiles, int32_t lag, int32_t mat_workers, int32_t vec_workers,
+                                int64_t* stats) {
+  if (!counts || !seg_tiles || Ep < 1 || lag < 0 || mat_workers < 1 || vec_workers < 1) return MOE_ERR_INVALID_ARG;
+  std::vector<int> mb_start(Ep + 1, 0), mblk_expert;
+  for (int e = 0; e < Ep; ++e) {
+    const int m = (counts[e] + BLOCK_M - 1) / BLOCK_M;
+    mb_start[e + 1] = mb_start[e] + m;
+    for (int q = 0; q < m; ++q) mblk_expert.push_back(e);
+  }
+  const int M = mb_start[Ep];
+  mblk_expert.push_back(0);
+  SchedParams sp;
+  memset(&sp, 0, sizeof sp);
+  sp.is_bwd = is_bwd; sp.lag = lag; sp.Ep = Ep; sp.T = T; sp.k = k;
+  for (int i = 0; i < SCHED_MAX_SEG; ++i) sp.seg_tiles[i] = seg_tiles[i];
+  std::vector<int> step_start(M + lag + 1, 0);
+  for (int i = 0; i < M + lag; ++i)
+    step_start[i + 1] = step_start[i] + step_tiles(sp, i, M, mblk_expert.data(), mb_start.data());
+  const int total = step_start[M + lag], vtotal = vec_total(sp, M);
+  std::vector<long> ctr(ctr_ints(M + 1), 0);
+  // 1. coverage and ticket order of producers
+  std::vector<int> seg0_last_ticket(M, -1), seg0_count(M, 0), lag_count(M, 0);
+  std::vector<int> w2_count(Ep, 0), w1_count(Ep, 0);
+  for (int t = 0; t < total; ++t) {
+    const MatTile m = decode_matrix_ticket(sp, t, M, step_start.data(), mblk_expert.data(), mb_start.data());
+    if (m.e < 0 || m.e >= Ep || m.idx < 0 || m.idx >= sp.seg_tiles[m.slot]) return 10;
+    if (m.slot == 0) { seg0_last_ticket[m.mb] = t; seg0_count[m.mb]++; }
+    else if (m.mb >= 0) { lag_count[m.mb]++; if (seg0_last_ticket[m.mb] < 0 || seg0_count[m.mb] != sp.seg_tiles[0]) return 11; }
+    else if (m.slot == 1) w2_count[m.e]++;
+    else {
+      w1_count[m.e]++;
+      for (int q = 0; q < m.dep_count; ++q)
+        if (seg0_count[m.dep_first + q] != sp.seg_tiles[0]) return 12;  // a producer with a larger ticket
+    }
+  }
+  for (int mb = 0; mb < M; ++mb)
+    if (seg0_count[mb] != sp.seg_tiles[0] || lag_count[mb] != (is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1])) return 13;
+  if (is_bwd)
+    for (int e = 0; e < Ep; ++e) {
+      const int want = counts[e] > 0 ? 1 : 0;
+      if (w2_count[e] != want * sp.seg_tiles[1] || w1_count[e] != want * sp.seg_tiles[3]) return 14;
+    }
+  // 2. consumption by a bounded number of workers
+  struct Worker { bool holding = false; MatTile m; VecTask v; };
+  std::vector<Worker> mw(mat_workers), vw(vec_workers);
+  int next_mat = 0, next_vec = 0, done_mat = 0, done_vec = 0;
+  long rounds = 0, stalls = 0;
+  while (done_mat < total || done_vec < vtotal) {
+    bool progress = false;
+    for (auto& wk : mw) {
+      if (!wk.holding && next_mat < total) {
+        wk.m = decode_matrix_ticket(sp, next_mat++, M, step_start.data(), mblk_expert.data(), mb_start.data());
+        wk.holding = true;
+        progress = true;
+      }
+      if (!wk.holding) continue;
+      bool ready = true;
+      for (int q = 0; q < wk.m.dep_count; ++q) {
+        const int mb = wk.m.dep_first + q;
+        if (ctr[wk.m.dep_base == 0 ? ctr_gather(mb) : ctr_act(mb)] < wk.m.dep_thr) ready = false;
+      }
+      if (!ready) { ++stalls; continue; }
+      if (wk.m.trig_base == 1) ctr[ctr_act(wk.m.mb)] += EPI_WARPS;
+      if (wk.m.trig_base == 2) ctr[CTR_DONE] += EPI_WARPS;
+      if (wk.m.trig_also_ag) ctr[CTR_AG_DONE] += EPI_WARPS;
+      wk.holding = false;
+      ++done_mat;
+      progress = true;
+    }
+    for (auto& wk : vw) {
+      if (!wk.holding && next_vec < vtotal) {
+        wk.v = decode_vector_ticket(sp, next_vec++, M);
+        wk.holding = true;
+        progress = true;
+      }
+      if (!wk.holding) continue;
+      if (wk.v.dep && ctr[wk.v.dep == 2 ? CTR_DONE : CTR_AG_DONE] < wk.v.dep_thr) { ++stalls; continue; }
+      if (wk.v.op == VEC_GATHER) ctr[ctr_gather(wk.v.idx / GATHER_SUB)] += 1;
+      wk.holding = false;
+      ++done_vec;
+      progress = true;
+    }
+    ++rounds;
+    if (!progress) return 20;  // deadlock
+  }
+  // 3. every counter ends exactly at its threshold
+  for (int mb = 0; mb < M; ++mb)
+    if (ctr[ctr_gather(mb)] != GATHER_SUB || ctr[ctr_act(mb)] != (long)EPI_WARPS * sp.seg_tiles[0]) return 30;
+  if (ctr[CTR_DONE] != (long)EPI_WARPS * M * (is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1])) return 31;
+  if (is_bwd && ctr[CTR_AG_DONE] != (long)EPI_WARPS * M * sp.seg_tiles[0]) return 32;
+  if (stats) { stats[0] = total; stats[1] = vtotal; stats[2] = rounds; stats[3] = stalls; }
   return MOE_OK;
 }
 

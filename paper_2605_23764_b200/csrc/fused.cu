@@ -1,0 +1,460 @@
+// The single persistent, dependency-driven launch of the forward (and of the backward) layer.
+//
+// One cooperative grid of one CTA per SM runs the whole operator chain.  Per CTA:
+//   warp 0      matrix-queue producer: takes the next ticket of the matrix queue, decodes the tile,
+//               publishes it to the CTA's other roles, polls the tile's dependent counters, then
+//               streams its operands through TMA;
+//   warp 1      tcgen05.mma issuer (and TMEM owner);
+//   warps 2-5   epilogue: TMEM -> fused element-wise math -> TMA store, then the tile's trigger
+//               counter once the stores are complete;
+//   warps 6-9   vector workers: take tickets of the vector queue (permute-gather, zero-fill of
+//               weight gradients of experts without rows, routing-weight gradient, combine).
+// This is the paper's unified runtime (Section 4.4) restated for one SM: matrix and vector work
+// progress concurrently inside one launch, ordered only by event counters with static thresholds
+// (Section 4.3).  The tile math is the same code the one-launch-per-operator mode runs.
+#include <cooperative_groups.h>
+
+#include <vector>
+
+#include "gemm_tile.cuh"
+#include "schedule.h"
+
+namespace moe {
+
+constexpr int FUSED_THREADS = GEMM_THREADS + 128;  // + 4 vector warps
+constexpr int RING = 4;                            // published-tile ring depth
+
+struct TileSlot {
+  int op, slot, e, row0, n0, m0, nkb, nb;
+  int trig_idx;   // counter index to bump per epilogue warp, -1 = none
+  int trig_ag;    // also bump the global act_grad counter
+  int pad[2];
+};
+
+struct __align__(16) FusedShared {
+  GemmBarriers bars;
+  uint64_t tk_full[RING];
+  uint64_t tk_empty[RING];
+  TileSlot ring[RING];
+};
+
+constexpr size_t FUSED_SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + 4 * OUT_STAGE_BYTES +
+                                    sizeof(FusedShared);
+static_assert(FUSED_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+// ---------------------------------------------------------------- schedule prefix + counter reset
+// One block: step_start[i] = tickets before step i (i in [0, M+lag]); counters zeroed.
+__global__ void __launch_bounds__(1024) build_schedule_kernel(SchedParams sp, LayoutView lv, int* step_start,
+                                                              int* ctr, int ctr_count) {
+  __shared__ int warp_sums[32];
+  __shared__ int carry_s;
+  const int M = lv.meta[0];
+  const int n = M + sp.lag;
+  for (int i = threadIdx.x; i < ctr_count; i += blockDim.x) ctr[i] = 0;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int base = 0; base < n; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int v = i < n ? step_tiles(sp, i, M, lv.mblk_expert, lv.mb_start) : 0;
+    int incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      int o = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += o;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_sums[lane];
+      int wi = w;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        int o = __shfl_up_sync(0xffffffffu, wi, off);
+        if (lane >= off) wi += o;
+      }
+      warp_sums[lane] = wi - w;  // exclusive
+    }
+    __syncthreads();
+    const int carry = carry_s;
+    const int excl = carry + warp_sums[warp] + incl - v;
+    if (i < n) step_start[i] = excl;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry_s = excl + v;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) step_start[n] = carry_s;
+}
+
+// ---------------------------------------------------------------- vector work (one warp per task)
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ void vec_gather(const FusedArgs& fa, int task, int lane) {
+  const int mb = task / GATHER_SUB, sub = task - mb * GATHER_SUB;
+  const LayoutView& lv = fa.lv;
+  const int e = lv.mblk_expert[mb];
+  const int cnt = lv.counts[e], pad0 = lv.pad_off[e], off0 = lv.offsets[e];
+  const int nvec = fa.d >> 3;
+  const int k = fa.sp.k;
+  for (int r = 0; r < BLOCK_M / GATHER_SUB; ++r) {
+    const int p = mb * BLOCK_M + sub * (BLOCK_M / GATHER_SUB) + r;
+    const int local = p - pad0;
+    uint4* out = reinterpret_cast<uint4*>(fa.gather_dst + (size_t)p * fa.d);
+    if (local < cnt) {
+      const int slot = lv.src_of[off0 + local];
+      const int t = slot / fa.kp, j = slot - t * fa.kp;
+      const uint4* in = reinterpret_cast<const uint4*>(fa.gather_src + (size_t)t * fa.d);
+      int v = lane;
+      for (; v + 96 < nvec; v += 128) {
+        uint4 a = ldg_nc_v4(in + v), b = ldg_nc_v4(in + v + 32), c = ldg_nc_v4(in + v + 64),
+              dd = ldg_nc_v4(in + v + 96);
+        out[v] = a; out[v + 32] = b; out[v + 64] = c; out[v + 96] = dd;
+      }
+      for (; v < nvec; v += 32) out[v] = ldg_nc_v4(in + v);
+      if (fa.prow_w && lane == 0) fa.prow_w[p] = j < k ? fa.topk_w[(size_t)t * k + j] : 1.0f;
+    } else {
+      for (int v = lane; v < nvec; v += 32) out[v] = make_uint4(0, 0, 0, 0);
+      if (fa.prow_w && lane == 0) fa.prow_w[p] = 0.0f;
+    }
+  }
+}
+
+__device__ __forceinline__ void vec_combine(const FusedArgs& fa, int task, int lane) {
+  const int nvec = fa.d >> 3, kp = fa.kp, T = fa.sp.T;
+  const int t1 = min(T, (task + 1) * COMBINE_TOKENS);
+  for (int t = task * COMBINE_TOKENS; t < t1; ++t) {
+    for (int v = lane; v < nvec; v += 32) {
+      float acc[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+      for (int j = 0; j < kp; ++j) {
+        const int p = fa.lv.prow_of[(size_t)t * kp + j];
+        if (p < 0) continue;
+        // plain (coherent) load: these rows were written earlier in this same launch
+        const uint4 r = *(reinterpret_cast<const uint4*>(fa.combine_rows + (size_t)p * fa.d) + v);
+        acc[0] += bf16lo(r.x); acc[1] += bf16hi(r.x);
+        acc[2] += bf16lo(r.y); acc[3] += bf16hi(r.y);
+        acc[4] += bf16lo(r.z); acc[5] += bf16hi(r.z);
+        acc[6] += bf16lo(r.w); acc[7] += bf16hi(r.w);
+      }
+      uint4 o;
+      o.x = pack_bf16x2(acc[0], acc[1]);
+      o.y = pack_bf16x2(acc[2], acc[3]);
+      o.z = pack_bf16x2(acc[4], acc[5]);
+      o.w = pack_bf16x2(acc[6], acc[7]);
+      reinterpret_cast<uint4*>(fa.combine_out + (size_t)t * fa.d)[v] = o;
+    }
+  }
+}
+
+__device__ __forceinline__ void vec_dw(const FusedArgs& fa, int task, int lane) {
+  if (!fa.d_topk_w) return;
+  const int k = fa.sp.k, n = fa.sp.T * k;
+  for (int i = task * DW_SLOTS + lane; i < min(n, (task + 1) * DW_SLOTS); i += 32) {
+    const int t = i / k, j = i - t * k;
+    const int p = fa.lv.prow_of[(size_t)t * fa.kp + j];
+    float s = 0.f;
+    if (p >= 0)
+      for (int q = 0; q < fa.dw_nparts; ++q) s += fa.dw_partial[(size_t)p * fa.dw_nparts + q];
+    fa.d_topk_w[i] = s;
+  }
+}
+
+__device__ __forceinline__ void vec_zero(const FusedArgs& fa, int task, int lane) {
+  const int e = task / ZERO_CHUNKS, ch = task - e * ZERO_CHUNKS;
+  if (fa.lv.counts[e] != 0) return;  // only experts without rows: their weight gradients are exact zeros
+  uint4* s1 = reinterpret_cast<uint4*>(fa.dW1) + (size_t)e * fa.dW1_slab_vec;
+  uint4* s2 = reinterpret_cast<uint4*>(fa.dW2) + (size_t)e * fa.dW2_slab_vec;
+  const uint4 z = make_uint4(0, 0, 0, 0);
+  for (size_t v = fa.dW1_slab_vec * ch / ZERO_CHUNKS + lane; v < fa.dW1_slab_vec * (ch + 1) / ZERO_CHUNKS; v += 32)
+    s1[v] = z;
+  for (size_t v = fa.dW2_slab_vec * ch / ZERO_CHUNKS + lane; v < fa.dW2_slab_vec * (ch + 1) / ZERO_CHUNKS; v += 32)
+    s2[v] = z;
+}
+
+// ---------------------------------------------------------------- matrix-role dispatch on the operator
+template <bool BWD>
+__device__ __forceinline__ void fused_load_stage(const FusedArgs& fa, const TileSlot& ts, const Tile& tl, int kb,
+                                                 uint8_t* sA, uint8_t* sB, uint64_t* bar) {
+  const GemmArgs& g = fa.op[ts.slot];
+  if (!BWD) {
+    if (ts.op == GEMM_GATE_UP) load_stage<GEMM_GATE_UP>(g, tl, kb, sA, sB, bar);
+    else load_stage<GEMM_DOWN>(g, tl, kb, sA, sB, bar);
+  } else {
+    if (ts.op == GEMM_ACT_GRAD) load_stage<GEMM_ACT_GRAD>(g, tl, kb, sA, sB, bar);
+    else if (ts.op == GEMM_GATE_GRAD) load_stage<GEMM_GATE_GRAD>(g, tl, kb, sA, sB, bar);
+    else load_stage<GEMM_WGRAD>(g, tl, kb, sA, sB, bar);
+  }
+}
+template <bool BWD>
+__device__ __forceinline__ void fused_mma(int op, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first) {
+  if (!BWD) {
+    mma_kblock<GEMM_GATE_UP>(d_tmem, a_addr, b_addr, first);  // GATE_UP and DOWN: same operand layouts
+  } else {
+    if (op == GEMM_WGRAD) mma_kblock<GEMM_WGRAD>(d_tmem, a_addr, b_addr, first);
+    else mma_kblock<GEMM_ACT_GRAD>(d_tmem, a_addr, b_addr, first);  // ACT_GRAD and GATE_GRAD alike
+  }
+}
+template <bool BWD>
+__device__ __forceinline__ void fused_epilogue(const FusedArgs& fa, const TileSlot& ts, const Tile& tl,
+                                               uint32_t tmem_acc, int quad, int lane, uint8_t* stg) {
+  const GemmArgs& g = fa.op[ts.slot];
+  if (!BWD) {
+    if (ts.op == GEMM_GATE_UP) epilogue_tile<GEMM_GATE_UP>(g, tl, tmem_acc, quad, lane, stg);
+    else epilogue_tile<GEMM_DOWN>(g, tl, tmem_acc, quad, lane, stg);
+  } else {
+    if (ts.op == GEMM_ACT_GRAD) epilogue_tile<GEMM_ACT_GRAD>(g, tl, tmem_acc, quad, lane, stg);
+    else if (ts.op == GEMM_GATE_GRAD) epilogue_tile<GEMM_GATE_GRAD>(g, tl, tmem_acc, quad, lane, stg);
+    else epilogue_tile<GEMM_WGRAD>(g, tl, tmem_acc, quad, lane, stg);
+  }
+}
+
+__device__ __forceinline__ Tile slot_tile(const TileSlot& ts) {
+  Tile tl;
+  tl.e = ts.e; tl.row0 = ts.row0; tl.n0 = ts.n0; tl.m0 = ts.m0; tl.nkb = ts.nkb; tl.nb = ts.nb;
+  return tl;
+}
+
+// ---------------------------------------------------------------- the kernel
+template <bool BWD>
+__global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_constant__ FusedArgs fa) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + STAGES * A_STAGE_BYTES;
+  uint8_t* sOut = smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES);
+  FusedShared* sh = reinterpret_cast<FusedShared*>(sOut + 4 * OUT_STAGE_BYTES);
+  GemmBarriers* bars = &sh->bars;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WaitCtl wc{fa.status, fa.budget_ns};
+  const int M = fa.lv.meta[0];
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&bars->full[s], 1);
+      mbar_init(&bars->empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&bars->tmem_full[s], 1);
+      mbar_init(&bars->tmem_empty[s], EPI_WARPS);
+    }
+    mbar_init(&bars->drain, 1);
+    for (int s = 0; s < RING; ++s) {
+      mbar_init(&sh->tk_full[s], 1);
+      mbar_init(&sh->tk_empty[s], 1 + EPI_WARPS);  // the MMA issuer and every epilogue warp release a slot
+    }
+    mbar_fence_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc(&bars->tmem_base, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------ matrix-queue producer
+    if (lane == 0) {
+      const int total = fa.step_start[M + fa.sp.lag];
+      uint32_t it = 0, n = 0;
+      bool ok = true;
+      while (ok) {
+        const int t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
+        TileSlot ts;
+        MatTile mt;
+        if (t >= total) {
+          ts.op = -1; ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
+          ts.trig_idx = -1; ts.trig_ag = 0;
+        } else {
+          mt = decode_matrix_ticket(fa.sp, t, M, fa.step_start, fa.lv.mblk_expert, fa.lv.mb_start);
+          const GemmArgs& g = fa.op[mt.slot];
+          ts.op = mt.op; ts.slot = mt.slot; ts.e = mt.e;
+          if (mt.op == GEMM_WGRAD) {
+            const int mbw = mt.idx / g.n_tiles_n;
+            ts.nb = mt.idx - mbw * g.n_tiles_n;
+            ts.m0 = mbw * BLOCK_M;
+            ts.n0 = ts.nb * BN;
+            ts.row0 = fa.lv.mb_start[mt.e] * BLOCK_M;
+            ts.nkb = (fa.lv.counts[mt.e] + BK - 1) / BK;
+          } else {
+            ts.nb = mt.idx;
+            ts.m0 = 0;
+            ts.n0 = mt.idx * (mt.op == GEMM_GATE_UP ? BN / 2 : BN);
+            ts.row0 = mt.mb * BLOCK_M;
+            ts.nkb = (g.K + BK - 1) / BK;
+          }
+          ts.trig_idx = mt.trig_base == 1 ? ctr_act(mt.mb) : (mt.trig_base == 2 ? CTR_DONE : -1);
+          ts.trig_ag = mt.trig_also_ag;
+        }
+        const int rs = n % RING;
+        if (!mbar_wait(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) break;
+        sh->ring[rs] = ts;
+        mbar_arrive(&sh->tk_full[rs]);  // release: the slot's contents are visible to the waiters
+        ++n;
+        if (ts.op < 0) break;
+        // dependent event(s): poll until every producer counter has reached its threshold
+        for (int q = 0; q < mt.dep_count && ok; ++q) {
+          const int mbq = mt.dep_first + q;
+          const int* c = fa.ctr + (mt.dep_base == 0 ? ctr_gather(mbq) : ctr_act(mbq));
+          ok = counter_wait(c, mt.dep_thr, wc, t);
+        }
+        if (!ok) break;
+        fence_proxy_async();  // the producers' writes must be seen by the TMA loads that follow
+        const Tile tl = slot_tile(ts);
+        for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
+          fused_load_stage<BWD>(fa, ts, tl, kb, sA + s * A_STAGE_BYTES, sB + s * B_STAGE_BYTES, &bars->full[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, acc_it = 0, n = 0;
+      bool ok = true;
+      while (ok) {
+        const int rs = n % RING;
+        if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -1)) break;
+        const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb;
+        mbar_arrive(&sh->tk_empty[rs]);
+        ++n;
+        if (op < 0) break;
+        if (nkb == 0) continue;
+        const int as = acc_it & 1;
+        if (!mbar_wait(&bars->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, n)) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + as * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGES;
+          if (!mbar_wait(&bars->full[s], (it / STAGES) & 1, wc, SITE_FULL, n)) { ok = false; break; }
+          tc_fence_after_sync();
+          fused_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * B_STAGE_BYTES), kb == 0);
+          tc_commit(&bars->empty[s]);
+        }
+        if (!ok) break;
+        tc_commit(&bars->tmem_full[as]);
+        ++acc_it;
+      }
+      if (*reinterpret_cast<volatile int*>(&fa.status->abort)) {
+        tc_commit(&bars->drain);
+        const WaitCtl shortwc{fa.status, 20ull * 1000 * 1000};
+        mbar_wait(&bars->drain, 0, shortwc, SITE_DRAIN, 0);
+      }
+    }
+  } else if (warp < 2 + EPI_WARPS) {
+    // ------------------------------------------------ epilogue warps
+    const int quad = warp & 3;
+    uint8_t* stg = sOut + quad * OUT_STAGE_BYTES;
+    uint32_t acc_it = 0, n = 0;
+    while (true) {
+      const int rs = n % RING;
+      if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -2)) break;
+      const TileSlot ts = sh->ring[rs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->tk_empty[rs]);
+      ++n;
+      if (ts.op < 0) break;
+      const Tile tl = slot_tile(ts);
+      if (ts.nkb == 0) {
+        fused_epilogue<BWD>(fa, ts, tl, 0, quad, lane, stg);
+      } else {
+        const int as = acc_it & 1;
+        if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, n)) break;
+        tc_fence_after_sync();
+        fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->tmem_empty[as]);
+        ++acc_it;
+      }
+      if (ts.trig_idx >= 0) {
+        // trigger event: only after this warp's part of the tile is readable by everyone
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_wait_all();
+          fence_proxy_async();
+          counter_signal(fa.ctr + ts.trig_idx, 1);
+          if (ts.trig_ag) counter_signal(fa.ctr + CTR_AG_DONE, 1);
+        }
+      }
+    }
+    if (lane == 0) tma_store_wait_all();
+  } else {
+    // ------------------------------------------------ vector workers
+    const int vtotal = vec_total(fa.sp, M);
+    while (true) {
+      int t = 0;
+      if (lane == 0) t = atomicAdd(&fa.ctr[CTR_VEC_TICKET], 1);
+      t = __shfl_sync(0xffffffffu, t, 0);
+      if (t >= vtotal) break;
+      const VecTask v = decode_vector_ticket(fa.sp, t, M);
+      if (v.dep) {
+        int ok = 1;
+        if (lane == 0) ok = counter_wait(fa.ctr + (v.dep == 2 ? CTR_DONE : CTR_AG_DONE), v.dep_thr, wc, t) ? 1 : 0;
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+      }
+      if (v.op == VEC_GATHER) {
+        vec_gather(fa, v.idx, lane);
+        __syncwarp();
+        if (lane == 0) counter_signal(fa.ctr + ctr_gather(v.idx / GATHER_SUB), 1);
+      } else if (v.op == VEC_COMBINE) {
+        vec_combine(fa, v.idx, lane);
+      } else if (BWD && v.op == VEC_DW) {
+        vec_dw(fa, v.idx, lane);
+      } else if (BWD && v.op == VEC_ZERO) {
+        vec_zero(fa, v.idx, lane);
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  if (*reinterpret_cast<volatile int*>(&fa.status->abort)) __nanosleep(200000);
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ---------------------------------------------------------------- host side
+cudaError_t launch_build_schedule(const SchedParams& sp, const LayoutView& lv, int* step_start, int* ctr,
+                                  int ctr_count, cudaStream_t s, int* launches) {
+  build_schedule_kernel<<<1, 1024, 0, s>>>(sp, lv, step_start, ctr, ctr_count);
+  ++*launches;
+  return cudaGetLastError();
+}
+
+template <bool BWD>
+static cudaError_t launch_fused_t(const FusedArgs& fa, int num_sms, cudaStream_t s) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(fused_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)FUSED_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  void* params[] = {const_cast<FusedArgs*>(&fa)};
+  // cooperative: the launch fails rather than run with CTAs that are not all resident
+  return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(fused_kernel<BWD>), dim3(num_sms), dim3(FUSED_THREADS),
+                                     params, FUSED_SMEM_BYTES, s);
+}
+
+cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, cudaStream_t s, int* launches) {
+  ++*launches;
+  return bwd ? launch_fused_t<true>(fa, num_sms, s) : launch_fused_t<false>(fa, num_sms, s);
+}
+
+}  // namespace moe

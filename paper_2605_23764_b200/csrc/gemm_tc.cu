@@ -1,284 +1,17 @@
-// Grouped GEMMs of the MoE-FFN layer on the sm_100a tensor cores.
+// Grouped GEMMs of the MoE-FFN layer, one launch per operator (the operator-by-operator mode).
 //
 // One persistent, warp-specialised kernel body serves the five GEMM-shaped operators of the layer
 // (forward GMM1+SwiGLU, GMM2; backward act_grad+SwiGLU_grad, gate_grad, and the two weight
 // gradients).  Per CTA: warp 0 = TMA producer (one elected lane), warp 1 = tcgen05.mma issuer (one
-// elected lane; the warp also owns the TMEM allocation), warps 2..5 = epilogue (TMEM -> registers
-// -> fused element-wise math -> swizzled shared staging -> TMA store).  Operands travel global ->
-// shared through TMA into a 4-stage ring of 128-byte-swizzled tiles; accumulators live in TMEM,
-// double-buffered (2 x 256 columns) so the epilogue of tile i overlaps the main loop of tile i+1.
-//
-// Tiles never straddle experts: rows live in a padded row space where every expert segment starts
-// on a multiple of 128 (the paper's rule that vector tiles align with GMM row partitions and that
-// the reduction dimension stays intact, Section 4.2).
-#include "moe_internal.h"
+// elected lane; the warp also owns the TMEM allocation), warps 2..5 = epilogue.  Operands travel
+// global -> shared through TMA into a 4-stage ring of 128-byte-swizzled tiles; accumulators live in
+// TMEM, double-buffered (2 x 256 columns) so the epilogue of tile i overlaps the main loop of tile
+// i+1.  Tiles are assigned round-robin over the CTAs.
+#include "gemm_tile.cuh"
 
 namespace moe {
 
-constexpr int BN = 256;                       // accumulator columns per tile
-constexpr int BK = 64;                        // reduction elements per stage (one 128-byte swizzle row)
-constexpr int STAGES = 4;
-constexpr int A_STAGE_BYTES = BLOCK_M * BK * 2;  // 16 KB
-constexpr int B_STAGE_BYTES = BN * BK * 2;       // 32 KB
-constexpr int MN_BOX_BYTES = 64 * BK * 2;        // one [64 k][64 mn] box of an MN-major operand
-constexpr int GEMM_THREADS = 192;
-constexpr int TMEM_COLS = 512;
-constexpr int OUT_BOX_BYTES = 32 * 64 * 2;       // epilogue staging box: 32 rows x 64 bf16 columns
-constexpr int OUT_STAGE_BYTES = 2 * OUT_BOX_BYTES;  // per epilogue warp: two boxes
-
-struct __align__(8) GemmBarriers {
-  uint64_t full[STAGES];
-  uint64_t empty[STAGES];
-  uint64_t tmem_full[2];
-  uint64_t tmem_empty[2];
-  uint64_t drain;
-  uint32_t tmem_base;
-  uint32_t pad;
-};
-
-constexpr size_t GEMM_SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
-                                   4 * OUT_STAGE_BYTES + sizeof(GemmBarriers);
-static_assert(GEMM_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 size_t gemm_smem_bytes() { return GEMM_SMEM_BYTES; }
-
-struct Tile {
-  int e;      // expert
-  int row0;   // row-space modes: first padded row of the M-block; WGRAD: first padded row of the expert
-  int n0;     // first output column of the tile
-  int m0;     // WGRAD: first output row (within the expert's slab)
-  int nkb;    // k-blocks of the main loop (may be 0 for an expert without rows in WGRAD)
-  int nb;     // column-tile index (ACT_GRAD partials)
-};
-
-template <int MODE>
-__device__ __forceinline__ int total_tiles(const GemmArgs& a) {
-  if (MODE == GEMM_WGRAD) return a.Ep * a.n_tiles_m * a.n_tiles_n;
-  return a.meta[0] * a.n_tiles_n;
-}
-
-// Tile order.  Row-space modes: expert-major; inside an expert the column tile is the slow index
-// and the M-block the fast one, so CTAs running at the same time share one slab of weights (read
-// from HBM once, then from L2) while the expert's rows stay L2-resident.
-template <int MODE>
-__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int t) {
-  Tile tl;
-  if (MODE == GEMM_WGRAD) {
-    const int per_e = a.n_tiles_m * a.n_tiles_n;
-    tl.e = t / per_e;
-    const int r = t - tl.e * per_e;
-    const int mb = r / a.n_tiles_n;
-    tl.nb = r - mb * a.n_tiles_n;
-    tl.m0 = mb * BLOCK_M;
-    tl.n0 = tl.nb * BN;
-    tl.row0 = a.mb_start[tl.e] * BLOCK_M;
-    tl.nkb = (a.counts[tl.e] + BK - 1) / BK;
-  } else {
-    const int e = a.mblk_expert[t / a.n_tiles_n];
-    const int ms = a.mb_start[e];
-    const int mcount = a.mb_start[e + 1] - ms;
-    const int local = t - ms * a.n_tiles_n;
-    tl.nb = local / mcount;
-    const int mbl = local - tl.nb * mcount;
-    tl.e = e;
-    tl.row0 = (ms + mbl) * BLOCK_M;
-    tl.n0 = tl.nb * (MODE == GEMM_GATE_UP ? BN / 2 : BN);
-    tl.m0 = 0;
-    tl.nkb = (a.K + BK - 1) / BK;
-  }
-  return tl;
-}
-
-// ---------------------------------------------------------------- producer: TMA loads of one k-block
-template <int MODE>
-__device__ __forceinline__ void load_stage(const GemmArgs& a, const Tile& tl, int kb, uint8_t* sA, uint8_t* sB,
-                                           uint64_t* bar) {
-  const int k0 = kb * BK;
-  if (MODE == GEMM_WGRAD) {
-    // both operands MN-major: boxes of [64 rows of the expert][64 columns]
-    mbar_expect_tx(bar, 2 * MN_BOX_BYTES + 4 * MN_BOX_BYTES);
-#pragma unroll
-    for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * MN_BOX_BYTES, &a.tmA, tl.m0 + j * 64, tl.row0 + k0, bar);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + j * 64, tl.row0 + k0, bar);
-    return;
-  }
-  mbar_expect_tx(bar, A_STAGE_BYTES + B_STAGE_BYTES);
-  tma_load_2d(sA, &a.tmA, k0, tl.row0, bar);  // A: [128 rows][64 k], K-major
-  const int brow = tl.e * a.b_rows_per_expert;
-  if (MODE == GEMM_GATE_UP) {
-    tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);                          // gate rows -> columns 0..127
-    tma_load_2d(sB + B_STAGE_BYTES / 2, &a.tmB, k0, brow + a.F + tl.n0, bar);  // up rows   -> columns 128..255
-  } else if (MODE == GEMM_DOWN) {
-    tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);  // [256 rows of W_down][64 k], K-major
-  } else {
-    // ACT_GRAD / GATE_GRAD: B = forward weight read along its rows (reduction) -> MN-major boxes
-#pragma unroll
-    for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + j * 64, brow + k0, bar);
-  }
-}
-
-// ---------------------------------------------------------------- epilogues
-// Each epilogue warp owns 32 rows of the tile (its TMEM lane quadrant) and a private staging area of
-// two [32 rows][64 columns] bf16 boxes in the 128-byte-swizzled layout the store tensor maps expect.
-// A thread (= one row) writes 16-byte chunks at chunk index (j ^ (row & 7)): conflict-free.
-__device__ __forceinline__ void stage8(uint8_t* box, int lane, int j, const float* v) {
-  uint4 q = make_uint4(pack_bf16x2(v[0], v[1]), pack_bf16x2(v[2], v[3]), pack_bf16x2(v[4], v[5]),
-                       pack_bf16x2(v[6], v[7]));
-  *reinterpret_cast<uint4*>(box + lane * 128 + ((j ^ (lane & 7)) << 4)) = q;
-}
-__device__ __forceinline__ void load8_bf16(const uint16_t* p, float* v) {
-  uint4 r;
-  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
-  v[0] = bf16lo(r.x); v[1] = bf16hi(r.x); v[2] = bf16lo(r.y); v[3] = bf16hi(r.y);
-  v[4] = bf16lo(r.z); v[5] = bf16hi(r.z); v[6] = bf16lo(r.w); v[7] = bf16hi(r.w);
-}
-__device__ __forceinline__ float sigmoidf_fast(float g) { return 1.0f / (1.0f + __expf(-g)); }
-
-// Before refilling the staging area: the previous stores must have finished reading it.
-__device__ __forceinline__ void staging_acquire(int lane) {
-  if (lane == 0) tma_store_wait_read();
-  __syncwarp();
-}
-// After filling: publish the writes to the async proxy; lane 0 then issues the stores.
-__device__ __forceinline__ void staging_release() {
-  fence_proxy_async_smem();
-  __syncwarp();
-}
-
-template <int MODE>
-__device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl, uint32_t tmem_acc, int quad,
-                                              int lane, uint8_t* stg) {
-  const uint32_t trow = tmem_acc + (static_cast<uint32_t>(quad * 32) << 16);
-  uint8_t* box0 = stg;
-  uint8_t* box1 = stg + OUT_BOX_BYTES;
-  if (MODE == GEMM_GATE_UP) {
-    const int prow0 = tl.row0 + quad * 32;             // first padded row of this warp's slab
-    const float w = a.prow_w[prow0 + lane];
-    // round 1: A = w * silu(g) * u, 128 columns
-    staging_acquire(lane);
-    for (int c = 0; c < BN / 2; c += 16) {
-      float g[16], u[16], act[16];
-      tmem_ld16(trow + c, g);
-      tmem_ld16(trow + BN / 2 + c, u);
-      tmem_ld_wait();
-#pragma unroll
-      for (int i = 0; i < 16; ++i) act[i] = w * (g[i] * sigmoidf_fast(g[i]) * u[i]);
-      uint8_t* box = (c < 64) ? box0 : box1;
-      stage8(box, lane, (c & 63) >> 3, act);
-      stage8(box, lane, ((c & 63) >> 3) + 1, act + 8);
-    }
-    staging_release();
-    if (lane == 0) {
-      tma_store_2d(&a.tmOut0, tl.n0, prow0, box0);
-      if (tl.n0 + 64 < a.F) tma_store_2d(&a.tmOut0, tl.n0 + 64, prow0, box1);
-      tma_store_commit();
-    }
-    if (a.save_h) {
-      // rounds 2, 3: the pre-activations, kept for the backward pass (H viewed as [row][gate|up][F])
-#pragma unroll 1
-      for (int half = 0; half < 2; ++half) {
-        staging_acquire(lane);
-        for (int c = 0; c < BN / 2; c += 16) {
-          float v[16];
-          tmem_ld16(trow + half * (BN / 2) + c, v);
-          tmem_ld_wait();
-          uint8_t* box = (c < 64) ? box0 : box1;
-          stage8(box, lane, (c & 63) >> 3, v);
-          stage8(box, lane, ((c & 63) >> 3) + 1, v + 8);
-        }
-        staging_release();
-        if (lane == 0) {
-          tma_store_3d(&a.tmOut1, tl.n0, half, prow0, box0);
-          if (tl.n0 + 64 < a.F) tma_store_3d(&a.tmOut1, tl.n0 + 64, half, prow0, box1);
-          tma_store_commit();
-        }
-      }
-    }
-  } else if (MODE == GEMM_ACT_GRAD) {
-    const int prow0 = tl.row0 + quad * 32;
-    const size_t p = (size_t)prow0 + lane;
-    const float w = a.prow_w[p];
-    const uint16_t* hrow = a.in0 + p * a.ld_in0;
-    float part = 0.f;
-    // 64 columns of F per round: box0 <- d(gate), box1 <- d(up)
-#pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += 64) {
-      if (tl.n0 + c0 >= a.F) break;  // uniform: whole round outside the tensor
-      staging_acquire(lane);
-#pragma unroll
-      for (int c = 0; c < 64; c += 16) {
-        float da[16];
-        tmem_ld16(trow + c0 + c, da);
-        tmem_ld_wait();
-#pragma unroll
-        for (int h = 0; h < 16; h += 8) {
-          const int col = tl.n0 + c0 + c + h;
-          float g[8], u[8], dg[8], du[8];
-          if (col < a.F) {
-            load8_bf16(hrow + col, g);
-            load8_bf16(hrow + a.F + col, u);
-          } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) g[i] = u[i] = 0.f;
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const float s = sigmoidf_fast(g[i]);
-            const float gs = g[i] * s;
-            part += da[h + i] * (gs * u[i]);        // <dA_unweighted, a>: gradient of the routing weight
-            const float dav = w * da[h + i];        // backward Dispatch's weight, applied here
-            dg[i] = dav * u[i] * (s * (1.0f + g[i] * (1.0f - s)));
-            du[i] = dav * gs;
-          }
-          stage8(box0, lane, (c + h) >> 3, dg);
-          stage8(box1, lane, (c + h) >> 3, du);
-        }
-      }
-      staging_release();
-      if (lane == 0) {
-        tma_store_3d(&a.tmOut0, tl.n0 + c0, 0, prow0, box0);
-        tma_store_3d(&a.tmOut0, tl.n0 + c0, 1, prow0, box1);
-        tma_store_commit();
-      }
-    }
-    if (a.dw_partial) a.dw_partial[p * a.n_tiles_n + tl.nb] = part;
-  } else {
-    // plain bf16 store of the accumulator: DOWN (Y), GATE_GRAD (dXp), WGRAD (dW)
-    const int y0 = (MODE == GEMM_WGRAD ? tl.m0 : tl.row0) + quad * 32;
-#pragma unroll 1
-    for (int c0 = 0; c0 < BN; c0 += 128) {
-      if (tl.n0 + c0 >= a.N) break;
-      if (MODE == GEMM_WGRAD && y0 >= a.M) break;
-      staging_acquire(lane);
-#pragma unroll
-      for (int c = 0; c < 128; c += 32) {
-        float v[32];
-        if (MODE == GEMM_WGRAD && tl.nkb == 0) {
-#pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0.f;
-        } else {
-          tmem_ld16(trow + c0 + c, v);
-          tmem_ld16(trow + c0 + c + 16, v + 16);
-          tmem_ld_wait();
-        }
-        uint8_t* box = (c < 64) ? box0 : box1;
-#pragma unroll
-        for (int h = 0; h < 32; h += 8) stage8(box, lane, ((c & 63) + h) >> 3, v + h);
-      }
-      staging_release();
-      if (lane == 0) {
-        if (MODE == GEMM_WGRAD) {
-          tma_store_3d(&a.tmOut0, tl.n0 + c0, y0, tl.e, box0);
-          if (tl.n0 + c0 + 64 < a.N) tma_store_3d(&a.tmOut0, tl.n0 + c0 + 64, y0, tl.e, box1);
-        } else {
-          tma_store_2d(&a.tmOut0, tl.n0 + c0, y0, box0);
-          if (tl.n0 + c0 + 64 < a.N) tma_store_2d(&a.tmOut0, tl.n0 + c0 + 64, y0, box1);
-        }
-        tma_store_commit();
-      }
-    }
-  }
-}
 
 // ---------------------------------------------------------------- the kernel
 template <int MODE>
@@ -318,8 +51,6 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
   const int total = total_tiles<MODE>(a);
-  constexpr bool A_MN = (MODE == GEMM_WGRAD);
-  constexpr bool B_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD || MODE == GEMM_WGRAD);
 
   if (warp == 0) {
     // ------------------------------------------------ TMA producer
@@ -339,7 +70,6 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_bf16(BLOCK_M, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
       uint32_t it = 0, acc_it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
@@ -355,17 +85,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait(&bars->full[s], ph, wc, SITE_FULL, t)) { ok = false; break; }
           tc_fence_after_sync();
-          const uint32_t a_addr = smem_u32(sA + s * A_STAGE_BYTES);
-          const uint32_t b_addr = smem_u32(sB + s * B_STAGE_BYTES);
-#pragma unroll
-          for (int k16 = 0; k16 < BK / 16; ++k16) {
-            // K-major: 16 k-elements = 32 bytes inside the swizzled row; MN-major: 16 k-rows of 128 bytes
-            const uint64_t da = A_MN ? make_smem_desc(a_addr + k16 * 2048, MN_BOX_BYTES, 1024)
-                                     : make_smem_desc(a_addr + k16 * 32, 16, 1024);
-            const uint64_t db = B_MN ? make_smem_desc(b_addr + k16 * 2048, MN_BOX_BYTES, 1024)
-                                     : make_smem_desc(b_addr + k16 * 32, 16, 1024);
-            tc_mma_bf16(d_tmem, da, db, idesc, (kb | k16) != 0);
-          }
+          mma_kblock<MODE>(d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * B_STAGE_BYTES), kb == 0);
           tc_commit(&bars->empty[s]);  // frees the smem stage once these MMAs have read it
         }
         if (!ok) break;

@@ -7,6 +7,7 @@
 #include <stdint.h>
 
 #include "common.cuh"
+#include "schedule.h"
 
 namespace moe {
 
@@ -97,5 +98,40 @@ struct GemmArgs {
 
 cudaError_t launch_gemm(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
 size_t gemm_smem_bytes();
+
+// ---- fused.cu (the single persistent dependency-driven launch)
+// Everything one fused launch needs: the operators' GEMM arguments (one per schedule segment), the
+// schedule, the counters, and the tensors of the vector tasks.
+struct FusedArgs {
+  GemmArgs op[SCHED_MAX_SEG];
+  SchedParams sp;
+  LayoutView lv;
+  const int* step_start;
+  int* ctr;
+  int d, kp;
+  // gather (Dispatch / backward Dispatch)
+  const uint16_t* gather_src;
+  uint16_t* gather_dst;
+  const float* topk_w;
+  float* prow_w;            // written by the forward gather only (may be NULL)
+  // combine (Combine / backward Combine)
+  const uint16_t* combine_rows;
+  uint16_t* combine_out;
+  // backward extras
+  const float* dw_partial;
+  int dw_nparts;
+  float* d_topk_w;          // may be NULL
+  uint16_t* dW1;
+  uint16_t* dW2;
+  size_t dW1_slab_vec, dW2_slab_vec;  // 16-byte vectors per expert slab
+  DevStatus* status;
+  uint64_t budget_ns;
+};
+
+
+// step_start[i] = matrix-queue tickets before step i; also zeroes the counter block.
+cudaError_t launch_build_schedule(const SchedParams& sp, const LayoutView& lv, int* step_start, int* ctr,
+                                  int ctr_count, cudaStream_t s, int* launches);
+cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, cudaStream_t s, int* launches);
 
 }  // namespace moe

@@ -1,0 +1,179 @@
+// The static tile schedule of the single persistent launch: two ticket-ordered queues (matrix
+// tiles and vector tasks, the counterparts of the paper's CTQ and VTQ, Section 4.3), the dependent
+// and trigger counters of every tile with their static thresholds, and the decode from a ticket to
+// a tile.  Plain host/device code without CUDA calls, so the same functions drive the kernels and
+// the CPU-side simulation that checks the schedule for deadlock freedom.
+//
+// Matrix queue.  "Steps" run over the M-blocks of the padded row space in order (= expert order).
+// Forward step i holds the gate+up tiles of M-block i and the down tiles of M-block i-lag; the lag
+// keeps a consumer's producers several hundred tickets ahead, so its dependency is normally already
+// met when its ticket comes up, while the intermediate it reads is still L2-resident (the paper's
+// producer/consumer placement, Section 4.4).  Backward step i holds act_grad tiles of M-block i,
+// the w2_grad tiles of the expert that ends at M-block i (they share the gathered upstream
+// gradient: the paper's cache-guided GMM interleaving, Section 4.5), gate_grad tiles of M-block
+// i-lag and the w1_grad tiles of the expert ending there (they share dH).
+//
+// Every tile's producers have smaller tickets in their queue; queues are consumed in ticket
+// order by workers that are all resident, hence no deadlock (Section 4.3, correctness argument).
+#pragma once
+
+#include <stdint.h>
+
+#ifdef __CUDACC__
+#define MOE_HD __host__ __device__ __forceinline__
+#else
+#define MOE_HD inline
+#endif
+
+namespace moe {
+
+constexpr int SCHED_MAX_SEG = 4;
+constexpr int GATHER_SUB = 4;          // vector sub-tasks per M-block gather (32 rows each)
+constexpr int EPI_WARPS = 4;           // epilogue warps per matrix tile; each signals once
+constexpr int COMBINE_TOKENS = 16;     // tokens per combine task
+constexpr int ZERO_CHUNKS = 64;        // zero-fill tasks per expert slab pair (only empty experts do work)
+constexpr int DW_SLOTS = 1024;         // routing-weight-gradient entries per task
+
+// op codes of matrix tiles (values = GemmMode) and vector tasks
+enum VecOp : int { VEC_GATHER = 0, VEC_ZERO = 1, VEC_DW = 2, VEC_COMBINE = 3, VEC_NONE = -1 };
+
+struct SchedParams {
+  int is_bwd;
+  int lag;                 // in M-blocks
+  int Ep;
+  int T, k;
+  // tiles per M-block (row-space operators) / per expert (weight gradients), per segment:
+  //   forward : seg0 = gate+up (per M-block), seg1 = down (per M-block, lagged)
+  //   backward: seg0 = act_grad (per M-block), seg1 = w2_grad (per expert, at its last M-block),
+  //             seg2 = gate_grad (per M-block, lagged), seg3 = w1_grad (per expert, lagged)
+  int seg_tiles[SCHED_MAX_SEG];
+  int wgrad_tn[2];         // column tiles of w2_grad / w1_grad (to split a per-expert index)
+};
+
+// tiles of step i given the layout (M = number of M-blocks)
+MOE_HD int step_tiles(const SchedParams& sp, int i, int M, const int* mblk_expert, const int* mb_start) {
+  int n = 0;
+  const int j = i - sp.lag;
+  if (i < M) {
+    n += sp.seg_tiles[0];
+    if (sp.is_bwd && i + 1 == mb_start[mblk_expert[i] + 1]) n += sp.seg_tiles[1];
+  }
+  if (j >= 0 && j < M) {
+    if (!sp.is_bwd) {
+      n += sp.seg_tiles[1];
+    } else {
+      n += sp.seg_tiles[2];
+      if (j + 1 == mb_start[mblk_expert[j] + 1]) n += sp.seg_tiles[3];
+    }
+  }
+  return n;
+}
+
+struct MatTile {
+  int op;        // GemmMode, or -1 = end of queue
+  int slot;      // which GemmArgs of the launch (segment index)
+  int e;
+  int mb;        // M-block (row-space operators) or -1
+  int idx;       // tile index inside the segment
+  // dependency: every counter dep_ctr[dep_first .. dep_first+dep_count) must reach dep_thr
+  int dep_base;  // 0 = gather counters, 1 = activation counters
+  int dep_first, dep_count, dep_thr;
+  // trigger: counter incremented once per epilogue warp after the tile's stores are complete
+  int trig_base; // 1 = activation counter of mb, 2 = global done counter, -1 = none
+  int trig_also_ag;  // backward act_grad also bumps the global act_grad counter
+};
+
+// Decode ticket t (0 <= t < step_start[M+lag]) into a tile.
+MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, int M, const int* step_start,
+                                    const int* mblk_expert, const int* mb_start) {
+  int lo = 0, hi = M + sp.lag - 1;  // last step whose start <= t
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (step_start[mid] <= t) lo = mid; else hi = mid - 1;
+  }
+  const int i = lo, j = i - sp.lag;
+  int r = t - step_start[i];
+  MatTile m;
+  m.trig_also_ag = 0;
+  if (i < M) {
+    if (r < sp.seg_tiles[0]) {
+      m.slot = 0; m.op = sp.is_bwd ? 2 /*ACT_GRAD*/ : 0 /*GATE_UP*/;
+      m.mb = i; m.e = mblk_expert[i]; m.idx = r;
+      m.dep_base = 0; m.dep_first = i; m.dep_count = 1; m.dep_thr = GATHER_SUB;
+      m.trig_base = 1; m.trig_also_ag = sp.is_bwd;
+      return m;
+    }
+    r -= sp.seg_tiles[0];
+    if (sp.is_bwd && i + 1 == mb_start[mblk_expert[i] + 1]) {
+      if (r < sp.seg_tiles[1]) {
+        const int e = mblk_expert[i];
+        m.slot = 1; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = e; m.idx = r;
+        m.dep_base = 0; m.dep_first = mb_start[e]; m.dep_count = mb_start[e + 1] - mb_start[e];
+        m.dep_thr = GATHER_SUB; m.trig_base = -1;
+        return m;
+      }
+      r -= sp.seg_tiles[1];
+    }
+  }
+  // lagged segments of M-block j
+  if (!sp.is_bwd) {
+    m.slot = 1; m.op = 1 /*DOWN*/; m.mb = j; m.e = mblk_expert[j]; m.idx = r;
+    m.dep_base = 1; m.dep_first = j; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
+    m.trig_base = 2;
+    return m;
+  }
+  if (r < sp.seg_tiles[2]) {
+    m.slot = 2; m.op = 3 /*GATE_GRAD*/; m.mb = j; m.e = mblk_expert[j]; m.idx = r;
+    m.dep_base = 1; m.dep_first = j; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
+    m.trig_base = 2;
+    return m;
+  }
+  r -= sp.seg_tiles[2];
+  const int e = mblk_expert[j];
+  m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = e; m.idx = r;
+  m.dep_base = 1; m.dep_first = mb_start[e]; m.dep_count = mb_start[e + 1] - mb_start[e];
+  m.dep_thr = EPI_WARPS * sp.seg_tiles[0]; m.trig_base = -1;
+  return m;
+}
+
+// ---------------------------------------------------------------- vector queue
+struct VecTask {
+  int op;       // VecOp
+  int idx;      // task index inside its kind
+  int dep;      // 0 = none, 2 = global done counter, 3 = global act_grad counter
+  int dep_thr;
+};
+
+MOE_HD int vec_total(const SchedParams& sp, int M) {
+  int n = GATHER_SUB * M + (sp.T + COMBINE_TOKENS - 1) / COMBINE_TOKENS;
+  if (sp.is_bwd) n += sp.Ep * ZERO_CHUNKS + (sp.T * sp.k + DW_SLOTS - 1) / DW_SLOTS;
+  return n;
+}
+
+MOE_HD VecTask decode_vector_ticket(const SchedParams& sp, int t, int M) {
+  VecTask v;
+  v.dep = 0; v.dep_thr = 0;
+  if (t < GATHER_SUB * M) { v.op = VEC_GATHER; v.idx = t; return v; }
+  t -= GATHER_SUB * M;
+  if (sp.is_bwd) {
+    if (t < sp.Ep * ZERO_CHUNKS) { v.op = VEC_ZERO; v.idx = t; return v; }
+    t -= sp.Ep * ZERO_CHUNKS;
+    const int ndw = (sp.T * sp.k + DW_SLOTS - 1) / DW_SLOTS;
+    if (t < ndw) {
+      v.op = VEC_DW; v.idx = t; v.dep = 3; v.dep_thr = EPI_WARPS * M * sp.seg_tiles[0];
+      return v;
+    }
+    t -= ndw;
+  }
+  v.op = VEC_COMBINE; v.idx = t; v.dep = 2;
+  v.dep_thr = EPI_WARPS * M * (sp.is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1]);
+  return v;
+}
+
+// Layout of the counter block in device memory (ints).
+constexpr int CTR_MAT_TICKET = 0, CTR_VEC_TICKET = 1, CTR_DONE = 2, CTR_AG_DONE = 3, CTR_PER_MB = 8;
+MOE_HD int ctr_gather(int mb) { return CTR_PER_MB + 2 * mb; }
+MOE_HD int ctr_act(int mb) { return CTR_PER_MB + 2 * mb + 1; }
+MOE_HD int ctr_ints(int cap_mblocks) { return CTR_PER_MB + 2 * cap_mblocks; }
+
+}  // namespace moe

@@ -12,7 +12,7 @@ from workloads import configs
 pytestmark = pytest.mark.gpu
 
 
-def _bwd_case(T, d, E, k, S, F, seed, renorm=True, serial=True):
+def _bwd_case(T, d, E, k, S, F, seed, renorm=True, serial=False):
     x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, seed)
     layer = MoeLayer(T, d, E, k, S, F, renorm=renorm, save_for_bwd=True, serial=serial)
     ids, w = layer.route(logits)
@@ -38,14 +38,16 @@ def _bwd_case(T, d, E, k, S, F, seed, renorm=True, serial=True):
     (515, 128, 3, 1, 2, 320),
     (64, 512, 40, 4, 0, 72),
 ])
-def test_small_shapes(T, d, E, k, S, F):
-    _bwd_case(T, d, E, k, S, F, seed=T + F)
+@pytest.mark.parametrize("serial", [False, True])
+def test_small_shapes(T, d, E, k, S, F, serial):
+    _bwd_case(T, d, E, k, S, F, seed=T + F, serial=serial)
 
 
-def test_config0_full():
+@pytest.mark.parametrize("serial", [False, True])
+def test_config0_full(serial):
     c = configs.CONFIGS[0]
     inp = configs.make_inputs(c, "cuda")
-    layer = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=True, serial=True)
+    layer = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=True, serial=serial)
     ids, w = layer.route(inp["logits"])
     layer.ffn_fwd(inp["x"], ids, w, inp["W_gate_up"], inp["W_down"])
     dx, dW1, dW2, dw = layer.ffn_bwd(inp["dout"], inp["x"], ids, w, inp["W_gate_up"], inp["W_down"])
@@ -72,35 +74,50 @@ def test_backward_needs_a_saved_forward():
     layer.close()
 
 
-def test_repeat_runs_are_bit_identical():
+def test_repeat_runs_and_launch_modes_are_bit_identical():
+    """Five runs of the persistent launch and one of the operator-by-operator launches give the same
+    bits: the tile math is shared and every reduction has a fixed order (a cheap race detector)."""
     T, d, E, k, S, F = 700, 256, 16, 4, 1, 256
     x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, 77)
-    layer = MoeLayer(T, d, E, k, S, F, save_for_bwd=True, serial=True)
-    ids, w = layer.route(logits)
     first = None
-    for _ in range(5):
-        out = layer.ffn_fwd(x, ids, w, W1, W2)
-        res = (out,) + layer.ffn_bwd(dout, x, ids, w, W1, W2)
-        res = [r.clone() for r in res]
-        if first is None:
-            first = res
-        else:
-            for a, b in zip(first, res):
-                assert torch.equal(a, b)
-    layer.close()
+    for serial, reps in ((False, 5), (True, 1)):
+        layer = MoeLayer(T, d, E, k, S, F, save_for_bwd=True, serial=serial)
+        ids, w = layer.route(logits)
+        for _ in range(reps):
+            out = layer.ffn_fwd(x, ids, w, W1, W2)
+            res = (out,) + layer.ffn_bwd(dout, x, ids, w, W1, W2)
+            res = [r.clone() for r in res]
+            assert layer.status() == (0, 0)
+            if first is None:
+                first = res
+            else:
+                for a, b in zip(first, res):
+                    assert torch.equal(a, b)
+        assert layer.launches() == (7 if serial else 2)
+        layer.close()
 
 
 def test_training_config_full_size_sampled():
     cfg = configs.CONFIGS[4]
     inp = configs.make_inputs(cfg, "cuda")
     x, W1, W2, dout = inp["x"], inp["W_gate_up"], inp["W_down"], inp["dout"]
-    layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=True, serial=True)
+    layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=True)
     ids, w = layer.route(inp["logits"])
     out = layer.ffn_fwd(x, ids, w, W1, W2)
     dx, dW1, dW2, dw = layer.ffn_bwd(dout, x, ids, w, W1, W2)
     torch.cuda.synchronize()
     assert layer.status() == (0, 0)
     ids_c, w_c = ids.cpu(), w.cpu()
+    # the operator-by-operator launches give the same bits (checksums: the gradients are 45 GB)
+    sums = [t.view(torch.int16).to(torch.int64).sum().item() for t in (out, dx, dW1, dW2)]
+    other = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=True, serial=True)
+    out2 = other.ffn_fwd(x, ids, w, W1, W2)
+    other.ffn_bwd(dout, x, ids, w, W1, W2, dx=dx, dW_gate_up=dW1, dW_down=dW2, d_topk_w=torch.empty_like(dw))
+    assert other.status() == (0, 0)
+    sums2 = [t.view(torch.int16).to(torch.int64).sum().item() for t in (out2, dx, dW1, dW2)]
+    assert sums == sums2, "fused and serial launches disagree"
+    other.close()
+    del out2
     # sampled tokens: out, dx and d_topk_w need only the token's own k experts
     g = torch.Generator().manual_seed(cfg.seed)
     toks = sorted(set(torch.randint(0, cfg.T, (10,), generator=g).tolist()) | {0, cfg.T - 1})

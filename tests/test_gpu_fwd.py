@@ -12,7 +12,7 @@ from workloads import configs
 pytestmark = pytest.mark.gpu
 
 
-def _fwd_case(T, d, E, k, S, F, seed, renorm=True, serial=True, stages=True):
+def _fwd_case(T, d, E, k, S, F, seed, renorm=True, serial=False, stages=True):
     x, W1, W2, logits, _ = small_problem(T, d, E, k, S, F, seed)
     layer = MoeLayer(T, d, E, k, S, F, renorm=renorm, save_for_bwd=True, serial=serial)
     ids, w = layer.route(logits)
@@ -36,10 +36,11 @@ def _fwd_case(T, d, E, k, S, F, seed, renorm=True, serial=True, stages=True):
     return out
 
 
-def test_config0_stagewise():
+@pytest.mark.parametrize("serial", [False, True])
+def test_config0(serial):
     c = configs.CONFIGS[0]
     inp = configs.make_inputs(c, "cuda")
-    layer = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=True, serial=True)
+    layer = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=True, serial=serial)
     ids, w = layer.route(inp["logits"])
     out = layer.ffn_fwd(inp["x"], ids, w, inp["W_gate_up"], inp["W_down"])
     ref = oracle.fwd(inp["x"], ids.cpu(), w.cpu(), inp["W_gate_up"], inp["W_down"])
@@ -55,14 +56,15 @@ def test_config0_stagewise():
     (515, 128, 3, 1, 2, 320),     # experts spanning several M-blocks, shared experts
     (64, 512, 40, 4, 0, 72),      # more experts than rows per expert: many empty / tiny segments
 ])
-def test_small_shapes_stagewise(T, d, E, k, S, F):
-    _fwd_case(T, d, E, k, S, F, seed=T + F)
+@pytest.mark.parametrize("serial", [False, True])
+def test_small_shapes_stagewise(T, d, E, k, S, F, serial):
+    _fwd_case(T, d, E, k, S, F, seed=T + F, serial=serial)
 
 
 def test_single_expert_is_dense_ffn():
     T, d, F = 384, 192, 256
     x, W1, W2, _, _ = small_problem(T, d, 1, 1, 0, F, 5)
-    layer = MoeLayer(T, d, 1, 1, 0, F, serial=True)
+    layer = MoeLayer(T, d, 1, 1, 0, F)
     ids = torch.zeros(T, 1, dtype=torch.int32, device="cuda")
     w = torch.ones(T, 1, dtype=torch.float32, device="cuda")
     out = layer.ffn_fwd(x, ids, w, W1, W2)
@@ -75,7 +77,7 @@ def test_single_expert_is_dense_ffn():
 def test_zero_weights_and_empty_batch():
     T, d, E, k, F = 100, 64, 4, 2, 64
     x, W1, W2, logits, _ = small_problem(T, d, E, k, 0, F, 9)
-    layer = MoeLayer(T, d, E, k, 0, F, serial=True)
+    layer = MoeLayer(T, d, E, k, 0, F)
     ids, w = layer.route(logits)
     out = layer.ffn_fwd(x, ids, torch.zeros_like(w), W1, W2)
     assert torch.count_nonzero(out).item() == 0
@@ -88,15 +90,21 @@ def test_zero_weights_and_empty_batch():
     layer.close()
 
 
-def _sampled_tokens_check(cfg, n_tokens=24):
+def _sampled_tokens_check(cfg, n_tokens=24, serial=False):
     """Full-size forward on the GPU; the oracle evaluates a sample of tokens one by one."""
     inp = configs.make_inputs(cfg, "cuda")
-    layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, serial=True)
+    layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, serial=serial)
     ids, w = layer.route(inp["logits"])
     out = layer.ffn_fwd(inp["x"], ids, w, inp["W_gate_up"], inp["W_down"])
     torch.cuda.synchronize()
     assert layer.status() == (0, 0)
     assert torch.isfinite(out.float()).all()
+    if not serial:  # the one-launch-per-operator mode must give the same bits (same tile math)
+        other = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, serial=True)
+        out_serial = other.ffn_fwd(inp["x"], ids, w, inp["W_gate_up"], inp["W_down"])
+        assert other.status() == (0, 0)
+        assert torch.equal(out, out_serial), "fused and serial launches disagree"
+        other.close()
     ids_c, w_c = ids.cpu(), w.cpu()
     counts = torch.bincount(ids_c.flatten().long(), minlength=cfg.E)
     order = torch.argsort(counts)
