@@ -111,7 +111,7 @@ struct Carve {
 // Byte offsets of every workspace tensor.
 struct WsPlan {
   size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
-      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, total;
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, stats, total;
   int cap_rows, nblk_max, ntn_act, ctr_count;
 };
 
@@ -152,8 +152,9 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.st_dw = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_logits = c.take(sizeof(float) * (size_t)s.T_max * s.E);
   p.ctr_count = ctr_ints((int)(cap / BLOCK_M) + 1);
-  p.step_start = c.take(sizeof(int) * (cap / BLOCK_M + SCHED_LAG_MAX + 4));
+  p.step_start = c.take(sizeof(int) * (size_t)(Ep + SCHED_LAG_MAX + 4));
   p.ctr = c.take(sizeof(int) * (size_t)p.ctr_count);
+  p.stats = c.take(sizeof(long long) * 32 * 256);
   p.total = c.off;
   return p;
 }
@@ -170,7 +171,7 @@ struct moe_ctx {
   int launches = 0;
   int saved_T = -1;  // T of the forward whose tensors are in the workspace (-1: none)
   uint64_t budget_ns = 2000ull * 1000 * 1000;
-  int sched_lag = 8;  // M-blocks between a producer step and its consumer step in the matrix queue
+  int sched_lag = 0;  // experts between a producer step and its consumer step; 0 = choose from the shape
   cudaStream_t last_stream = nullptr;
   // optional per-operator timing
   bool profiling = false;
@@ -362,7 +363,6 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
   SchedParams sp;
   memset(&sp, 0, sizeof sp);
   sp.is_bwd = bwd ? 1 : 0;
-  sp.lag = c->sched_lag;
   sp.Ep = s.E + s.n_shared;
   sp.T = T;
   sp.k = s.k;
@@ -371,12 +371,20 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
     sp.seg_tiles[1] = (s.d + 255) / 256;
   } else {
     sp.seg_tiles[0] = c->plan.ntn_act;
-    sp.wgrad_tn[0] = (s.F + 255) / 256;
-    sp.seg_tiles[1] = ((s.d + 127) / 128) * sp.wgrad_tn[0];
+    sp.seg_tiles[1] = (s.d + 127) / 128;       // w2_grad: strips of 128 rows of dW_down
+    sp.strip_tiles[0] = (s.F + 255) / 256;
     sp.seg_tiles[2] = (s.d + 255) / 256;
-    sp.wgrad_tn[1] = (s.d + 255) / 256;
-    sp.seg_tiles[3] = ((2 * s.F + 127) / 128) * sp.wgrad_tn[1];
+    sp.seg_tiles[3] = (2 * s.F + 127) / 128;   // w1_grad: strips of 128 rows of dW_gate_up
+    sp.strip_tiles[1] = (s.d + 255) / 256;
   }
+  // lag: enough experts that a consumer's producers are about two grid-fulls of tickets ahead
+  const long rows = (long)T * (s.k + s.n_shared);
+  const int avg_m = (int)((rows / sp.Ep + BLOCK_M - 1) / BLOCK_M) > 0 ? (int)((rows / sp.Ep + BLOCK_M - 1) / BLOCK_M) : 1;
+  const int per_step = avg_m * sp.seg_tiles[0] + (bwd ? sp.seg_tiles[1] : 0);
+  int lag = (2 * c->num_sms + per_step - 1) / per_step;
+  if (lag < 1) lag = 1;
+  if (lag > SCHED_LAG_MAX) lag = SCHED_LAG_MAX;
+  sp.lag = c->sched_lag > 0 ? c->sched_lag : lag;
   return sp;
 }
 
@@ -391,6 +399,7 @@ FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
   fa.ctr = c->at<int>(p.ctr);
   fa.d = s.d;
   fa.kp = s.k + s.n_shared;
+  fa.stats = c->at<long long>(p.stats);
   fa.status = c->status();
   fa.budget_ns = c->budget_ns;
   return fa;
@@ -793,6 +802,7 @@ int moe_debug_buffer(moe_ctx* c, int which, void** ptr, size_t* elems) {
     case MOE_BUF_DH: if (!train) return MOE_ERR_STATE; off = p.dH; n = cap * 2 * s.F; break;
     case MOE_BUF_DXP: off = p.Y; n = cap * s.d; break;
     case MOE_BUF_META: off = p.meta; n = 8; break;
+    case 14: off = p.stats; n = 2 * 32 * 256; break;  // diagnostic builds: wait accounting (int64 as int32 pairs)
     default: return MOE_ERR_INVALID_ARG;
   }
   *ptr = c->ws + off;
@@ -807,31 +817,27 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
                                 const int32_t* seg_tiles, int32_t lag, int32_t mat_workers, int32_t vec_workers,
                                 int64_t* stats) {
   if (!counts || !seg_tiles || Ep < 1 || lag < 0 || mat_workers < 1 || vec_workers < 1) return MOE_ERR_INVALID_ARG;
-  std::vector<int> mb_start(Ep + 1, 0), mblk_expert;
-  for (int e = 0; e < Ep; ++e) {
-    const int m = (counts[e] + BLOCK_M - 1) / BLOCK_M;
-    mb_start[e + 1] = mb_start[e] + m;
-    for (int q = 0; q < m; ++q) mblk_expert.push_back(e);
-  }
+  std::vector<int> mb_start(Ep + 1, 0);
+  for (int e = 0; e < Ep; ++e) mb_start[e + 1] = mb_start[e] + (counts[e] + BLOCK_M - 1) / BLOCK_M;
   const int M = mb_start[Ep];
-  mblk_expert.push_back(0);
   SchedParams sp;
   memset(&sp, 0, sizeof sp);
   sp.is_bwd = is_bwd; sp.lag = lag; sp.Ep = Ep; sp.T = T; sp.k = k;
   for (int i = 0; i < SCHED_MAX_SEG; ++i) sp.seg_tiles[i] = seg_tiles[i];
-  std::vector<int> step_start(M + lag + 1, 0);
-  for (int i = 0; i < M + lag; ++i)
-    step_start[i + 1] = step_start[i] + step_tiles(sp, i, M, mblk_expert.data(), mb_start.data());
-  const int total = step_start[M + lag], vtotal = vec_total(sp, M);
+  sp.strip_tiles[0] = sp.strip_tiles[1] = 1;
+  std::vector<int> step_start(Ep + lag + 1, 0);
+  for (int i = 0; i < Ep + lag; ++i) step_start[i + 1] = step_start[i] + step_tiles(sp, i, mb_start.data());
+  const int total = step_start[Ep + lag], vtotal = vec_total(sp, M);
   std::vector<long> ctr(ctr_ints(M + 1), 0);
   // 1. coverage and ticket order of producers
-  std::vector<int> seg0_last_ticket(M, -1), seg0_count(M, 0), lag_count(M, 0);
+  std::vector<int> seg0_count(M + 1, 0), lag_count(M + 1, 0);
   std::vector<int> w2_count(Ep, 0), w1_count(Ep, 0);
   for (int t = 0; t < total; ++t) {
-    const MatTile m = decode_matrix_ticket(sp, t, M, step_start.data(), mblk_expert.data(), mb_start.data());
+    const MatTile m = decode_matrix_ticket(sp, t, step_start.data(), mb_start.data());
     if (m.e < 0 || m.e >= Ep || m.idx < 0 || m.idx >= sp.seg_tiles[m.slot]) return 10;
-    if (m.slot == 0) { seg0_last_ticket[m.mb] = t; seg0_count[m.mb]++; }
-    else if (m.mb >= 0) { lag_count[m.mb]++; if (seg0_last_ticket[m.mb] < 0 || seg0_count[m.mb] != sp.seg_tiles[0]) return 11; }
+    if (m.mb >= 0 && (m.mb < mb_start[m.e] || m.mb >= mb_start[m.e + 1])) return 10;
+    if (m.slot == 0) seg0_count[m.mb]++;
+    else if (m.mb >= 0) { lag_count[m.mb]++; if (seg0_count[m.mb] != sp.seg_tiles[0]) return 11; }
     else if (m.slot == 1) w2_count[m.e]++;
     else {
       w1_count[m.e]++;
@@ -855,7 +861,7 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
     bool progress = false;
     for (auto& wk : mw) {
       if (!wk.holding && next_mat < total) {
-        wk.m = decode_matrix_ticket(sp, next_mat++, M, step_start.data(), mblk_expert.data(), mb_start.data());
+        wk.m = decode_matrix_ticket(sp, next_mat++, step_start.data(), mb_start.data());
         wk.holding = true;
         progress = true;
       }

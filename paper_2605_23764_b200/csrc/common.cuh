@@ -98,8 +98,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
 
 // Bounded acquire-poll of a dependency counter in global memory until it reaches `threshold`
 // (the paper's "dependent event", Section 4.3).
-__device__ __forceinline__ bool counter_wait(const int* ctr, int threshold, const WaitCtl& wc, int tile) {
+__device__ __forceinline__ bool counter_wait(const int* ctr, int threshold, const WaitCtl& wc, int tile,
+                                             uint32_t max_sleep_ns = 512) {
   uint64_t t0 = 0;
+  uint32_t sleep_ns = 32;
   for (uint32_t spin = 0;; ++spin) {
     int v;
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(ctr) : "memory");
@@ -113,7 +115,8 @@ __device__ __forceinline__ bool counter_wait(const int* ctr, int threshold, cons
         return false;
       }
     }
-    __nanosleep(64);
+    __nanosleep(sleep_ns);  // back off: pollers must not crowd the L2 slice that holds the counter
+    if (sleep_ns < max_sleep_ns) sleep_ns <<= 1;
   }
 }
 

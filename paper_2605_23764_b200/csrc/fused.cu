@@ -7,8 +7,9 @@
 //   warp 1      tcgen05.mma issuer (and TMEM owner);
 //   warps 2-5   epilogue: TMEM -> fused element-wise math -> TMA store, then the tile's trigger
 //               counter once the stores are complete;
-//   warps 6-9   vector workers: take tickets of the vector queue (permute-gather, zero-fill of
-//               weight gradients of experts without rows, routing-weight gradient, combine).
+//   warps 6-13  vector workers: take tickets of the vector queue (permute-gather, zero-fill of
+//               weight gradients of experts without rows, routing-weight gradient, combine); the
+//               matrix-role warps join them when the matrix queue is exhausted.
 // This is the paper's unified runtime (Section 4.4) restated for one SM: matrix and vector work
 // progress concurrently inside one launch, ordered only by event counters with static thresholds
 // (Section 4.3).  The tile math is the same code the one-launch-per-operator mode runs.
@@ -21,7 +22,22 @@
 
 namespace moe {
 
-constexpr int FUSED_THREADS = GEMM_THREADS + 128;  // + 4 vector warps
+// Optional per-CTA wait accounting (diagnostic builds only: -DMOE_STATS).
+#ifdef MOE_STATS
+#define ST_DECL long long st_t0 = clock64(), st_acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long st_mark = st_t0
+#define ST_MARK() st_mark = clock64()
+#define ST_ADD(i) do { long long _n = clock64(); st_acc[i] += _n - st_mark; st_mark = _n; } while (0)
+#define ST_FLUSH(base, n) do { if (fa.stats) { for (int _i = 0; _i < (n); ++_i) fa.stats[blockIdx.x * 32 + (base) + _i] = st_acc[_i]; \
+                               fa.stats[blockIdx.x * 32 + (base) + (n)] = clock64() - st_t0; } } while (0)
+#else
+#define ST_DECL
+#define ST_MARK()
+#define ST_ADD(i)
+#define ST_FLUSH(base, n)
+#endif
+
+constexpr int VEC_WARPS = 8;
+constexpr int FUSED_THREADS = GEMM_THREADS + 32 * VEC_WARPS;
 constexpr int RING = 4;                            // published-tile ring depth
 
 struct TileSlot {
@@ -35,6 +51,9 @@ struct __align__(16) FusedShared {
   GemmBarriers bars;
   uint64_t tk_full[RING];
   uint64_t tk_empty[RING];
+  uint64_t vec_ready[2];  // one-shot: the global "all tiles done" conditions the vector tail waits for
+  int vec_poller[2];      // which warp polls the global counter on behalf of the CTA
+  int pad[2];
   TileSlot ring[RING];
 };
 
@@ -43,20 +62,19 @@ constexpr size_t FUSED_SMEM_BYTES = 1024 + (size_t)STAGES * (A_STAGE_BYTES + B_S
 static_assert(FUSED_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 // ---------------------------------------------------------------- schedule prefix + counter reset
-// One block: step_start[i] = tickets before step i (i in [0, M+lag]); counters zeroed.
+// One block: step_start[i] = tickets before step i (i in [0, Ep+lag]); counters zeroed.
 __global__ void __launch_bounds__(1024) build_schedule_kernel(SchedParams sp, LayoutView lv, int* step_start,
                                                               int* ctr, int ctr_count) {
   __shared__ int warp_sums[32];
   __shared__ int carry_s;
-  const int M = lv.meta[0];
-  const int n = M + sp.lag;
+  const int n = sp.Ep + sp.lag;
   for (int i = threadIdx.x; i < ctr_count; i += blockDim.x) ctr[i] = 0;
   if (threadIdx.x == 0) carry_s = 0;
   __syncthreads();
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int base = 0; base < n; base += blockDim.x) {
     const int i = base + threadIdx.x;
-    const int v = i < n ? step_tiles(sp, i, M, lv.mblk_expert, lv.mb_start) : 0;
+    const int v = i < n ? step_tiles(sp, i, lv.mb_start) : 0;
     int incl = v;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -111,10 +129,12 @@ __device__ __forceinline__ void vec_gather(const FusedArgs& fa, int task, int la
       const int t = slot / fa.kp, j = slot - t * fa.kp;
       const uint4* in = reinterpret_cast<const uint4*>(fa.gather_src + (size_t)t * fa.d);
       int v = lane;
-      for (; v + 96 < nvec; v += 128) {
-        uint4 a = ldg_nc_v4(in + v), b = ldg_nc_v4(in + v + 32), c = ldg_nc_v4(in + v + 64),
-              dd = ldg_nc_v4(in + v + 96);
-        out[v] = a; out[v + 32] = b; out[v + 64] = c; out[v + 96] = dd;
+      for (; v + 224 < nvec; v += 256) {
+        uint4 q[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) q[u] = ldg_nc_v4(in + v + 32 * u);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) out[v + 32 * u] = q[u];
       }
       for (; v < nvec; v += 32) out[v] = ldg_nc_v4(in + v);
       if (fa.prow_w && lane == 0) fa.prow_w[p] = j < k ? fa.topk_w[(size_t)t * k + j] : 1.0f;
@@ -133,15 +153,24 @@ __device__ __forceinline__ void vec_combine(const FusedArgs& fa, int task, int l
       float acc[8];
 #pragma unroll
       for (int q = 0; q < 8; ++q) acc[q] = 0.f;
-      for (int j = 0; j < kp; ++j) {
-        const int p = fa.lv.prow_of[(size_t)t * kp + j];
-        if (p < 0) continue;
-        // plain (coherent) load: these rows were written earlier in this same launch
-        const uint4 r = *(reinterpret_cast<const uint4*>(fa.combine_rows + (size_t)p * fa.d) + v);
-        acc[0] += bf16lo(r.x); acc[1] += bf16hi(r.x);
-        acc[2] += bf16lo(r.y); acc[3] += bf16hi(r.y);
-        acc[4] += bf16lo(r.z); acc[5] += bf16hi(r.z);
-        acc[6] += bf16lo(r.w); acc[7] += bf16hi(r.w);
+      for (int j0 = 0; j0 < kp; j0 += 8) {
+        uint4 r[8];
+        // eight independent row loads in flight; plain (coherent) loads: the rows were written
+        // earlier in this same launch
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int j = j0 + u;
+          const int p = j < kp ? fa.lv.prow_of[(size_t)t * kp + j] : -1;
+          r[u] = p >= 0 ? *(reinterpret_cast<const uint4*>(fa.combine_rows + (size_t)p * fa.d) + v)
+                        : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          acc[0] += bf16lo(r[u].x); acc[1] += bf16hi(r[u].x);
+          acc[2] += bf16lo(r[u].y); acc[3] += bf16hi(r[u].y);
+          acc[4] += bf16lo(r[u].z); acc[5] += bf16hi(r[u].z);
+          acc[6] += bf16lo(r[u].w); acc[7] += bf16hi(r[u].w);
+        }
       }
       uint4 o;
       o.x = pack_bf16x2(acc[0], acc[1]);
@@ -250,6 +279,10 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
       mbar_init(&sh->tk_full[s], 1);
       mbar_init(&sh->tk_empty[s], 1 + EPI_WARPS);  // the MMA issuer and every epilogue warp release a slot
     }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh->vec_ready[s], 1);
+      sh->vec_poller[s] = 0;
+    }
     mbar_fence_init();
     fence_proxy_async();
   }
@@ -265,25 +298,46 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
   if (warp == 0) {
     // ------------------------------------------------ matrix-queue producer
     if (lane == 0) {
-      const int total = fa.step_start[M + fa.sp.lag];
+      const int total = fa.step_start[fa.sp.Ep + fa.sp.lag];
       uint32_t it = 0, n = 0;
       bool ok = true;
+      ST_DECL;
+      int next_t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
       while (ok) {
-        const int t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
+        ST_MARK();
+        const int t = next_t;
         TileSlot ts;
-        MatTile mt;
+        ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
+        ts.trig_idx = -1; ts.trig_ag = 0;
         if (t >= total) {
-          ts.op = -1; ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
-          ts.trig_idx = -1; ts.trig_ag = 0;
-        } else {
-          mt = decode_matrix_ticket(fa.sp, t, M, fa.step_start, fa.lv.mblk_expert, fa.lv.mb_start);
-          const GemmArgs& g = fa.op[mt.slot];
-          ts.op = mt.op; ts.slot = mt.slot; ts.e = mt.e;
+          // end of the queue: tell the other roles
+          ts.op = -1;
+          const int rs = n % RING;
+          if (!mbar_wait(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) break;
+          sh->ring[rs] = ts;
+          mbar_arrive(&sh->tk_full[rs]);
+          break;
+        }
+        const MatTile mt = decode_matrix_ticket(fa.sp, t, fa.step_start, fa.lv.mb_start);
+        const GemmArgs& g = fa.op[mt.slot];
+        ST_ADD(0);  // ticket + decode
+        // dependent event(s): poll until every producer counter has reached its threshold
+        for (int q = 0; q < mt.dep_count && ok; ++q) {
+          const int mbq = mt.dep_first + q;
+          const int* c = fa.ctr + (mt.dep_base == 0 ? ctr_gather(mbq) : ctr_act(mbq));
+          ok = counter_wait(c, mt.dep_thr, wc, t);
+        }
+        if (!ok) break;
+        fence_proxy_async();  // the producers' writes must be seen by the TMA loads that follow
+        ST_ADD(1);  // dependency wait
+        ts.op = mt.op; ts.slot = mt.slot; ts.e = mt.e;
+        ts.trig_idx = mt.trig_base == 1 ? ctr_act(mt.mb) : (mt.trig_base == 2 ? CTR_DONE : -1);
+        ts.trig_ag = mt.trig_also_ag;
+        for (int gi = 0; gi < mt.group && ok; ++gi) {
           if (mt.op == GEMM_WGRAD) {
-            const int mbw = mt.idx / g.n_tiles_n;
-            ts.nb = mt.idx - mbw * g.n_tiles_n;
-            ts.m0 = mbw * BLOCK_M;
-            ts.n0 = ts.nb * BN;
+            ts.nb = gi;                       // one 128-row block of the gradient, column tile gi
+            ts.m0 = mt.idx * BLOCK_M;
+            ts.n0 = gi * BN;
             ts.row0 = fa.lv.mb_start[mt.e] * BLOCK_M;
             ts.nkb = (fa.lv.counts[mt.e] + BK - 1) / BK;
           } else {
@@ -293,39 +347,40 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
             ts.row0 = mt.mb * BLOCK_M;
             ts.nkb = (g.K + BK - 1) / BK;
           }
-          ts.trig_idx = mt.trig_base == 1 ? ctr_act(mt.mb) : (mt.trig_base == 2 ? CTR_DONE : -1);
-          ts.trig_ag = mt.trig_also_ag;
-        }
-        const int rs = n % RING;
-        if (!mbar_wait(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) break;
-        sh->ring[rs] = ts;
-        mbar_arrive(&sh->tk_full[rs]);  // release: the slot's contents are visible to the waiters
-        ++n;
-        if (ts.op < 0) break;
-        // dependent event(s): poll until every producer counter has reached its threshold
-        for (int q = 0; q < mt.dep_count && ok; ++q) {
-          const int mbq = mt.dep_first + q;
-          const int* c = fa.ctr + (mt.dep_base == 0 ? ctr_gather(mbq) : ctr_act(mbq));
-          ok = counter_wait(c, mt.dep_thr, wc, t);
-        }
-        if (!ok) break;
-        fence_proxy_async();  // the producers' writes must be seen by the TMA loads that follow
-        const Tile tl = slot_tile(ts);
-        for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
-          const int s = it % STAGES;
-          if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
-          fused_load_stage<BWD>(fa, ts, tl, kb, sA + s * A_STAGE_BYTES, sB + s * B_STAGE_BYTES, &bars->full[s]);
+          const int rs = n % RING;
+          if (!mbar_wait(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
+          sh->ring[rs] = ts;
+          mbar_arrive(&sh->tk_full[rs]);  // release: the slot's contents are visible to the waiters
+          ++n;
+          ST_ADD(2);  // ring slot wait
+          const Tile tl = slot_tile(ts);
+          const int kb_prefetch = (gi + 1 == mt.group) ? max(0, ts.nkb - 8) : -1;
+          for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
+            // take the next ticket shortly before this ticket's loads end: the atomic's round trip
+            // hides behind the last k-blocks, and tiles with adjacent tickets (which share an
+            // operand through L2) still start close together in time
+            if (kb == kb_prefetch) next_t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
+            const int s = it % STAGES;
+            if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
+            ST_ADD(3);  // stage wait (back-pressure from the tensor core: the healthy state)
+            fused_load_stage<BWD>(fa, ts, tl, kb, sA + s * A_STAGE_BYTES, sB + s * B_STAGE_BYTES, &bars->full[s]);
+            ST_ADD(4);  // issue
+          }
         }
       }
+      ST_FLUSH(0, 5);
     }
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer
     if (lane == 0) {
       uint32_t it = 0, acc_it = 0, n = 0;
       bool ok = true;
+      ST_DECL;
       while (ok) {
         const int rs = n % RING;
+        ST_MARK();
         if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -1)) break;
+        ST_ADD(0);  // waiting for a published tile
         const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb;
         mbar_arrive(&sh->tk_empty[rs]);
         ++n;
@@ -333,19 +388,23 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
         if (nkb == 0) continue;
         const int as = acc_it & 1;
         if (!mbar_wait(&bars->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, n)) break;
+        ST_ADD(1);  // accumulator not yet drained by the epilogue
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + as * BN;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGES;
           if (!mbar_wait(&bars->full[s], (it / STAGES) & 1, wc, SITE_FULL, n)) { ok = false; break; }
+          ST_ADD(2);  // operands not yet in shared memory (starved)
           tc_fence_after_sync();
           fused_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * B_STAGE_BYTES), kb == 0);
           tc_commit(&bars->empty[s]);
+          ST_ADD(3);  // issue
         }
         if (!ok) break;
         tc_commit(&bars->tmem_full[as]);
         ++acc_it;
       }
+      ST_FLUSH(8, 4);
       if (*reinterpret_cast<volatile int*>(&fa.status->abort)) {
         tc_commit(&bars->drain);
         const WaitCtl shortwc{fa.status, 20ull * 1000 * 1000};
@@ -357,9 +416,12 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
     const int quad = warp & 3;
     uint8_t* stg = sOut + quad * OUT_STAGE_BYTES;
     uint32_t acc_it = 0, n = 0;
+    ST_DECL;
     while (true) {
       const int rs = n % RING;
+      ST_MARK();
       if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -2)) break;
+      ST_ADD(0);
       const TileSlot ts = sh->ring[rs];
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->tk_empty[rs]);
@@ -371,12 +433,14 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
       } else {
         const int as = acc_it & 1;
         if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, n)) break;
+        ST_ADD(1);  // waiting for the accumulator
         tc_fence_after_sync();
         fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->tmem_empty[as]);
         ++acc_it;
+        ST_ADD(2);  // epilogue work
       }
       if (ts.trig_idx >= 0) {
         // trigger event: only after this warp's part of the tile is readable by everyone
@@ -387,11 +451,19 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
           counter_signal(fa.ctr + ts.trig_idx, 1);
           if (ts.trig_ag) counter_signal(fa.ctr + CTR_AG_DONE, 1);
         }
+        __syncwarp();
+        ST_ADD(3);  // trigger (store completion + signal)
       }
     }
+    if (quad == 0 && lane == 0) ST_FLUSH(16, 4);
     if (lane == 0) tma_store_wait_all();
-  } else {
-    // ------------------------------------------------ vector workers
+  }
+
+  // ------------------------------------------------ vector workers: the dedicated warps from the
+  // start, every other warp once its matrix role has reached the end of the matrix queue (the
+  // tail of the vector queue -- combine -- then runs on the whole SM)
+  __syncwarp();
+  if (!*reinterpret_cast<volatile int*>(&fa.status->abort)) {
     const int vtotal = vec_total(fa.sp, M);
     while (true) {
       int t = 0;
@@ -400,9 +472,20 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
       if (t >= vtotal) break;
       const VecTask v = decode_vector_ticket(fa.sp, t, M);
       if (v.dep) {
+        // A global completion counter: one warp of the CTA polls it (slowly), the others sleep on a
+        // shared-memory barrier -- a thousand warps spinning on one L2 line would slow every load.
+        const int kind = v.dep == 2 ? 0 : 1;
         int ok = 1;
-        if (lane == 0) ok = counter_wait(fa.ctr + (v.dep == 2 ? CTR_DONE : CTR_AG_DONE), v.dep_thr, wc, t) ? 1 : 0;
+        if (lane == 0) {
+          if (atomicExch(&sh->vec_poller[kind], 1) == 0) {
+            ok = counter_wait(fa.ctr + (kind == 0 ? CTR_DONE : CTR_AG_DONE), v.dep_thr, wc, t, 2000) ? 1 : 0;
+            if (ok) mbar_arrive(&sh->vec_ready[kind]);
+          } else {
+            ok = mbar_wait(&sh->vec_ready[kind], 0, wc, SITE_DEP, t) ? 1 : 0;
+          }
+        }
         ok = __shfl_sync(0xffffffffu, ok, 0);
+        __syncwarp();
         if (!ok) break;
       }
       if (v.op == VEC_GATHER) {

@@ -124,6 +124,7 @@ struct FusedArgs {
   uint16_t* dW1;
   uint16_t* dW2;
   size_t dW1_slab_vec, dW2_slab_vec;  // 16-byte vectors per expert slab
+  long long* stats;         // diagnostic builds: per-CTA wait accounting [grid][32]
   DevStatus* status;
   uint64_t budget_ns;
 };

@@ -4,14 +4,15 @@
 // a tile.  Plain host/device code without CUDA calls, so the same functions drive the kernels and
 // the CPU-side simulation that checks the schedule for deadlock freedom.
 //
-// Matrix queue.  "Steps" run over the M-blocks of the padded row space in order (= expert order).
-// Forward step i holds the gate+up tiles of M-block i and the down tiles of M-block i-lag; the lag
-// keeps a consumer's producers several hundred tickets ahead, so its dependency is normally already
-// met when its ticket comes up, while the intermediate it reads is still L2-resident (the paper's
-// producer/consumer placement, Section 4.4).  Backward step i holds act_grad tiles of M-block i,
-// the w2_grad tiles of the expert that ends at M-block i (they share the gathered upstream
-// gradient: the paper's cache-guided GMM interleaving, Section 4.5), gate_grad tiles of M-block
-// i-lag and the w1_grad tiles of the expert ending there (they share dH).
+// Matrix queue.  "Steps" run over the experts in order.  Forward step i holds the gate+up tiles of
+// expert i (column tile slow, M-block fast: tiles in flight together share one slab of weights)
+// and the down tiles of expert i-lag; the lag keeps a consumer's producers a few hundred tickets
+// ahead, so its dependency is normally met when its ticket comes up while the intermediate it reads
+// is still L2-resident (the paper's producer/consumer placement, Section 4.4).  Backward step i
+// holds the act_grad tiles of expert i and its w2_grad strips (they share the gathered upstream
+// gradient: the paper's cache-guided GMM interleaving, Section 4.5), then the gate_grad tiles of
+// expert i-lag and its w1_grad strips (they share dH).  A weight-gradient ticket is a strip: one
+// 128-row block of the gradient across all its column tiles.
 //
 // Every tile's producers have smaller tickets in their queue; queues are consumed in ticket
 // order by workers that are all resident, hence no deadlock (Section 4.3, correctness argument).
@@ -28,9 +29,9 @@
 namespace moe {
 
 constexpr int SCHED_MAX_SEG = 4;
-constexpr int GATHER_SUB = 4;          // vector sub-tasks per M-block gather (32 rows each)
+constexpr int GATHER_SUB = 8;          // vector sub-tasks per M-block gather (16 rows each)
 constexpr int EPI_WARPS = 4;           // epilogue warps per matrix tile; each signals once
-constexpr int COMBINE_TOKENS = 16;     // tokens per combine task
+constexpr int COMBINE_TOKENS = 2;      // tokens per combine task
 constexpr int ZERO_CHUNKS = 64;        // zero-fill tasks per expert slab pair (only empty experts do work)
 constexpr int DW_SLOTS = 1024;         // routing-weight-gradient entries per task
 
@@ -39,42 +40,47 @@ enum VecOp : int { VEC_GATHER = 0, VEC_ZERO = 1, VEC_DW = 2, VEC_COMBINE = 3, VE
 
 struct SchedParams {
   int is_bwd;
-  int lag;                 // in M-blocks
+  int lag;                 // in experts
   int Ep;
   int T, k;
-  // tiles per M-block (row-space operators) / per expert (weight gradients), per segment:
-  //   forward : seg0 = gate+up (per M-block), seg1 = down (per M-block, lagged)
-  //   backward: seg0 = act_grad (per M-block), seg1 = w2_grad (per expert, at its last M-block),
-  //             seg2 = gate_grad (per M-block, lagged), seg3 = w1_grad (per expert, lagged)
+  // tickets per M-block (row-space operators) / per expert (weight-gradient strips), per segment:
+  //   forward : seg0 = gate+up (column tiles per M-block), seg1 = down (per M-block, lagged)
+  //   backward: seg0 = act_grad (per M-block), seg1 = w2_grad strips (per expert),
+  //             seg2 = gate_grad (per M-block, lagged), seg3 = w1_grad strips (per expert, lagged)
   int seg_tiles[SCHED_MAX_SEG];
-  int wgrad_tn[2];         // column tiles of w2_grad / w1_grad (to split a per-expert index)
+  int strip_tiles[2];      // column tiles in one w2_grad / w1_grad strip
 };
 
-// tiles of step i given the layout (M = number of M-blocks)
-MOE_HD int step_tiles(const SchedParams& sp, int i, int M, const int* mblk_expert, const int* mb_start) {
+MOE_HD int expert_mblocks(const int* mb_start, int e) { return mb_start[e + 1] - mb_start[e]; }
+
+// tickets of step i
+MOE_HD int step_tiles(const SchedParams& sp, int i, const int* mb_start) {
   int n = 0;
   const int j = i - sp.lag;
-  if (i < M) {
-    n += sp.seg_tiles[0];
-    if (sp.is_bwd && i + 1 == mb_start[mblk_expert[i] + 1]) n += sp.seg_tiles[1];
+  if (i < sp.Ep) {
+    const int m = expert_mblocks(mb_start, i);
+    n += m * sp.seg_tiles[0];
+    if (sp.is_bwd && m > 0) n += sp.seg_tiles[1];
   }
-  if (j >= 0 && j < M) {
+  if (j >= 0 && j < sp.Ep) {
+    const int m = expert_mblocks(mb_start, j);
     if (!sp.is_bwd) {
-      n += sp.seg_tiles[1];
+      n += m * sp.seg_tiles[1];
     } else {
-      n += sp.seg_tiles[2];
-      if (j + 1 == mb_start[mblk_expert[j] + 1]) n += sp.seg_tiles[3];
+      n += m * sp.seg_tiles[2];
+      if (m > 0) n += sp.seg_tiles[3];
     }
   }
   return n;
 }
 
 struct MatTile {
-  int op;        // GemmMode, or -1 = end of queue
+  int op;        // GemmMode
   int slot;      // which GemmArgs of the launch (segment index)
   int e;
   int mb;        // M-block (row-space operators) or -1
-  int idx;       // tile index inside the segment
+  int idx;       // column tile (row-space operators) / strip index = 128-row block of the gradient
+  int group;     // tiles processed under this ticket (1, or the strip's column tiles)
   // dependency: every counter dep_ctr[dep_first .. dep_first+dep_count) must reach dep_thr
   int dep_base;  // 0 = gather counters, 1 = activation counters
   int dep_first, dep_count, dep_thr;
@@ -83,10 +89,9 @@ struct MatTile {
   int trig_also_ag;  // backward act_grad also bumps the global act_grad counter
 };
 
-// Decode ticket t (0 <= t < step_start[M+lag]) into a tile.
-MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, int M, const int* step_start,
-                                    const int* mblk_expert, const int* mb_start) {
-  int lo = 0, hi = M + sp.lag - 1;  // last step whose start <= t
+// Decode ticket t (0 <= t < step_start[Ep+lag]) into a tile (or strip).
+MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, const int* step_start, const int* mb_start) {
+  int lo = 0, hi = sp.Ep + sp.lag - 1;  // last step whose start <= t
   while (lo < hi) {
     int mid = (lo + hi + 1) >> 1;
     if (step_start[mid] <= t) lo = mid; else hi = mid - 1;
@@ -95,43 +100,46 @@ MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, int M, const i
   int r = t - step_start[i];
   MatTile m;
   m.trig_also_ag = 0;
-  if (i < M) {
-    if (r < sp.seg_tiles[0]) {
+  m.group = 1;
+  if (i < sp.Ep) {
+    const int mc = expert_mblocks(mb_start, i);
+    if (r < mc * sp.seg_tiles[0]) {
       m.slot = 0; m.op = sp.is_bwd ? 2 /*ACT_GRAD*/ : 0 /*GATE_UP*/;
-      m.mb = i; m.e = mblk_expert[i]; m.idx = r;
-      m.dep_base = 0; m.dep_first = i; m.dep_count = 1; m.dep_thr = GATHER_SUB;
+      m.idx = r / mc; m.mb = mb_start[i] + (r - m.idx * mc); m.e = i;
+      m.dep_base = 0; m.dep_first = m.mb; m.dep_count = 1; m.dep_thr = GATHER_SUB;
       m.trig_base = 1; m.trig_also_ag = sp.is_bwd;
       return m;
     }
-    r -= sp.seg_tiles[0];
-    if (sp.is_bwd && i + 1 == mb_start[mblk_expert[i] + 1]) {
+    r -= mc * sp.seg_tiles[0];
+    if (sp.is_bwd && mc > 0) {
       if (r < sp.seg_tiles[1]) {
-        const int e = mblk_expert[i];
-        m.slot = 1; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = e; m.idx = r;
-        m.dep_base = 0; m.dep_first = mb_start[e]; m.dep_count = mb_start[e + 1] - mb_start[e];
-        m.dep_thr = GATHER_SUB; m.trig_base = -1;
+        m.slot = 1; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = i; m.idx = r; m.group = sp.strip_tiles[0];
+        m.dep_base = 0; m.dep_first = mb_start[i]; m.dep_count = mc; m.dep_thr = GATHER_SUB;
+        m.trig_base = -1;
         return m;
       }
       r -= sp.seg_tiles[1];
     }
   }
-  // lagged segments of M-block j
+  // lagged segments of expert j
+  const int mc = expert_mblocks(mb_start, j);
   if (!sp.is_bwd) {
-    m.slot = 1; m.op = 1 /*DOWN*/; m.mb = j; m.e = mblk_expert[j]; m.idx = r;
-    m.dep_base = 1; m.dep_first = j; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
+    m.slot = 1; m.op = 1 /*DOWN*/; m.e = j;
+    m.idx = r / mc; m.mb = mb_start[j] + (r - m.idx * mc);
+    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
     m.trig_base = 2;
     return m;
   }
-  if (r < sp.seg_tiles[2]) {
-    m.slot = 2; m.op = 3 /*GATE_GRAD*/; m.mb = j; m.e = mblk_expert[j]; m.idx = r;
-    m.dep_base = 1; m.dep_first = j; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
+  if (r < mc * sp.seg_tiles[2]) {
+    m.slot = 2; m.op = 3 /*GATE_GRAD*/; m.e = j;
+    m.idx = r / mc; m.mb = mb_start[j] + (r - m.idx * mc);
+    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
     m.trig_base = 2;
     return m;
   }
-  r -= sp.seg_tiles[2];
-  const int e = mblk_expert[j];
-  m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = e; m.idx = r;
-  m.dep_base = 1; m.dep_first = mb_start[e]; m.dep_count = mb_start[e + 1] - mb_start[e];
+  r -= mc * sp.seg_tiles[2];
+  m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = j; m.idx = r; m.group = sp.strip_tiles[1];
+  m.dep_base = 1; m.dep_first = mb_start[j]; m.dep_count = mc;
   m.dep_thr = EPI_WARPS * sp.seg_tiles[0]; m.trig_base = -1;
   return m;
 }

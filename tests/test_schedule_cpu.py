@@ -14,8 +14,7 @@ def _lib():
 def _seg(is_bwd, d, F):
     if not is_bwd:
         return [(F + 127) // 128, (d + 255) // 256, 0, 0]
-    tn2, tn1 = (F + 255) // 256, (d + 255) // 256
-    return [(F + 255) // 256, ((d + 127) // 128) * tn2, (d + 255) // 256, ((2 * F + 127) // 128) * tn1]
+    return [(F + 255) // 256, (d + 127) // 128, (d + 255) // 256, (2 * F + 127) // 128]
 
 
 @pytest.mark.parametrize("is_bwd", [0, 1])
