@@ -2,6 +2,7 @@
 // sequences of the forward and backward layer.  Argument marshalling and planning only; every
 // step of the layer runs in the kernels of route_layout.cu, permute.cu and gemm_tc.cu.
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <string>
@@ -110,7 +111,7 @@ struct Carve {
 
 // Byte offsets of every workspace tensor.
 struct WsPlan {
-  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
+  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
       dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, stats, total;
   int cap_rows, nblk_max, ntn_act, ctr_count;
 };
@@ -133,6 +134,8 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.pad_off = c.take(sizeof(int) * (Ep + 1));
   p.mb_start = c.take(sizeof(int) * (Ep + 1));
   p.mblk_expert = c.take(sizeof(int) * (cap / BLOCK_M + 1));
+  p.pair_start = c.take(sizeof(int) * (Ep + 1));
+  p.pblk_expert = c.take(sizeof(int) * (cap / BLOCK_M + 1));
   p.blk_hist = c.take(sizeof(int) * (size_t)p.nblk_max * Ep);
   p.row_of = c.take(sizeof(int) * (slots + 1));
   p.src_of = c.take(sizeof(int) * (slots + 1));
@@ -189,7 +192,7 @@ struct moe_ctx {
   // tensor maps of the caller's weights, re-encoded when the pointers change
   const void* w1_ptr = nullptr;
   const void* w2_ptr = nullptr;
-  CUtensorMap tm_W1_k, tm_W2_k, tm_W1_mn, tm_W2_mn;
+  CUtensorMap tm_W1_k, tm_W2_k, tm_W2_k128, tm_W1_mn, tm_W2_mn;
   // store maps: workspace tensors (fixed) and the caller's weight gradients (re-encoded on change)
   CUtensorMap ts_A, ts_H, ts_Y, ts_dH;
   const void* dw1_ptr = nullptr;
@@ -209,6 +212,8 @@ struct moe_ctx {
     lv.pad_off = at<int>(plan.pad_off);
     lv.mb_start = at<int>(plan.mb_start);
     lv.mblk_expert = at<int>(plan.mblk_expert);
+    lv.pair_start = at<int>(plan.pair_start);
+    lv.pblk_expert = at<int>(plan.pblk_expert);
     lv.meta = at<int>(plan.meta);
     lv.blk_hist = at<int>(plan.blk_hist);
     return lv;
@@ -248,6 +253,7 @@ int encode_weight_maps(moe_ctx* c, const uint16_t* W1, const uint16_t* W2) {
   }
   if (W2 != c->w2_ptr) {
     if ((rc = encode_2d(&c->tm_W2_k, W2, Ep * s.d, s.F, 256, 64))) return rc;
+    if ((rc = encode_2d(&c->tm_W2_k128, W2, Ep * s.d, s.F, 128, 64))) return rc;
     if ((rc = encode_2d(&c->tm_W2_mn, W2, Ep * s.d, s.F, 64, 64))) return rc;
     c->w2_ptr = W2;
   }
@@ -262,6 +268,9 @@ GemmArgs base_args(const moe_ctx* c) {
   g.mb_start = lv.mb_start;
   g.counts = lv.counts;
   g.meta = lv.meta;
+  g.pair_start = lv.pair_start;
+  g.pblk_expert = lv.pblk_expert;
+  g.cap_rows = c->plan.cap_rows;
   g.Ep = c->shape.E + c->shape.n_shared;
   g.F = c->shape.F;
   g.status = c->status();
@@ -356,6 +365,19 @@ GemmArgs args_wgrad_gate_up(const moe_ctx* c) {
   return g;
 }
 
+// Diagnostic knob: MOE_B200_SINGLE_CTA_GEMM=1 runs the one-launch-per-operator mode on the single-CTA
+// tiles (the ones the persistent launch uses) instead of CTA pairs.
+bool single_cta_gemm() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("MOE_B200_SINGLE_CTA_GEMM");
+    v = (e && e[0] == '1') ? 1 : 0;
+  }
+  return v == 1;
+}
+#define LAUNCH_GEMM_SERIAL(mode, args, sms, st, launches) \
+  (single_cta_gemm() ? launch_gemm(mode, args, sms, st, launches) : launch_gemm2(mode, args, sms, st, launches))
+
 bool serial_mode(const moe_ctx* c) { return (c->shape.flags & MOE_FLAG_SERIAL_LAUNCH) != 0; }
 
 SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
@@ -425,11 +447,13 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     }
     {
       Phase ph(c, MOE_PHASE_GEMM_GATE_UP, st);
-      MOE_CUDA(launch_gemm(GEMM_GATE_UP, args_gate_up(c), c->num_sms, st, &c->launches));
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_GATE_UP, args_gate_up(c), c->num_sms, st, &c->launches));
     }
     {
       Phase ph(c, MOE_PHASE_GEMM_DOWN, st);
-      MOE_CUDA(launch_gemm(GEMM_DOWN, args_down(c), c->num_sms, st, &c->launches));
+      GemmArgs g = args_down(c);
+      if (!single_cta_gemm()) g.tmB = c->tm_W2_k128;  // each CTA of a pair loads 128 of the tile's 256 rows
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_DOWN, g, c->num_sms, st, &c->launches));
     }
     {
       Phase ph(c, MOE_PHASE_COMBINE, st);
@@ -480,7 +504,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     }
     {
       Phase ph(c, MOE_PHASE_ACT_GRAD, st);
-      MOE_CUDA(launch_gemm(GEMM_ACT_GRAD, args_act_grad(c, d_w != nullptr), c->num_sms, st, &c->launches));
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_ACT_GRAD, args_act_grad(c, d_w != nullptr), c->num_sms, st, &c->launches));
     }
     if (d_w) {
       Phase ph(c, MOE_PHASE_DW_REDUCE, st);
@@ -488,15 +512,15 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     }
     {
       Phase ph(c, MOE_PHASE_WGRAD_DOWN, st);
-      MOE_CUDA(launch_gemm(GEMM_WGRAD, args_wgrad_down(c), c->num_sms, st, &c->launches));
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_WGRAD, args_wgrad_down(c), c->num_sms, st, &c->launches));
     }
     {
       Phase ph(c, MOE_PHASE_GATE_GRAD, st);
-      MOE_CUDA(launch_gemm(GEMM_GATE_GRAD, args_gate_grad(c), c->num_sms, st, &c->launches));
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_GATE_GRAD, args_gate_grad(c), c->num_sms, st, &c->launches));
     }
     {
       Phase ph(c, MOE_PHASE_WGRAD_GATE_UP, st);
-      MOE_CUDA(launch_gemm(GEMM_WGRAD, args_wgrad_gate_up(c), c->num_sms, st, &c->launches));
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_WGRAD, args_wgrad_gate_up(c), c->num_sms, st, &c->launches));
     }
     {  // backward Combine
       Phase ph(c, MOE_PHASE_BWD_COMBINE, st);

@@ -15,7 +15,10 @@ namespace moe {
 
 constexpr int BN = 256;                       // accumulator columns per tile
 constexpr int BK = 64;                        // reduction elements per stage (one 128-byte swizzle row)
-constexpr int STAGES = 4;
+#ifndef MOE_STAGES
+#define MOE_STAGES 4
+#endif
+constexpr int STAGES = MOE_STAGES;
 constexpr int A_STAGE_BYTES = BLOCK_M * BK * 2;  // 16 KB
 constexpr int B_STAGE_BYTES = BN * BK * 2;       // 32 KB
 constexpr int MN_BOX_BYTES = 64 * BK * 2;        // one [64 k][64 mn] box of an MN-major operand

@@ -37,7 +37,9 @@ struct LayoutView {
   int* pad_off;      // [Ep+1]  first padded row of each expert (multiple of BLOCK_M)
   int* mb_start;     // [Ep+1]  first M-block of each expert
   int* mblk_expert;  // [R_pad_max / BLOCK_M] expert of each M-block
-  int* meta;         // [8]     {num_mblocks, R_pad, rows, 0...}
+  int* pair_start;   // [Ep+1]  first M-block pair of each expert (pairs = ceil(M-blocks / 2))
+  int* pblk_expert;  // [pairs] expert of each M-block pair
+  int* meta;         // [8]     {num_mblocks, R_pad, rows, num_pairs, 0...}
   int* blk_hist;     // [nblk][Ep] per-block histograms, then per-block exclusive prefixes
 };
 
@@ -78,6 +80,9 @@ struct GemmArgs {
   const int* mb_start;
   const int* counts;
   const int* meta;
+  const int* pair_start;   // CTA-pair kernels: first M-block pair of each expert
+  const int* pblk_expert;  // CTA-pair kernels: expert of each M-block pair
+  int cap_rows;            // rows of the padded row space (a row coordinate >= cap_rows reads zeros)
   int Ep;
   int n_tiles_n;       // tiles along N per M-block (row-space modes) / per expert (WGRAD)
   int n_tiles_m;       // WGRAD only: tiles along M per expert
@@ -98,6 +103,8 @@ struct GemmArgs {
 
 cudaError_t launch_gemm(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
 size_t gemm_smem_bytes();
+// ---- gemm_tc2.cu: the same operators on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles)
+cudaError_t launch_gemm2(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
 
 // ---- fused.cu (the single persistent dependency-driven launch)
 // Everything one fused launch needs: the operators' GEMM arguments (one per schedule segment), the
