@@ -399,10 +399,9 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
     sp.seg_tiles[3] = (2 * s.F + 127) / 128;   // w1_grad: strips of 128 rows of dW_gate_up
     sp.strip_tiles[1] = (s.d + 255) / 256;
   }
-  // lag: enough experts that a consumer's producers are about two grid-fulls of tickets ahead
-  const long rows = (long)T * (s.k + s.n_shared);
-  const int avg_m = (int)((rows / sp.Ep + BLOCK_M - 1) / BLOCK_M) > 0 ? (int)((rows / sp.Ep + BLOCK_M - 1) / BLOCK_M) : 1;
-  const int per_step = avg_m * sp.seg_tiles[0] + (bwd ? sp.seg_tiles[1] : 0);
+  // lag: enough experts that a consumer's producers are about two grid-fulls of tickets ahead even
+  // when every expert in between holds a single M-block (skewed routing has many such experts)
+  const int per_step = sp.seg_tiles[0] + (bwd ? sp.seg_tiles[1] : 0);
   int lag = (2 * c->num_sms + per_step - 1) / per_step;
   if (lag < 1) lag = 1;
   if (lag > SCHED_LAG_MAX) lag = SCHED_LAG_MAX;

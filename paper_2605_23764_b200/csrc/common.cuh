@@ -77,14 +77,18 @@ struct WaitCtl {
 };
 
 // Bounded wait on an mbarrier phase.  Returns false (after recording MOE_ERR_TIMEOUT, or because
-// another role already aborted) instead of spinning forever.
+// another role already aborted) instead of spinning forever.  `sleep_ns` > 0 makes the waiter back
+// off between polls: a warp that spins takes issue slots from the warps of its scheduler, and the
+// single-thread MMA issuer and loader are among them.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitCtl& wc, int site,
-                                          int tile) {
+                                          int tile, uint32_t sleep_ns = 0) {
   if (mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = 0;
+  const uint32_t check = sleep_ns ? 63u : 1023u;
   for (uint32_t spin = 1;; ++spin) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((spin & 1023u) == 0) {
+    if (sleep_ns) __nanosleep(sleep_ns);
+    if ((spin & check) == 0) {
       if (*reinterpret_cast<volatile int*>(&wc.status->abort)) return false;
       uint64_t now = globaltimer_ns();
       if (t0 == 0) t0 = now;

@@ -1,9 +1,9 @@
 // The single persistent, dependency-driven launch of the forward (and of the backward) layer.
 //
 // One cooperative grid of one CTA per SM runs the whole operator chain.  Per CTA:
-//   warp 0      matrix-queue producer: takes the next ticket of the matrix queue, decodes the tile,
-//               publishes it to the CTA's other roles, polls the tile's dependent counters, then
-//               streams its operands through TMA;
+//   warp 14     scheduler: takes the next ticket of the matrix queue, decodes the tile, polls the
+//               tile's dependent counters, then publishes it to the CTA's other roles;
+//   warp 0      loader: streams the published tile's operands through TMA (one box per lane);
 //   warp 1      tcgen05.mma issuer (and TMEM owner);
 //   warps 2-5   epilogue: TMEM -> fused element-wise math -> TMA store, then the tile's trigger
 //               counter once the stores are complete;
@@ -36,21 +36,28 @@ namespace moe {
 #define ST_FLUSH(base, n)
 #endif
 
-constexpr int VEC_WARPS = 8;
-constexpr int FUSED_THREADS = GEMM_THREADS + 32 * VEC_WARPS;
+#ifndef MOE_VEC_WARPS
+#define MOE_VEC_WARPS 8
+#endif
+constexpr int VEC_WARPS = MOE_VEC_WARPS;
+constexpr int SCHED_WARP = 6 + VEC_WARPS;         // the last warp
+constexpr int FUSED_THREADS = GEMM_THREADS + 32 * VEC_WARPS + 32;
+constexpr int SCHED_AHEAD_KB = 24;                // k-blocks of a ticket left when the next one is fetched
 constexpr int RING = 4;                            // published-tile ring depth
 
 struct TileSlot {
   int op, slot, e, row0, n0, m0, nkb, nb;
   int trig_idx;   // counter index to bump per epilogue warp, -1 = none
   int trig_ag;    // also bump the global act_grad counter
-  int pad[2];
+  int go_kb;      // k-block at which the loader tells the scheduler to fetch the next ticket (-1: not in this tile)
+  int pad;
 };
 
 struct __align__(16) FusedShared {
   GemmBarriers bars;
   uint64_t tk_full[RING];
   uint64_t tk_empty[RING];
+  uint64_t sched_go;      // loader -> scheduler: fetch the next ticket
   uint64_t vec_ready[2];  // one-shot: the global "all tiles done" conditions the vector tail waits for
   int vec_poller[2];      // which warp polls the global counter on behalf of the CTA
   int pad[2];
@@ -210,15 +217,15 @@ __device__ __forceinline__ void vec_zero(const FusedArgs& fa, int task, int lane
 // ---------------------------------------------------------------- matrix-role dispatch on the operator
 template <bool BWD>
 __device__ __forceinline__ void fused_load_stage(const FusedArgs& fa, const TileSlot& ts, const Tile& tl, int kb,
-                                                 uint8_t* sA, uint8_t* sB, uint64_t* bar) {
+                                                 uint8_t* sA, uint8_t* sB, uint64_t* bar, int lane) {
   const GemmArgs& g = fa.op[ts.slot];
   if (!BWD) {
-    if (ts.op == GEMM_GATE_UP) load_stage<GEMM_GATE_UP>(g, tl, kb, sA, sB, bar);
-    else load_stage<GEMM_DOWN>(g, tl, kb, sA, sB, bar);
+    if (ts.op == GEMM_GATE_UP) load_stage_lanes<GEMM_GATE_UP>(g, tl, kb, sA, sB, bar, lane);
+    else load_stage_lanes<GEMM_DOWN>(g, tl, kb, sA, sB, bar, lane);
   } else {
-    if (ts.op == GEMM_ACT_GRAD) load_stage<GEMM_ACT_GRAD>(g, tl, kb, sA, sB, bar);
-    else if (ts.op == GEMM_GATE_GRAD) load_stage<GEMM_GATE_GRAD>(g, tl, kb, sA, sB, bar);
-    else load_stage<GEMM_WGRAD>(g, tl, kb, sA, sB, bar);
+    if (ts.op == GEMM_ACT_GRAD) load_stage_lanes<GEMM_ACT_GRAD>(g, tl, kb, sA, sB, bar, lane);
+    else if (ts.op == GEMM_GATE_GRAD) load_stage_lanes<GEMM_GATE_GRAD>(g, tl, kb, sA, sB, bar, lane);
+    else load_stage_lanes<GEMM_WGRAD>(g, tl, kb, sA, sB, bar, lane);
   }
 }
 template <bool BWD>
@@ -277,8 +284,9 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
     mbar_init(&bars->drain, 1);
     for (int s = 0; s < RING; ++s) {
       mbar_init(&sh->tk_full[s], 1);
-      mbar_init(&sh->tk_empty[s], 1 + EPI_WARPS);  // the MMA issuer and every epilogue warp release a slot
+      mbar_init(&sh->tk_empty[s], 2 + EPI_WARPS);  // loader, MMA issuer and every epilogue warp release a slot
     }
+    mbar_init(&sh->sched_go, 1);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sh->vec_ready[s], 1);
       sh->vec_poller[s] = 0;
@@ -295,80 +303,98 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
   tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
 
-  if (warp == 0) {
-    // ------------------------------------------------ matrix-queue producer
+  if (warp == SCHED_WARP) {
+    // ------------------------------------------------ scheduler: ticket, decode, dependent events
+    // It runs ahead of the loader by at most the ring depth inside one ticket, and takes the NEXT
+    // ticket only when the loader signals that the current one is about to run out of k-blocks: the
+    // atomic, the decode and the counter polls hide behind those last loads, while tiles with
+    // adjacent tickets (which share an operand through L2) still start close together in time.
     if (lane == 0) {
       const int total = fa.step_start[fa.sp.Ep + fa.sp.lag];
-      uint32_t it = 0, n = 0;
+      uint32_t n = 0, go_n = 0;
+      int cursor = 0;  // step of the previous ticket: tickets of one CTA only grow
       bool ok = true;
       ST_DECL;
-      int next_t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
       while (ok) {
         ST_MARK();
-        const int t = next_t;
+        const int t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
         TileSlot ts;
         ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
-        ts.trig_idx = -1; ts.trig_ag = 0;
+        ts.trig_idx = -1; ts.trig_ag = 0; ts.go_kb = -1;
         if (t >= total) {
-          // end of the queue: tell the other roles
-          ts.op = -1;
+          ts.op = -1;  // end of the queue: tell the other roles
           const int rs = n % RING;
           if (!mbar_wait(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) break;
           sh->ring[rs] = ts;
           mbar_arrive(&sh->tk_full[rs]);
           break;
         }
-        const MatTile mt = decode_matrix_ticket(fa.sp, t, fa.step_start, fa.lv.mb_start);
+        while (fa.step_start[cursor + 1] <= t) ++cursor;
+        const MatTile mt = decode_matrix_ticket_at(fa.sp, t, cursor, fa.step_start, fa.lv.mb_start);
         const GemmArgs& g = fa.op[mt.slot];
         ST_ADD(0);  // ticket + decode
-        // dependent event(s): poll until every producer counter has reached its threshold
         for (int q = 0; q < mt.dep_count && ok; ++q) {
           const int mbq = mt.dep_first + q;
           const int* c = fa.ctr + (mt.dep_base == 0 ? ctr_gather(mbq) : ctr_act(mbq));
           ok = counter_wait(c, mt.dep_thr, wc, t);
         }
         if (!ok) break;
-        fence_proxy_async();  // the producers' writes must be seen by the TMA loads that follow
         ST_ADD(1);  // dependency wait
         ts.op = mt.op; ts.slot = mt.slot; ts.e = mt.e;
         ts.trig_idx = mt.trig_base == 1 ? ctr_act(mt.mb) : (mt.trig_base == 2 ? CTR_DONE : -1);
         ts.trig_ag = mt.trig_also_ag;
+        const int nkb = mt.op == GEMM_WGRAD ? (fa.lv.counts[mt.e] + BK - 1) / BK : (g.K + BK - 1) / BK;
         for (int gi = 0; gi < mt.group && ok; ++gi) {
           if (mt.op == GEMM_WGRAD) {
             ts.nb = gi;                       // one 128-row block of the gradient, column tile gi
             ts.m0 = mt.idx * BLOCK_M;
             ts.n0 = gi * BN;
             ts.row0 = fa.lv.mb_start[mt.e] * BLOCK_M;
-            ts.nkb = (fa.lv.counts[mt.e] + BK - 1) / BK;
           } else {
             ts.nb = mt.idx;
             ts.m0 = 0;
             ts.n0 = mt.idx * (mt.op == GEMM_GATE_UP ? BN / 2 : BN);
             ts.row0 = mt.mb * BLOCK_M;
-            ts.nkb = (g.K + BK - 1) / BK;
           }
+          ts.nkb = nkb;
+          // the k-block of this tile at which SCHED_AHEAD_KB k-blocks of the ticket remain
+          const int after = (mt.group - 1 - gi) * nkb;
+          ts.go_kb = -1;
+          if (after < SCHED_AHEAD_KB && (after + nkb >= SCHED_AHEAD_KB || gi == 0))
+            ts.go_kb = max(0, nkb - (SCHED_AHEAD_KB - after));
           const int rs = n % RING;
           if (!mbar_wait(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
           sh->ring[rs] = ts;
           mbar_arrive(&sh->tk_full[rs]);  // release: the slot's contents are visible to the waiters
           ++n;
-          ST_ADD(2);  // ring slot wait
-          const Tile tl = slot_tile(ts);
-          const int kb_prefetch = (gi + 1 == mt.group) ? max(0, ts.nkb - 8) : -1;
-          for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
-            // take the next ticket shortly before this ticket's loads end: the atomic's round trip
-            // hides behind the last k-blocks, and tiles with adjacent tickets (which share an
-            // operand through L2) still start close together in time
-            if (kb == kb_prefetch) next_t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
-            const int s = it % STAGES;
-            if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
-            ST_ADD(3);  // stage wait (back-pressure from the tensor core: the healthy state)
-            fused_load_stage<BWD>(fa, ts, tl, kb, sA + s * A_STAGE_BYTES, sB + s * B_STAGE_BYTES, &bars->full[s]);
-            ST_ADD(4);  // issue
-          }
         }
+        ST_ADD(2);  // ring slot waits
+        if (!ok || !mbar_wait(&sh->sched_go, go_n & 1, wc, SITE_DEP, t, 200)) break;
+        ++go_n;
+        ST_ADD(3);  // waiting for the loader's signal (the healthy state)
       }
-      ST_FLUSH(0, 5);
+      ST_FLUSH(0, 4);
+    }
+  } else if (warp == 0) {
+    // ------------------------------------------------ loader: TMA boxes of each k-block, one per lane
+    uint32_t it = 0, n = 0;
+    bool ok = true;
+    while (ok) {
+      const int rs = n % RING;
+      if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -3)) break;
+      const TileSlot ts = sh->ring[rs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->tk_empty[rs]);
+      ++n;
+      if (ts.op < 0) break;
+      fence_proxy_async();  // the producers' writes (acquired by the scheduler) must be seen by the TMA loads
+      const Tile tl = slot_tile(ts);
+      for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
+        if (kb == ts.go_kb && lane == 0) mbar_arrive(&sh->sched_go);
+        const int s = it % STAGES;
+        if (!mbar_wait(&bars->empty[s], ((it / STAGES) & 1) ^ 1, wc, SITE_EMPTY, n)) { ok = false; break; }
+        fused_load_stage<BWD>(fa, ts, tl, kb, sA + s * A_STAGE_BYTES, sB + s * B_STAGE_BYTES, &bars->full[s], lane);
+      }
     }
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer
@@ -420,7 +446,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
     while (true) {
       const int rs = n % RING;
       ST_MARK();
-      if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -2)) break;
+      if (!mbar_wait(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -2, 100)) break;
       ST_ADD(0);
       const TileSlot ts = sh->ring[rs];
       __syncwarp();
@@ -432,7 +458,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
         fused_epilogue<BWD>(fa, ts, tl, 0, quad, lane, stg);
       } else {
         const int as = acc_it & 1;
-        if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, n)) break;
+        if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, n, 100)) break;
         ST_ADD(1);  // waiting for the accumulator
         tc_fence_after_sync();
         fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);
@@ -481,7 +507,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
             ok = counter_wait(fa.ctr + (kind == 0 ? CTR_DONE : CTR_AG_DONE), v.dep_thr, wc, t, 2000) ? 1 : 0;
             if (ok) mbar_arrive(&sh->vec_ready[kind]);
           } else {
-            ok = mbar_wait(&sh->vec_ready[kind], 0, wc, SITE_DEP, t) ? 1 : 0;
+            ok = mbar_wait(&sh->vec_ready[kind], 0, wc, SITE_DEP, t, 4000) ? 1 : 0;
           }
         }
         ok = __shfl_sync(0xffffffffu, ok, 0);

@@ -117,6 +117,33 @@ __device__ __forceinline__ void load_stage(const GemmArgs& a, const Tile& tl, in
   }
 }
 
+// The same loads issued by a whole warp, one box per lane (a single thread needs several hundred
+// cycles to issue the five or six boxes of a k-block).  All lanes call it; lane 0 arms the barrier.
+template <int MODE>
+__device__ __forceinline__ void load_stage_lanes(const GemmArgs& a, const Tile& tl, int kb, uint8_t* sA, uint8_t* sB,
+                                                 uint64_t* bar, int lane) {
+  const int k0 = kb * BK;
+  if (lane == 0)
+    mbar_expect_tx(bar, MODE == GEMM_WGRAD ? 6 * MN_BOX_BYTES : A_STAGE_BYTES + B_STAGE_BYTES);
+  __syncwarp();
+  if (MODE == GEMM_WGRAD) {
+    if (lane < 2) tma_load_2d(sA + lane * MN_BOX_BYTES, &a.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
+    else if (lane < 6) tma_load_2d(sB + (lane - 2) * MN_BOX_BYTES, &a.tmB, tl.n0 + (lane - 2) * 64, tl.row0 + k0, bar);
+    return;
+  }
+  const int brow = tl.e * a.b_rows_per_expert;
+  if (lane == 0) {
+    tma_load_2d(sA, &a.tmA, k0, tl.row0, bar);
+  } else if (MODE == GEMM_GATE_UP) {
+    if (lane == 1) tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);
+    else if (lane == 2) tma_load_2d(sB + B_STAGE_BYTES / 2, &a.tmB, k0, brow + a.F + tl.n0, bar);
+  } else if (MODE == GEMM_DOWN) {
+    if (lane == 1) tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);
+  } else {
+    if (lane < 5) tma_load_2d(sB + (lane - 1) * MN_BOX_BYTES, &a.tmB, tl.n0 + (lane - 1) * 64, brow + k0, bar);
+  }
+}
+
 // ---------------------------------------------------------------- epilogues
 // Each epilogue warp owns 32 rows of the tile (its TMEM lane quadrant) and a private staging area of
 // two [32 rows][64 columns] bf16 boxes in the 128-byte-swizzled layout the store tensor maps expect.

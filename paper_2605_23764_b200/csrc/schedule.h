@@ -89,14 +89,10 @@ struct MatTile {
   int trig_also_ag;  // backward act_grad also bumps the global act_grad counter
 };
 
-// Decode ticket t (0 <= t < step_start[Ep+lag]) into a tile (or strip).
-MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, const int* step_start, const int* mb_start) {
-  int lo = 0, hi = sp.Ep + sp.lag - 1;  // last step whose start <= t
-  while (lo < hi) {
-    int mid = (lo + hi + 1) >> 1;
-    if (step_start[mid] <= t) lo = mid; else hi = mid - 1;
-  }
-  const int i = lo, j = i - sp.lag;
+// Decode ticket t of step i (step_start[i] <= t < step_start[i+1]) into a tile (or strip).
+MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, const int* step_start,
+                                       const int* mb_start) {
+  const int j = i - sp.lag;
   int r = t - step_start[i];
   MatTile m;
   m.trig_also_ag = 0;
@@ -142,6 +138,16 @@ MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, const int* ste
   m.dep_base = 1; m.dep_first = mb_start[j]; m.dep_count = mc;
   m.dep_thr = EPI_WARPS * sp.seg_tiles[0]; m.trig_base = -1;
   return m;
+}
+
+// Decode ticket t (0 <= t < step_start[Ep+lag]) into a tile (or strip).
+MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, const int* step_start, const int* mb_start) {
+  int lo = 0, hi = sp.Ep + sp.lag - 1;  // last step whose start <= t
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if (step_start[mid] <= t) lo = mid; else hi = mid - 1;
+  }
+  return decode_matrix_ticket_at(sp, t, lo, step_start, mb_start);
 }
 
 // ---------------------------------------------------------------- vector queue
