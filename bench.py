@@ -57,7 +57,9 @@ def phase_work(cfg, train):
         "gemm_down": (2.0 * R * F * d, R * F * bf + W2 + R * d * bf),
         "combine": (0.0, R * d * bf + T * d * bf),
     }
+    work["fused_fwd"] = (6.0 * R * d * F, W1 + W2 + 2 * T * d * bf + (R * 2 * F * bf if train else 0))
     if train:
+        work["fused_bwd"] = (12.0 * R * d * F, 3 * (W1 + W2) + 2 * T * d * bf + R * 2 * F * bf + R * (d + F) * bf)
         work.update({
             "bwd_gather": (0.0, T * d * bf + R * d * bf),
             "act_grad": (2.0 * R * d * F, R * d * bf + W2 + R * 2 * F * bf * 2),
@@ -245,7 +247,7 @@ def workload_desc(cfg, train, args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=4, help="index into BASELINE.json configs (default: the training step)")
     ap.add_argument("--serial", action="store_true", help="one kernel launch per operator instead of the fused launch")
@@ -253,6 +255,7 @@ def main():
     ap.add_argument("--fwd-only", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-compare", action="store_true", help="skip timing the other launch mode")
     ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -292,87 +295,105 @@ def main():
     if cfg.weight_bytes() <= 4e8:
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
 
-    launches = 0
+    def measure(lay):
+        """W warm-up steps, then K timed steps back to back (CUDA events on the launching stream; the
+        per-operator events inside the library are read after each call).  -> dict"""
+        def step(count=False, phases=None):
+            n = 0
+            B.moe_route(lay.ctx, logits, T, ids, w)
+            n += lay.launches()
+            if phases is not None:
+                phases.update(B.moe_get_phase_ms(lay.ctx))
+            B.moe_ffn_fwd(lay.ctx, x, ids, w, W1, W2, out, T)
+            n += lay.launches()
+            if phases is not None:
+                phases.update(B.moe_get_phase_ms(lay.ctx))
+            if train:
+                B.moe_ffn_bwd(lay.ctx, dout, x, ids, w, W1, W2, dx, dW1, dW2, dw, T)
+                n += lay.launches()
+                if phases is not None:
+                    phases.update(B.moe_get_phase_ms(lay.ctx))
+            return n
 
-    def step():
-        nonlocal launches
-        B.moe_route(layer.ctx, logits, T, ids, w)
-        launches += layer.launches()
-        B.moe_ffn_fwd(layer.ctx, x, ids, w, W1, W2, out, T)
-        launches += layer.launches()
-        if train:
-            B.moe_ffn_bwd(layer.ctx, dout, x, ids, w, W1, W2, dx, dW1, dW2, dw, T)
-            launches += layer.launches()
+        for _ in range(args.warmup):
+            step()
+        torch.cuda.synchronize()
+        assert lay.status() == (0, 0), "device-side error during warm-up"
+        B.moe_set_profiling(lay.ctx, True)
+        phase_sum, n_launch = {}, 0
+        sampler = ClockSampler(local)
+        sampler.start()
+        barrier(world)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        flush_ms = 0.0
+        ev0.record()
+        for _ in range(args.steps):
+            if flush is not None:
+                f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                f0.record(); flush.zero_(); f1.record()
+            ph = {}
+            n_launch += step(phases=ph)
+            for kname, v in ph.items():
+                phase_sum[kname] = phase_sum.get(kname, 0.0) + v
+            if flush is not None:
+                f1.synchronize()
+                flush_ms += f0.elapsed_time(f1)
+        ev1.record()
+        barrier(world)
+        clk = sampler.stop()
+        elapsed = max_over_ranks(ev0.elapsed_time(ev1) - flush_ms, world)
+        B.moe_set_profiling(lay.ctx, False)
+        code, detail = lay.status()
+        assert code == 0, f"device-side error {code} detail {detail:#x}"
+        ms = elapsed / args.steps
+        return {"ms_per_step": ms, "value": world * step_flops(cfg, train) / (ms * 1e-3) / 1e12,
+                "phases_ms": {k: v / args.steps for k, v in phase_sum.items()}, "launches": n_launch, "clocks": clk,
+                "timed_ms": elapsed}
 
-    # ---- device-resident timing --------------------------------------------------------------
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    assert layer.status() == (0, 0), "device-side error during warm-up"
-    B.moe_set_profiling(layer.ctx, True)
-    phase_sum, launches = {}, 0
-    sampler = ClockSampler(local)
-    sampler.start()
-    barrier(world)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    flush_ms = 0.0
-    ev0.record()
-    for _ in range(args.steps):
-        if flush is not None:
-            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            f0.record(); flush.zero_(); f1.record()
-        B.moe_route(layer.ctx, logits, T, ids, w)
-        launches += layer.launches()
-        ph = B.moe_get_phase_ms(layer.ctx)
-        B.moe_ffn_fwd(layer.ctx, x, ids, w, W1, W2, out, T)
-        launches += layer.launches()
-        ph.update(B.moe_get_phase_ms(layer.ctx))
-        if train:
-            B.moe_ffn_bwd(layer.ctx, dout, x, ids, w, W1, W2, dx, dW1, dW2, dw, T)
-            launches += layer.launches()
-            ph.update(B.moe_get_phase_ms(layer.ctx))
-        for kname, v in ph.items():
-            phase_sum[kname] = phase_sum.get(kname, 0.0) + v
-        if flush is not None:
-            f1.synchronize()
-            flush_ms += f0.elapsed_time(f1)
-    ev1.record()
-    barrier(world)
-    clocks = sampler.stop()
-    elapsed_ms = ev0.elapsed_time(ev1) - flush_ms
-    elapsed_ms = max_over_ranks(elapsed_ms, world)
-    B.moe_set_profiling(layer.ctx, False)
-    code, detail = layer.status()
-    assert code == 0, f"device-side error {code} detail {detail:#x}"
-    ms_per_step = elapsed_ms / args.steps
-    flops = step_flops(cfg, train)
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
-
-    # ---- roofline of the dominant kernel --------------------------------------------------------
-    work = phase_work(cfg, train)
-    phases_ms = {k: v / args.steps for k, v in phase_sum.items()}
-    peak_tf = peaks["bf16_tflops_sustained"] if ms_per_step * args.steps > 500 else peaks["bf16_tflops"]
-    peak_gb = peaks["hbm_gbs"]
-    dom = max((k for k in phases_ms if k in work), key=lambda k: phases_ms[k], default=None)
-    roofline = None
-    if dom:
-        fl, by = work[dom]
-        t_s = phases_ms[dom] * 1e-3
-        tensor_bound = fl / (peak_tf * 1e12) >= by / (peak_gb * 1e9)
-        if tensor_bound:
-            roofline = {"kernel": dom, "bound": "tensor", "achieved": fl / t_s / 1e12, "peak": peak_tf,
-                        "unit": "TFLOP/s"}
-        else:
-            roofline = {"kernel": dom, "bound": "hbm", "achieved": by / t_s / 1e9, "peak": peak_gb, "unit": "GB/s"}
-        roofline["frac"] = roofline["achieved"] / roofline["peak"]
-        roofline["peak_source"] = peaks["source"] + (" sustained" if peak_tf == peaks.get("bf16_tflops_sustained")
-                                                     and tensor_bound else "")
-        roofline["traffic"] = ncu_traffic(dom, cfg)
-        roofline["launch_ms"] = phases_ms[dom]
-    t_roof = max(flops / (peak_tf * 1e12), step_min_bytes(cfg, train) / (peak_gb * 1e9))
-    step_roofline = {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step,
+    def rooflines(res):
+        """Roofline of the operator with the largest time, and of the whole step."""
+        work = phase_work(cfg, train)
+        phases_ms = res["phases_ms"]
+        peak_tf = peaks["bf16_tflops_sustained"] if res["timed_ms"] > 500 else peaks["bf16_tflops"]
+        peak_gb = peaks["hbm_gbs"]
+        dom = max((k for k in phases_ms if k in work), key=lambda k: phases_ms[k], default=None)
+        roof = None
+        if dom:
+            fl, by = work[dom]
+            t_s = phases_ms[dom] * 1e-3
+            tensor_bound = fl / (peak_tf * 1e12) >= by / (peak_gb * 1e9)
+            if tensor_bound:
+                roof = {"kernel": dom, "bound": "tensor", "achieved": fl / t_s / 1e12, "peak": peak_tf, "unit": "TFLOP/s"}
+            else:
+                roof = {"kernel": dom, "bound": "hbm", "achieved": by / t_s / 1e9, "peak": peak_gb, "unit": "GB/s"}
+            roof["frac"] = roof["achieved"] / roof["peak"]
+            roof["peak_source"] = peaks["source"] + ((" sustained" if peak_tf == peaks.get("bf16_tflops_sustained")
+                                                      else " burst") if tensor_bound else "")
+            roof["traffic"] = ncu_traffic(dom, cfg)
+            roof["launch_ms"] = phases_ms[dom]
+        flops = step_flops(cfg, train)
+        t_roof = max(flops / (peak_tf * 1e12), step_min_bytes(cfg, train) / (peak_gb * 1e9))
+        step_roof = {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / res["ms_per_step"],
                      "flop_ms": flops / (peak_tf * 1e12) * 1e3,
                      "hbm_ms": step_min_bytes(cfg, train) / (peak_gb * 1e9) * 1e3}
+        return roof, step_roof
+
+    # ---- device-resident timing: the chosen launch mode, then the other one for comparison ----------
+    res = measure(layer)
+    ms_per_step, value, launches, clocks, phases_ms = (res["ms_per_step"], res["value"], res["launches"],
+                                                       res["clocks"], res["phases_ms"])
+    flops = step_flops(cfg, train)
+    roofline, step_roofline = rooflines(res)
+    other = None
+    if not args.no_compare:
+        other_layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=train,
+                               serial=not args.serial)
+        r2 = measure(other_layer)
+        roof2, step2 = rooflines(r2)
+        other = {"launch": "fused persistent" if args.serial else "serial kernels (one launch per operator)",
+                 "ms_per_step": r2["ms_per_step"], "value": r2["value"], "phases_ms": r2["phases_ms"],
+                 "roofline": roof2, "step_roofline": step2, "clocks": r2["clocks"]}
+        other_layer.close()
 
     # ---- end to end through the host-buffer entry points ------------------------------------------
     e2e = None
@@ -428,11 +449,12 @@ def main():
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": workload_desc(cfg, train, args), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "step_roofline": step_roofline, "phases_ms": phases_ms,
-            "cpu_baseline": cpu_baseline,
+            "other_launch_mode": other, "cpu_baseline": cpu_baseline,
         }
         per_step = launches / max(1, args.steps)
-        line["config"]["launch"] = ("fused persistent" if per_step <= (4 if train else 3)
-                                    else "serial kernels (one launch per operator)")
+        line["config"]["launch"] = ("serial kernels (one launch per operator)" if args.serial else
+                                    "fused persistent (one launch each for forward and backward, after the "
+                                    "index-only layout and schedule kernels)")
         line["config"]["launches_per_step"] = per_step
         print(json.dumps(line), flush=True)
     layer.close()

@@ -239,7 +239,7 @@ __device__ __forceinline__ void fused_mma(int op, uint32_t d_tmem, uint32_t a_ad
 }
 template <bool BWD>
 __device__ __forceinline__ void fused_epilogue(const FusedArgs& fa, const TileSlot& ts, const Tile& tl,
-                                               uint32_t tmem_acc, int quad, int lane, uint8_t* stg) {
+                                               uint32_t tmem_acc, int quad, int lane, Staging& stg) {
   const GemmArgs& g = fa.op[ts.slot];
   if (!BWD) {
     if (ts.op == GEMM_GATE_UP) epilogue_tile<GEMM_GATE_UP>(g, tl, tmem_acc, quad, lane, stg);
@@ -440,7 +440,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
   } else if (warp < 2 + EPI_WARPS) {
     // ------------------------------------------------ epilogue warps
     const int quad = warp & 3;
-    uint8_t* stg = sOut + quad * OUT_STAGE_BYTES;
+    Staging stg{sOut + quad * OUT_STAGE_BYTES, 1, 0};
     uint32_t acc_it = 0, n = 0;
     ST_DECL;
     while (true) {

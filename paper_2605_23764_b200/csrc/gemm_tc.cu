@@ -102,7 +102,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_kernel(const __g
   } else {
     // ------------------------------------------------ epilogue warps
     const int quad = warp & 3;  // TMEM lane quadrant this warp may access
-    uint8_t* stg = sOut + quad * OUT_STAGE_BYTES;
+    Staging stg{sOut + quad * OUT_STAGE_BYTES, 1, 0};
     uint32_t acc_it = 0;
     for (int t = blockIdx.x; t < total; t += gridDim.x) {
       const Tile tl = decode_tile<MODE>(a, t);

@@ -20,7 +20,8 @@
 
 namespace moe {
 
-constexpr int STAGES2 = 6;
+constexpr int STAGES2 = 5;                                       // 5 x 32 KB operand stages ...
+constexpr int OUT_BUFS2 = 2;                                     // ... and double-buffered epilogue staging
 constexpr int HALF_B_BYTES = B_STAGE_BYTES / 2;                 // 16 KB: this CTA's half of the B tile
 constexpr int STAGE2_BYTES = A_STAGE_BYTES + HALF_B_BYTES;      // 32 KB
 
@@ -34,7 +35,8 @@ struct __align__(8) PairBarriers {
   uint32_t pad;
 };
 
-constexpr size_t GEMM2_SMEM_BYTES = 1024 + (size_t)STAGES2 * STAGE2_BYTES + 4 * OUT_STAGE_BYTES + sizeof(PairBarriers);
+constexpr size_t GEMM2_SMEM_BYTES =
+    1024 + (size_t)STAGES2 * STAGE2_BYTES + 4 * OUT_BUFS2 * OUT_STAGE_BYTES + sizeof(PairBarriers);
 static_assert(GEMM2_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 struct PairTile {
@@ -134,7 +136,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
   uint8_t* sA = smem;                                  // [STAGES2][16 KB]
   uint8_t* sB = smem + STAGES2 * A_STAGE_BYTES;        // [STAGES2][16 KB]
   uint8_t* sOut = smem + STAGES2 * STAGE2_BYTES;
-  PairBarriers* bars = reinterpret_cast<PairBarriers*>(sOut + 4 * OUT_STAGE_BYTES);
+  PairBarriers* bars = reinterpret_cast<PairBarriers*>(sOut + 4 * OUT_BUFS2 * OUT_STAGE_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();
@@ -215,7 +217,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
   } else {
     // ------------------------------------------------ epilogue warps (both CTAs, own rows)
     const int quad = warp & 3;
-    uint8_t* stg = sOut + quad * OUT_STAGE_BYTES;
+    Staging stg{sOut + quad * OUT_BUFS2 * OUT_STAGE_BYTES, OUT_BUFS2, 0};
     uint32_t acc_it = 0;
     for (int t = pair; t < total; t += npairs) {
       const PairTile pt = decode_pair_tile<MODE>(a, t, rank);

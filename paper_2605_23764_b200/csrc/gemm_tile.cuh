@@ -162,9 +162,22 @@ __device__ __forceinline__ void load8_bf16(const uint16_t* p, float* v) {
 __device__ __forceinline__ float sigmoidf_fast(float g) { return 1.0f / (1.0f + __expf(-g)); }
 
 // Before refilling the staging area: the previous stores must have finished reading it.
-__device__ __forceinline__ void staging_acquire(int lane) {
-  if (lane == 0) tma_store_wait_read();
+// `nbuf` staging areas are used round-robin: with two, the stores of one round drain while the next
+// round is being filled.
+struct Staging {
+  uint8_t* base;
+  uint32_t nbuf;   // 1 or 2 areas of OUT_STAGE_BYTES
+  uint32_t round;
+};
+__device__ __forceinline__ uint8_t* staging_acquire(Staging& sg, int lane) {
+  if (lane == 0) {
+    if (sg.nbuf == 2) tma_store_wait_read1();
+    else tma_store_wait_read();
+  }
   __syncwarp();
+  uint8_t* area = sg.base + (sg.round % sg.nbuf) * OUT_STAGE_BYTES;
+  ++sg.round;
+  return area;
 }
 // After filling: publish the writes to the async proxy; lane 0 then issues the stores.
 __device__ __forceinline__ void staging_release() {
@@ -174,15 +187,14 @@ __device__ __forceinline__ void staging_release() {
 
 template <int MODE>
 __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl, uint32_t tmem_acc, int quad,
-                                              int lane, uint8_t* stg) {
+                                              int lane, Staging& sg) {
   const uint32_t trow = tmem_acc + (static_cast<uint32_t>(quad * 32) << 16);
-  uint8_t* box0 = stg;
-  uint8_t* box1 = stg + OUT_BOX_BYTES;
+  uint8_t *box0, *box1;
   if (MODE == GEMM_GATE_UP) {
     const int prow0 = tl.row0 + quad * 32;             // first padded row of this warp's slab
     const float w = a.prow_w[prow0 + lane];
     // round 1: A = w * silu(g) * u, 128 columns
-    staging_acquire(lane);
+    box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
     for (int c = 0; c < BN / 2; c += 16) {
       float g[16], u[16], act[16];
       tmem_ld16(trow + c, g);
@@ -204,7 +216,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
       // rounds 2, 3: the pre-activations, kept for the backward pass (H viewed as [row][gate|up][F])
 #pragma unroll 1
       for (int half = 0; half < 2; ++half) {
-        staging_acquire(lane);
+        box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
         for (int c = 0; c < BN / 2; c += 16) {
           float v[16];
           tmem_ld16(trow + half * (BN / 2) + c, v);
@@ -231,7 +243,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += 64) {
       if (tl.n0 + c0 >= a.F) break;  // uniform: whole round outside the tensor
-      staging_acquire(lane);
+      box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
 #pragma unroll
       for (int c = 0; c < 64; c += 16) {
         float da[16];
@@ -276,7 +288,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
     for (int c0 = 0; c0 < BN; c0 += 128) {
       if (tl.n0 + c0 >= a.N) break;
       if (MODE == GEMM_WGRAD && y0 >= a.M) break;
-      staging_acquire(lane);
+      box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
 #pragma unroll
       for (int c = 0; c < 128; c += 32) {
         float v[32];
