@@ -195,12 +195,12 @@ int moe_debug_buffer(moe_ctx* ctx, int which, void** ptr, size_t* elems);
  * given per-expert row counts[Ep] it builds the matrix and vector queues, verifies that every tile
  * appears once and after all of its producers, lets mat_workers + vec_workers workers consume the
  * queues in ticket order blocking on the counters, and verifies that every counter ends at its
- * threshold.  seg_tiles[4] = tickets per M-block / per expert of each schedule segment, lag in
- * experts.  Returns 0, or a positive code naming the violated property (20 = deadlock).
+ * threshold.  seg_tiles[4] = tickets per M-block (or per M-block pair when `pair` is set: two CTAs
+ * on one 256-row tile) / per expert of each schedule segment, lag in experts.  Returns 0, or a positive code naming the violated property (20 = deadlock).
  * stats[4] (may be NULL) = {matrix tiles, vector tasks, scheduler rounds, stalled polls}.  Needs no GPU. */
 int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t is_bwd,
                                 const int32_t* seg_tiles, int32_t lag, int32_t mat_workers,
-                                int32_t vec_workers, int64_t* stats);
+                                int32_t vec_workers, int32_t pair, int64_t* stats);
 
 /* Dispatch layout for callers that cannot allocate device memory (no counterpart in the paper:
  * this is a convenience of this library).  Who needs it: code that runs where cudaMalloc is not

@@ -70,7 +70,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_get_phase_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.moe_route_host.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.moe_layout_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
-    lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, i32, vp]
+    lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, vp]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -223,13 +223,13 @@ def moe_layout_noalloc(topk_ids, T, E, k, n_shared, counts, offsets, row_of, src
                                              _dev(status2, i32, "status2"), _stream()), "moe_layout_noalloc")
 
 
-def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_workers, vec_workers):
+def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_workers, vec_workers, pair=False):
     """Host-only schedule check; returns (code, stats) with code 0 = schedule is sound."""
     c = (ctypes.c_int32 * len(counts))(*[int(v) for v in counts])
     seg = (ctypes.c_int32 * 4)(*[int(v) for v in seg_tiles])
     stats = (ctypes.c_int64 * 4)()
     rc = load_library().moe_debug_simulate_schedule(c, len(counts), T, k, int(is_bwd), seg, lag, mat_workers,
-                                                    vec_workers, stats)
+                                                    vec_workers, int(bool(pair)), stats)
     return rc, list(stats)
 
 

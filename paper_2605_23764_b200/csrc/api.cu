@@ -385,6 +385,7 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
   SchedParams sp;
   memset(&sp, 0, sizeof sp);
   sp.is_bwd = bwd ? 1 : 0;
+  sp.pair = single_cta_gemm() ? 0 : 1;
   sp.Ep = s.E + s.n_shared;
   sp.T = T;
   sp.k = s.k;
@@ -393,10 +394,11 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
     sp.seg_tiles[1] = (s.d + 255) / 256;
   } else {
     sp.seg_tiles[0] = c->plan.ntn_act;
-    sp.seg_tiles[1] = (s.d + 127) / 128;       // w2_grad: strips of 128 rows of dW_down
+    const int strip_rows = sp.pair ? 256 : 128;  // rows of the gradient one ticket covers
+    sp.seg_tiles[1] = (s.d + strip_rows - 1) / strip_rows;       // w2_grad strips
     sp.strip_tiles[0] = (s.F + 255) / 256;
     sp.seg_tiles[2] = (s.d + 255) / 256;
-    sp.seg_tiles[3] = (2 * s.F + 127) / 128;   // w1_grad: strips of 128 rows of dW_gate_up
+    sp.seg_tiles[3] = (2 * s.F + strip_rows - 1) / strip_rows;   // w1_grad strips
     sp.strip_tiles[1] = (s.d + 255) / 256;
   }
   // lag: enough experts that a consumer's producers are about two grid-fulls of tickets ahead even
@@ -463,6 +465,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     FusedArgs fa = fused_base(c, false, T);
     fa.op[0] = args_gate_up(c);
     fa.op[1] = args_down(c);
+    if (fa.sp.pair) fa.op[1].tmB = c->tm_W2_k128;
     fa.gather_src = x;
     fa.gather_dst = c->at<uint16_t>(p.Xp);
     fa.topk_w = w;
@@ -838,14 +841,14 @@ int moe_debug_buffer(moe_ctx* c, int which, void** ptr, size_t* elems) {
 // consume them in ticket order, each blocking on its tile's dependent counters.
 int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t is_bwd,
                                 const int32_t* seg_tiles, int32_t lag, int32_t mat_workers, int32_t vec_workers,
-                                int64_t* stats) {
+                                int32_t pair, int64_t* stats) {
   if (!counts || !seg_tiles || Ep < 1 || lag < 0 || mat_workers < 1 || vec_workers < 1) return MOE_ERR_INVALID_ARG;
   std::vector<int> mb_start(Ep + 1, 0);
   for (int e = 0; e < Ep; ++e) mb_start[e + 1] = mb_start[e] + (counts[e] + BLOCK_M - 1) / BLOCK_M;
   const int M = mb_start[Ep];
   SchedParams sp;
   memset(&sp, 0, sizeof sp);
-  sp.is_bwd = is_bwd; sp.lag = lag; sp.Ep = Ep; sp.T = T; sp.k = k;
+  sp.is_bwd = is_bwd; sp.lag = lag; sp.Ep = Ep; sp.T = T; sp.k = k; sp.pair = pair ? 1 : 0;
   for (int i = 0; i < SCHED_MAX_SEG; ++i) sp.seg_tiles[i] = seg_tiles[i];
   sp.strip_tiles[0] = sp.strip_tiles[1] = 1;
   std::vector<int> step_start(Ep + lag + 1, 0);
@@ -859,8 +862,11 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
     const MatTile m = decode_matrix_ticket(sp, t, step_start.data(), mb_start.data());
     if (m.e < 0 || m.e >= Ep || m.idx < 0 || m.idx >= sp.seg_tiles[m.slot]) return 10;
     if (m.mb >= 0 && (m.mb < mb_start[m.e] || m.mb >= mb_start[m.e + 1])) return 10;
-    if (m.slot == 0) seg0_count[m.mb]++;
-    else if (m.mb >= 0) { lag_count[m.mb]++; if (seg0_count[m.mb] != sp.seg_tiles[0]) return 11; }
+    if (m.mb >= 0 && (m.mb_count < 1 || m.mb_count > (pair ? 2 : 1) || m.mb + m.mb_count > mb_start[m.e + 1])) return 10;
+    if (m.slot == 0) { for (int q = 0; q < m.mb_count; ++q) seg0_count[m.mb + q]++; }
+    else if (m.mb >= 0) {
+      for (int q = 0; q < m.mb_count; ++q) { lag_count[m.mb + q]++; if (seg0_count[m.mb + q] != sp.seg_tiles[0]) return 11; }
+    }
     else if (m.slot == 1) w2_count[m.e]++;
     else {
       w1_count[m.e]++;
@@ -895,9 +901,11 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
         if (ctr[wk.m.dep_base == 0 ? ctr_gather(mb) : ctr_act(mb)] < wk.m.dep_thr) ready = false;
       }
       if (!ready) { ++stalls; continue; }
-      if (wk.m.trig_base == 1) ctr[ctr_act(wk.m.mb)] += EPI_WARPS;
-      if (wk.m.trig_base == 2) ctr[CTR_DONE] += EPI_WARPS;
-      if (wk.m.trig_also_ag) ctr[CTR_AG_DONE] += EPI_WARPS;
+      for (int q = 0; q < wk.m.mb_count; ++q) {  // every real M-block of the tile signals (an idle half does not)
+        if (wk.m.trig_base == 1) ctr[ctr_act(wk.m.mb + q)] += EPI_WARPS;
+        if (wk.m.trig_base == 2) ctr[CTR_DONE] += EPI_WARPS;
+        if (wk.m.trig_also_ag) ctr[CTR_AG_DONE] += EPI_WARPS;
+      }
       wk.holding = false;
       ++done_mat;
       progress = true;

@@ -17,7 +17,7 @@
 
 #include <vector>
 
-#include "gemm_tile.cuh"
+#include "gemm_pair.cuh"
 #include "schedule.h"
 
 namespace moe {
@@ -257,6 +257,51 @@ __device__ __forceinline__ Tile slot_tile(const TileSlot& ts) {
   return tl;
 }
 
+// ---------------------------------------------------------------- vector-queue consumer (one warp)
+template <bool BWD>
+__device__ __forceinline__ void vector_worker_loop(const FusedArgs& fa, uint64_t* vec_ready, int* vec_poller,
+                                                   const WaitCtl& wc, int M, int lane) {
+  if (!*reinterpret_cast<volatile int*>(&fa.status->abort)) {
+    const int vtotal = vec_total(fa.sp, M);
+    while (true) {
+      int t = 0;
+      if (lane == 0) t = atomicAdd(&fa.ctr[CTR_VEC_TICKET], 1);
+      t = __shfl_sync(0xffffffffu, t, 0);
+      if (t >= vtotal) break;
+      const VecTask v = decode_vector_ticket(fa.sp, t, M);
+      if (v.dep) {
+        // A global completion counter: one warp of the CTA polls it (slowly), the others sleep on a
+        // shared-memory barrier -- a thousand warps spinning on one L2 line would slow every load.
+        const int kind = v.dep == 2 ? 0 : 1;
+        int ok = 1;
+        if (lane == 0) {
+          if (atomicExch(&vec_poller[kind], 1) == 0) {
+            ok = counter_wait(fa.ctr + (kind == 0 ? CTR_DONE : CTR_AG_DONE), v.dep_thr, wc, t, 2000) ? 1 : 0;
+            if (ok) mbar_arrive(&vec_ready[kind]);
+          } else {
+            ok = mbar_wait(&vec_ready[kind], 0, wc, SITE_DEP, t, 4000) ? 1 : 0;
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        __syncwarp();
+        if (!ok) break;
+      }
+      if (v.op == VEC_GATHER) {
+        vec_gather(fa, v.idx, lane);
+        __syncwarp();
+        if (lane == 0) counter_signal(fa.ctr + ctr_gather(v.idx / GATHER_SUB), 1);
+      } else if (v.op == VEC_COMBINE) {
+        vec_combine(fa, v.idx, lane);
+      } else if (BWD && v.op == VEC_DW) {
+        vec_dw(fa, v.idx, lane);
+      } else if (BWD && v.op == VEC_ZERO) {
+        vec_zero(fa, v.idx, lane);
+      }
+    }
+  }
+
+}
+
 // ---------------------------------------------------------------- the kernel
 template <bool BWD>
 __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_constant__ FusedArgs fa) {
@@ -489,44 +534,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
   // start, every other warp once its matrix role has reached the end of the matrix queue (the
   // tail of the vector queue -- combine -- then runs on the whole SM)
   __syncwarp();
-  if (!*reinterpret_cast<volatile int*>(&fa.status->abort)) {
-    const int vtotal = vec_total(fa.sp, M);
-    while (true) {
-      int t = 0;
-      if (lane == 0) t = atomicAdd(&fa.ctr[CTR_VEC_TICKET], 1);
-      t = __shfl_sync(0xffffffffu, t, 0);
-      if (t >= vtotal) break;
-      const VecTask v = decode_vector_ticket(fa.sp, t, M);
-      if (v.dep) {
-        // A global completion counter: one warp of the CTA polls it (slowly), the others sleep on a
-        // shared-memory barrier -- a thousand warps spinning on one L2 line would slow every load.
-        const int kind = v.dep == 2 ? 0 : 1;
-        int ok = 1;
-        if (lane == 0) {
-          if (atomicExch(&sh->vec_poller[kind], 1) == 0) {
-            ok = counter_wait(fa.ctr + (kind == 0 ? CTR_DONE : CTR_AG_DONE), v.dep_thr, wc, t, 2000) ? 1 : 0;
-            if (ok) mbar_arrive(&sh->vec_ready[kind]);
-          } else {
-            ok = mbar_wait(&sh->vec_ready[kind], 0, wc, SITE_DEP, t, 4000) ? 1 : 0;
-          }
-        }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        __syncwarp();
-        if (!ok) break;
-      }
-      if (v.op == VEC_GATHER) {
-        vec_gather(fa, v.idx, lane);
-        __syncwarp();
-        if (lane == 0) counter_signal(fa.ctr + ctr_gather(v.idx / GATHER_SUB), 1);
-      } else if (v.op == VEC_COMBINE) {
-        vec_combine(fa, v.idx, lane);
-      } else if (BWD && v.op == VEC_DW) {
-        vec_dw(fa, v.idx, lane);
-      } else if (BWD && v.op == VEC_ZERO) {
-        vec_zero(fa, v.idx, lane);
-      }
-    }
-  }
+  vector_worker_loop<BWD>(fa, sh->vec_ready, sh->vec_poller, wc, M, lane);
 
   // ---------------------------------------------------------------- teardown
   if (*reinterpret_cast<volatile int*>(&fa.status->abort)) __nanosleep(200000);
@@ -536,6 +544,326 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, TMEM_COLS);
   }
+}
+
+// =====================================================================================================
+// The same persistent launch on CTA pairs: a cluster of two CTAs shares every matrix tile
+// (tcgen05 cta_group::2, 256 x 256; see gemm_pair.cuh).  The even CTA owns the scheduler, the MMA
+// issuer and every barrier the MMA issuer waits on; it publishes each tile into the tile rings of
+// both CTAs (the odd CTA's copy over the cluster's shared-memory network).  Loaders and epilogue
+// warps run in both CTAs on their own half of the tile; vector workers are per CTA as before.
+// =====================================================================================================
+constexpr int STAGESP = 6;  // 6 x 32 KB operand stages per CTA
+
+struct __align__(16) PairShared {
+  uint64_t full[STAGESP];      // even CTA: bytes of both CTAs' loads
+  uint64_t empty[STAGESP];     // each CTA: the stage's MMAs are complete (multicast commit)
+  uint64_t tmem_full[2];       // each CTA: accumulator ready (multicast commit)
+  uint64_t tmem_empty[2];      // even CTA: the 8 epilogue warps of the pair have drained it
+  uint64_t drain;
+  uint64_t tk_full[RING];      // each CTA: a tile has been published into this CTA's ring
+  uint64_t tk_empty[RING];     // even CTA: every consumer of both CTAs has read the slot
+  uint64_t sched_go;           // even CTA: loader -> scheduler
+  uint64_t vec_ready[2];
+  int vec_poller[2];
+  uint32_t tmem_base;
+  uint32_t pad;
+  TileSlot ring[RING];
+};
+
+constexpr size_t FUSEDP_SMEM_BYTES = 1024 + (size_t)STAGESP * STAGE2_BYTES + 4 * OUT_STAGE_BYTES + sizeof(PairShared);
+static_assert(FUSEDP_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+constexpr int PAIR_TK_EMPTY_COUNT = (2 + EPI_WARPS) + (1 + EPI_WARPS);  // even: loader, MMA, epilogue; odd: loader, epilogue
+
+template <bool BWD>
+__device__ __forceinline__ void fusedp_load_stage(const FusedArgs& fa, const TileSlot& ts, const Tile& tl, int kb,
+                                                  int rank, uint8_t* sA, uint8_t* sB, uint64_t* bar, int lane) {
+  const GemmArgs& g = fa.op[ts.slot];
+  if (!BWD) {
+    if (ts.op == GEMM_GATE_UP) load_stage_pair_lanes<GEMM_GATE_UP>(g, tl, kb, rank, sA, sB, bar, lane);
+    else load_stage_pair_lanes<GEMM_DOWN>(g, tl, kb, rank, sA, sB, bar, lane);
+  } else {
+    if (ts.op == GEMM_ACT_GRAD) load_stage_pair_lanes<GEMM_ACT_GRAD>(g, tl, kb, rank, sA, sB, bar, lane);
+    else if (ts.op == GEMM_GATE_GRAD) load_stage_pair_lanes<GEMM_GATE_GRAD>(g, tl, kb, rank, sA, sB, bar, lane);
+    else load_stage_pair_lanes<GEMM_WGRAD>(g, tl, kb, rank, sA, sB, bar, lane);
+  }
+}
+template <bool BWD>
+__device__ __forceinline__ void fusedp_mma(int op, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first) {
+  if (!BWD) {
+    mma_kblock_pair<GEMM_GATE_UP>(d_tmem, a_addr, b_addr, first);
+  } else {
+    if (op == GEMM_WGRAD) mma_kblock_pair<GEMM_WGRAD>(d_tmem, a_addr, b_addr, first);
+    else mma_kblock_pair<GEMM_ACT_GRAD>(d_tmem, a_addr, b_addr, first);
+  }
+}
+
+// Publish one tile into the ring slot `rs` of CTA `rank` (through the cluster address space, also for
+// the even CTA itself) and signal that CTA's consumers.
+__device__ __forceinline__ void publish_slot(PairShared* sh, int rs, uint32_t rank, const TileSlot& ts) {
+  const uint32_t dst = map_to_rank(smem_u32(&sh->ring[rs]), rank);
+  const uint4* src = reinterpret_cast<const uint4*>(&ts);
+  static_assert(sizeof(TileSlot) == 48, "TileSlot is published as three 16-byte stores");
+  st_cluster_v4(dst, src[0]);
+  st_cluster_v4(dst + 16, src[1]);
+  st_cluster_v4(dst + 32, src[2]);
+  mbar_arrive_cluster_addr(map_to_rank(smem_u32(&sh->tk_full[rs]), rank));
+}
+
+template <bool BWD>
+__global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __grid_constant__ FusedArgs fa) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem;
+  uint8_t* sB = smem + STAGESP * A_STAGE_BYTES;
+  uint8_t* sOut = smem + STAGESP * STAGE2_BYTES;
+  PairShared* sh = reinterpret_cast<PairShared*>(sOut + 4 * OUT_STAGE_BYTES);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)cluster_ctarank();
+  const WaitCtl wc{fa.status, fa.budget_ns};
+  const int M = fa.lv.meta[0];
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGESP; ++s) {
+      mbar_init(&sh->full[s], 1);
+      mbar_init(&sh->empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sh->tmem_full[s], 1);
+      mbar_init(&sh->tmem_empty[s], 2 * EPI_WARPS);
+      mbar_init(&sh->vec_ready[s], 1);
+      sh->vec_poller[s] = 0;
+    }
+    mbar_init(&sh->drain, 1);
+    for (int s = 0; s < RING; ++s) {
+      mbar_init(&sh->tk_full[s], 1);
+      mbar_init(&sh->tk_empty[s], PAIR_TK_EMPTY_COUNT);
+    }
+    mbar_init(&sh->sched_go, 1);
+    mbar_fence_init();
+    fence_proxy_async();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(&sh->tmem_base, TMEM_COLS);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = sh->tmem_base;
+
+  if (warp == SCHED_WARP && rank == 0) {
+    // ------------------------------------------------ scheduler (even CTA): tickets of the pair
+    if (lane == 0) {
+      const int total = fa.step_start[fa.sp.Ep + fa.sp.lag];
+      uint32_t n = 0, go_n = 0;
+      int cursor = 0;
+      bool ok = true;
+      while (ok) {
+        const int t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
+        TileSlot ts;
+        ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
+        ts.trig_idx = -1; ts.trig_ag = 0; ts.go_kb = -1; ts.pad = 0;
+        if (t >= total) {
+          ts.op = -1;
+          const int rs = n % RING;
+          if (!mbar_wait_cluster(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) break;
+          publish_slot(sh, rs, 0, ts);
+          publish_slot(sh, rs, 1, ts);
+          break;
+        }
+        while (fa.step_start[cursor + 1] <= t) ++cursor;
+        const MatTile mt = decode_matrix_ticket_at(fa.sp, t, cursor, fa.step_start, fa.lv.mb_start);
+        const GemmArgs& g = fa.op[mt.slot];
+        for (int q = 0; q < mt.dep_count && ok; ++q) {
+          const int mbq = mt.dep_first + q;
+          const int* c = fa.ctr + (mt.dep_base == 0 ? ctr_gather(mbq) : ctr_act(mbq));
+          ok = counter_wait(c, mt.dep_thr, wc, t);
+        }
+        if (!ok) break;
+        ts.op = mt.op; ts.slot = mt.slot; ts.e = mt.e;
+        ts.trig_ag = mt.trig_also_ag;
+        const int nkb = mt.op == GEMM_WGRAD ? (fa.lv.counts[mt.e] + BK - 1) / BK : (g.K + BK - 1) / BK;
+        ts.nkb = nkb;
+        for (int gi = 0; gi < mt.group && ok; ++gi) {
+          const int after = (mt.group - 1 - gi) * nkb;
+          ts.go_kb = -1;
+          if (after < SCHED_AHEAD_KB && (after + nkb >= SCHED_AHEAD_KB || gi == 0))
+            ts.go_kb = max(0, nkb - (SCHED_AHEAD_KB - after));
+          const int rs = n % RING;
+          if (!mbar_wait_cluster(&sh->tk_empty[rs], ((n / RING) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {  // the slot as CTA r of the pair sees it
+            TileSlot tr = ts;
+            if (mt.op == GEMM_WGRAD) {
+              tr.nb = gi;
+              tr.m0 = (2 * mt.idx + r) * BLOCK_M;  // this CTA's 128 rows of the 256-row strip
+              tr.n0 = gi * BN;
+              tr.row0 = fa.lv.mb_start[mt.e] * BLOCK_M;
+              tr.pad = tr.m0 >= g.M;               // nothing to store: the strip's second half is outside dW
+              tr.trig_idx = -1;
+            } else {
+              const bool idle = r >= mt.mb_count;
+              tr.nb = mt.idx;
+              tr.m0 = 0;
+              tr.n0 = mt.idx * (mt.op == GEMM_GATE_UP ? BN / 2 : BN);
+              tr.row0 = idle ? g.cap_rows : (mt.mb + r) * BLOCK_M;  // rows beyond the tensor read as zeros
+              tr.pad = idle;
+              tr.trig_idx = idle ? -1 : (mt.trig_base == 1 ? ctr_act(mt.mb + r) : (mt.trig_base == 2 ? CTR_DONE : -1));
+              if (idle) tr.trig_ag = 0;
+            }
+            publish_slot(sh, rs, r, tr);
+          }
+          ++n;
+        }
+        if (!ok || !mbar_wait(&sh->sched_go, go_n & 1, wc, SITE_DEP, t, 200)) break;
+        ++go_n;
+      }
+    }
+  } else if (warp == 0) {
+    // ------------------------------------------------ loader (both CTAs): own rows of A, own half of B
+    uint32_t it = 0, n = 0;
+    bool ok = true;
+    while (ok) {
+      const int rs = n % RING;
+      if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -3)) break;
+      const TileSlot ts = sh->ring[rs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(&sh->tk_empty[rs]);
+      ++n;
+      if (ts.op < 0) break;
+      fence_proxy_async();
+      const Tile tl = slot_tile(ts);
+      for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
+        if (kb == ts.go_kb && lane == 0 && rank == 0) mbar_arrive(&sh->sched_go);
+        const int s = it % STAGESP;
+        if (!mbar_wait(&sh->empty[s], ((it / STAGESP) & 1) ^ 1, wc, SITE_EMPTY, n)) { ok = false; break; }
+        fusedp_load_stage<BWD>(fa, ts, tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s], lane);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer (even CTA)
+    if (lane == 0 && rank == 0) {
+      uint32_t it = 0, acc_it = 0, n = 0;
+      bool ok = true;
+      while (ok) {
+        const int rs = n % RING;
+        if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -1)) break;
+        const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb;
+        mbar_arrive(&sh->tk_empty[rs]);
+        ++n;
+        if (op < 0) break;
+        if (nkb == 0) continue;
+        const int as = acc_it & 1;
+        if (!mbar_wait_cluster(&sh->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, n)) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + as * BN;
+        for (int kb = 0; kb < nkb; ++kb, ++it) {
+          const int s = it % STAGESP;
+          if (!mbar_wait(&sh->full[s], (it / STAGESP) & 1, wc, SITE_FULL, n)) { ok = false; break; }
+          tc_fence_after_sync();
+          fusedp_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0);
+          tc_commit_pair(&sh->empty[s]);
+        }
+        if (!ok) break;
+        tc_commit_pair(&sh->tmem_full[as]);
+        ++acc_it;
+      }
+      if (*reinterpret_cast<volatile int*>(&fa.status->abort)) {
+        tc_commit_pair(&sh->drain);
+        const WaitCtl shortwc{fa.status, 20ull * 1000 * 1000};
+        mbar_wait(&sh->drain, 0, shortwc, SITE_DRAIN, 0);
+      }
+    }
+  } else if (warp < 2 + EPI_WARPS) {
+    // ------------------------------------------------ epilogue warps (both CTAs, own rows)
+    const int quad = warp & 3;
+    Staging stg{sOut + quad * OUT_STAGE_BYTES, 1, 0};
+    uint32_t acc_it = 0, n = 0;
+    while (true) {
+      const int rs = n % RING;
+      if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -2, 100)) break;
+      const TileSlot ts = sh->ring[rs];
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(&sh->tk_empty[rs]);
+      ++n;
+      if (ts.op < 0) break;
+      const Tile tl = slot_tile(ts);
+      const bool idle = ts.pad != 0;
+      if (ts.nkb != 0) {
+        const int as = acc_it & 1;
+        if (!mbar_wait(&sh->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, n, 100)) break;
+        tc_fence_after_sync();
+        if (!idle) fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_leader(&sh->tmem_empty[as]);
+        ++acc_it;
+      }
+      if (ts.trig_idx >= 0) {
+        __syncwarp();
+        if (lane == 0) {
+          tma_store_wait_all();
+          fence_proxy_async();
+          counter_signal(fa.ctr + ts.trig_idx, 1);
+          if (ts.trig_ag) counter_signal(fa.ctr + CTR_AG_DONE, 1);
+        }
+        __syncwarp();
+      }
+    }
+    if (lane == 0) tma_store_wait_all();
+  }
+
+  // ------------------------------------------------ vector workers (per CTA, as in the single-CTA kernel)
+  __syncwarp();
+  vector_worker_loop<BWD>(fa, sh->vec_ready, sh->vec_poller, wc, M, lane);
+
+  // ---------------------------------------------------------------- teardown
+  if (*reinterpret_cast<volatile int*>(&fa.status->abort)) __nanosleep(200000);
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA leaves while its partner may still read its shared memory or signal it
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
+template <bool BWD>
+static cudaError_t launch_fused_pair_t(const FusedArgs& fa, int num_sms, cudaStream_t s) {
+  static bool attr_set = false;
+  static int max_pairs = 0;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(fused_pair_kernel<BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)FUSEDP_SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof cfg);
+  cfg.gridDim = dim3((num_sms / 2) * 2);
+  cfg.blockDim = dim3(FUSED_THREADS);
+  cfg.dynamicSmemBytes = FUSEDP_SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;  // the launch fails rather than run with CTAs that are not all resident
+  attr[1].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  if (max_pairs == 0) {
+    int n = 0;
+    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, fused_pair_kernel<BWD>, &cfg);
+    if (e != cudaSuccess) return e;
+    max_pairs = n > 0 ? n : 1;
+  }
+  if (2 * max_pairs < (int)cfg.gridDim.x) cfg.gridDim = dim3(2 * max_pairs);
+  return cudaLaunchKernelEx(&cfg, fused_pair_kernel<BWD>, fa);
 }
 
 // ---------------------------------------------------------------- host side
@@ -563,6 +891,7 @@ static cudaError_t launch_fused_t(const FusedArgs& fa, int num_sms, cudaStream_t
 
 cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, cudaStream_t s, int* launches) {
   ++*launches;
+  if (fa.sp.pair) return bwd ? launch_fused_pair_t<true>(fa, num_sms, s) : launch_fused_pair_t<false>(fa, num_sms, s);
   return bwd ? launch_fused_t<true>(fa, num_sms, s) : launch_fused_t<false>(fa, num_sms, s);
 }
 

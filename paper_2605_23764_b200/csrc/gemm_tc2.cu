@@ -16,14 +16,12 @@
 #include <stdio.h>
 #include <stdlib.h>
 
-#include "gemm_tile.cuh"
+#include "gemm_pair.cuh"
 
 namespace moe {
 
 constexpr int STAGES2 = 5;                                       // 5 x 32 KB operand stages ...
 constexpr int OUT_BUFS2 = 2;                                     // ... and double-buffered epilogue staging
-constexpr int HALF_B_BYTES = B_STAGE_BYTES / 2;                 // 16 KB: this CTA's half of the B tile
-constexpr int STAGE2_BYTES = A_STAGE_BYTES + HALF_B_BYTES;      // 32 KB
 
 struct __align__(8) PairBarriers {
   uint64_t full[STAGES2];     // used in the even CTA: bytes of both CTAs' loads
@@ -84,49 +82,6 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmArgs& a, int t, i
     tl.nkb = (a.K + BK - 1) / BK;
   }
   return pt;
-}
-
-// This CTA's loads of one k-block: its 128 rows of A and its half of B.  Completion bytes go to the
-// even CTA's barrier.
-template <int MODE>
-__device__ __forceinline__ void load_stage_pair(const GemmArgs& a, const Tile& tl, int kb, int rank, uint8_t* sA,
-                                                uint8_t* sB, uint64_t* bar) {
-  const int k0 = kb * BK;
-  if (MODE == GEMM_WGRAD) {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) tma_load_2d_pair(sA + j * MN_BOX_BYTES, &a.tmA, tl.m0 + j * 64, tl.row0 + k0, bar);
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-      tma_load_2d_pair(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + (2 * rank + j) * 64, tl.row0 + k0, bar);
-    return;
-  }
-  tma_load_2d_pair(sA, &a.tmA, k0, tl.row0, bar);
-  const int brow = tl.e * a.b_rows_per_expert;
-  if (MODE == GEMM_GATE_UP) {
-    // accumulator columns 0..127 = gate (even CTA's half of B), 128..255 = up (odd CTA's half)
-    tma_load_2d_pair(sB, &a.tmB, k0, brow + rank * a.F + tl.n0, bar);
-  } else if (MODE == GEMM_DOWN) {
-    tma_load_2d_pair(sB, &a.tmB, k0, brow + tl.n0 + rank * (BN / 2), bar);
-  } else {
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-      tma_load_2d_pair(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + (2 * rank + j) * 64, brow + k0, bar);
-  }
-}
-
-template <int MODE>
-__device__ __forceinline__ void mma_kblock_pair(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first_kblock) {
-  constexpr bool A_MN = (MODE == GEMM_WGRAD);
-  constexpr bool B_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD || MODE == GEMM_WGRAD);
-  constexpr uint32_t idesc = make_idesc_bf16(2 * BLOCK_M, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
-#pragma unroll
-  for (int k16 = 0; k16 < BK / 16; ++k16) {
-    const uint64_t da = A_MN ? make_smem_desc(a_addr + k16 * 2048, MN_BOX_BYTES, 1024)
-                             : make_smem_desc(a_addr + k16 * 32, 16, 1024);
-    const uint64_t db = B_MN ? make_smem_desc(b_addr + k16 * 2048, MN_BOX_BYTES, 1024)
-                             : make_smem_desc(b_addr + k16 * 32, 16, 1024);
-    tc_mma_bf16_pair(d_tmem, da, db, idesc, !(first_kblock && k16 == 0));
-  }
 }
 
 template <int MODE>

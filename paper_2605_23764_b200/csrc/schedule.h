@@ -40,6 +40,7 @@ enum VecOp : int { VEC_GATHER = 0, VEC_ZERO = 1, VEC_DW = 2, VEC_COMBINE = 3, VE
 
 struct SchedParams {
   int is_bwd;
+  int pair;                // 1: a row-space ticket covers a PAIR of M-blocks (two CTAs on a 256-row tile)
   int lag;                 // in experts
   int Ep;
   int T, k;
@@ -52,18 +53,23 @@ struct SchedParams {
 };
 
 MOE_HD int expert_mblocks(const int* mb_start, int e) { return mb_start[e + 1] - mb_start[e]; }
+// row-space scheduling units of an expert: its M-blocks, or its M-block pairs
+MOE_HD int expert_units(const SchedParams& sp, const int* mb_start, int e) {
+  const int m = expert_mblocks(mb_start, e);
+  return sp.pair ? (m + 1) >> 1 : m;
+}
 
 // tickets of step i
 MOE_HD int step_tiles(const SchedParams& sp, int i, const int* mb_start) {
   int n = 0;
   const int j = i - sp.lag;
   if (i < sp.Ep) {
-    const int m = expert_mblocks(mb_start, i);
+    const int m = expert_units(sp, mb_start, i);
     n += m * sp.seg_tiles[0];
     if (sp.is_bwd && m > 0) n += sp.seg_tiles[1];
   }
   if (j >= 0 && j < sp.Ep) {
-    const int m = expert_mblocks(mb_start, j);
+    const int m = expert_units(sp, mb_start, j);
     if (!sp.is_bwd) {
       n += m * sp.seg_tiles[1];
     } else {
@@ -78,7 +84,8 @@ struct MatTile {
   int op;        // GemmMode
   int slot;      // which GemmArgs of the launch (segment index)
   int e;
-  int mb;        // M-block (row-space operators) or -1
+  int mb;        // first M-block of the tile (row-space operators) or -1
+  int mb_count;  // M-blocks of the tile: 1, or 2 for a full pair
   int idx;       // column tile (row-space operators) / strip index = 128-row block of the gradient
   int group;     // tiles processed under this ticket (1, or the strip's column tiles)
   // dependency: every counter dep_ctr[dep_first .. dep_first+dep_count) must reach dep_thr
@@ -97,16 +104,20 @@ MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, cons
   MatTile m;
   m.trig_also_ag = 0;
   m.group = 1;
+  m.mb_count = 0;
+  const int stride = sp.pair ? 2 : 1;  // M-blocks per row-space unit
   if (i < sp.Ep) {
-    const int mc = expert_mblocks(mb_start, i);
-    if (r < mc * sp.seg_tiles[0]) {
+    const int uc = expert_units(sp, mb_start, i), mc = expert_mblocks(mb_start, i);
+    if (r < uc * sp.seg_tiles[0]) {
       m.slot = 0; m.op = sp.is_bwd ? 2 /*ACT_GRAD*/ : 0 /*GATE_UP*/;
-      m.idx = r / mc; m.mb = mb_start[i] + (r - m.idx * mc); m.e = i;
-      m.dep_base = 0; m.dep_first = m.mb; m.dep_count = 1; m.dep_thr = GATHER_SUB;
+      m.idx = r / uc;
+      const int u = r - m.idx * uc;
+      m.mb = mb_start[i] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride; m.e = i;
+      m.dep_base = 0; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = GATHER_SUB;
       m.trig_base = 1; m.trig_also_ag = sp.is_bwd;
       return m;
     }
-    r -= mc * sp.seg_tiles[0];
+    r -= uc * sp.seg_tiles[0];
     if (sp.is_bwd && mc > 0) {
       if (r < sp.seg_tiles[1]) {
         m.slot = 1; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = i; m.idx = r; m.group = sp.strip_tiles[0];
@@ -118,22 +129,18 @@ MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, cons
     }
   }
   // lagged segments of expert j
-  const int mc = expert_mblocks(mb_start, j);
-  if (!sp.is_bwd) {
-    m.slot = 1; m.op = 1 /*DOWN*/; m.e = j;
-    m.idx = r / mc; m.mb = mb_start[j] + (r - m.idx * mc);
-    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
+  const int uc = expert_units(sp, mb_start, j), mc = expert_mblocks(mb_start, j);
+  if (!sp.is_bwd || r < uc * sp.seg_tiles[2]) {
+    const int seg = sp.is_bwd ? 2 : 1;
+    m.slot = seg; m.op = sp.is_bwd ? 3 /*GATE_GRAD*/ : 1 /*DOWN*/; m.e = j;
+    m.idx = r / uc;
+    const int u = r - m.idx * uc;
+    m.mb = mb_start[j] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride;
+    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
     m.trig_base = 2;
     return m;
   }
-  if (r < mc * sp.seg_tiles[2]) {
-    m.slot = 2; m.op = 3 /*GATE_GRAD*/; m.e = j;
-    m.idx = r / mc; m.mb = mb_start[j] + (r - m.idx * mc);
-    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = 1; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
-    m.trig_base = 2;
-    return m;
-  }
-  r -= mc * sp.seg_tiles[2];
+  r -= uc * sp.seg_tiles[2];
   m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = j; m.idx = r; m.group = sp.strip_tiles[1];
   m.dep_base = 1; m.dep_first = mb_start[j]; m.dep_count = mc;
   m.dep_thr = EPI_WARPS * sp.seg_tiles[0]; m.trig_base = -1;

@@ -17,10 +17,11 @@ def _seg(is_bwd, d, F):
     return [(F + 255) // 256, (d + 127) // 128, (d + 255) // 256, (2 * F + 127) // 128]
 
 
+@pytest.mark.parametrize("pair", [False, True])
 @pytest.mark.parametrize("is_bwd", [0, 1])
 @pytest.mark.parametrize("workers", [(1, 1), (3, 2), (148, 592)])
 @pytest.mark.parametrize("lag", [0, 1, 8])
-def test_schedule_is_sound(is_bwd, workers, lag):
+def test_schedule_is_sound(is_bwd, workers, lag, pair):
     rng = np.random.default_rng(lag * 7 + is_bwd)
     cases = [
         rng.integers(0, 700, 24),                      # mixed sizes
@@ -31,9 +32,11 @@ def test_schedule_is_sound(is_bwd, workers, lag):
     ]
     for counts in cases:
         T = max(1, int(counts.sum()) // 2)
-        rc, stats = binding.moe_debug_simulate_schedule(counts, T, 2, is_bwd, _seg(is_bwd, 520, 264), lag, *workers)
+        rc, stats = binding.moe_debug_simulate_schedule(counts, T, 2, is_bwd, _seg(is_bwd, 520, 264), lag, *workers,
+                                                        pair=pair)
         assert rc == 0, (counts.tolist(), rc)
-        M = int(((counts + 127) // 128).sum())
+        mblocks = (counts + 127) // 128
+        M = int(((mblocks + 1) // 2).sum()) if pair else int(mblocks.sum())
         seg = _seg(is_bwd, 520, 264)
         want = M * (seg[0] + (seg[2] if is_bwd else seg[1]))
         if is_bwd:
@@ -46,5 +49,7 @@ def test_training_config_schedule():
     rng = np.random.default_rng(4)
     counts = rng.binomial(65536, 1 / 256, 256)
     for is_bwd in (0, 1):
-        rc, stats = binding.moe_debug_simulate_schedule(counts, 8192, 8, is_bwd, _seg(is_bwd, 7168, 2048), 8, 148, 592)
-        assert rc == 0
+        for pair in (False, True):
+            rc, stats = binding.moe_debug_simulate_schedule(counts, 8192, 8, is_bwd, _seg(is_bwd, 7168, 2048), 8, 148,
+                                                            592, pair=pair)
+            assert rc == 0
