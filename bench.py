@@ -147,13 +147,21 @@ def barrier(world):
     torch.cuda.synchronize()
 
 
-def max_over_ranks(v, world):
+def max_over_ranks(v, world, device="cuda"):
+    """The slowest rank's time: replicas are independent, the job is as slow as its slowest one."""
     if world == 1:
         return v
     import torch.distributed as dist
-    t = torch.tensor([v], dtype=torch.float64, device="cuda")
+    t = torch.tensor([v], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def replica_throughput(local_ms_per_step, flops_per_replica_step, world, device="cuda"):
+    """Whole-job TFLOP/s of `world` independent replicas (weak scaling): all ranks' work over the
+    slowest rank's time."""
+    ms = max_over_ranks(local_ms_per_step, world, device)
+    return world * flops_per_replica_step / (ms * 1e-3) / 1e12, ms
 
 
 # ----------------------------------------------------------------------------------------------
@@ -341,12 +349,13 @@ def main():
         ev1.record()
         barrier(world)
         clk = sampler.stop()
-        elapsed = max_over_ranks(ev0.elapsed_time(ev1) - flush_ms, world)
+        local_ms = (ev0.elapsed_time(ev1) - flush_ms) / args.steps
+        value_all, ms = replica_throughput(local_ms, step_flops(cfg, train), world)
+        elapsed = ms * args.steps
         B.moe_set_profiling(lay.ctx, False)
         code, detail = lay.status()
         assert code == 0, f"device-side error {code} detail {detail:#x}"
-        ms = elapsed / args.steps
-        return {"ms_per_step": ms, "value": world * step_flops(cfg, train) / (ms * 1e-3) / 1e12,
+        return {"ms_per_step": ms, "value": value_all,
                 "phases_ms": {k: v / args.steps for k, v in phase_sum.items()}, "launches": n_launch, "clocks": clk,
                 "timed_ms": elapsed}
 

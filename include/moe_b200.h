@@ -190,6 +190,12 @@ enum {
 };
 int moe_debug_buffer(moe_ctx* ctx, int which, void** ptr, size_t* elems);
 
+/* Failure-handling test hook: with on != 0 the persistent launches of this context wait for one more
+ * producer signal than will ever arrive (a threshold nothing reaches).  The bounded waits then run
+ * out after the wait budget, the kernel records MOE_ERR_TIMEOUT and returns normally (no trap, no
+ * hang); moe_get_status reports it and the context stays usable once the hook is switched off. */
+int moe_debug_set_unreachable_dependency(moe_ctx* ctx, int32_t on);
+
 /* Host-only check of the static tile schedule of the single persistent launch (Section 4.3: tasks
  * ordered in static queues, dependent/trigger event counters with static thresholds).  For the
  * given per-expert row counts[Ep] it builds the matrix and vector queues, verifies that every tile

@@ -21,7 +21,7 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
            "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
-           "moe_debug_simulate_schedule"]
+           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -71,6 +71,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_route_host.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.moe_layout_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, vp]
+    lib.moe_debug_set_unreachable_dependency.argtypes = [vp, i32]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -231,6 +232,11 @@ def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_worker
     rc = load_library().moe_debug_simulate_schedule(c, len(counts), T, k, int(is_bwd), seg, lag, mat_workers,
                                                     vec_workers, int(bool(pair)), stats)
     return rc, list(stats)
+
+
+def moe_debug_set_unreachable_dependency(ctx, on: bool):
+    _check(load_library().moe_debug_set_unreachable_dependency(ctx, 1 if on else 0),
+           "moe_debug_set_unreachable_dependency")
 
 
 class _DevView:

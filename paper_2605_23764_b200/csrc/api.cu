@@ -174,6 +174,7 @@ struct moe_ctx {
   int launches = 0;
   int saved_T = -1;  // T of the forward whose tensors are in the workspace (-1: none)
   uint64_t budget_ns = 2000ull * 1000 * 1000;
+  int dep_extra = 0;  // test hook: makes the activation dependencies of the persistent launch unreachable
   int sched_lag = 0;  // experts between a producer step and its consumer step; 0 = choose from the shape
   cudaStream_t last_stream = nullptr;
   // optional per-operator timing
@@ -386,6 +387,7 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
   memset(&sp, 0, sizeof sp);
   sp.is_bwd = bwd ? 1 : 0;
   sp.pair = single_cta_gemm() ? 0 : 1;
+  sp.dep_extra = c->dep_extra;
   sp.Ep = s.E + s.n_shared;
   sp.T = T;
   sp.k = s.k;
@@ -803,6 +805,12 @@ int moe_get_phase_ms(moe_ctx* c, float* ms) {
       MOE_CUDA(cudaEventElapsedTime(&ms[i], c->ev_start[i], c->ev_stop[i]));
     }
   }
+  return MOE_OK;
+}
+
+int moe_debug_set_unreachable_dependency(moe_ctx* c, int32_t on) {
+  if (!c) return MOE_ERR_INVALID_ARG;
+  c->dep_extra = on ? 1 : 0;
   return MOE_OK;
 }
 

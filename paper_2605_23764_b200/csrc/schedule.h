@@ -50,6 +50,7 @@ struct SchedParams {
   //             seg2 = gate_grad (per M-block, lagged), seg3 = w1_grad strips (per expert, lagged)
   int seg_tiles[SCHED_MAX_SEG];
   int strip_tiles[2];      // column tiles in one w2_grad / w1_grad strip
+  int dep_extra;           // test hook: added to the activation-counter thresholds (> 0 = never reached)
 };
 
 MOE_HD int expert_mblocks(const int* mb_start, int e) { return mb_start[e + 1] - mb_start[e]; }
@@ -136,14 +137,14 @@ MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, cons
     m.idx = r / uc;
     const int u = r - m.idx * uc;
     m.mb = mb_start[j] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride;
-    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = EPI_WARPS * sp.seg_tiles[0];
+    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = EPI_WARPS * sp.seg_tiles[0] + sp.dep_extra;
     m.trig_base = 2;
     return m;
   }
   r -= uc * sp.seg_tiles[2];
   m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = j; m.idx = r; m.group = sp.strip_tiles[1];
   m.dep_base = 1; m.dep_first = mb_start[j]; m.dep_count = mc;
-  m.dep_thr = EPI_WARPS * sp.seg_tiles[0]; m.trig_base = -1;
+  m.dep_thr = EPI_WARPS * sp.seg_tiles[0] + sp.dep_extra; m.trig_base = -1;
   return m;
 }
 

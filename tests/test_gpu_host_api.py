@@ -1,0 +1,53 @@
+"""The host-buffer entry points (pinned host activations in, host results out) and the per-operator
+timing calls give the same results as the device-buffer calls."""
+import pytest
+import torch
+
+from paper_2605_23764_b200 import MoeLayer, binding as B
+from tests.gpu_util import small_problem
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_host_buffer_calls_match_device_calls(serial):
+    T, d, E, k, S, F = 333, 192, 12, 3, 1, 160
+    x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, 21)
+    layer = MoeLayer(T, d, E, k, S, F, renorm=True, save_for_bwd=True, serial=serial)
+    ids, w = layer.route(logits)
+    out = layer.ffn_fwd(x, ids, w, W1, W2)
+    dx, dW1, dW2, dw = layer.ffn_bwd(dout, x, ids, w, W1, W2)
+    torch.cuda.synchronize()
+
+    pin = dict(pin_memory=True)
+    lh, xh, doh = logits.cpu().pin_memory(), x.cpu().pin_memory(), dout.cpu().pin_memory()
+    idh = torch.empty(T, k, dtype=torch.int32, **pin)
+    wh = torch.empty(T, k, dtype=torch.float32, **pin)
+    oh = torch.empty(T, d, dtype=torch.bfloat16, **pin)
+    dxh = torch.empty(T, d, dtype=torch.bfloat16, **pin)
+    dwh = torch.empty(T, k, dtype=torch.float32, **pin)
+    dW1b, dW2b = torch.empty_like(W1), torch.empty_like(W2)
+    B.moe_route_host(layer.ctx, lh, T, idh, wh)
+    B.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, W1, W2, oh, T)
+    B.moe_ffn_bwd_host(layer.ctx, doh, W1, W2, dxh, dW1b, dW2b, dwh, T)
+    torch.cuda.synchronize()
+    assert layer.status() == (0, 0)
+    assert torch.equal(idh, ids.cpu()) and torch.equal(wh, w.cpu())
+    assert torch.equal(oh, out.cpu()) and torch.equal(dxh, dx.cpu()) and torch.equal(dwh, dw.cpu())
+    assert torch.equal(dW1b, dW1) and torch.equal(dW2b, dW2)
+    layer.close()
+
+
+def test_phase_times_are_reported_per_operator():
+    T, d, E, k, S, F = 512, 256, 8, 2, 0, 256
+    x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, 5)
+    for serial, want in ((True, {"layout", "gather", "gemm_gate_up", "gemm_down", "combine"}),
+                         (False, {"layout", "fused_fwd"})):
+        layer = MoeLayer(T, d, E, k, S, F, serial=serial)
+        ids, w = layer.route(logits)
+        B.moe_set_profiling(layer.ctx, True)
+        layer.ffn_fwd(x, ids, w, W1, W2)
+        ph = B.moe_get_phase_ms(layer.ctx)
+        assert set(ph) == want and all(v > 0 for v in ph.values())
+        assert layer.launches() == (7 if serial else 5)
+        layer.close()
