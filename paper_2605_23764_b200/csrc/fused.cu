@@ -49,8 +49,9 @@ struct TileSlot {
   int op, slot, e, row0, n0, m0, nkb, nb;
   int trig_idx;   // counter index to bump per epilogue warp, -1 = none
   int trig_ag;    // also bump the global act_grad counter
-  int go_kb;      // k-block at which the loader tells the scheduler to fetch the next ticket (-1: not in this tile)
-  int pad;
+  short go_kb;    // k-block at which the loader tells the scheduler to fetch the next ticket (-1: not in this tile)
+  short pad;      // CTA-pair kernel: this CTA's half of the tile is idle (no rows / outside the gradient)
+  int krows;      // weight gradients: rows of the expert (the reduction length)
 };
 
 struct __align__(16) FusedShared {
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
         const int t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
         TileSlot ts;
         ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
-        ts.trig_idx = -1; ts.trig_ag = 0; ts.go_kb = -1;
+        ts.trig_idx = -1; ts.trig_ag = 0; ts.go_kb = -1; ts.pad = 0; ts.krows = 0;
         if (t >= total) {
           ts.op = -1;  // end of the queue: tell the other roles
           const int rs = n % RING;
@@ -402,6 +403,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
             ts.row0 = mt.mb * BLOCK_M;
           }
           ts.nkb = nkb;
+          ts.krows = mt.op == GEMM_WGRAD ? fa.lv.counts[mt.e] : 0;
           // the k-block of this tile at which SCHED_AHEAD_KB k-blocks of the ticket remain
           const int after = (mt.group - 1 - gi) * nkb;
           ts.go_kb = -1;
@@ -589,11 +591,12 @@ __device__ __forceinline__ void fusedp_load_stage(const FusedArgs& fa, const Til
   }
 }
 template <bool BWD>
-__device__ __forceinline__ void fusedp_mma(int op, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first) {
+__device__ __forceinline__ void fusedp_mma(int op, uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first,
+                                           int k16_steps) {
   if (!BWD) {
     mma_kblock_pair<GEMM_GATE_UP>(d_tmem, a_addr, b_addr, first);
   } else {
-    if (op == GEMM_WGRAD) mma_kblock_pair<GEMM_WGRAD>(d_tmem, a_addr, b_addr, first);
+    if (op == GEMM_WGRAD) mma_kblock_pair<GEMM_WGRAD>(d_tmem, a_addr, b_addr, first, k16_steps);
     else mma_kblock_pair<GEMM_ACT_GRAD>(d_tmem, a_addr, b_addr, first);
   }
 }
@@ -665,7 +668,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         const int t = atomicAdd(&fa.ctr[CTR_MAT_TICKET], 1);
         TileSlot ts;
         ts.slot = 0; ts.e = 0; ts.row0 = 0; ts.n0 = 0; ts.m0 = 0; ts.nkb = 0; ts.nb = 0;
-        ts.trig_idx = -1; ts.trig_ag = 0; ts.go_kb = -1; ts.pad = 0;
+        ts.trig_idx = -1; ts.trig_ag = 0; ts.go_kb = -1; ts.pad = 0; ts.krows = 0;
         if (t >= total) {
           ts.op = -1;
           const int rs = n % RING;
@@ -687,6 +690,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         ts.trig_ag = mt.trig_also_ag;
         const int nkb = mt.op == GEMM_WGRAD ? (fa.lv.counts[mt.e] + BK - 1) / BK : (g.K + BK - 1) / BK;
         ts.nkb = nkb;
+        ts.krows = mt.op == GEMM_WGRAD ? fa.lv.counts[mt.e] : 0;
         for (int gi = 0; gi < mt.group && ok; ++gi) {
           const int after = (mt.group - 1 - gi) * nkb;
           ts.go_kb = -1;
@@ -751,7 +755,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
       while (ok) {
         const int rs = n % RING;
         if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -1)) break;
-        const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb;
+        const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb, krows = sh->ring[rs].krows;
         mbar_arrive(&sh->tk_empty[rs]);
         ++n;
         if (op < 0) break;
@@ -764,7 +768,8 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
           const int s = it % STAGESP;
           if (!mbar_wait(&sh->full[s], (it / STAGESP) & 1, wc, SITE_FULL, n)) { ok = false; break; }
           tc_fence_after_sync();
-          fusedp_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0);
+          fusedp_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0,
+                          op == GEMM_WGRAD ? k16_steps_of(krows, kb) : BK / 16);
           tc_commit_pair(&sh->empty[s]);
         }
         if (!ok) break;

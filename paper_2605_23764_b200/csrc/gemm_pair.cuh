@@ -38,8 +38,15 @@ __device__ __forceinline__ void load_stage_pair(const GemmArgs& a, const Tile& t
   }
 }
 
+// 16-row MMA steps needed in k-block kb of a reduction over `rows` rows
+__device__ __forceinline__ int k16_steps_of(int rows, int kb) {
+  const int left = rows - kb * BK;
+  return left >= BK ? BK / 16 : (left + 15) / 16;
+}
+
 template <int MODE>
-__device__ __forceinline__ void mma_kblock_pair(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first_kblock) {
+__device__ __forceinline__ void mma_kblock_pair(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first_kblock,
+                                                int k16_steps = BK / 16) {
   constexpr bool A_MN = (MODE == GEMM_WGRAD);
   constexpr bool B_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD || MODE == GEMM_WGRAD);
   constexpr uint32_t idesc = make_idesc_bf16(2 * BLOCK_M, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
@@ -49,7 +56,9 @@ __device__ __forceinline__ void mma_kblock_pair(uint32_t d_tmem, uint32_t a_addr
                              : make_smem_desc(a_addr + k16 * 32, 16, 1024);
     const uint64_t db = B_MN ? make_smem_desc(b_addr + k16 * 2048, MN_BOX_BYTES, 1024)
                              : make_smem_desc(b_addr + k16 * 32, 16, 1024);
-    tc_mma_bf16_pair(d_tmem, da, db, idesc, !(first_kblock && k16 == 0));
+    // the last k-block of a weight gradient may hold fewer than 64 rows of the expert: the 16-row
+    // steps that would only multiply zero padding are not issued
+    if (k16 < k16_steps) tc_mma_bf16_pair(d_tmem, da, db, idesc, !(first_kblock && k16 == 0));
   }
 }
 

@@ -156,7 +156,8 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
           const int s = it % STAGES2;
           if (!mbar_wait(&bars->full[s], (it / STAGES2) & 1, wc, SITE_FULL, t)) { ok = false; break; }
           tc_fence_after_sync();
-          mma_kblock_pair<MODE>(d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0);
+          mma_kblock_pair<MODE>(d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0,
+                                MODE == GEMM_WGRAD ? k16_steps_of(a.counts[pt.tl.e], kb) : BK / 16);
           tc_commit_pair(&bars->empty[s]);   // frees the stage in both CTAs
         }
         if (!ok) break;

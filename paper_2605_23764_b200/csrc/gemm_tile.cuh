@@ -290,19 +290,21 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
       if (MODE == GEMM_WGRAD && y0 >= a.M) break;
       box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
 #pragma unroll
-      for (int c = 0; c < 128; c += 32) {
-        float v[32];
+      for (int c = 0; c < 128; c += 64) {
+        // 64 columns per TMEM round trip (one wait per box): fewer round trips keep this epilogue
+        // shorter than the four-or-five-k-block main loop of a weight-gradient tile
+        float v[64];
         if (MODE == GEMM_WGRAD && tl.nkb == 0) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) v[i] = 0.f;
+          for (int i = 0; i < 64; ++i) v[i] = 0.f;
         } else {
-          tmem_ld16(trow + c0 + c, v);
-          tmem_ld16(trow + c0 + c + 16, v + 16);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) tmem_ld16(trow + c0 + c + 16 * q, v + 16 * q);
           tmem_ld_wait();
         }
         uint8_t* box = (c < 64) ? box0 : box1;
 #pragma unroll
-        for (int h = 0; h < 32; h += 8) stage8(box, lane, ((c & 63) + h) >> 3, v + h);
+        for (int h = 0; h < 64; h += 8) stage8(box, lane, h >> 3, v + h);
       }
       staging_release();
       if (lane == 0) {
