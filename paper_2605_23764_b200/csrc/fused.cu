@@ -743,7 +743,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
       for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
         if (kb == ts.go_kb && lane == 0 && rank == 0) mbar_arrive(&sh->sched_go);
         const int s = it % STAGESP;
-        if (!mbar_wait(&sh->empty[s], ((it / STAGESP) & 1) ^ 1, wc, SITE_EMPTY, n)) { ok = false; break; }
+        if (!mbar_wait(&sh->empty[s], ((it / STAGESP) & 1) ^ 1, wc, SITE_EMPTY, n, 50)) { ok = false; break; }
         fusedp_load_stage<BWD>(fa, ts, tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s], lane);
       }
     }
@@ -752,9 +752,12 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
     if (lane == 0 && rank == 0) {
       uint32_t it = 0, acc_it = 0, n = 0;
       bool ok = true;
+      ST_DECL;
       while (ok) {
         const int rs = n % RING;
+        ST_MARK();
         if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -1)) break;
+        ST_ADD(0);  // waiting for a published tile
         const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb, krows = sh->ring[rs].krows;
         mbar_arrive(&sh->tk_empty[rs]);
         ++n;
@@ -762,20 +765,24 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         if (nkb == 0) continue;
         const int as = acc_it & 1;
         if (!mbar_wait_cluster(&sh->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, n)) break;
+        ST_ADD(1);  // accumulator not yet drained by the epilogues
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + as * BN;
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGESP;
           if (!mbar_wait(&sh->full[s], (it / STAGESP) & 1, wc, SITE_FULL, n)) { ok = false; break; }
+          ST_ADD(2);  // operands not yet in shared memory
           tc_fence_after_sync();
           fusedp_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0,
                           op == GEMM_WGRAD ? k16_steps_of(krows, kb) : BK / 16);
           tc_commit_pair(&sh->empty[s]);
+          ST_ADD(op == GEMM_WGRAD ? 4 : 3);  // issue (includes back-pressure of the tensor pipe)
         }
         if (!ok) break;
         tc_commit_pair(&sh->tmem_full[as]);
         ++acc_it;
       }
+      ST_FLUSH(8, 5);
       if (*reinterpret_cast<volatile int*>(&fa.status->abort)) {
         tc_commit_pair(&sh->drain);
         const WaitCtl shortwc{fa.status, 20ull * 1000 * 1000};

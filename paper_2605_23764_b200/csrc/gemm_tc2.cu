@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
         const PairTile pt = decode_pair_tile<MODE>(a, t, rank);
         for (int kb = 0; kb < pt.tl.nkb; ++kb, ++it) {
           const int s = it % STAGES2;
-          if (!mbar_wait(&bars->empty[s], ((it / STAGES2) & 1) ^ 1, wc, SITE_EMPTY, t)) { ok = false; break; }
+          if (!mbar_wait(&bars->empty[s], ((it / STAGES2) & 1) ^ 1, wc, SITE_EMPTY, t, 50)) { ok = false; break; }
           if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * STAGE2_BYTES);  // the bytes of both CTAs
           load_stage_pair<MODE>(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s]);
         }
@@ -182,7 +182,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
         continue;
       }
       const int as = acc_it & 1;
-      if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, t)) break;
+      if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, t, 200)) break;  // back off: idle epilogue warps must not take issue slots and power
       tc_fence_after_sync();
       if (!pt.idle) epilogue_tile<MODE>(a, pt.tl, tmem_base + as * BN, quad, lane, stg);
       tc_fence_before_sync();
