@@ -46,18 +46,19 @@ EncodeTiledFn get_encode_fn() {
 // bf16 tensor of `rank` dimensions (dims[0] innermost, strides in bytes for dims 1..), 128-byte
 // swizzle, zero fill outside the tensor on loads, clipping on stores.
 int encode_tiled(CUtensorMap* tm, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
-                 const uint32_t* box) {
+                 const uint32_t* box, bool swizzle = true) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) {
     g_cuda_error = "cuTensorMapEncodeTiled entry point not available";
     return MOE_ERR_CUDA;
   }
-  cuuint64_t gdim[3], gstr[2];
-  cuuint32_t bx[3], estr[3] = {1, 1, 1};
+  cuuint64_t gdim[5], gstr[4];
+  cuuint32_t bx[5], estr[5] = {1, 1, 1, 1, 1};
   for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; }
   for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides[i];
   CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void*>(base), gdim, gstr, bx, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     char buf[200];
@@ -83,6 +84,26 @@ int encode_halves(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t F) 
   const uint64_t dims[3] = {F, 2, rows}, strides[2] = {F * 2, 2 * F * 2};
   const uint32_t box[3] = {64, 1, 32};
   return encode_tiled(tm, base, 3, dims, strides, box);
+}
+
+// Store maps of the token-column tiles: un-swizzled boxes of 32 rows x `box_cols` columns.
+int encode_2d_plain(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t cols, uint32_t box_cols) {
+  const uint64_t dims[2] = {cols, rows}, strides[1] = {cols * 2};
+  const uint32_t box[2] = {box_cols, 32};
+  return encode_tiled(tm, base, 2, dims, strides, box, false);
+}
+int encode_halves_plain(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t F, uint32_t box_cols) {
+  const uint64_t dims[3] = {F, 2, rows}, strides[2] = {F * 2, 2 * F * 2};
+  const uint32_t box[3] = {box_cols, 1, 32};
+  return encode_tiled(tm, base, 3, dims, strides, box, false);
+}
+// Load map of W_gate_up viewed as [Ep][F/16 groups][gate | up][16 rows][d]: one box brings, for four
+// groups of 16 features, the 16 gate rows followed by the 16 up rows (needs F % 16 == 0).
+int encode_gate_up_rows(CUtensorMap* tm, const void* base, uint64_t Ep, uint64_t F, uint64_t d) {
+  const uint64_t dims[5] = {d, 16, 2, F / 16, Ep};
+  const uint64_t strides[4] = {d * 2, F * d * 2, 16 * d * 2, 2 * F * d * 2};
+  const uint32_t box[5] = {64, 16, 2, 4, 1};
+  return encode_tiled(tm, base, 5, dims, strides, box);
 }
 
 // Store map of a weight-gradient tensor [Ep][M][N]: box 32 rows x 64 columns inside one expert slab.
@@ -141,7 +162,7 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.src_of = c.take(sizeof(int) * (slots + 1));
   p.prow_of = c.take(sizeof(int) * (slots + 1));
   p.prow_w = c.take(sizeof(float) * cap);
-  p.dw_partial = c.take(train ? sizeof(float) * cap * p.ntn_act : 0);
+  p.dw_partial = c.take(train ? sizeof(float) * cap * p.ntn_act * DW_PARTS_PER_TILE : 0);
   p.Xp = c.take(2 * cap * s.d);
   p.H = c.take(train ? 2 * cap * 2 * s.F : 0);
   p.A = c.take(2 * cap * s.F);
@@ -194,8 +215,12 @@ struct moe_ctx {
   const void* w1_ptr = nullptr;
   const void* w2_ptr = nullptr;
   CUtensorMap tm_W1_k, tm_W2_k, tm_W2_k128, tm_W1_mn, tm_W2_mn;
+  CUtensorMap tm_W1_gu;  // token-column tiles: 16 gate rows + 16 up rows per box
   // store maps: workspace tensors (fixed) and the caller's weight gradients (re-encoded on change)
   CUtensorMap ts_A, ts_H, ts_Y, ts_dH;
+  // token-column tiles: token operands with 64-row and 16-row boxes, un-swizzled store maps
+  CUtensorMap tk_Xp[3], tk_A[3], tk_dOutp[3], tk_dH[3];
+  CUtensorMap tp_A, tp_H, tp_Y, tp_dH;
   const void* dw1_ptr = nullptr;
   const void* dw2_ptr = nullptr;
   CUtensorMap ts_dW1, ts_dW2;
@@ -250,6 +275,7 @@ int encode_weight_maps(moe_ctx* c, const uint16_t* W1, const uint16_t* W2) {
   if (W1 != c->w1_ptr) {
     if ((rc = encode_2d(&c->tm_W1_k, W1, Ep * 2 * s.F, s.d, 128, 64))) return rc;
     if ((rc = encode_2d(&c->tm_W1_mn, W1, Ep * 2 * s.F, s.d, 64, 64))) return rc;
+    if (s.F % 16 == 0 && (rc = encode_gate_up_rows(&c->tm_W1_gu, W1, Ep, s.F, s.d))) return rc;
     c->w1_ptr = W1;
   }
   if (W2 != c->w2_ptr) {
@@ -376,8 +402,47 @@ bool single_cta_gemm() {
   }
   return v == 1;
 }
-#define LAUNCH_GEMM_SERIAL(mode, args, sms, st, launches) \
-  (single_cta_gemm() ? launch_gemm(mode, args, sms, st, launches) : launch_gemm2(mode, args, sms, st, launches))
+// Diagnostic knob: MOE_B200_TOKEN_ROW_TILES=1 keeps the tokens on the accumulator rows (256-row tiles
+// padded per expert) in the row-space GEMMs of the CTA-pair kernels.
+bool token_col_tiles() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("MOE_B200_TOKEN_ROW_TILES");
+    v = (e && e[0] == '1') ? 0 : 1;
+  }
+  return v == 1 && !single_cta_gemm();
+}
+bool token_col_tiles(const moe_ctx* c) { return token_col_tiles() && c->shape.F % 16 == 0; }
+// Rewrites the arguments of a row-space operator for the token-column tiles: tmA/tmTok16 = tokens,
+// tmB = weights, un-swizzled store maps.
+GemmArgs to_token_cols(const moe_ctx* c, GemmMode mode, GemmArgs g) {
+  switch (mode) {
+    case GEMM_GATE_UP:
+      g.tmA = c->tm_Xp_k; memcpy(g.tmTok, c->tk_Xp, sizeof g.tmTok); g.tmB = c->tm_W1_gu;
+      g.tmOut0 = c->tp_A; g.tmOut1 = c->tp_H;
+      break;
+    case GEMM_DOWN:
+      g.tmA = c->tm_A_k; memcpy(g.tmTok, c->tk_A, sizeof g.tmTok); g.tmB = c->tm_W2_k128;
+      g.tmOut0 = c->tp_Y;
+      break;
+    case GEMM_ACT_GRAD:
+      g.tmA = c->tm_dOutp_k; memcpy(g.tmTok, c->tk_dOutp, sizeof g.tmTok);
+      g.tmOut0 = c->tp_dH;
+      break;
+    case GEMM_GATE_GRAD:
+      g.tmA = c->tm_dH_k; memcpy(g.tmTok, c->tk_dH, sizeof g.tmTok);
+      g.tmOut0 = c->tp_Y;
+      break;
+    default: break;
+  }
+  return g;
+}
+cudaError_t launch_gemm_serial(const moe_ctx* c, GemmMode mode, const GemmArgs& args, cudaStream_t st, int* launches) {
+  if (single_cta_gemm()) return launch_gemm(mode, args, c->num_sms, st, launches);
+  if (mode != GEMM_WGRAD && token_col_tiles(c)) return launch_gemm3(mode, to_token_cols(c, mode, args), c->num_sms, st, launches);
+  return launch_gemm2(mode, args, c->num_sms, st, launches);
+}
+#define LAUNCH_GEMM_SERIAL(mode, args, sms, st, launches) launch_gemm_serial(c, mode, args, st, launches)
 
 bool serial_mode(const moe_ctx* c) { return (c->shape.flags & MOE_FLAG_SERIAL_LAUNCH) != 0; }
 
@@ -512,7 +577,8 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     }
     if (d_w) {
       Phase ph(c, MOE_PHASE_DW_REDUCE, st);
-      MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), p.ntn_act, dm, lv, d_w, st, &c->launches));
+      MOE_CUDA(launch_dw_reduce(c->at<float>(p.dw_partial), token_col_tiles(c) ? p.ntn_act * DW_PARTS_PER_TILE : p.ntn_act,
+                                dm, lv, d_w, st, &c->launches));
     }
     {
       Phase ph(c, MOE_PHASE_WGRAD_DOWN, st);
@@ -614,6 +680,17 @@ int moe_create(moe_ctx** out, const moe_shape* shape, void* workspace, size_t wo
   if (!rc && train) rc = encode_2d(&c->tm_A_mn, c->ws + p.A, cap, s.F, 64, 64);
   if (!rc && train) rc = encode_2d(&c->tm_dH_mn, c->ws + p.dH, cap, 2 * s.F, 64, 64);
   if (!rc && train) rc = encode_2d(&c->tm_Xp_mn, c->ws + p.Xp, cap, s.d, 64, 64);
+  for (int i = 0; i < 3 && !rc; ++i) {
+    const uint32_t br = 64u >> i;
+    rc = encode_2d(&c->tk_Xp[i], c->ws + p.Xp, cap, s.d, br, 64);
+    if (!rc) rc = encode_2d(&c->tk_A[i], c->ws + p.A, cap, s.F, br, 64);
+    if (!rc && train) rc = encode_2d(&c->tk_dOutp[i], c->ws + p.dOutp, cap, s.d, br, 64);
+    if (!rc && train) rc = encode_2d(&c->tk_dH[i], c->ws + p.dH, cap, 2 * s.F, br, 64);
+  }
+  if (!rc) rc = encode_2d_plain(&c->tp_A, c->ws + p.A, cap, s.F, 16);
+  if (!rc) rc = encode_2d_plain(&c->tp_Y, c->ws + p.Y, cap, s.d, 32);
+  if (!rc && train) rc = encode_halves_plain(&c->tp_H, c->ws + p.H, cap, s.F, 16);
+  if (!rc && train) rc = encode_halves_plain(&c->tp_dH, c->ws + p.dH, cap, s.F, 32);
   if (rc) {
     if (c->owns_ws) cudaFree(c->ws);
     delete c;

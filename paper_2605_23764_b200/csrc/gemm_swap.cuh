@@ -1,0 +1,285 @@
+// Token-column tiles of the row-space grouped GEMMs (GMM1+SwiGLU, GMM2, act_grad, gate_grad) on CTA
+// pairs.  The weights take the 256 accumulator ROWS of a pair (128 per CTA, the A operand of
+// tcgen05.mma) and the expert's tokens the accumulator COLUMNS (the B operand, 32..256 per tile in
+// steps of 32, half of them in each CTA's shared memory).  The MMA time of a tile then follows the
+// number of tokens it really holds: an expert with n tokens costs ceil(n / 256) tiles of about
+// n / ceil(n / 256) tokens each instead of ceil(n / 256) full 256-row tiles.
+//
+// The accumulator arrives transposed (TMEM lane = output feature, column = token); the epilogues
+// write it back token-major through small un-swizzled staging boxes and TMA stores.
+#pragma once
+
+#include <cuda_bf16.h>
+
+#include "gemm_pair.cuh"
+
+namespace moe {
+
+constexpr int TOK_GRAIN = 32;                    // tokens per tile: a multiple of 32 (16 rows of B per CTA)
+constexpr int W_STAGE_BYTES = A_STAGE_BYTES;     // 128 weight rows (or 2 MN-major boxes) x 64 k: 16 KB
+constexpr int SW_SLOT_BYTES = 4096;              // one staging slot of an epilogue warp
+#ifndef MOE_SW_SLOTS
+#define MOE_SW_SLOTS 2
+#endif
+constexpr int SW_SLOTS = MOE_SW_SLOTS;           // ring of slots per warp
+
+struct SwapTile {
+  int e;      // expert
+  int row0;   // first padded row of the tile's tokens
+  int ntok;   // tokens (accumulator columns) of the tile, multiple of TOK_GRAIN
+  int n0;     // first output feature of the pair (GATE_UP: of the 128 gate/up feature pairs)
+  int nb;     // feature-tile index
+  int nkb;    // k-blocks
+};
+
+// Features per pair tile: GATE_UP holds 64 gate + 64 up rows per CTA = 128 features per pair.
+template <int MODE>
+__device__ __forceinline__ int swap_tile_features() { return MODE == GEMM_GATE_UP ? 128 : 256; }
+
+// Token range of the pl-th of `pcount` tiles of an expert with n tokens whose segment starts at seg_row0.
+__device__ __forceinline__ void token_tile_range(int n, int pcount, int pl, int seg_row0, int* row0, int* ntok) {
+  const int n32 = (n + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);
+  const int tn = ((n + pcount - 1) / pcount + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);  // even split, <= 256
+  *row0 = seg_row0 + pl * tn;
+  const int left = n32 - pl * tn;
+  *ntok = left < tn ? left : tn;
+}
+
+// Tile order: expert-major; inside an expert the feature tile is the slow index and the token tile
+// the fast one (tiles running at the same time share one slab of weights in L2).
+template <int MODE>
+__device__ __forceinline__ SwapTile decode_swap_tile(const GemmArgs& a, int t) {
+  SwapTile st;
+  const int e = a.pblk_expert[t / a.n_tiles_n];
+  const int ps = a.pair_start[e];
+  const int pcount = a.pair_start[e + 1] - ps;   // ceil(n / 256) token tiles
+  const int local = t - ps * a.n_tiles_n;
+  st.nb = local / pcount;
+  const int pl = local - st.nb * pcount;
+  st.e = e;
+  token_tile_range(a.counts[e], pcount, pl, a.mb_start[e] * BLOCK_M, &st.row0, &st.ntok);
+  st.n0 = st.nb * swap_tile_features<MODE>();
+  st.nkb = (a.K + BK - 1) / BK;
+  return st;
+}
+
+__device__ __forceinline__ uint32_t swap_stage_tx_bytes(int ntok) {
+  return 2u * (uint32_t)(W_STAGE_BYTES + (ntok >> 1) * BK * 2);   // both CTAs: weights + half of the tokens
+}
+
+// This CTA's loads of one k-block are split over two producer warps, one box per lane (issuing a TMA
+// box costs its thread on the order of a hundred cycles, and a k-block of a short tile only lasts a
+// few hundred).  Tokens: rows [row0 + rank * ntok/2, + ntok/2) as one box per set bit of ntok/2
+// (128, 64, 32, 16 rows).  The even CTA's weight producer arms the barrier for both CTAs' bytes.
+__device__ __forceinline__ void load_tokens_swap(const GemmArgs& a, const SwapTile& st, int kb, int rank, uint8_t* sT,
+                                                 uint64_t* bar, int lane) {
+  if (lane >= 4) return;
+  const int half = st.ntok >> 1;
+  const int size = 128 >> lane;                 // lane 0: 128-row box ... lane 3: 16-row box
+  if (!(half & size)) return;
+  const int before = half & ~(2 * size - 1);    // rows covered by the larger boxes
+  const CUtensorMap* m = lane == 0 ? &a.tmA : &a.tmTok[lane - 1];
+  tma_load_2d_pair(sT + before * (BK * 2), m, kb * BK, st.row0 + rank * half + before, bar);
+}
+template <int MODE>
+__device__ __forceinline__ void load_weights_swap(const GemmArgs& a, const SwapTile& st, int kb, int rank, uint8_t* sW,
+                                                  uint64_t* bar, int lane) {
+  const int k0 = kb * BK;
+  if (lane == 0 && rank == 0) mbar_expect_tx(bar, swap_stage_tx_bytes(st.ntok));
+  __syncwarp();
+  const int brow = st.e * a.b_rows_per_expert;
+  if (MODE == GEMM_GATE_UP) {
+    // one box [4 groups][gate | up][16 rows][64 k]: per epilogue warp 16 gate rows, then the 16 up rows
+    // of the same features (W_gate_up viewed as [Ep][F/16][2][16][d])
+    if (lane == 0) tma_load_5d_pair(sW, &a.tmB, k0, 0, 0, (st.n0 + rank * 64) >> 4, st.e, bar);
+  } else if (MODE == GEMM_DOWN) {
+    if (lane == 0) tma_load_2d_pair(sW, &a.tmB, k0, brow + st.n0 + rank * 128, bar);
+  } else {
+    // ACT_GRAD / GATE_GRAD: the forward weight read along its rows -> two MN-major [64 k][64 features] boxes
+    if (lane < 2) tma_load_2d_pair(sW + lane * MN_BOX_BYTES, &a.tmB, st.n0 + (2 * rank + lane) * 64, brow + k0, bar);
+  }
+}
+
+// One 64-deep k-block: D[256 features x ntok tokens] (+)= W . X^T.  w_lo / t_lo: low descriptor words of
+// the stage's weight and token tiles (smem_desc_lo); the issuing thread only adds the k-step.
+template <int MODE>
+__device__ __forceinline__ void mma_kblock_swap(uint32_t d_tmem, uint32_t w_lo, uint32_t t_lo, uint32_t idesc,
+                                                bool first_kblock) {
+  constexpr bool W_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD);
+  constexpr uint32_t hi = smem_desc_hi(1024);
+  constexpr uint32_t wstep = W_MN ? (2048 >> 4) : (32 >> 4);   // 16 k-rows of an MN-major box / 32 bytes of a K-major row
+#pragma unroll
+  for (int k16 = 0; k16 < BK / 16; ++k16)
+    tc_mma_bf16_pair_lohi(d_tmem, w_lo + k16 * wstep, hi, t_lo + k16 * 2, hi, idesc, !(first_kblock && k16 == 0));
+}
+template <int MODE>
+__device__ __forceinline__ uint32_t swap_w_desc_lo(uint32_t w_addr) {
+  constexpr bool W_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD);
+  return smem_desc_lo(w_addr, W_MN ? MN_BOX_BYTES : 16);
+}
+template <int MODE>
+__device__ __forceinline__ uint32_t swap_idesc(int ntok) {
+  constexpr bool W_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD);
+  return make_idesc_bf16(2 * BLOCK_M, ntok, W_MN ? 1 : 0, 0);
+}
+
+// ---------------------------------------------------------------- staging ring of an epilogue warp
+struct SwStaging {
+  uint8_t* base;     // SW_SLOTS slots of SW_SLOT_BYTES
+  uint32_t round;
+};
+__device__ __forceinline__ uint8_t* sw_acquire(SwStaging& sg, int lane) {
+  if (lane == 0) tma_store_wait_read_n<SW_SLOTS - 1>();   // the slot's previous stores have read it
+  __syncwarp();
+  uint8_t* slot = sg.base + (sg.round % SW_SLOTS) * SW_SLOT_BYTES;
+  ++sg.round;
+  return slot;
+}
+__device__ __forceinline__ uint16_t bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ float bf16_to_f32(uint16_t h) { return __uint_as_float(static_cast<uint32_t>(h) << 16); }
+__device__ __forceinline__ uint16_t ld_nc_u16(const uint16_t* p) {
+  uint16_t v;
+  asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+  return v;
+}
+
+
+// ---------------------------------------------------------------- epilogues (transposed accumulator)
+// Warp `quad` of CTA `rank` owns TMEM lanes 32*quad .. 32*quad+31 (32 output features) and walks the
+// tile's tokens 32 columns at a time.  A thread (= one feature) writes one bf16 per token into a
+// staging box laid out [token][feature]; lane 0 stores the box with TMA (clipped at the tensor edge).
+template <int MODE>
+__device__ __forceinline__ void epilogue_swap(const GemmArgs& a, const SwapTile& st, uint32_t tmem_acc, int rank,
+                                              int quad, int lane, SwStaging& sg) {
+  const uint32_t trow = tmem_acc + (static_cast<uint32_t>(quad * 32) << 16);
+  if (MODE == GEMM_DOWN || MODE == GEMM_GATE_GRAD) {
+    const int f0 = st.n0 + rank * 128 + quad * 32;   // first output column of this warp
+    if (f0 >= a.N) return;
+#pragma unroll 1
+    for (int c0 = 0; c0 < st.ntok; c0 += 32) {
+      float v[32];
+      tmem_ld16(trow + c0, v);
+      tmem_ld16(trow + c0 + 16, v + 16);
+      tmem_ld_wait();
+      uint8_t* box = sw_acquire(sg, lane);
+      uint16_t* col = reinterpret_cast<uint16_t*>(box) + lane;   // [32 tokens][32 features]
+#pragma unroll
+      for (int j = 0; j < 32; ++j) col[j * 32] = bf16_bits(v[j]);
+      staging_release();
+      if (lane == 0) {
+        tma_store_2d(&a.tmOut0, f0, st.row0 + c0, box);
+        tma_store_commit();
+      }
+    }
+  } else if (MODE == GEMM_GATE_UP) {
+    // lanes 0..15: gate pre-activations of 16 features, lanes 16..31: up pre-activations of the same
+    // features.  For a token pair (j, j+1) the halves swap one value: the low half finishes token j,
+    // the high half token j+1.
+    const int fl = lane & 15;
+    const bool hi = lane >= 16;
+    const int fw0 = st.n0 + rank * 64 + quad * 16;   // first feature of this warp
+    if (fw0 >= a.F) return;
+#pragma unroll 1
+    for (int c0 = 0; c0 < st.ntok; c0 += 32) {
+      float v[32];
+      tmem_ld16(trow + c0, v);
+      tmem_ld16(trow + c0 + 16, v + 16);
+      const float wl = a.prow_w[st.row0 + c0 + lane];   // routing weight of token c0 + lane
+      tmem_ld_wait();
+      uint8_t* box = sw_acquire(sg, lane);
+      uint16_t* abox = reinterpret_cast<uint16_t*>(box);           // A: [32 tokens][16 features]
+      uint16_t* hbox = reinterpret_cast<uint16_t*>(box + 1024 + (hi ? 1024 : 0));   // H gate / H up
+#pragma unroll
+      for (int j = 0; j < 32; j += 2) {
+        const float send = hi ? v[j] : v[j + 1];
+        const float recv = __shfl_xor_sync(0xffffffffu, send, 16);
+        const float g = hi ? recv : v[j];
+        const float u = hi ? v[j + 1] : recv;
+        const int tj = j + (hi ? 1 : 0);
+        const float w = __shfl_sync(0xffffffffu, wl, tj);
+        abox[tj * 16 + fl] = bf16_bits(w * (g * sigmoidf_fast(g) * u));
+      }
+      if (a.save_h) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) hbox[j * 16 + fl] = bf16_bits(v[j]);
+      }
+      staging_release();
+      if (lane == 0) {
+        tma_store_2d(&a.tmOut0, fw0, st.row0 + c0, box);
+        if (a.save_h) {
+          tma_store_3d(&a.tmOut1, fw0, 0, st.row0 + c0, box + 1024);
+          tma_store_3d(&a.tmOut1, fw0, 1, st.row0 + c0, box + 2048);
+        }
+        tma_store_commit();
+      }
+    }
+  } else if (MODE == GEMM_ACT_GRAD) {
+    const int f0 = st.n0 + rank * 128 + quad * 32;
+    const int f = f0 + lane;
+    const int nparts = a.n_tiles_n * DW_PARTS_PER_TILE;
+    const int slot = (st.nb * 2 + rank) * 4 + quad;
+    if (f0 >= a.F) {
+      // no features here: the partial slots of this warp still take part in the reduction
+      if (a.dw_partial)
+        for (int j = lane; j < st.ntok; j += 32) a.dw_partial[(size_t)(st.row0 + j) * nparts + slot] = 0.f;
+      return;
+    }
+    const bool fvalid = f < a.F;
+    const uint16_t* hcol = a.in0 + (fvalid ? f : 0);
+#pragma unroll 1
+    for (int c0 = 0; c0 < st.ntok; c0 += 32) {
+      const float wl = a.prow_w[st.row0 + c0 + lane];
+      uint8_t* box = sw_acquire(sg, lane);
+      uint16_t* gbox = reinterpret_cast<uint16_t*>(box) + lane;          // d(gate): [32 tokens][32 features]
+      uint16_t* ubox = reinterpret_cast<uint16_t*>(box + 2048) + lane;   // d(up)
+#pragma unroll 1
+      for (int h = 0; h < 32; h += 16) {
+        float da[16], part[16];
+        tmem_ld16(trow + c0 + h, da);
+        uint16_t gr[16], ur[16];
+        const uint16_t* hp = hcol + (size_t)(st.row0 + c0 + h) * a.ld_in0;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          gr[j] = fvalid ? ld_nc_u16(hp + (size_t)j * a.ld_in0) : (uint16_t)0;
+          ur[j] = fvalid ? ld_nc_u16(hp + (size_t)j * a.ld_in0 + a.F) : (uint16_t)0;
+        }
+        tmem_ld_wait();
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float g = bf16_to_f32(gr[j]), u = bf16_to_f32(ur[j]);
+          const float s = sigmoidf_fast(g);
+          const float gs = g * s;
+          part[j] = da[j] * (gs * u);                 // <dA_unweighted, a>: gradient of the routing weight
+          const float w = __shfl_sync(0xffffffffu, wl, h + j);
+          const float dav = w * da[j];                // backward Dispatch's weight, applied here
+          gbox[(h + j) * 32] = bf16_bits(dav * u * (s * (1.0f + g * (1.0f - s))));
+          ubox[(h + j) * 32] = bf16_bits(dav * gs);
+        }
+        if (a.dw_partial) {
+          // sum over the warp's 32 features: a transposing butterfly leaves token (lane >> 1) in each lane
+#pragma unroll
+          for (int off = 16, n = 8; off >= 2; off >>= 1, n >>= 1) {
+            const bool up = (lane & off) != 0;
+#pragma unroll
+            for (int i = 0; i < n; ++i) {
+              const float keep = up ? part[i + n] : part[i];
+              const float send = up ? part[i] : part[i + n];
+              part[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+            }
+          }
+          part[0] += __shfl_xor_sync(0xffffffffu, part[0], 1);
+          if ((lane & 1) == 0)
+            a.dw_partial[(size_t)(st.row0 + c0 + h + (lane >> 1)) * nparts + slot] = part[0];
+        }
+      }
+      staging_release();
+      if (lane == 0) {
+        tma_store_3d(&a.tmOut0, f0, 0, st.row0 + c0, box);
+        tma_store_3d(&a.tmOut0, f0, 1, st.row0 + c0, box + 2048);
+        tma_store_commit();
+      }
+    }
+  }
+}
+
+}  // namespace moe

@@ -75,6 +75,7 @@ struct GemmArgs {
   CUtensorMap tmB;     // B operand
   CUtensorMap tmOut0;  // store map of out0: [rows][N] (2-D), [rows][2][F] (dH), or [Ep][M][N] (WGRAD)
   CUtensorMap tmOut1;  // GATE_UP: store map of H as [rows][2][F]
+  CUtensorMap tmTok[3]; // token-column tiles (gemm_tc3.cu): the token operand with 64-, 32- and 16-row boxes (tmA: 128)
   // tile table
   const int* mblk_expert;
   const int* mb_start;
@@ -105,6 +106,11 @@ cudaError_t launch_gemm(GemmMode mode, const GemmArgs& a, int num_sms, cudaStrea
 size_t gemm_smem_bytes();
 // ---- gemm_tc2.cu: the same operators on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles)
 cudaError_t launch_gemm2(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
+
+// ---- gemm_tc3.cu: the row-space operators with the tokens as accumulator COLUMNS (weights take the
+// 256 accumulator rows of a CTA pair), so a tile's MMA time follows the expert's real token count
+cudaError_t launch_gemm3(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
+constexpr int DW_PARTS_PER_TILE = 8;  // routing-weight gradient partials per (row, column tile): 2 CTAs x 4 warps
 
 // ---- fused.cu (the single persistent dependency-driven launch)
 // Everything one fused launch needs: the operators' GEMM arguments (one per schedule segment), the
