@@ -201,8 +201,10 @@ int moe_debug_set_unreachable_dependency(moe_ctx* ctx, int32_t on);
  * given per-expert row counts[Ep] it builds the matrix and vector queues, verifies that every tile
  * appears once and after all of its producers, lets mat_workers + vec_workers workers consume the
  * queues in ticket order blocking on the counters, and verifies that every counter ends at its
- * threshold.  seg_tiles[4] = tickets per M-block (or per M-block pair when `pair` is set: two CTAs
- * on one 256-row tile) / per expert of each schedule segment, lag in experts.  Returns 0, or a positive code naming the violated property (20 = deadlock).
+ * threshold.  seg_tiles[4] = tickets per M-block (or per unit of one or two M-blocks when `pair` is
+ * set: two CTAs on one tile; pair = 1: token-row tiles, units (0,1),(2,3),..; pair = 2: token-column
+ * tiles, balanced units, 8 instead of 4 signals per M-block and column tile) / per expert of each
+ * schedule segment, lag in experts.  Returns 0, or a positive code naming the violated property (20 = deadlock).
  * stats[4] (may be NULL) = {matrix tiles, vector tasks, scheduler rounds, stalled polls}.  Needs no GPU. */
 int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t is_bwd,
                                 const int32_t* seg_tiles, int32_t lag, int32_t mat_workers,

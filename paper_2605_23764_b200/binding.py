@@ -224,13 +224,14 @@ def moe_layout_noalloc(topk_ids, T, E, k, n_shared, counts, offsets, row_of, src
                                              _dev(status2, i32, "status2"), _stream()), "moe_layout_noalloc")
 
 
-def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_workers, vec_workers, pair=False):
-    """Host-only schedule check; returns (code, stats) with code 0 = schedule is sound."""
+def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_workers, vec_workers, pair=0):
+    """Host-only schedule check; returns (code, stats) with code 0 = schedule is sound.
+    pair: 0 = one CTA per tile, 1 = CTA pairs on token-row tiles, 2 = CTA pairs on token-column tiles."""
     c = (ctypes.c_int32 * len(counts))(*[int(v) for v in counts])
     seg = (ctypes.c_int32 * 4)(*[int(v) for v in seg_tiles])
     stats = (ctypes.c_int64 * 4)()
     rc = load_library().moe_debug_simulate_schedule(c, len(counts), T, k, int(is_bwd), seg, lag, mat_workers,
-                                                    vec_workers, int(bool(pair)), stats)
+                                                    vec_workers, int(pair), stats)
     return rc, list(stats)
 
 

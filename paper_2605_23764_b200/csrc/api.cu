@@ -452,6 +452,8 @@ SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
   memset(&sp, 0, sizeof sp);
   sp.is_bwd = bwd ? 1 : 0;
   sp.pair = single_cta_gemm() ? 0 : 1;
+  sp.tokcol = token_col_tiles(c) ? 1 : 0;
+  sp.sig = sp.tokcol ? 2 * EPI_WARPS : EPI_WARPS;
   sp.dep_extra = c->dep_extra;
   sp.Ep = s.E + s.n_shared;
   sp.T = T;
@@ -533,6 +535,10 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     fa.op[0] = args_gate_up(c);
     fa.op[1] = args_down(c);
     if (fa.sp.pair) fa.op[1].tmB = c->tm_W2_k128;
+    if (fa.sp.tokcol) {
+      fa.op[0] = to_token_cols(c, GEMM_GATE_UP, fa.op[0]);
+      fa.op[1] = to_token_cols(c, GEMM_DOWN, fa.op[1]);
+    }
     fa.gather_src = x;
     fa.gather_dst = c->at<uint16_t>(p.Xp);
     fa.topk_w = w;
@@ -608,6 +614,11 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     fa.combine_out = dx;
     fa.dw_partial = c->at<float>(p.dw_partial);
     fa.dw_nparts = p.ntn_act;
+    if (fa.sp.tokcol) {
+      fa.op[0] = to_token_cols(c, GEMM_ACT_GRAD, fa.op[0]);
+      fa.op[2] = to_token_cols(c, GEMM_GATE_GRAD, fa.op[2]);
+      fa.dw_nparts = p.ntn_act * DW_PARTS_PER_TILE;
+    }
     fa.d_topk_w = d_w;
     fa.dW1 = dW1;
     fa.dW2 = dW2;
@@ -934,6 +945,8 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
   SchedParams sp;
   memset(&sp, 0, sizeof sp);
   sp.is_bwd = is_bwd; sp.lag = lag; sp.Ep = Ep; sp.T = T; sp.k = k; sp.pair = pair ? 1 : 0;
+  sp.tokcol = pair == 2 ? 1 : 0;
+  sp.sig = sp.tokcol ? 2 * EPI_WARPS : EPI_WARPS;
   for (int i = 0; i < SCHED_MAX_SEG; ++i) sp.seg_tiles[i] = seg_tiles[i];
   sp.strip_tiles[0] = sp.strip_tiles[1] = 1;
   std::vector<int> step_start(Ep + lag + 1, 0);
@@ -987,9 +1000,9 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
       }
       if (!ready) { ++stalls; continue; }
       for (int q = 0; q < wk.m.mb_count; ++q) {  // every real M-block of the tile signals (an idle half does not)
-        if (wk.m.trig_base == 1) ctr[ctr_act(wk.m.mb + q)] += EPI_WARPS;
-        if (wk.m.trig_base == 2) ctr[CTR_DONE] += EPI_WARPS;
-        if (wk.m.trig_also_ag) ctr[CTR_AG_DONE] += EPI_WARPS;
+        if (wk.m.trig_base == 1) ctr[ctr_act(wk.m.mb + q)] += sp.sig;
+        if (wk.m.trig_base == 2) ctr[CTR_DONE] += sp.sig;
+        if (wk.m.trig_also_ag) ctr[CTR_AG_DONE] += sp.sig;
       }
       wk.holding = false;
       ++done_mat;
@@ -1013,9 +1026,9 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
   }
   // 3. every counter ends exactly at its threshold
   for (int mb = 0; mb < M; ++mb)
-    if (ctr[ctr_gather(mb)] != GATHER_SUB || ctr[ctr_act(mb)] != (long)EPI_WARPS * sp.seg_tiles[0]) return 30;
-  if (ctr[CTR_DONE] != (long)EPI_WARPS * M * (is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1])) return 31;
-  if (is_bwd && ctr[CTR_AG_DONE] != (long)EPI_WARPS * M * sp.seg_tiles[0]) return 32;
+    if (ctr[ctr_gather(mb)] != GATHER_SUB || ctr[ctr_act(mb)] != (long)sp.sig * sp.seg_tiles[0]) return 30;
+  if (ctr[CTR_DONE] != (long)sp.sig * M * (is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1])) return 31;
+  if (is_bwd && ctr[CTR_AG_DONE] != (long)sp.sig * M * sp.seg_tiles[0]) return 32;
   if (stats) { stats[0] = total; stats[1] = vtotal; stats[2] = rounds; stats[3] = stalls; }
   return MOE_OK;
 }

@@ -17,7 +17,7 @@
 
 #include <vector>
 
-#include "gemm_pair.cuh"
+#include "gemm_swap.cuh"
 #include "schedule.h"
 
 namespace moe {
@@ -41,7 +41,8 @@ namespace moe {
 #endif
 constexpr int VEC_WARPS = MOE_VEC_WARPS;
 constexpr int SCHED_WARP = 6 + VEC_WARPS;         // the last warp
-constexpr int FUSED_THREADS = GEMM_THREADS + 32 * VEC_WARPS + 32;
+constexpr int TOK_WARP = SCHED_WARP + 1;            // CTA-pair kernel, token-column tiles: TMA producer of the tokens
+constexpr int FUSED_THREADS = GEMM_THREADS + 32 * VEC_WARPS + 64;
 constexpr int SCHED_AHEAD_KB = 24;                // k-blocks of a ticket left when the next one is fetched
 constexpr int RING = 4;                            // published-tile ring depth
 
@@ -52,6 +53,7 @@ struct TileSlot {
   short go_kb;    // k-block at which the loader tells the scheduler to fetch the next ticket (-1: not in this tile)
   short pad;      // CTA-pair kernel: this CTA's half of the tile is idle (no rows / outside the gradient)
   int krows;      // weight gradients: rows of the expert (the reduction length)
+                  // token-column tiles (row-space operators): m0 = tokens of the tile, krows = its M-blocks
 };
 
 struct __align__(16) FusedShared {
@@ -575,7 +577,7 @@ struct __align__(16) PairShared {
 
 constexpr size_t FUSEDP_SMEM_BYTES = 1024 + (size_t)STAGESP * STAGE2_BYTES + 4 * OUT_STAGE_BYTES + sizeof(PairShared);
 static_assert(FUSEDP_SMEM_BYTES <= 227 * 1024, "shared memory budget");
-constexpr int PAIR_TK_EMPTY_COUNT = (2 + EPI_WARPS) + (1 + EPI_WARPS);  // even: loader, MMA, epilogue; odd: loader, epilogue
+constexpr int PAIR_TK_EMPTY_COUNT = (3 + EPI_WARPS) + (2 + EPI_WARPS);  // even: 2 loaders, MMA, epilogue; odd: 2 loaders, epilogue
 
 template <bool BWD>
 __device__ __forceinline__ void fusedp_load_stage(const FusedArgs& fa, const TileSlot& ts, const Tile& tl, int kb,
@@ -598,6 +600,53 @@ __device__ __forceinline__ void fusedp_mma(int op, uint32_t d_tmem, uint32_t a_a
   } else {
     if (op == GEMM_WGRAD) mma_kblock_pair<GEMM_WGRAD>(d_tmem, a_addr, b_addr, first, k16_steps);
     else mma_kblock_pair<GEMM_ACT_GRAD>(d_tmem, a_addr, b_addr, first);
+  }
+}
+
+// ---- token-column tiles (gemm_swap.cuh) in the persistent launch
+__device__ __forceinline__ bool slot_is_tokcol(const FusedArgs& fa, int op) { return fa.sp.tokcol && op != GEMM_WGRAD; }
+__device__ __forceinline__ SwapTile slot_swap_tile(const TileSlot& ts) {
+  SwapTile st;
+  st.e = ts.e; st.row0 = ts.row0; st.ntok = ts.m0; st.n0 = ts.n0; st.nb = ts.nb; st.nkb = ts.nkb;
+  return st;
+}
+template <bool BWD>
+__device__ __forceinline__ void fusedp_load_weights_swap(const FusedArgs& fa, const TileSlot& ts, const SwapTile& st,
+                                                         int kb, int rank, uint8_t* sW, uint64_t* bar, int lane) {
+  const GemmArgs& g = fa.op[ts.slot];
+  if (!BWD) {
+    if (ts.op == GEMM_GATE_UP) load_weights_swap<GEMM_GATE_UP>(g, st, kb, rank, sW, bar, lane);
+    else load_weights_swap<GEMM_DOWN>(g, st, kb, rank, sW, bar, lane);
+  } else {
+    load_weights_swap<GEMM_ACT_GRAD>(g, st, kb, rank, sW, bar, lane);  // ACT_GRAD and GATE_GRAD alike
+  }
+}
+template <bool BWD>
+__device__ __forceinline__ void fusedp_epilogue_swap(const FusedArgs& fa, const TileSlot& ts, const SwapTile& st,
+                                                     uint32_t tmem_acc, int rank, int quad, int lane, SwStaging& sg) {
+  const GemmArgs& g = fa.op[ts.slot];
+  if (!BWD) {
+    if (ts.op == GEMM_GATE_UP) epilogue_swap<GEMM_GATE_UP>(g, st, tmem_acc, rank, quad, lane, sg);
+    else epilogue_swap<GEMM_DOWN>(g, st, tmem_acc, rank, quad, lane, sg);
+  } else {
+    if (ts.op == GEMM_ACT_GRAD) epilogue_swap<GEMM_ACT_GRAD>(g, st, tmem_acc, rank, quad, lane, sg);
+    else epilogue_swap<GEMM_GATE_GRAD>(g, st, tmem_acc, rank, quad, lane, sg);
+  }
+}
+static_assert(SW_SLOTS * SW_SLOT_BYTES == OUT_STAGE_BYTES, "both epilogue kinds share one staging area per warp");
+// Weight-gradient stage split over the two loader warps (warp 0: the A boxes and the byte count,
+// TOK_WARP: this CTA's B boxes), so that both warps take part in every stage of the launch: a warp
+// that only waited on a stage's barrier could fall two phases behind it, where a parity wait is no
+// longer meaningful.
+__device__ __forceinline__ void fusedp_load_wgrad_part(const GemmArgs& g, const Tile& tl, int kb, int rank, uint8_t* sA,
+                                                       uint8_t* sB, uint64_t* bar, int lane, bool tok_warp) {
+  const int k0 = kb * BK;
+  if (!tok_warp) {
+    if (lane == 0 && rank == 0) mbar_expect_tx(bar, 2 * STAGE2_BYTES);
+    __syncwarp();
+    if (lane < 2) tma_load_2d_pair(sA + lane * MN_BOX_BYTES, &g.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
+  } else {
+    if (lane < 2) tma_load_2d_pair(sB + lane * MN_BOX_BYTES, &g.tmB, tl.n0 + (2 * rank + lane) * 64, tl.row0 + k0, bar);
   }
 }
 
@@ -708,6 +757,19 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
               tr.row0 = fa.lv.mb_start[mt.e] * BLOCK_M;
               tr.pad = tr.m0 >= g.M;               // nothing to store: the strip's second half is outside dW
               tr.trig_idx = -1;
+            } else if (fa.sp.tokcol) {
+              // token-column tile: both CTAs work on all its tokens (each on its half of the features)
+              const int n32 = (fa.lv.counts[mt.e] + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);
+              const int first = mt.mb - fa.lv.mb_start[mt.e];
+              int end = (first + mt.mb_count) * BLOCK_M;
+              if (end > n32) end = n32;
+              tr.nb = mt.idx;
+              tr.m0 = end - first * BLOCK_M;           // tokens of the tile
+              tr.krows = mt.mb_count;
+              tr.n0 = mt.idx * (mt.op == GEMM_GATE_UP ? 128 : 256);
+              tr.row0 = mt.mb * BLOCK_M;
+              tr.pad = 0;
+              tr.trig_idx = mt.trig_base == 1 ? ctr_act(mt.mb) : (mt.trig_base == 2 ? CTR_DONE : -1);
             } else {
               const bool idle = r >= mt.mb_count;
               tr.nb = mt.idx;
@@ -726,9 +788,10 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         ++go_n;
       }
     }
-  } else if (warp == 0) {
-    // ------------------------------------------------ loader (both CTAs): own rows of A, own half of B
-    uint32_t it = 0, n = 0;
+  } else if (warp == 0 || warp == TOK_WARP) {
+    // ------------------------------------------------ loaders (both CTAs).  Warp 0: own rows of A and own half
+    // of B of a token-row tile, or the weights of a token-column tile; TOK_WARP: the tokens of a token-column tile.
+    uint32_t s = 0, ph = 1, n = 0;
     bool ok = true;
     while (ok) {
       const int rs = n % RING;
@@ -739,12 +802,26 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
       ++n;
       if (ts.op < 0) break;
       fence_proxy_async();
+      const bool tokcol = slot_is_tokcol(fa, ts.op);
       const Tile tl = slot_tile(ts);
-      for (int kb = 0; kb < ts.nkb; ++kb, ++it) {
-        if (kb == ts.go_kb && lane == 0 && rank == 0) mbar_arrive(&sh->sched_go);
-        const int s = it % STAGESP;
-        if (!mbar_wait(&sh->empty[s], ((it / STAGESP) & 1) ^ 1, wc, SITE_EMPTY, n, 50)) { ok = false; break; }
-        fusedp_load_stage<BWD>(fa, ts, tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s], lane);
+      const SwapTile st = slot_swap_tile(ts);
+      if (warp == TOK_WARP && !fa.sp.tokcol) continue;   // token-row tiles: warp 0 loads everything
+      for (int kb = 0; kb < ts.nkb; ++kb) {
+        if (warp == 0 && kb == ts.go_kb && lane == 0 && rank == 0) mbar_arrive(&sh->sched_go);
+        int go = 1;
+        if (lane == 0) go = mbar_wait(&sh->empty[s], ph, wc, SITE_EMPTY, n, 50) ? 1 : 0;
+        go = __shfl_sync(0xffffffffu, go, 0);
+        if (!go) { ok = false; break; }
+        if (!fa.sp.tokcol)
+          fusedp_load_stage<BWD>(fa, ts, tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s], lane);
+        else if (!tokcol)   // a weight-gradient tile between token-column tiles
+          fusedp_load_wgrad_part(fa.op[ts.slot], tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s],
+                                 lane, warp == TOK_WARP);
+        else if (warp == 0)
+          fusedp_load_weights_swap<BWD>(fa, ts, st, kb, rank, sA + s * A_STAGE_BYTES, &sh->full[s], lane);
+        else
+          load_tokens_swap(fa.op[ts.slot], st, kb, rank, sB + s * HALF_B_BYTES, &sh->full[s], lane);
+        if (++s == STAGESP) { s = 0; ph ^= 1; }
       }
     }
   } else if (warp == 1) {
@@ -758,7 +835,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         ST_MARK();
         if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -1)) break;
         ST_ADD(0);  // waiting for a published tile
-        const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb, krows = sh->ring[rs].krows;
+        const int op = sh->ring[rs].op, nkb = sh->ring[rs].nkb, krows = sh->ring[rs].krows, ntok = sh->ring[rs].m0;
         mbar_arrive(&sh->tk_empty[rs]);
         ++n;
         if (op < 0) break;
@@ -768,13 +845,20 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         ST_ADD(1);  // accumulator not yet drained by the epilogues
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + as * BN;
+        const bool tokcol = slot_is_tokcol(fa, op);
+        const uint32_t idesc = swap_idesc<BWD ? GEMM_ACT_GRAD : GEMM_GATE_UP>(ntok);
         for (int kb = 0; kb < nkb; ++kb, ++it) {
           const int s = it % STAGESP;
           if (!mbar_wait(&sh->full[s], (it / STAGESP) & 1, wc, SITE_FULL, n)) { ok = false; break; }
           ST_ADD(2);  // operands not yet in shared memory
           tc_fence_after_sync();
-          fusedp_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0,
-                          op == GEMM_WGRAD ? k16_steps_of(krows, kb) : BK / 16);
+          if (tokcol)
+            mma_kblock_swap<BWD ? GEMM_ACT_GRAD : GEMM_GATE_UP>(
+                d_tmem, swap_w_desc_lo<BWD ? GEMM_ACT_GRAD : GEMM_GATE_UP>(smem_u32(sA + s * A_STAGE_BYTES)),
+                smem_desc_lo(smem_u32(sB + s * HALF_B_BYTES), 16), idesc, kb == 0);
+          else
+            fusedp_mma<BWD>(op, d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0,
+                            op == GEMM_WGRAD ? k16_steps_of(krows, kb) : BK / 16);
           tc_commit_pair(&sh->empty[s]);
           ST_ADD(op == GEMM_WGRAD ? 4 : 3);  // issue (includes back-pressure of the tensor pipe)
         }
@@ -804,11 +888,20 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
       if (ts.op < 0) break;
       const Tile tl = slot_tile(ts);
       const bool idle = ts.pad != 0;
+      const bool tokcol = slot_is_tokcol(fa, ts.op);
       if (ts.nkb != 0) {
         const int as = acc_it & 1;
         if (!mbar_wait(&sh->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, n, 100)) break;
         tc_fence_after_sync();
-        if (!idle) fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);
+        if (tokcol) {
+          // the staging area changes hands between the two epilogue kinds: let the earlier stores finish reading
+          if (lane == 0) tma_store_wait_read();
+          __syncwarp();
+          SwStaging sg{sOut + quad * OUT_STAGE_BYTES, 0};
+          fusedp_epilogue_swap<BWD>(fa, ts, slot_swap_tile(ts), tmem_base + as * BN, rank, quad, lane, sg);
+        } else if (!idle) {
+          fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);
+        }
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive_leader(&sh->tmem_empty[as]);
@@ -819,8 +912,15 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         if (lane == 0) {
           tma_store_wait_all();
           fence_proxy_async();
-          counter_signal(fa.ctr + ts.trig_idx, 1);
-          if (ts.trig_ag) counter_signal(fa.ctr + CTR_AG_DONE, 1);
+          if (tokcol) {
+            // this warp stored its features of every row of the tile's M-blocks (ts.krows of them)
+            if (ts.trig_idx == CTR_DONE) counter_signal(fa.ctr + CTR_DONE, ts.krows);
+            else for (int q = 0; q < ts.krows; ++q) counter_signal(fa.ctr + ts.trig_idx + 2 * q, 1);
+            if (ts.trig_ag) counter_signal(fa.ctr + CTR_AG_DONE, ts.krows);
+          } else {
+            counter_signal(fa.ctr + ts.trig_idx, 1);
+            if (ts.trig_ag) counter_signal(fa.ctr + CTR_AG_DONE, 1);
+          }
         }
         __syncwarp();
       }

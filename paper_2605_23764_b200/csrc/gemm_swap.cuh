@@ -2,8 +2,7 @@
 // pairs.  The weights take the 256 accumulator ROWS of a pair (128 per CTA, the A operand of
 // tcgen05.mma) and the expert's tokens the accumulator COLUMNS (the B operand, 32..256 per tile in
 // steps of 32, half of them in each CTA's shared memory).  The MMA time of a tile then follows the
-// number of tokens it really holds: an expert with n tokens costs ceil(n / 256) tiles of about
-// n / ceil(n / 256) tokens each instead of ceil(n / 256) full 256-row tiles.
+// number of tokens it really holds instead of the padded 256 rows of a token-row tile.
 //
 // The accumulator arrives transposed (TMEM lane = output feature, column = token); the epilogues
 // write it back token-major through small un-swizzled staging boxes and TMA stores.
@@ -36,28 +35,26 @@ struct SwapTile {
 template <int MODE>
 __device__ __forceinline__ int swap_tile_features() { return MODE == GEMM_GATE_UP ? 128 : 256; }
 
-// Token range of the pl-th of `pcount` tiles of an expert with n tokens whose segment starts at seg_row0.
-__device__ __forceinline__ void token_tile_range(int n, int pcount, int pl, int seg_row0, int* row0, int* ntok) {
-  const int n32 = (n + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);
-  const int tn = ((n + pcount - 1) / pcount + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);  // even split, <= 256
-  *row0 = seg_row0 + pl * tn;
-  const int left = n32 - pl * tn;
-  *ntok = left < tn ? left : tn;
-}
-
 // Tile order: expert-major; inside an expert the feature tile is the slow index and the token tile
-// the fast one (tiles running at the same time share one slab of weights in L2).
+// the fast one (tiles running at the same time share one slab of weights in L2).  Token tiles are the
+// expert's balanced units of one or two M-blocks (schedule.h), cut at the expert's last 32-row group.
 template <int MODE>
 __device__ __forceinline__ SwapTile decode_swap_tile(const GemmArgs& a, int t) {
   SwapTile st;
   const int e = a.pblk_expert[t / a.n_tiles_n];
   const int ps = a.pair_start[e];
-  const int pcount = a.pair_start[e + 1] - ps;   // ceil(n / 256) token tiles
+  const int pcount = a.pair_start[e + 1] - ps;   // units = ceil(M-blocks / 2)
   const int local = t - ps * a.n_tiles_n;
   st.nb = local / pcount;
   const int pl = local - st.nb * pcount;
   st.e = e;
-  token_tile_range(a.counts[e], pcount, pl, a.mb_start[e] * BLOCK_M, &st.row0, &st.ntok);
+  int first, count;
+  balanced_unit(a.mb_start[e + 1] - a.mb_start[e], pl, &first, &count);
+  const int n32 = (a.counts[e] + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);
+  int end = (first + count) * BLOCK_M;
+  if (end > n32) end = n32;
+  st.row0 = (a.mb_start[e] + first) * BLOCK_M;
+  st.ntok = end - first * BLOCK_M;
   st.n0 = st.nb * swap_tile_features<MODE>();
   st.nkb = (a.K + BK - 1) / BK;
   return st;

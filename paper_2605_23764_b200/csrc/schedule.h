@@ -51,7 +51,26 @@ struct SchedParams {
   int seg_tiles[SCHED_MAX_SEG];
   int strip_tiles[2];      // column tiles in one w2_grad / w1_grad strip
   int dep_extra;           // test hook: added to the activation-counter thresholds (> 0 = never reached)
+  int tokcol;              // 1 (with pair): token-column tiles, balanced units of one or two M-blocks
+  int sig;                 // signals one (M-block, column tile) sends to its counters: EPI_WARPS, or
+                           // 2 * EPI_WARPS when the epilogue warps of both CTAs of a pair cover every row
 };
+
+// Token-column tiles: the ceil(mc / 2) row-space units of an expert with mc M-blocks.  An odd count
+// does not leave a lone M-block at the end (a tile of a few tokens still streams the whole weight
+// tile): the single block sits before the last unit, which takes the last full block and the tail.
+MOE_HD void balanced_unit(int mc, int u, int* first, int* count) {
+  const int uc = (mc + 1) >> 1;
+  *first = 2 * u;
+  *count = 2;
+  if ((mc & 1) == 0) return;
+  if (u == uc - 1) {
+    if (mc == 1) { *first = 0; *count = 1; }
+    else *first = 2 * u - 1;
+  } else if (u == uc - 2) {
+    *count = 1;
+  }
+}
 
 MOE_HD int expert_mblocks(const int* mb_start, int e) { return mb_start[e + 1] - mb_start[e]; }
 // row-space scheduling units of an expert: its M-blocks, or its M-block pairs
@@ -114,6 +133,7 @@ MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, cons
       m.idx = r / uc;
       const int u = r - m.idx * uc;
       m.mb = mb_start[i] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride; m.e = i;
+      if (sp.pair && sp.tokcol) { int f, c; balanced_unit(mc, u, &f, &c); m.mb = mb_start[i] + f; m.mb_count = c; }
       m.dep_base = 0; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = GATHER_SUB;
       m.trig_base = 1; m.trig_also_ag = sp.is_bwd;
       return m;
@@ -137,14 +157,15 @@ MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, cons
     m.idx = r / uc;
     const int u = r - m.idx * uc;
     m.mb = mb_start[j] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride;
-    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = EPI_WARPS * sp.seg_tiles[0] + sp.dep_extra;
+    if (sp.pair && sp.tokcol) { int f, c; balanced_unit(mc, u, &f, &c); m.mb = mb_start[j] + f; m.mb_count = c; }
+    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = sp.sig * sp.seg_tiles[0] + sp.dep_extra;
     m.trig_base = 2;
     return m;
   }
   r -= uc * sp.seg_tiles[2];
   m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = j; m.idx = r; m.group = sp.strip_tiles[1];
   m.dep_base = 1; m.dep_first = mb_start[j]; m.dep_count = mc;
-  m.dep_thr = EPI_WARPS * sp.seg_tiles[0] + sp.dep_extra; m.trig_base = -1;
+  m.dep_thr = sp.sig * sp.seg_tiles[0] + sp.dep_extra; m.trig_base = -1;
   return m;
 }
 
@@ -182,13 +203,13 @@ MOE_HD VecTask decode_vector_ticket(const SchedParams& sp, int t, int M) {
     t -= sp.Ep * ZERO_CHUNKS;
     const int ndw = (sp.T * sp.k + DW_SLOTS - 1) / DW_SLOTS;
     if (t < ndw) {
-      v.op = VEC_DW; v.idx = t; v.dep = 3; v.dep_thr = EPI_WARPS * M * sp.seg_tiles[0];
+      v.op = VEC_DW; v.idx = t; v.dep = 3; v.dep_thr = sp.sig * M * sp.seg_tiles[0];
       return v;
     }
     t -= ndw;
   }
   v.op = VEC_COMBINE; v.idx = t; v.dep = 2;
-  v.dep_thr = EPI_WARPS * M * (sp.is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1]);
+  v.dep_thr = sp.sig * M * (sp.is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1]);
   return v;
 }
 

@@ -17,7 +17,7 @@ def _seg(is_bwd, d, F):
     return [(F + 255) // 256, (d + 127) // 128, (d + 255) // 256, (2 * F + 127) // 128]
 
 
-@pytest.mark.parametrize("pair", [False, True])
+@pytest.mark.parametrize("pair", [0, 1, 2])
 @pytest.mark.parametrize("is_bwd", [0, 1])
 @pytest.mark.parametrize("workers", [(1, 1), (3, 2), (148, 592)])
 @pytest.mark.parametrize("lag", [0, 1, 8])
@@ -44,12 +44,21 @@ def test_schedule_is_sound(is_bwd, workers, lag, pair):
         assert stats[0] == want
 
 
+def test_balanced_units_cover_every_mblock_once():
+    """Token-column tiles: the units of an expert (one or two M-blocks each) partition its M-blocks, and a
+    lone M-block never comes last when there are three or more."""
+    for n in list(range(0, 1200, 7)) + [128, 256, 257, 384, 385, 512, 640, 641]:
+        counts = np.array([n, 1, 300])
+        rc, stats = binding.moe_debug_simulate_schedule(counts, 64, 2, 0, [3, 2, 0, 0], 1, 5, 7, pair=2)
+        assert rc == 0, (n, rc)
+
+
 def test_training_config_schedule():
     """Config-4-like counts (256 experts, ~256 rows each) with the launch's real worker counts."""
     rng = np.random.default_rng(4)
     counts = rng.binomial(65536, 1 / 256, 256)
     for is_bwd in (0, 1):
-        for pair in (False, True):
+        for pair in (0, 1, 2):
             rc, stats = binding.moe_debug_simulate_schedule(counts, 8192, 8, is_bwd, _seg(is_bwd, 7168, 2048), 8, 148,
                                                             592, pair=pair)
             assert rc == 0
