@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the Dispatch->Combine MoE-FFN layer on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--serial] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--launch auto|fused|serial] [--impl reference]
 
 One step = one pass of the whole hot path on one batch of seeded synthetic input: routing,
 forward (dispatch layout, permute-gather, grouped GEMM gate+up with SwiGLU, grouped GEMM down,
@@ -246,7 +246,7 @@ def run_reference(args, cfg, train):
 def workload_desc(cfg, train, args):
     return {"workload": cfg.name, "T": cfg.T, "d": cfg.d, "E": cfg.E, "top_k": cfg.k, "shared": cfg.S, "F": cfg.F,
             "pass": "route+fwd+bwd" if train else "route+fwd",
-            "launch": "serial kernels" if args.serial else "fused persistent",
+            "launch": "serial kernels" if getattr(args, "launch", "") == "serial" else "fused persistent",
             "l2": "weights and expert-ordered activations exceed the 126 MB L2 (no flush needed)"
             if cfg.weight_bytes() > 4e8 else "L2 flushed between timed steps"}
 
@@ -258,7 +258,10 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", type=int, default=4, help="index into BASELINE.json configs (default: the training step)")
-    ap.add_argument("--serial", action="store_true", help="one kernel launch per operator instead of the fused launch")
+    ap.add_argument("--launch", default="auto", choices=["auto", "fused", "serial"],
+                    help="fused: one persistent launch per pass; serial: one launch per operator; auto (default): "
+                         "time both, report the faster as the headline and the other beside it")
+    ap.add_argument("--serial", action="store_true", help="same as --launch serial")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--fwd-only", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -267,6 +270,10 @@ def main():
     ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.serial:
+        args.launch = "serial"
+    if args.launch == "auto" and args.no_compare:
+        args.launch = "serial"
 
     cfg = configs.CONFIGS[args.config]
     if args.small:
@@ -290,8 +297,9 @@ def main():
     inp = configs.make_inputs(cfg, "cuda")
     x, W1, W2, logits = inp["x"], inp["W_gate_up"], inp["W_down"], inp["logits"]
     dout = inp.get("dout")
-    layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=train,
-                     serial=args.serial)
+    def make_layer(mode):
+        return MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=train,
+                        serial=(mode == "serial"))
     T = cfg.T
     ids = torch.empty(T, cfg.k, dtype=torch.int32, device="cuda")
     w = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
@@ -387,22 +395,29 @@ def main():
                      "hbm_ms": step_min_bytes(cfg, train) / (peak_gb * 1e9) * 1e3}
         return roof, step_roof
 
-    # ---- device-resident timing: the chosen launch mode, then the other one for comparison ----------
-    res = measure(layer)
+    # ---- device-resident timing of the launch modes (max over ranks: every rank sees the same numbers) ----
+    launch_names = {"serial": "serial kernels (one launch per operator)",
+                    "fused": "fused persistent (one launch each for forward and backward, after the index-only "
+                             "layout and schedule kernels)"}
+    modes = ["fused", "serial"] if args.launch == "auto" else (
+        [args.launch] if args.no_compare else [args.launch, "serial" if args.launch == "fused" else "fused"])
+    layers = {m: make_layer(m) for m in modes}
+    results = {m: measure(layers[m]) for m in modes}
+    head = min(modes, key=lambda m: results[m]["ms_per_step"]) if args.launch == "auto" else args.launch
+    layer, res = layers[head], results[head]
     ms_per_step, value, launches, clocks, phases_ms = (res["ms_per_step"], res["value"], res["launches"],
                                                        res["clocks"], res["phases_ms"])
     flops = step_flops(cfg, train)
     roofline, step_roofline = rooflines(res)
     other = None
-    if not args.no_compare:
-        other_layer = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=train,
-                               serial=not args.serial)
-        r2 = measure(other_layer)
+    for m in modes:
+        if m == head:
+            continue
+        r2 = results[m]
         roof2, step2 = rooflines(r2)
-        other = {"launch": "fused persistent" if args.serial else "serial kernels (one launch per operator)",
-                 "ms_per_step": r2["ms_per_step"], "value": r2["value"], "phases_ms": r2["phases_ms"],
-                 "roofline": roof2, "step_roofline": step2, "clocks": r2["clocks"]}
-        other_layer.close()
+        other = {"launch": launch_names[m], "ms_per_step": r2["ms_per_step"], "value": r2["value"],
+                 "phases_ms": r2["phases_ms"], "roofline": roof2, "step_roofline": step2, "clocks": r2["clocks"]}
+        layers[m].close()
 
     # ---- end to end through the host-buffer entry points ------------------------------------------
     e2e = None
@@ -461,9 +476,9 @@ def main():
             "other_launch_mode": other, "cpu_baseline": cpu_baseline,
         }
         per_step = launches / max(1, args.steps)
-        line["config"]["launch"] = ("serial kernels (one launch per operator)" if args.serial else
-                                    "fused persistent (one launch each for forward and backward, after the "
-                                    "index-only layout and schedule kernels)")
+        line["config"]["launch"] = launch_names[head]
+        line["config"]["launch_choice"] = ("faster of the two launch modes, both timed" if args.launch == "auto"
+                                           else "requested")
         line["config"]["launches_per_step"] = per_step
         print(json.dumps(line), flush=True)
     layer.close()
