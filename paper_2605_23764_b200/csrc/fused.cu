@@ -634,22 +634,6 @@ __device__ __forceinline__ void fusedp_epilogue_swap(const FusedArgs& fa, const 
   }
 }
 static_assert(SW_SLOTS * SW_SLOT_BYTES == OUT_STAGE_BYTES, "both epilogue kinds share one staging area per warp");
-// Weight-gradient stage split over the two loader warps (warp 0: the A boxes and the byte count,
-// TOK_WARP: this CTA's B boxes), so that both warps take part in every stage of the launch: a warp
-// that only waited on a stage's barrier could fall two phases behind it, where a parity wait is no
-// longer meaningful.
-__device__ __forceinline__ void fusedp_load_wgrad_part(const GemmArgs& g, const Tile& tl, int kb, int rank, uint8_t* sA,
-                                                       uint8_t* sB, uint64_t* bar, int lane, bool tok_warp) {
-  const int k0 = kb * BK;
-  if (!tok_warp) {
-    if (lane == 0 && rank == 0) mbar_expect_tx(bar, 2 * STAGE2_BYTES);
-    __syncwarp();
-    if (lane < 2) tma_load_2d_pair(sA + lane * MN_BOX_BYTES, &g.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
-  } else {
-    if (lane < 2) tma_load_2d_pair(sB + lane * MN_BOX_BYTES, &g.tmB, tl.n0 + (2 * rank + lane) * 64, tl.row0 + k0, bar);
-  }
-}
-
 // Publish one tile into the ring slot `rs` of CTA `rank` (through the cluster address space, also for
 // the even CTA itself) and signal that CTA's consumers.
 __device__ __forceinline__ void publish_slot(PairShared* sh, int rs, uint32_t rank, const TileSlot& ts) {
@@ -815,7 +799,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
         if (!fa.sp.tokcol)
           fusedp_load_stage<BWD>(fa, ts, tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s], lane);
         else if (!tokcol)   // a weight-gradient tile between token-column tiles
-          fusedp_load_wgrad_part(fa.op[ts.slot], tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s],
+          load_wgrad_part(fa.op[ts.slot], tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s],
                                  lane, warp == TOK_WARP);
         else if (warp == 0)
           fusedp_load_weights_swap<BWD>(fa, ts, st, kb, rank, sA + s * A_STAGE_BYTES, &sh->full[s], lane);

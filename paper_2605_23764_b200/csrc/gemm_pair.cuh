@@ -90,4 +90,21 @@ __device__ __forceinline__ void load_stage_pair_lanes(const GemmArgs& a, const T
   }
 }
 
+// A weight-gradient stage split over two loader warps (the first: this CTA's A boxes and the byte
+// count; the second: its B boxes): issuing a TMA box costs the issuing warp on the order of a hundred
+// cycles, and four boxes in one warp take about as long as the k-block's MMAs.  Both warps take part
+// in every stage, so neither can fall two phases behind a stage's barrier (where a parity wait is no
+// longer meaningful).
+__device__ __forceinline__ void load_wgrad_part(const GemmArgs& g, const Tile& tl, int kb, int rank, uint8_t* sA,
+                                                uint8_t* sB, uint64_t* bar, int lane, bool second_warp) {
+  const int k0 = kb * BK;
+  if (!second_warp) {
+    if (lane == 0 && rank == 0) mbar_expect_tx(bar, 2 * STAGE2_BYTES);
+    __syncwarp();
+    if (lane < 2) tma_load_2d_pair(sA + lane * MN_BOX_BYTES, &g.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
+  } else {
+    if (lane < 2) tma_load_2d_pair(sB + lane * MN_BOX_BYTES, &g.tmB, tl.n0 + (2 * rank + lane) * 64, tl.row0 + k0, bar);
+  }
+}
+
 }  // namespace moe

@@ -84,8 +84,10 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmArgs& a, int t, i
   return pt;
 }
 
+constexpr int GEMM2_THREADS = GEMM_THREADS + 32;   // warp 6: second TMA producer of the weight gradients
+
 template <int MODE>
-__global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(const __grid_constant__ GemmArgs a) {
+__global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(const __grid_constant__ GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem;                                  // [STAGES2][16 KB]
@@ -125,19 +127,23 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
   const uint32_t tmem_base = bars->tmem_base;
   const int total = total_pair_tiles<MODE>(a);
 
-  if (warp == 0) {
-    // ------------------------------------------------ TMA producer (both CTAs)
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int t = pair; t < total && ok; t += npairs) {
-        const PairTile pt = decode_pair_tile<MODE>(a, t, rank);
-        for (int kb = 0; kb < pt.tl.nkb; ++kb, ++it) {
-          const int s = it % STAGES2;
-          if (!mbar_wait(&bars->empty[s], ((it / STAGES2) & 1) ^ 1, wc, SITE_EMPTY, t, 50)) { ok = false; break; }
-          if (rank == 0) mbar_expect_tx(&bars->full[s], 2 * STAGE2_BYTES);  // the bytes of both CTAs
-          load_stage_pair<MODE>(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s]);
-        }
+  if (warp == 0 || (warp == 6 && MODE == GEMM_WGRAD)) {
+    // ------------------------------------------------ TMA producers (both CTAs, one box per lane); the
+    // weight gradients split each stage over two warps
+    uint32_t s = 0, ph = 1;
+    bool ok = true;
+    for (int t = pair; t < total && ok; t += npairs) {
+      const PairTile pt = decode_pair_tile<MODE>(a, t, rank);
+      for (int kb = 0; kb < pt.tl.nkb; ++kb) {
+        int go = 1;
+        if (lane == 0) go = mbar_wait(&bars->empty[s], ph, wc, SITE_EMPTY, t, 50) ? 1 : 0;
+        go = __shfl_sync(0xffffffffu, go, 0);
+        if (!go) { ok = false; break; }
+        if (MODE == GEMM_WGRAD)
+          load_wgrad_part(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s], lane, warp == 6);
+        else
+          load_stage_pair_lanes<MODE>(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s], lane);
+        if (++s == STAGES2) { s = 0; ph ^= 1; }
       }
     }
   } else if (warp == 1) {
@@ -170,7 +176,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 1) grouped_gemm_pair_kernel(cons
         mbar_wait(&bars->drain, 0, shortwc, SITE_DRAIN, 0);
       }
     }
-  } else {
+  } else if (warp < 6) {
     // ------------------------------------------------ epilogue warps (both CTAs, own rows)
     const int quad = warp & 3;
     Staging stg{sOut + quad * OUT_BUFS2 * OUT_STAGE_BYTES, OUT_BUFS2, 0};
@@ -217,7 +223,7 @@ static cudaError_t launch_pair_mode(const GemmArgs& a, int num_sms, cudaStream_t
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((num_sms / 2) * 2);
-  cfg.blockDim = dim3(GEMM_THREADS);
+  cfg.blockDim = dim3(GEMM2_THREADS);
   cfg.dynamicSmemBytes = GEMM2_SMEM_BYTES;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
