@@ -412,6 +412,16 @@ bool token_col_tiles() {
   }
   return v == 1 && !single_cta_gemm();
 }
+// Diagnostic knob: MOE_B200_WGRAD_PER_TILE=1 runs the weight gradients tile by tile (both operands
+// streamed for every tile) instead of strip by strip with a resident A operand.
+bool wgrad_strips_on() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("MOE_B200_WGRAD_PER_TILE");
+    v = (e && e[0] == '1') ? 0 : 1;
+  }
+  return v == 1;
+}
 bool token_col_tiles(const moe_ctx* c) { return token_col_tiles() && c->shape.F % 16 == 0; }
 // Rewrites the arguments of a row-space operator for the token-column tiles: tmA/tmTok16 = tokens,
 // tmB = weights, un-swizzled store maps.
@@ -439,6 +449,7 @@ GemmArgs to_token_cols(const moe_ctx* c, GemmMode mode, GemmArgs g) {
 }
 cudaError_t launch_gemm_serial(const moe_ctx* c, GemmMode mode, const GemmArgs& args, cudaStream_t st, int* launches) {
   if (single_cta_gemm()) return launch_gemm(mode, args, c->num_sms, st, launches);
+  if (mode == GEMM_WGRAD && wgrad_strips_on()) return launch_wgrad_strips(args, c->num_sms, st, launches);
   if (mode != GEMM_WGRAD && token_col_tiles(c)) return launch_gemm3(mode, to_token_cols(c, mode, args), c->num_sms, st, launches);
   return launch_gemm2(mode, args, c->num_sms, st, launches);
 }

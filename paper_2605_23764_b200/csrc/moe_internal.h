@@ -110,6 +110,8 @@ cudaError_t launch_gemm2(GemmMode mode, const GemmArgs& a, int num_sms, cudaStre
 // ---- gemm_tc3.cu: the row-space operators with the tokens as accumulator COLUMNS (weights take the
 // 256 accumulator rows of a CTA pair), so a tile's MMA time follows the expert's real token count
 cudaError_t launch_gemm3(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
+// ---- gemm_wgrad.cu: weight gradients strip by strip, the strip's A operand resident in shared memory
+cudaError_t launch_wgrad_strips(const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
 constexpr int DW_PARTS_PER_TILE = 8;  // routing-weight gradient partials per (row, column tile): 2 CTAs x 4 warps
 
 // ---- fused.cu (the single persistent dependency-driven launch)
