@@ -557,7 +557,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_kernel(const __grid_co
 // both CTAs (the odd CTA's copy over the cluster's shared-memory network).  Loaders and epilogue
 // warps run in both CTAs on their own half of the tile; vector workers are per CTA as before.
 // =====================================================================================================
-constexpr int STAGESP = 6;  // 6 x 32 KB operand stages per CTA
+constexpr int STAGESP = 5;  // 5 x 32 KB operand stages per CTA
 
 struct __align__(16) PairShared {
   uint64_t full[STAGESP];      // even CTA: bytes of both CTAs' loads
@@ -575,7 +575,8 @@ struct __align__(16) PairShared {
   TileSlot ring[RING];
 };
 
-constexpr size_t FUSEDP_SMEM_BYTES = 1024 + (size_t)STAGESP * STAGE2_BYTES + 4 * OUT_STAGE_BYTES + sizeof(PairShared);
+constexpr size_t FUSEDP_SMEM_BYTES =
+    1024 + (size_t)STAGESP * STAGE2_BYTES + 4 * OUT_STAGE_BYTES + 4 * SW_SCRATCH_BYTES + sizeof(PairShared);
 static_assert(FUSEDP_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 constexpr int PAIR_TK_EMPTY_COUNT = (3 + EPI_WARPS) + (2 + EPI_WARPS);  // even: 2 loaders, MMA, epilogue; odd: 2 loaders, epilogue
 
@@ -653,7 +654,8 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
   uint8_t* sA = smem;
   uint8_t* sB = smem + STAGESP * A_STAGE_BYTES;
   uint8_t* sOut = smem + STAGESP * STAGE2_BYTES;
-  PairShared* sh = reinterpret_cast<PairShared*>(sOut + 4 * OUT_STAGE_BYTES);
+  uint8_t* sScr = sOut + 4 * OUT_STAGE_BYTES;   // act_grad epilogue: 4 KB per epilogue warp
+  PairShared* sh = reinterpret_cast<PairShared*>(sScr + 4 * SW_SCRATCH_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();
@@ -881,7 +883,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
           // the staging area changes hands between the two epilogue kinds: let the earlier stores finish reading
           if (lane == 0) tma_store_wait_read();
           __syncwarp();
-          SwStaging sg{sOut + quad * OUT_STAGE_BYTES, 0};
+          SwStaging sg{sOut + quad * OUT_STAGE_BYTES, 0, sScr + quad * SW_SCRATCH_BYTES};
           fusedp_epilogue_swap<BWD>(fa, ts, slot_swap_tile(ts), tmem_base + as * BN, rank, quad, lane, sg);
         } else if (!idle) {
           fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);

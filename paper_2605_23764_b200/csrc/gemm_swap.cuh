@@ -124,7 +124,9 @@ __device__ __forceinline__ uint32_t swap_idesc(int ntok) {
 struct SwStaging {
   uint8_t* base;     // SW_SLOTS slots of SW_SLOT_BYTES
   uint32_t round;
+  uint8_t* scratch;  // act_grad: 4 KB of this warp (two halves of [gate | up][16 tokens][32 features])
 };
+constexpr int SW_SCRATCH_BYTES = 4096;
 __device__ __forceinline__ uint8_t* sw_acquire(SwStaging& sg, int lane) {
   if (lane == 0) tma_store_wait_read_n<SW_SLOTS - 1>();   // the slot's previous stores have read it
   __syncwarp();
@@ -134,10 +136,10 @@ __device__ __forceinline__ uint8_t* sw_acquire(SwStaging& sg, int lane) {
 }
 __device__ __forceinline__ uint16_t bf16_bits(float x) { return __bfloat16_as_ushort(__float2bfloat16_rn(x)); }
 __device__ __forceinline__ float bf16_to_f32(uint16_t h) { return __uint_as_float(static_cast<uint32_t>(h) << 16); }
-__device__ __forceinline__ uint16_t ld_nc_u16(const uint16_t* p) {
-  uint16_t v;
-  asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
-  return v;
+__device__ __forceinline__ uint4 ld_nc_v4(const uint16_t* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+  return r;
 }
 
 
@@ -212,7 +214,6 @@ __device__ __forceinline__ void epilogue_swap(const GemmArgs& a, const SwapTile&
     }
   } else if (MODE == GEMM_ACT_GRAD) {
     const int f0 = st.n0 + rank * 128 + quad * 32;
-    const int f = f0 + lane;
     const int nparts = a.n_tiles_n * DW_PARTS_PER_TILE;
     const int slot = (st.nb * 2 + rank) * 4 + quad;
     if (f0 >= a.F) {
@@ -221,59 +222,84 @@ __device__ __forceinline__ void epilogue_swap(const GemmArgs& a, const SwapTile&
         for (int j = lane; j < st.ntok; j += 32) a.dw_partial[(size_t)(st.row0 + j) * nparts + slot] = 0.f;
       return;
     }
-    const bool fvalid = f < a.F;
-    const uint16_t* hcol = a.in0 + (fvalid ? f : 0);
+    // The saved pre-activations of 16 tokens x 32 features (gate and up: 1 KB each) come in as four
+    // 16-byte loads per lane (lane -> token (lane + 32 i) / 4, features 8 (lane % 4) ..), are parked in
+    // this warp's scratch [gate | up][16 tokens][32 features] and read back one feature column per lane.
+    // The loads of the next 16 tokens are in flight while the current ones are worked on.
+    const int part = lane & 3;
+    const bool cvalid = f0 + part * 8 < a.F;     // F % 8 == 0: a 16-byte chunk is inside or outside as a whole
+    const uint16_t* hbase = a.in0 + (size_t)st.row0 * a.ld_in0 + f0 + part * 8;
+    uint4 pre[4];
+    auto fetch = [&](int tok0) {
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int t = (lane + 32 * i) >> 2;
+        const uint16_t* p = hbase + (size_t)(tok0 + t) * a.ld_in0;
+        pre[2 * i] = cvalid ? ld_nc_v4(p) : make_uint4(0, 0, 0, 0);
+        pre[2 * i + 1] = cvalid ? ld_nc_v4(p + a.F) : make_uint4(0, 0, 0, 0);
+      }
+    };
+    fetch(0);
+    uint8_t* box = nullptr;
+    float wl = 0.f;
 #pragma unroll 1
-    for (int c0 = 0; c0 < st.ntok; c0 += 32) {
-      const float wl = a.prow_w[st.row0 + c0 + lane];
-      uint8_t* box = sw_acquire(sg, lane);
+    for (int h0 = 0; h0 < st.ntok; h0 += 16) {
+      const int hh = h0 & 16;   // which half of the 32-token staging box
+      if (hh == 0) {
+        box = sw_acquire(sg, lane);
+        wl = a.prow_w[st.row0 + h0 + lane];
+      }
+      uint8_t* scr = sg.scratch + (((h0 >> 4) & 1) ? 2048 : 0);
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        const int t = (lane + 32 * i) >> 2;
+        *reinterpret_cast<uint4*>(scr + t * 64 + part * 16) = pre[2 * i];
+        *reinterpret_cast<uint4*>(scr + 1024 + t * 64 + part * 16) = pre[2 * i + 1];
+      }
+      if (h0 + 16 < st.ntok) fetch(h0 + 16);
+      float da[16], pr[16];
+      tmem_ld16(trow + h0, da);
+      __syncwarp();
+      tmem_ld_wait();
       uint16_t* gbox = reinterpret_cast<uint16_t*>(box) + lane;          // d(gate): [32 tokens][32 features]
       uint16_t* ubox = reinterpret_cast<uint16_t*>(box + 2048) + lane;   // d(up)
-#pragma unroll 1
-      for (int h = 0; h < 32; h += 16) {
-        float da[16], part[16];
-        tmem_ld16(trow + c0 + h, da);
-        uint16_t gr[16], ur[16];
-        const uint16_t* hp = hcol + (size_t)(st.row0 + c0 + h) * a.ld_in0;
+      const uint16_t* gs16 = reinterpret_cast<const uint16_t*>(scr) + lane;
+      const uint16_t* us16 = reinterpret_cast<const uint16_t*>(scr + 1024) + lane;
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          gr[j] = fvalid ? ld_nc_u16(hp + (size_t)j * a.ld_in0) : (uint16_t)0;
-          ur[j] = fvalid ? ld_nc_u16(hp + (size_t)j * a.ld_in0 + a.F) : (uint16_t)0;
-        }
-        tmem_ld_wait();
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float g = bf16_to_f32(gr[j]), u = bf16_to_f32(ur[j]);
-          const float s = sigmoidf_fast(g);
-          const float gs = g * s;
-          part[j] = da[j] * (gs * u);                 // <dA_unweighted, a>: gradient of the routing weight
-          const float w = __shfl_sync(0xffffffffu, wl, h + j);
-          const float dav = w * da[j];                // backward Dispatch's weight, applied here
-          gbox[(h + j) * 32] = bf16_bits(dav * u * (s * (1.0f + g * (1.0f - s))));
-          ubox[(h + j) * 32] = bf16_bits(dav * gs);
-        }
-        if (a.dw_partial) {
-          // sum over the warp's 32 features: a transposing butterfly leaves token (lane >> 1) in each lane
-#pragma unroll
-          for (int off = 16, n = 8; off >= 2; off >>= 1, n >>= 1) {
-            const bool up = (lane & off) != 0;
-#pragma unroll
-            for (int i = 0; i < n; ++i) {
-              const float keep = up ? part[i + n] : part[i];
-              const float send = up ? part[i] : part[i + n];
-              part[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-            }
-          }
-          part[0] += __shfl_xor_sync(0xffffffffu, part[0], 1);
-          if ((lane & 1) == 0)
-            a.dw_partial[(size_t)(st.row0 + c0 + h + (lane >> 1)) * nparts + slot] = part[0];
-        }
+      for (int j = 0; j < 16; ++j) {
+        const float g = bf16_to_f32(gs16[j * 32]), u = bf16_to_f32(us16[j * 32]);
+        const float s = sigmoidf_fast(g);
+        const float gs = g * s;
+        pr[j] = da[j] * (gs * u);                   // <dA_unweighted, a>: gradient of the routing weight
+        const float w = __shfl_sync(0xffffffffu, wl, hh + j);
+        const float dav = w * da[j];                // backward Dispatch's weight, applied here
+        gbox[(hh + j) * 32] = bf16_bits(dav * u * (s * (1.0f + g * (1.0f - s))));
+        ubox[(hh + j) * 32] = bf16_bits(dav * gs);
       }
-      staging_release();
-      if (lane == 0) {
-        tma_store_3d(&a.tmOut0, f0, 0, st.row0 + c0, box);
-        tma_store_3d(&a.tmOut0, f0, 1, st.row0 + c0, box + 2048);
-        tma_store_commit();
+      if (a.dw_partial) {
+        // sum over the warp's 32 features: a transposing butterfly leaves token (lane >> 1) in each lane
+#pragma unroll
+        for (int off = 16, n = 8; off >= 2; off >>= 1, n >>= 1) {
+          const bool up = (lane & off) != 0;
+#pragma unroll
+          for (int i = 0; i < n; ++i) {
+            const float keep = up ? pr[i + n] : pr[i];
+            const float send = up ? pr[i] : pr[i + n];
+            pr[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+          }
+        }
+        pr[0] += __shfl_xor_sync(0xffffffffu, pr[0], 1);
+        if ((lane & 1) == 0) a.dw_partial[(size_t)(st.row0 + h0 + (lane >> 1)) * nparts + slot] = pr[0];
+      }
+      if (hh == 16) {
+        staging_release();
+        if (lane == 0) {
+          tma_store_3d(&a.tmOut0, f0, 0, st.row0 + h0 - 16, box);
+          tma_store_3d(&a.tmOut0, f0, 1, st.row0 + h0 - 16, box + 2048);
+          tma_store_commit();
+        }
+      } else {
+        __syncwarp();   // the scratch half written two rounds from now is the one just read
       }
     }
   }

@@ -12,7 +12,7 @@
 namespace moe {
 
 #ifndef MOE_STAGES3
-#define MOE_STAGES3 6
+#define MOE_STAGES3 5
 #endif
 constexpr int STAGES3 = MOE_STAGES3;   // 32 KB operand stages; the rest: 4 epilogue warps x staging ring
 
@@ -26,8 +26,8 @@ struct __align__(8) SwapBarriers {
   uint32_t pad;
 };
 
-constexpr size_t GEMM3_SMEM_BYTES =
-    1024 + (size_t)STAGES3 * STAGE2_BYTES + 4 * SW_SLOTS * SW_SLOT_BYTES + sizeof(SwapBarriers);
+constexpr size_t GEMM3_SMEM_BYTES = 1024 + (size_t)STAGES3 * STAGE2_BYTES + 4 * SW_SLOTS * SW_SLOT_BYTES +
+                                    4 * SW_SCRATCH_BYTES + sizeof(SwapBarriers);
 static_assert(GEMM3_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 #ifdef MOE_STATS3
@@ -50,7 +50,8 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
   uint8_t* sW = smem;                                   // [STAGES3][16 KB] weights
   uint8_t* sT = smem + STAGES3 * W_STAGE_BYTES;         // [STAGES3][16 KB] tokens (this CTA's half)
   uint8_t* sOut = smem + STAGES3 * STAGE2_BYTES;
-  SwapBarriers* bars = reinterpret_cast<SwapBarriers*>(sOut + 4 * SW_SLOTS * SW_SLOT_BYTES);
+  uint8_t* sScr = sOut + 4 * SW_SLOTS * SW_SLOT_BYTES;  // act_grad: per epilogue warp 4 KB for the saved pre-activations
+  SwapBarriers* bars = reinterpret_cast<SwapBarriers*>(sScr + 4 * SW_SCRATCH_BYTES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
   } else if (warp < 6) {
     // ------------------------------------------------ epilogue warps (both CTAs, own features)
     const int quad = warp & 3;
-    SwStaging sg{sOut + quad * SW_SLOTS * SW_SLOT_BYTES, 0};
+    SwStaging sg{sOut + quad * SW_SLOTS * SW_SLOT_BYTES, 0, sScr + quad * SW_SCRATCH_BYTES};
     uint32_t acc_it = 0;
     for (int t = pair; t < total; t += npairs) {
       const SwapTile st = decode_swap_tile<MODE>(a, t);
