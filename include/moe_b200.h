@@ -120,7 +120,14 @@ int moe_ffn_bwd(moe_ctx* ctx, const uint16_t* dout, const uint16_t* x, const int
  * asynchronous copies).  x/topk_ids/topk_w/dout are host pointers copied to the device inside the
  * call; out/dx/d_topk_w are host pointers filled from the device; weights and weight gradients
  * stay device pointers (model state is resident).  The call returns after enqueueing; the host
- * buffers are valid once `stream` has been synchronised. */
+ * output buffers are valid, and the host input buffers may be reused, once `stream` has been
+ * synchronised.  The large inputs (x_host, dout_host) travel on a copy-in stream of the context,
+ * started when the call is made: they must hold their final values at that moment (they are not
+ * ordered behind earlier work on `stream`), and the copy overlaps whatever the context still has
+ * running.  topk_ids_host / topk_w_host are copied in stream order, so the buffers a preceding
+ * moe_route_host on the same stream fills can be passed on without a synchronisation.  Results leave
+ * on a copy-out stream that `stream` joins before the call's work ends (dx_host while the last
+ * weight gradient is still being computed). */
 int moe_ffn_fwd_host(moe_ctx* ctx, const uint16_t* x_host, const int32_t* topk_ids_host,
                      const float* topk_w_host, const uint16_t* W_gate_up, const uint16_t* W_down,
                      uint16_t* out_host, int32_t T, void* stream);

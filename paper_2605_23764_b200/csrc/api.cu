@@ -133,7 +133,7 @@ struct Carve {
 // Byte offsets of every workspace tensor.
 struct WsPlan {
   size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
-      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, stats, total;
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, stats, total;
   int cap_rows, nblk_max, ntn_act, ctr_count;
 };
 
@@ -170,6 +170,7 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.dOutp = c.take(train ? 2 * cap * s.d : 0);
   p.dH = c.take(train ? 2 * cap * 2 * s.F : 0);
   p.st_x = c.take(2 * (size_t)s.T_max * s.d);
+  p.st_dout = c.take(train ? 2 * (size_t)s.T_max * s.d : 0);
   p.st_ids = c.take(sizeof(int) * (size_t)s.T_max * s.k);
   p.st_w = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_out = c.take(2 * (size_t)s.T_max * s.d);
@@ -185,6 +186,8 @@ WsPlan plan_workspace(const moe_shape& s) {
 
 }  // namespace
 
+constexpr int HOST_CHUNKS = 4;   // token chunks of a host-buffer result (combine + copy-out pipelined)
+
 struct moe_ctx {
   moe_shape shape;
   WsPlan plan;
@@ -198,6 +201,13 @@ struct moe_ctx {
   int dep_extra = 0;  // test hook: makes the activation dependencies of the persistent launch unreachable
   int sched_lag = 0;  // experts between a producer step and its consumer step; 0 = choose from the shape
   cudaStream_t last_stream = nullptr;
+  // host-buffer entry points: a copy-in stream (the next call's large input arrives while the previous
+  // call still computes) and a copy-out stream (the result leaves in token chunks behind the combine)
+  bool copy_ready = false;
+  cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+  cudaEvent_t ev_x_free = nullptr, ev_dout_free = nullptr, ev_h2d_done = nullptr, ev_d2h_done = nullptr;
+  cudaEvent_t ev_chunk[HOST_CHUNKS] = {};
+  bool x_used = false, dout_used = false;
   // optional per-operator timing
   bool profiling = false;
   bool events_made = false;
@@ -508,8 +518,43 @@ FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
   return fa;
 }
 
+int ensure_copy_streams(moe_ctx* c) {
+  if (c->copy_ready) return MOE_OK;
+  MOE_CUDA(cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking));
+  MOE_CUDA(cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
+  cudaEvent_t* evs[] = {&c->ev_x_free, &c->ev_dout_free, &c->ev_h2d_done, &c->ev_d2h_done};
+  for (cudaEvent_t* e : evs) MOE_CUDA(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+  for (int i = 0; i < HOST_CHUNKS; ++i) MOE_CUDA(cudaEventCreateWithFlags(&c->ev_chunk[i], cudaEventDisableTiming));
+  c->copy_ready = true;
+  return MOE_OK;
+}
+
+// Combine into `out` (device).  With `out_host` the tokens are combined in HOST_CHUNKS launches and
+// each chunk is copied out on the copy-out stream while the next one is being combined; the
+// launching stream then waits for the last copy, so the host buffer is complete once `st` is.
+int combine_and_maybe_copy_out(moe_ctx* c, const Dims& dm, const LayoutView& lv, uint16_t* out, uint16_t* out_host,
+                               cudaStream_t st) {
+  const WsPlan& p = c->plan;
+  if (!out_host || dm.T < HOST_CHUNKS * 64) {
+    MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+    if (out_host) MOE_CUDA(cudaMemcpyAsync(out_host, out, 2 * (size_t)dm.T * dm.d, cudaMemcpyDeviceToHost, st));
+    return MOE_OK;
+  }
+  for (int i = 0; i < HOST_CHUNKS; ++i) {
+    const int t0 = (int)((long)dm.T * i / HOST_CHUNKS), t1 = (int)((long)dm.T * (i + 1) / HOST_CHUNKS);
+    MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches, t0, t1));
+    MOE_CUDA(cudaEventRecord(c->ev_chunk[i], st));
+    MOE_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_chunk[i], 0));
+    MOE_CUDA(cudaMemcpyAsync(out_host + (size_t)t0 * dm.d, out + (size_t)t0 * dm.d, 2 * (size_t)(t1 - t0) * dm.d,
+                             cudaMemcpyDeviceToHost, c->d2h_stream));
+  }
+  MOE_CUDA(cudaEventRecord(c->ev_d2h_done, c->d2h_stream));
+  MOE_CUDA(cudaStreamWaitEvent(st, c->ev_d2h_done, 0));
+  return MOE_OK;
+}
+
 int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, const uint16_t* W1,
-            const uint16_t* W2, uint16_t* out, int T, cudaStream_t st) {
+            const uint16_t* W2, uint16_t* out, int T, cudaStream_t st, uint16_t* out_host = nullptr) {
   const WsPlan& p = c->plan;
   const Dims dm = c->dims(T);
   const LayoutView lv = c->layout();
@@ -538,7 +583,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     }
     {
       Phase ph(c, MOE_PHASE_COMBINE, st);
-      MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
+      if ((rc = combine_and_maybe_copy_out(c, dm, lv, out, out_host, st))) return rc;
     }
   } else {
     // one persistent launch: gather, GMM1+SwiGLU, GMM2 and combine tiles ordered by event counters
@@ -560,13 +605,14 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     MOE_CUDA(launch_build_schedule(fa.sp, lv, c->at<int>(p.step_start), c->at<int>(p.ctr), p.ctr_count, st,
                                    &c->launches));
     MOE_CUDA(launch_fused(false, fa, c->num_sms, st, &c->launches));
+    if (out_host) MOE_CUDA(cudaMemcpyAsync(out_host, out, 2 * (size_t)T * c->shape.d, cudaMemcpyDeviceToHost, st));
   }
   if (c->train()) c->saved_T = T;
   return MOE_OK;
 }
 
 int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t* W2, uint16_t* dx, uint16_t* dW1,
-            uint16_t* dW2, float* d_w, int T, cudaStream_t st) {
+            uint16_t* dW2, float* d_w, int T, cudaStream_t st, uint16_t* dx_host = nullptr) {
   const moe_shape& s = c->shape;
   const WsPlan& p = c->plan;
   const Dims dm = c->dims(T);
@@ -605,14 +651,22 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
       Phase ph(c, MOE_PHASE_GATE_GRAD, st);
       MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_GATE_GRAD, args_gate_grad(c), c->num_sms, st, &c->launches));
     }
+    {  // backward Combine: before the last weight gradient, which does not need dXp, so that with
+       // host buffers the copy of dx leaves on the copy-out stream while that GEMM runs
+      Phase ph(c, MOE_PHASE_BWD_COMBINE, st);
+      MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
+      if (dx_host) {
+        MOE_CUDA(cudaEventRecord(c->ev_chunk[0], st));
+        MOE_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_chunk[0], 0));
+        MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, c->d2h_stream));
+        MOE_CUDA(cudaEventRecord(c->ev_d2h_done, c->d2h_stream));
+      }
+    }
     {
       Phase ph(c, MOE_PHASE_WGRAD_GATE_UP, st);
       MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_WGRAD, args_wgrad_gate_up(c), c->num_sms, st, &c->launches));
     }
-    {  // backward Combine
-      Phase ph(c, MOE_PHASE_BWD_COMBINE, st);
-      MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, dx, st, &c->launches));
-    }
+    if (dx_host) MOE_CUDA(cudaStreamWaitEvent(st, c->ev_d2h_done, 0));  // dx_host is complete once `st` is
   } else {
     FusedArgs fa = fused_base(c, true, T);
     fa.op[0] = args_act_grad(c, d_w != nullptr);
@@ -639,6 +693,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     MOE_CUDA(launch_build_schedule(fa.sp, lv, c->at<int>(p.step_start), c->at<int>(p.ctr), p.ctr_count, st,
                                    &c->launches));
     MOE_CUDA(launch_fused(true, fa, c->num_sms, st, &c->launches));
+    if (dx_host) MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
   }
   return MOE_OK;
 }
@@ -729,6 +784,17 @@ int moe_destroy(moe_ctx* c) {
       cudaEventDestroy(c->ev_start[i]);
       cudaEventDestroy(c->ev_stop[i]);
     }
+  if (c->copy_ready) {
+    cudaStreamSynchronize(c->h2d_stream);
+    cudaStreamSynchronize(c->d2h_stream);
+    cudaStreamDestroy(c->h2d_stream);
+    cudaStreamDestroy(c->d2h_stream);
+    cudaEventDestroy(c->ev_x_free);
+    cudaEventDestroy(c->ev_dout_free);
+    cudaEventDestroy(c->ev_h2d_done);
+    cudaEventDestroy(c->ev_d2h_done);
+    for (int i = 0; i < HOST_CHUNKS; ++i) cudaEventDestroy(c->ev_chunk[i]);
+  }
   if (c->owns_ws) cudaFree(c->ws);
   delete c;
   return MOE_OK;
@@ -828,15 +894,23 @@ int moe_ffn_fwd_host(moe_ctx* c, const uint16_t* x_host, const int32_t* topk_ids
   if (T == 0) return MOE_OK;
   const moe_shape& s = c->shape;
   const WsPlan& p = c->plan;
-  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_x, x_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, st));
+  int rc = ensure_copy_streams(c);
+  if (rc) return rc;
+  // x goes in on the copy-in stream as soon as the previous forward has read its staging buffer:
+  // it overlaps whatever this context's earlier calls still have running on `st`
+  if (c->x_used) MOE_CUDA(cudaStreamWaitEvent(c->h2d_stream, c->ev_x_free, 0));
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_x, x_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, c->h2d_stream));
+  MOE_CUDA(cudaEventRecord(c->ev_h2d_done, c->h2d_stream));
   MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_ids, topk_ids_host, sizeof(int) * (size_t)T * s.k, cudaMemcpyHostToDevice,
                            st));
   MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_w, topk_w_host, sizeof(float) * (size_t)T * s.k, cudaMemcpyHostToDevice,
                            st));
-  int rc = run_fwd(c, c->at<uint16_t>(p.st_x), c->at<int32_t>(p.st_ids), c->at<float>(p.st_w), W_gate_up, W_down,
-                   c->at<uint16_t>(p.st_out), T, st);
+  MOE_CUDA(cudaStreamWaitEvent(st, c->ev_h2d_done, 0));
+  rc = run_fwd(c, c->at<uint16_t>(p.st_x), c->at<int32_t>(p.st_ids), c->at<float>(p.st_w), W_gate_up, W_down,
+               c->at<uint16_t>(p.st_out), T, st, out_host);
   if (rc) return rc;
-  MOE_CUDA(cudaMemcpyAsync(out_host, c->ws + p.st_out, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
+  MOE_CUDA(cudaEventRecord(c->ev_x_free, st));
+  c->x_used = true;
   return MOE_OK;
 }
 
@@ -851,12 +925,19 @@ int moe_ffn_bwd_host(moe_ctx* c, const uint16_t* dout_host, const uint16_t* W_ga
   c->begin_call(st);
   const moe_shape& s = c->shape;
   const WsPlan& p = c->plan;
-  // the staged x is dead after the forward's gather: its buffer receives dout
-  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_x, dout_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, st));
-  int rc = run_bwd(c, c->at<uint16_t>(p.st_x), W_gate_up, W_down, c->at<uint16_t>(p.st_out), dW_gate_up, dW_down,
-                   d_topk_w_host ? c->at<float>(p.st_dw) : nullptr, T, st);
+  int rc = ensure_copy_streams(c);
   if (rc) return rc;
-  MOE_CUDA(cudaMemcpyAsync(dx_host, c->ws + p.st_out, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
+  // dout has a staging buffer of its own and goes in on the copy-in stream: it arrives while the
+  // forward that was enqueued before this call is still computing
+  if (c->dout_used) MOE_CUDA(cudaStreamWaitEvent(c->h2d_stream, c->ev_dout_free, 0));
+  MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_dout, dout_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, c->h2d_stream));
+  MOE_CUDA(cudaEventRecord(c->ev_h2d_done, c->h2d_stream));
+  MOE_CUDA(cudaStreamWaitEvent(st, c->ev_h2d_done, 0));
+  rc = run_bwd(c, c->at<uint16_t>(p.st_dout), W_gate_up, W_down, c->at<uint16_t>(p.st_out), dW_gate_up, dW_down,
+               d_topk_w_host ? c->at<float>(p.st_dw) : nullptr, T, st, dx_host);
+  if (rc) return rc;
+  MOE_CUDA(cudaEventRecord(c->ev_dout_free, st));
+  c->dout_used = true;
   if (d_topk_w_host)
     MOE_CUDA(cudaMemcpyAsync(d_topk_w_host, c->ws + p.st_dw, sizeof(float) * (size_t)T * s.k,
                              cudaMemcpyDeviceToHost, st));

@@ -54,9 +54,10 @@ cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView&
 // of the row (1 for shared experts, 0 on padding rows).
 cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& dm, const LayoutView& lv,
                           uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches);
-// out[t] = sum_j rows[prow_of[t*kp+j]] in slot order, fp32 accumulate, bf16 result.
+// out[t] = sum_j rows[prow_of[t*kp+j]] in slot order, fp32 accumulate, bf16 result; tokens [t0, t1)
+// (t1 < 0: all).
 cudaError_t launch_combine(const uint16_t* rows, const Dims& dm, const LayoutView& lv, uint16_t* out,
-                           cudaStream_t s, int* launches);
+                           cudaStream_t s, int* launches, int t0 = 0, int t1 = -1);
 // d_topk_w[t][j] = sum_nb partial[prow_of[t*kp+j]][nb]
 cudaError_t launch_dw_reduce(const float* partial, int nparts, const Dims& dm, const LayoutView& lv,
                              float* d_topk_w, cudaStream_t s, int* launches);

@@ -53,11 +53,11 @@ cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& 
 
 // out[t][:] = sum_j rows[prow_of[t*kp+j]][:], j ascending, fp32 accumulation, one bf16 rounding.
 // Rows already carry their routing weight (it is applied where the activations are produced).
-__global__ void __launch_bounds__(PERM_THREADS) combine_rows_kernel(const uint16_t* __restrict__ rows, int T, int d,
-                                                                     int kp, const int* __restrict__ prow_of,
+__global__ void __launch_bounds__(PERM_THREADS) combine_rows_kernel(const uint16_t* __restrict__ rows, int t0, int t1,
+                                                                     int d, int kp, const int* __restrict__ prow_of,
                                                                      uint16_t* __restrict__ out) {
   const int nvec = d >> 3;
-  for (int t = blockIdx.x; t < T; t += gridDim.x) {
+  for (int t = t0 + blockIdx.x; t < t1; t += gridDim.x) {
     for (int v = threadIdx.x; v < nvec; v += PERM_THREADS) {
       float acc[8];
 #pragma unroll
@@ -82,10 +82,12 @@ __global__ void __launch_bounds__(PERM_THREADS) combine_rows_kernel(const uint16
 }
 
 cudaError_t launch_combine(const uint16_t* rows, const Dims& dm, const LayoutView& lv, uint16_t* out,
-                           cudaStream_t s, int* launches) {
-  int grid = dm.T < 148 * 16 ? dm.T : 148 * 16;
+                           cudaStream_t s, int* launches, int t0, int t1) {
+  if (t1 < 0) t1 = dm.T;
+  const int n = t1 - t0;
+  int grid = n < 148 * 16 ? n : 148 * 16;
   if (grid < 1) grid = 1;
-  combine_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(rows, dm.T, dm.d, dm.kp(), lv.prow_of, out);
+  combine_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(rows, t0, t1, dm.d, dm.kp(), lv.prow_of, out);
   ++*launches;
   return cudaGetLastError();
 }
