@@ -1,0 +1,57 @@
+"""Token-column tiles at their edges: experts whose token counts sit on and around the 32-token grain,
+the 128-row M-block and the 256-token tile, through forward and backward in both launch modes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_23764_b200 import MoeLayer
+from tests.gpu_util import assert_close_bf16
+
+pytestmark = pytest.mark.gpu
+
+# rows per expert: empty, one token, around 32, around one M-block, around one 256-token tile (one unit of two
+# M-blocks vs a single block followed by block + tail), three and five M-blocks, a long expert
+COUNTS = [0, 1, 31, 32, 33, 127, 128, 129, 160, 255, 256, 257, 300, 383, 384, 385, 513, 640, 1100, 0, 5]
+
+
+def _problem(d, F, seed):
+    counts = np.array(COUNTS)
+    E, T = len(counts), int(counts.sum())
+    g = torch.Generator().manual_seed(seed)
+    ids = torch.from_numpy(np.repeat(np.arange(E), counts).astype(np.int32))
+    ids = ids[torch.randperm(T, generator=g)].reshape(T, 1).contiguous()
+    w = (torch.rand(T, 1, generator=g) + 0.25).float()
+    x = torch.randn(T, d, generator=g).to(torch.bfloat16)
+    W1 = (torch.randn(E, 2 * F, d, generator=g) / d ** 0.5).to(torch.bfloat16)
+    W2 = (torch.randn(E, d, F, generator=g) / d ** 0.5).to(torch.bfloat16)
+    dout = torch.randn(T, d, generator=g).to(torch.bfloat16)
+    return T, E, [t.cuda() for t in (ids, w, x, W1, W2, dout)]
+
+
+@pytest.mark.parametrize("d,F", [(192, 80), (320, 256)])
+@pytest.mark.parametrize("serial", [False, True])
+def test_counts_on_tile_edges(d, F, serial):
+    T, E, (ids, w, x, W1, W2, dout) = _problem(d, F, seed=d + F)
+    layer = MoeLayer(T, d, E, 1, 0, F, renorm=False, save_for_bwd=True, serial=serial)
+    out = layer.ffn_fwd(x, ids, w, W1, W2)
+    dx, dW1, dW2, dw = layer.ffn_bwd(dout, x, ids, w, W1, W2)
+    torch.cuda.synchronize()
+    assert layer.status() == (0, 0)
+    ref_out = oracle.fwd(x, ids.cpu(), w.cpu(), W1, W2)
+    rdx, rdW1, rdW2, rdw = oracle.bwd(dout, x, ids.cpu(), w.cpu(), W1, W2)
+    assert_close_bf16(out, ref_out, "out")
+    assert_close_bf16(dx, rdx, "dx")
+    assert_close_bf16(dW1, rdW1, "dW_gate_up")
+    assert_close_bf16(dW2, rdW2, "dW_down")
+    assert_close_bf16(dw, rdw, "d_topk_w")
+    # every expert on its own: a wrong tile edge would hide in whole-tensor norms
+    for e, n in enumerate(COUNTS):
+        if n == 0:
+            assert torch.count_nonzero(dW1[e]).item() == 0 and torch.count_nonzero(dW2[e]).item() == 0
+        else:
+            assert_close_bf16(dW2[e], rdW2[e], f"dW_down[{e}] ({n} tokens)", max_rel=3e-2, mean_rel=8e-3)
+            tok = (ids[:, 0] == e).nonzero()[:, 0].cpu()
+            assert_close_bf16(out[tok], np.asarray(ref_out)[tok.numpy()], f"out of expert {e} ({n} tokens)",
+                              max_rel=3e-2, mean_rel=8e-3)
+    layer.close()
