@@ -55,3 +55,53 @@ def test_counts_on_tile_edges(d, F, serial):
             assert_close_bf16(out[tok], np.asarray(ref_out)[tok.numpy()], f"out of expert {e} ({n} tokens)",
                               max_rel=3e-2, mean_rel=8e-3)
     layer.close()
+
+
+def _check_against_oracle(T, d, E, k, F, ids, w, seed, serial):
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn(T, d, generator=g).to(torch.bfloat16).cuda()
+    W1 = (torch.randn(E, 2 * F, d, generator=g) / d ** 0.5).to(torch.bfloat16).cuda()
+    W2 = (torch.randn(E, d, F, generator=g) / d ** 0.5).to(torch.bfloat16).cuda()
+    dout = torch.randn(T, d, generator=g).to(torch.bfloat16).cuda()
+    layer = MoeLayer(T, d, E, k, 0, F, renorm=False, save_for_bwd=True, serial=serial)
+    out = layer.ffn_fwd(x, ids, w, W1, W2)
+    dx, dW1, dW2, dw = layer.ffn_bwd(dout, x, ids, w, W1, W2)
+    torch.cuda.synchronize()
+    assert layer.status() == (0, 0)
+    ref_out = oracle.fwd(x, ids.cpu(), w.cpu(), W1, W2)
+    rdx, rdW1, rdW2, rdw = oracle.bwd(dout, x, ids.cpu(), w.cpu(), W1, W2)
+    for got, ref, name in ((out, ref_out, "out"), (dx, rdx, "dx"), (dW1, rdW1, "dW_gate_up"), (dW2, rdW2, "dW_down"),
+                           (dw, rdw, "d_topk_w")):
+        assert_close_bf16(got, ref, name)
+    counts = np.bincount(ids.cpu().numpy().reshape(-1), minlength=E)
+    for e in np.nonzero(counts == 0)[0]:
+        assert torch.count_nonzero(dW1[e]).item() == 0 and torch.count_nonzero(dW2[e]).item() == 0
+    layer.close()
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_every_token_to_one_expert(serial):
+    """The degenerate routing: one expert holds all 1000 rows (eight M-blocks), the other seven none."""
+    T, d, E, F = 1000, 128, 8, 96
+    ids = torch.full((T, 1), 5, dtype=torch.int32).cuda()
+    w = torch.linspace(0.1, 1.0, T).reshape(T, 1).float().cuda()
+    _check_against_oracle(T, d, E, 1, F, ids, w, 11, serial)
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_top_k_equals_number_of_experts(serial):
+    """k = E: every expert receives every token."""
+    T, d, E, F = 300, 128, 4, 64
+    g = torch.Generator().manual_seed(5)
+    ids = torch.stack([torch.randperm(E, generator=g) for _ in range(T)]).to(torch.int32).cuda()
+    w = torch.softmax(torch.randn(T, E, generator=g), dim=1).float().cuda()
+    _check_against_oracle(T, d, E, E, F, ids, w, 12, serial)
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_more_experts_than_rows(serial):
+    """E > T k: at most six of the 64 experts hold a row."""
+    T, d, E, k, F = 3, 64, 64, 2, 32
+    ids = torch.tensor([[7, 40], [40, 63], [0, 7]], dtype=torch.int32).cuda()
+    w = torch.tensor([[0.7, 0.3], [0.5, 0.5], [0.9, 0.1]]).float().cuda()
+    _check_against_oracle(T, d, E, k, F, ids, w, 13, serial)
