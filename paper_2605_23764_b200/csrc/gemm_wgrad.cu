@@ -61,6 +61,17 @@ __device__ __forceinline__ Strip decode_strip(const GemmArgs& a, int s, int rank
   return st;
 }
 
+#ifdef MOE_STATS3
+__device__ long long g_stats_wg[160][8];
+#define SW_DECL long long sw_t = clock64(), sw_acc[4] = {0, 0, 0, 0}
+#define SW_LAP(i) do { const long long n_ = clock64(); sw_acc[i] += n_ - sw_t; sw_t = n_; } while (0)
+#define SW_FLUSH(base) do { for (int i_ = 0; i_ < 4; ++i_) g_stats_wg[blockIdx.x][(base) + i_] += sw_acc[i_]; } while (0)
+#else
+#define SW_DECL
+#define SW_LAP(i)
+#define SW_FLUSH(base)
+#endif
+
 __global__ void __launch_bounds__(WG_THREADS, 1) grouped_wgrad_pair_kernel(const __grid_constant__ GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -107,6 +118,7 @@ __global__ void __launch_bounds__(WG_THREADS, 1) grouped_wgrad_pair_kernel(const
     uint32_t s = 0, ph = 1;
     uint32_t a_ph = (1u << WG_STAGES) - 1;   // per A slot: parity to wait for before the next refill
     bool ok = true;
+    SW_DECL;
     for (int sp = pair; sp < total && ok; sp += npairs) {
       const Strip st = decode_strip(a, sp, rank);
       for (int nb = 0; nb < a.n_tiles_n && ok; ++nb) {
@@ -114,11 +126,13 @@ __global__ void __launch_bounds__(WG_THREADS, 1) grouped_wgrad_pair_kernel(const
         for (int kb = 0; kb < st.nkb; ++kb) {
           const int slot = st.resident ? kb : (int)s;
           int go = 1;
+          SW_LAP(1);
           if (lane == 0) {
             go = mbar_wait(&bars->empty[s], ph, wc, SITE_EMPTY, sp, 50) ? 1 : 0;
             if (go && warp == 0 && load_a) go = mbar_wait(&bars->a_empty[slot], (a_ph >> slot) & 1, wc, SITE_EMPTY, sp, 50) ? 1 : 0;
           }
           go = __shfl_sync(0xffffffffu, go, 0);
+          SW_LAP(0);
           if (!go) { ok = false; break; }
           const int k0 = kb * BK;
           if (warp == 0) {
@@ -137,22 +151,29 @@ __global__ void __launch_bounds__(WG_THREADS, 1) grouped_wgrad_pair_kernel(const
         }
       }
     }
+    SW_LAP(1);
+    if (lane == 0 && warp == 6) SW_FLUSH(4);   // [4] B producer: wait for a free stage, [5] issue
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer (even CTA only)
     if (lane == 0 && rank == 0) {
       uint32_t s = 0, ph = 0, acc_it = 0;
       bool ok = true;
+      SW_DECL;
       for (int sp = pair; sp < total && ok; sp += npairs) {
         const Strip st = decode_strip(a, sp, 0);
         if (st.nkb == 0) continue;
         for (int nb = 0; nb < a.n_tiles_n && ok; ++nb) {
           const int as = acc_it & 1;
+          SW_LAP(2);
           if (!mbar_wait(&bars->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, sp)) { ok = false; break; }
+          SW_LAP(0);
           tc_fence_after_sync();
           const uint32_t d_tmem = tmem_base + as * BN;
           const bool last_use = !st.resident || nb == a.n_tiles_n - 1;
           for (int kb = 0; kb < st.nkb; ++kb) {
+            SW_LAP(2);
             if (!mbar_wait(&bars->full[s], ph, wc, SITE_FULL, sp)) { ok = false; break; }
+            SW_LAP(1);
             tc_fence_after_sync();
             const int slot = st.resident ? kb : (int)s;
             mma_kblock_pair<GEMM_WGRAD>(d_tmem, smem_u32(sA + slot * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES),
@@ -166,6 +187,8 @@ __global__ void __launch_bounds__(WG_THREADS, 1) grouped_wgrad_pair_kernel(const
           ++acc_it;
         }
       }
+      SW_LAP(2);
+      SW_FLUSH(0);   // [0] wait tmem_empty, [1] wait operands, [2] issue
       if (!ok || *reinterpret_cast<volatile int*>(&a.status->abort)) {
         tc_commit_pair(&bars->drain);
         const WaitCtl shortwc{a.status, 20ull * 1000 * 1000};
@@ -244,5 +267,12 @@ cudaError_t launch_wgrad_strips(const GemmArgs& a, int num_sms, cudaStream_t s, 
   if (2 * max_pairs < (int)cfg.gridDim.x) cfg.gridDim = dim3(2 * max_pairs);
   return cudaLaunchKernelEx(&cfg, grouped_wgrad_pair_kernel, a);
 }
+
+#ifdef MOE_STATS3
+extern "C" int moe_debug_stats_wg(long long* host, int reset) {
+  if (reset) { static long long z[160][8]; return (int)cudaMemcpyToSymbol(g_stats_wg, z, sizeof z); }
+  return (int)cudaMemcpyFromSymbol(host, g_stats_wg, sizeof(long long) * 160 * 8);
+}
+#endif
 
 }  // namespace moe
