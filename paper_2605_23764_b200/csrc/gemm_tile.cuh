@@ -193,7 +193,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
   if (MODE == GEMM_GATE_UP) {
     const int prow0 = tl.row0 + quad * 32;             // first padded row of this warp's slab
     const float w = a.prow_w[prow0 + lane];
-    // round 1: A = w * silu(g) * u, 128 columns
+    // first pass over the accumulator: A = w * silu(g) * u, 128 columns
     box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
     for (int c = 0; c < BN / 2; c += 16) {
       float g[16], u[16], act[16];
@@ -213,7 +213,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
       tma_store_commit();
     }
     if (a.save_h) {
-      // rounds 2, 3: the pre-activations, kept for the backward pass (H viewed as [row][gate|up][F])
+      // second and third pass: the pre-activations, kept for the backward pass (H viewed as [row][gate|up][F])
 #pragma unroll 1
       for (int half = 0; half < 2; ++half) {
         box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
