@@ -779,9 +779,12 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
     // of B of a token-row tile, or the weights of a token-column tile; TOK_WARP: the tokens of a token-column tile.
     uint32_t s = 0, ph = 1, n = 0;
     bool ok = true;
+    ST_DECL;
     while (ok) {
       const int rs = n % RING;
+      ST_MARK();
       if (!mbar_wait_cluster(&sh->tk_full[rs], (n / RING) & 1, wc, SITE_FULL, -3)) break;
+      ST_ADD(0);  // loader: waiting for a published tile
       const TileSlot ts = sh->ring[rs];
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(&sh->tk_empty[rs]);
@@ -795,8 +798,10 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
       for (int kb = 0; kb < ts.nkb; ++kb) {
         if (warp == 0 && kb == ts.go_kb && lane == 0 && rank == 0) mbar_arrive(&sh->sched_go);
         int go = 1;
+        ST_ADD(2);  // loader: issuing loads, loop overhead
         if (lane == 0) go = mbar_wait(&sh->empty[s], ph, wc, SITE_EMPTY, n, 50) ? 1 : 0;
         go = __shfl_sync(0xffffffffu, go, 0);
+        ST_ADD(1);  // loader: waiting for a free stage
         if (!go) { ok = false; break; }
         if (!fa.sp.tokcol)
           fusedp_load_stage<BWD>(fa, ts, tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &sh->full[s], lane);
@@ -809,7 +814,9 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
           load_tokens_swap(fa.op[ts.slot], st, kb, rank, sB + s * HALF_B_BYTES, &sh->full[s], lane);
         if (++s == STAGESP) { s = 0; ph ^= 1; }
       }
+      ST_ADD(2);
     }
+    if (lane == 0 && rank == 0) ST_FLUSH(warp == 0 ? 16 : 20, 3);
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer (even CTA)
     if (lane == 0 && rank == 0) {
