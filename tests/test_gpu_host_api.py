@@ -51,3 +51,40 @@ def test_phase_times_are_reported_per_operator():
         assert set(ph) == want and all(v > 0 for v in ph.values())
         assert layer.launches() == (7 if serial else 5)
         layer.close()
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_back_to_back_host_steps_keep_their_own_inputs(serial):
+    """Three training steps through the host entry points with different inputs and no synchronisation in
+    between: the copy-in stream may run ahead of the compute stream, so a step's x / dout must not land in
+    the staging buffers before the previous step has read them."""
+    T, d, E, k, S, F = 1500, 256, 8, 2, 0, 128   # T >= 256: the chunked copy-out of the forward is in play
+    pin = dict(pin_memory=True)
+    layer = MoeLayer(T, d, E, k, S, F, renorm=True, save_for_bwd=True, serial=serial)
+    ref = MoeLayer(T, d, E, k, S, F, renorm=True, save_for_bwd=True, serial=serial)
+    steps = []
+    for i in range(3):
+        x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, 100 + i)
+        ids, w = ref.route(logits)
+        out = ref.ffn_fwd(x, ids, w, W1, W2)
+        dx, dW1, dW2, dw = ref.ffn_bwd(dout, x, ids, w, W1, W2)
+        steps.append(dict(x=x.cpu().pin_memory(), dout=dout.cpu().pin_memory(), ids=ids.cpu().pin_memory(),
+                          w=w.cpu().pin_memory(), W1=W1, W2=W2, out=out.cpu(), dx=dx.cpu(), dw=dw.cpu(),
+                          dW1=dW1.clone(), dW2=dW2.clone(),
+                          oh=torch.empty(T, d, dtype=torch.bfloat16, **pin),
+                          dxh=torch.empty(T, d, dtype=torch.bfloat16, **pin),
+                          dwh=torch.empty(T, k, dtype=torch.float32, **pin),
+                          gW1=torch.empty_like(W1), gW2=torch.empty_like(W2)))
+    torch.cuda.synchronize()
+    for s in steps:   # enqueue everything, synchronise once
+        B.moe_ffn_fwd_host(layer.ctx, s["x"], s["ids"], s["w"], s["W1"], s["W2"], s["oh"], T)
+        B.moe_ffn_bwd_host(layer.ctx, s["dout"], s["W1"], s["W2"], s["dxh"], s["gW1"], s["gW2"], s["dwh"], T)
+    torch.cuda.synchronize()
+    assert layer.status() == (0, 0)
+    for i, s in enumerate(steps):
+        assert torch.equal(s["oh"], s["out"]), f"step {i}: out"
+        assert torch.equal(s["dxh"], s["dx"]), f"step {i}: dx"
+        assert torch.equal(s["dwh"], s["dw"]), f"step {i}: d_topk_w"
+        assert torch.equal(s["gW1"], s["dW1"]) and torch.equal(s["gW2"], s["dW2"]), f"step {i}: weight gradients"
+    layer.close()
+    ref.close()
