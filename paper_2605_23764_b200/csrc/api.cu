@@ -569,7 +569,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     {
       Phase ph(c, MOE_PHASE_GATHER, st);
       MOE_CUDA(launch_gather(x, w, dm, lv, c->at<uint16_t>(p.Xp), c->at<float>(p.prow_w), p.cap_rows, st,
-                             &c->launches));
+                             &c->launches, c->status(), c->budget_ns));
     }
     {
       Phase ph(c, MOE_PHASE_GEMM_GATE_UP, st);
@@ -632,7 +632,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     {  // backward Dispatch: expert-ordered gather of the upstream gradient
       Phase ph(c, MOE_PHASE_BWD_GATHER, st);
       MOE_CUDA(launch_gather(dout, nullptr, dm, lv, c->at<uint16_t>(p.dOutp), nullptr, p.cap_rows, st,
-                             &c->launches));
+                             &c->launches, c->status(), c->budget_ns));
     }
     {
       Phase ph(c, MOE_PHASE_ACT_GRAD, st);

@@ -53,7 +53,8 @@ cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView&
 // Xp[p] = src[token of padded row p] (zeros on padding rows); optionally prow_w[p] = routing weight
 // of the row (1 for shared experts, 0 on padding rows).
 cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& dm, const LayoutView& lv,
-                          uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches);
+                          uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches,
+                          DevStatus* status = nullptr, uint64_t budget_ns = 0);
 // out[t] = sum_j rows[prow_of[t*kp+j]] in slot order, fp32 accumulate, bf16 result; tokens [t0, t1)
 // (t1 < 0: all).
 cudaError_t launch_combine(const uint16_t* rows, const Dims& dm, const LayoutView& lv, uint16_t* out,

@@ -1,6 +1,8 @@
 // Permute-gather (Dispatch / backward Dispatch on one GPU), combine (Combine / backward Combine)
 // and the small reduction that finishes the routing-weight gradient.  All three are pure
 // HBM-bandwidth work: 16-byte vector accesses, one row handled by one block at a time.
+#include <stdlib.h>
+
 #include "moe_internal.h"
 
 namespace moe {
@@ -42,12 +44,111 @@ __global__ void __launch_bounds__(PERM_THREADS) gather_rows_kernel(const uint16_
   }
 }
 
+// The same gather with bulk copies: one warp per SM, each of up to eight lanes runs its own
+// two-slot pipeline (row i+1 arrives in one shared-memory slot while row i leaves from the other):
+// whole rows move as single global -> shared and shared -> global bulk copies, up to 200 KB in
+// flight per SM, and no thread touches the data.  Padding rows leave from a zeroed slot.
+constexpr int GB_MAX_LANES = 8;
+constexpr int GB_SMEM_BUDGET = 216 * 1024;
+
+__global__ void __launch_bounds__(32) gather_rows_bulk_kernel(const uint16_t* __restrict__ src,
+                                                              const float* __restrict__ topk_w, int d, int k, int kp,
+                                                              LayoutView lv, uint16_t* __restrict__ dst,
+                                                              float* __restrict__ prow_w, int lanes, DevStatus* status,
+                                                              uint64_t budget_ns) {
+  extern __shared__ __align__(128) uint8_t gsm[];
+  __shared__ uint64_t full[2 * GB_MAX_LANES];
+  const int lane = threadIdx.x;
+  const uint32_t row_bytes = (uint32_t)d * 2;
+  uint8_t* zero_row = gsm;                                   // [row_bytes]
+  uint8_t* slots = gsm + row_bytes;                          // [lanes][2][row_bytes]
+  for (uint32_t i = lane; i < row_bytes / 16; i += 32) reinterpret_cast<uint4*>(zero_row)[i] = make_uint4(0, 0, 0, 0);
+  if (lane < 2 * GB_MAX_LANES) mbar_init(&full[lane], 1);
+  mbar_fence_init();
+  fence_proxy_async();
+  __syncwarp();
+  if (lane >= lanes) return;
+  const WaitCtl wc{status, budget_ns};
+  const int r_pad = lv.meta[1];
+  const int stride = gridDim.x * lanes;
+  uint8_t* my = slots + (size_t)lane * 2 * row_bytes;
+  // row -> source row (or -1 for a padding row); also writes the row's routing weight
+  auto source_of = [&](int p) -> long {
+    const int e = lv.mblk_expert[p / BLOCK_M];
+    const int local = p - lv.pad_off[e];
+    if (local >= lv.counts[e]) {
+      if (prow_w) prow_w[p] = 0.0f;
+      return -1;
+    }
+    const int slot = lv.src_of[lv.offsets[e] + local];
+    const int t = slot / kp, j = slot - t * kp;
+    if (prow_w) prow_w[p] = j < k ? topk_w[(size_t)t * k + j] : 1.0f;
+    return t;
+  };
+  auto load = [&](long t, int b) {
+    mbar_expect_tx(&full[2 * lane + b], row_bytes);
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(my + (size_t)b * row_bytes)), "l"(src + (size_t)t * d), "r"(row_bytes),
+                   "r"(smem_u32(&full[2 * lane + b]))
+                 : "memory");
+  };
+  int p = blockIdx.x * lanes + lane;
+  uint32_t n = 0, ph[2] = {0, 0};
+  long t_cur = p < r_pad ? source_of(p) : -1;
+  if (p < r_pad && t_cur >= 0) load(t_cur, 0);
+  for (; p < r_pad; p += stride, ++n) {
+    const int b = n & 1;
+    const int pn = p + stride;
+    const long t_next = pn < r_pad ? source_of(pn) : -1;
+    // the other slot is free once the previous row's store has read it
+    tma_store_wait_read();
+    if (pn < r_pad && t_next >= 0) load(t_next, b ^ 1);
+    const uint8_t* from = zero_row;
+    if (t_cur >= 0) {
+      if (!mbar_wait(&full[2 * lane + b], ph[b], wc, SITE_FULL, p)) break;
+      ph[b] ^= 1;
+      from = my + (size_t)b * row_bytes;
+    }
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst + (size_t)p * d), "r"(smem_u32(from)), "r"(row_bytes)
+                 : "memory");
+    tma_store_commit();
+    t_cur = t_next;
+  }
+  tma_store_wait_all();
+}
+
 cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& dm, const LayoutView& lv,
-                          uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches) {
+                          uint16_t* dst, float* prow_w, int rows_cap, cudaStream_t s, int* launches,
+                          DevStatus* status, uint64_t budget_ns) {
+  ++*launches;
+  const size_t row_bytes = (size_t)dm.d * 2;
+  int lanes = (int)((GB_SMEM_BUDGET - row_bytes) / (2 * row_bytes));
+  if (lanes > GB_MAX_LANES) lanes = GB_MAX_LANES;
+  static int bulk = -1;   // diagnostic knob: MOE_B200_GATHER_THREADS=1 keeps the copy in registers
+  if (bulk < 0) {
+    const char* e = getenv("MOE_B200_GATHER_THREADS");
+    bulk = (e && e[0] == '1') ? 0 : 1;
+  }
+  // rows of 8 KB and more: below that the per-row latency of the two-slot pipelines outweighs the gain
+  if (bulk && status && lanes >= 2 && row_bytes >= 8192 && row_bytes % 16 == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
+    const size_t smem = row_bytes * (1 + 2 * (size_t)lanes);
+    static size_t attr_bytes = 0;
+    if (smem > attr_bytes) {
+      cudaError_t e = cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      attr_bytes = smem;
+    }
+    int sms = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    gather_rows_bulk_kernel<<<sms, 32, smem, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w, lanes, status,
+                                                  budget_ns);
+    return cudaGetLastError();
+  }
   int grid = rows_cap < 148 * 16 ? rows_cap : 148 * 16;
   if (grid < 1) grid = 1;
   gather_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w);
-  ++*launches;
   return cudaGetLastError();
 }
 

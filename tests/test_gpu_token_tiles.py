@@ -105,3 +105,13 @@ def test_more_experts_than_rows(serial):
     ids = torch.tensor([[7, 40], [40, 63], [0, 7]], dtype=torch.int32).cuda()
     w = torch.tensor([[0.7, 0.3], [0.5, 0.5], [0.9, 0.1]]).float().cuda()
     _check_against_oracle(T, d, E, k, F, ids, w, 13, serial)
+
+
+def test_wide_rows_take_the_bulk_copy_gather():
+    """Rows of 8 KB and more are gathered with bulk copies (whole rows through shared-memory slots, padding
+    rows from a zeroed slot): d = 4096 with ragged expert segments, forward and backward."""
+    T, d, E, k, F = 700, 4096, 6, 2, 32
+    g = torch.Generator().manual_seed(3)
+    ids = torch.stack([torch.randperm(E, generator=g)[:k] for _ in range(T)]).to(torch.int32).cuda()
+    w = torch.softmax(torch.randn(T, k, generator=g), dim=1).float().cuda()
+    _check_against_oracle(T, d, E, k, F, ids, w, 14, serial=True)
