@@ -115,3 +115,20 @@ def test_wide_rows_take_the_bulk_copy_gather():
     ids = torch.stack([torch.randperm(E, generator=g)[:k] for _ in range(T)]).to(torch.int32).cuda()
     w = torch.softmax(torch.randn(T, k, generator=g), dim=1).float().cuda()
     _check_against_oracle(T, d, E, k, F, ids, w, 14, serial=True)
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_skewed_routing_forward_and_backward(serial):
+    """Zipf-like expert popularity with four unreachable experts: segments from empty to a few thousand rows
+    (streamed and resident weight-gradient strips, token tiles of one and two M-blocks side by side)."""
+    T, d, E, k, F = 2048, 512, 32, 4, 256
+    g = torch.Generator().manual_seed(21)
+    rank = torch.randperm(E, generator=g).float()
+    logits = torch.randn(T, E, generator=g) * 1.3 - 1.2 * torch.log(rank + 1.0)
+    logits[:, rank >= E - 4] = -1e4
+    top = torch.topk(logits, k, dim=1)
+    ids = top.indices.to(torch.int32).cuda()
+    w = torch.softmax(top.values, dim=1).float().cuda()
+    counts = np.bincount(ids.cpu().numpy().reshape(-1), minlength=E)
+    assert (counts == 0).sum() >= 4 and counts.max() > 640, counts
+    _check_against_oracle(T, d, E, k, F, ids, w, 22, serial)
