@@ -379,7 +379,13 @@ def main():
         """Roofline of the operator with the largest time, and of the whole step."""
         work = phase_work(cfg, train)
         phases_ms = res["phases_ms"]
-        peak_tf = peaks["bf16_tflops_sustained"] if res["timed_ms"] > 500 else peaks["bf16_tflops"]
+        # sustained peak for work timed inside a long, power-capped region (the clocks sampled during the timed
+        # steps say which): more than 0.5 s of timed work, or the power cap active with SM clocks a fifth or
+        # more below their maximum; burst peak otherwise
+        clk = res.get("clocks") or {}
+        capped = ("sw_power_cap" in (clk.get("reasons") or []) and clk.get("sm_mhz") and clk.get("sm_max_mhz")
+                  and clk["sm_mhz"] < 0.8 * clk["sm_max_mhz"])
+        peak_tf = peaks["bf16_tflops_sustained"] if (res["timed_ms"] > 500 or capped) else peaks["bf16_tflops"]
         peak_gb = peaks["hbm_gbs"]
         dom = max((k for k in phases_ms if k in work), key=lambda k: phases_ms[k], default=None)
         roof = None
