@@ -132,7 +132,7 @@ struct Carve {
 
 // Byte offsets of every workspace tensor.
 struct WsPlan {
-  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
+  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, work_start, wblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
       dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, stats, total;
   int cap_rows, nblk_max, ntn_act, ctr_count;
 };
@@ -157,6 +157,8 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.mblk_expert = c.take(sizeof(int) * (cap / BLOCK_M + 1));
   p.pair_start = c.take(sizeof(int) * (Ep + 1));
   p.pblk_expert = c.take(sizeof(int) * (cap / BLOCK_M + 1));
+  p.work_start = c.take(sizeof(int) * (Ep + 1));
+  p.wblk_expert = c.take(sizeof(int) * (cap / BLOCK_M + 1));
   p.blk_hist = c.take(sizeof(int) * (size_t)p.nblk_max * Ep);
   p.row_of = c.take(sizeof(int) * (slots + 1));
   p.src_of = c.take(sizeof(int) * (slots + 1));
@@ -250,6 +252,8 @@ struct moe_ctx {
     lv.mblk_expert = at<int>(plan.mblk_expert);
     lv.pair_start = at<int>(plan.pair_start);
     lv.pblk_expert = at<int>(plan.pblk_expert);
+    lv.work_start = at<int>(plan.work_start);
+    lv.wblk_expert = at<int>(plan.wblk_expert);
     lv.meta = at<int>(plan.meta);
     lv.blk_hist = at<int>(plan.blk_hist);
     return lv;
@@ -307,6 +311,8 @@ GemmArgs base_args(const moe_ctx* c) {
   g.meta = lv.meta;
   g.pair_start = lv.pair_start;
   g.pblk_expert = lv.pblk_expert;
+  g.work_start = lv.work_start;
+  g.wblk_expert = lv.wblk_expert;
   g.cap_rows = c->plan.cap_rows;
   g.Ep = c->shape.E + c->shape.n_shared;
   g.F = c->shape.F;

@@ -890,7 +890,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_pair_kernel(const __gr
           // the staging area changes hands between the two epilogue kinds: let the earlier stores finish reading
           if (lane == 0) tma_store_wait_read();
           __syncwarp();
-          SwStaging sg{sOut + quad * OUT_STAGE_BYTES, 0, sScr + quad * SW_SCRATCH_BYTES};
+          SwStaging sg{sOut + quad * OUT_STAGE_BYTES, 0, sScr + quad * SW_SCRATCH_BYTES, SW_SLOTS, SW_SLOT_BYTES};
           fusedp_epilogue_swap<BWD>(fa, ts, slot_swap_tile(ts), tmem_base + as * BN, rank, quad, lane, sg);
         } else if (!idle) {
           fused_epilogue<BWD>(fa, ts, tl, tmem_base + as * BN, quad, lane, stg);

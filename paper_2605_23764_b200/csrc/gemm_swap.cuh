@@ -35,29 +35,62 @@ struct SwapTile {
 template <int MODE>
 __device__ __forceinline__ int swap_tile_features() { return MODE == GEMM_GATE_UP ? 128 : 256; }
 
-// Tile order: expert-major; inside an expert the feature tile is the slow index and the token tile
-// the fast one (tiles running at the same time share one slab of weights in L2).  Token tiles are the
-// expert's balanced units of one or two M-blocks (schedule.h), cut at the expert's last 32-row group.
-template <int MODE>
-__device__ __forceinline__ SwapTile decode_swap_tile(const GemmArgs& a, int t) {
-  SwapTile st;
-  const int e = a.pblk_expert[t / a.n_tiles_n];
-  const int ps = a.pair_start[e];
-  const int pcount = a.pair_start[e + 1] - ps;   // units = ceil(M-blocks / 2)
-  const int local = t - ps * a.n_tiles_n;
-  st.nb = local / pcount;
-  const int pl = local - st.nb * pcount;
-  st.e = e;
+// Token tile `u` (a balanced unit of one or two M-blocks, schedule.h) of expert e, cut at the expert's
+// last 32-row group.
+__device__ __forceinline__ void unit_tokens(const GemmArgs& a, int e, int u, int* row0, int* ntok) {
   int first, count;
-  balanced_unit(a.mb_start[e + 1] - a.mb_start[e], pl, &first, &count);
+  balanced_unit(a.mb_start[e + 1] - a.mb_start[e], u, &first, &count);
   const int n32 = (a.counts[e] + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);
   int end = (first + count) * BLOCK_M;
   if (end > n32) end = n32;
-  st.row0 = (a.mb_start[e] + first) * BLOCK_M;
-  st.ntok = end - first * BLOCK_M;
-  st.n0 = st.nb * swap_tile_features<MODE>();
-  st.nkb = (a.K + BK - 1) / BK;
-  return st;
+  *row0 = (a.mb_start[e] + first) * BLOCK_M;
+  *ntok = end - first * BLOCK_M;
+}
+
+// One work item of the one-launch-per-operator kernel: a token tile, or -- in the operators that merge,
+// for an expert with an odd count of three or more M-blocks -- its last two token tiles (one block;
+// block + tail) under ONE k-loop: the weight stage is written to shared memory once and multiplied with
+// both token tiles into the two TMEM accumulators (shared-memory traffic bounds these kernels, and the
+// weights are the larger half of it).  For the epilogue warps the item is two consecutive tiles.
+// Only the operators with a short epilogue merge (down, gate_grad): with both accumulators in use the
+// epilogue of the second tile is exposed.
+struct SwapWork {
+  SwapTile a, b;
+  bool merged;
+};
+template <int MODE>
+__host__ __device__ constexpr bool swap_merges() { return MODE == GEMM_DOWN || MODE == GEMM_GATE_GRAD; }
+// token bytes of a stage per CTA: up to 128 rows, or (128 + 256) / 2 rows of a merged item
+template <int MODE>
+__host__ __device__ constexpr int tok_stage_bytes() { return (swap_merges<MODE>() ? 3 : 2) * 64 * BK * 2; }
+
+template <int MODE>
+__device__ __forceinline__ int total_swap_work(const GemmArgs& a) {
+  return (swap_merges<MODE>() ? a.meta[4] : a.meta[3]) * a.n_tiles_n;
+}
+
+// Item order: expert-major; inside an expert the feature tile is the slow index and the item the
+// fast one (items running at the same time share one slab of weights in L2).
+template <int MODE>
+__device__ __forceinline__ SwapWork decode_swap_work(const GemmArgs& a, int t) {
+  SwapWork w;
+  const int* start = swap_merges<MODE>() ? a.work_start : a.pair_start;
+  const int e = (swap_merges<MODE>() ? a.wblk_expert : a.pblk_expert)[t / a.n_tiles_n];
+  const int ws = start[e];
+  const int wcount = start[e + 1] - ws;
+  const int local = t - ws * a.n_tiles_n;
+  const int nb = local / wcount;
+  const int wi = local - nb * wcount;
+  const int mc = a.mb_start[e + 1] - a.mb_start[e];
+  w.merged = swap_merges<MODE>() && (mc & 1) && mc >= 3 && wi == wcount - 1;   // units wi and wi + 1
+  w.a.e = w.b.e = e;
+  w.a.nb = w.b.nb = nb;
+  w.a.n0 = w.b.n0 = nb * swap_tile_features<MODE>();
+  w.a.nkb = w.b.nkb = (a.K + BK - 1) / BK;
+  unit_tokens(a, e, wi, &w.a.row0, &w.a.ntok);
+  w.b.row0 = 0; w.b.ntok = 0;
+  if (w.merged) unit_tokens(a, e, wi + 1, &w.b.row0, &w.b.ntok);
+  return w;
 }
 
 __device__ __forceinline__ uint32_t swap_stage_tx_bytes(int ntok) {
@@ -70,7 +103,7 @@ __device__ __forceinline__ uint32_t swap_stage_tx_bytes(int ntok) {
 // (128, 64, 32, 16 rows).  The even CTA's weight producer arms the barrier for both CTAs' bytes.
 __device__ __forceinline__ void load_tokens_swap(const GemmArgs& a, const SwapTile& st, int kb, int rank, uint8_t* sT,
                                                  uint64_t* bar, int lane) {
-  if (lane >= 4) return;
+  if (lane < 0 || lane >= 4) return;
   const int half = st.ntok >> 1;
   const int size = 128 >> lane;                 // lane 0: 128-row box ... lane 3: 16-row box
   if (!(half & size)) return;
@@ -80,9 +113,9 @@ __device__ __forceinline__ void load_tokens_swap(const GemmArgs& a, const SwapTi
 }
 template <int MODE>
 __device__ __forceinline__ void load_weights_swap(const GemmArgs& a, const SwapTile& st, int kb, int rank, uint8_t* sW,
-                                                  uint64_t* bar, int lane) {
+                                                  uint64_t* bar, int lane, int ntok_total = -1) {
   const int k0 = kb * BK;
-  if (lane == 0 && rank == 0) mbar_expect_tx(bar, swap_stage_tx_bytes(st.ntok));
+  if (lane == 0 && rank == 0) mbar_expect_tx(bar, swap_stage_tx_bytes(ntok_total < 0 ? st.ntok : ntok_total));
   __syncwarp();
   const int brow = st.e * a.b_rows_per_expert;
   if (MODE == GEMM_GATE_UP) {
@@ -125,12 +158,17 @@ struct SwStaging {
   uint8_t* base;     // SW_SLOTS slots of SW_SLOT_BYTES
   uint32_t round;
   uint8_t* scratch;  // act_grad: 4 KB of this warp (two halves of [gate | up][16 tokens][32 features])
+  uint32_t slots;       // staging slots of this warp (1 or 2)
+  uint32_t slot_bytes;  // SW_SLOT_BYTES, or 2 KB in the plain-store operators that give room to the operand stages
 };
 constexpr int SW_SCRATCH_BYTES = 4096;
 __device__ __forceinline__ uint8_t* sw_acquire(SwStaging& sg, int lane) {
-  if (lane == 0) tma_store_wait_read_n<SW_SLOTS - 1>();   // the slot's previous stores have read it
+  if (lane == 0) {   // the slot's previous stores have read it
+    if (sg.slots == 1) tma_store_wait_read();
+    else tma_store_wait_read_n<SW_SLOTS - 1>();
+  }
   __syncwarp();
-  uint8_t* slot = sg.base + (sg.round % SW_SLOTS) * SW_SLOT_BYTES;
+  uint8_t* slot = sg.base + (sg.round % sg.slots) * sg.slot_bytes;
   ++sg.round;
   return slot;
 }

@@ -14,7 +14,8 @@ namespace moe {
 #ifndef MOE_STAGES3
 #define MOE_STAGES3 5
 #endif
-constexpr int STAGES3 = MOE_STAGES3;   // 32 KB operand stages; the rest: 4 epilogue warps x staging ring
+constexpr int STAGES3 = MOE_STAGES3;   // operand stages: 16 KB of weights + 16 KB of tokens (24 KB in the operators
+                                       // that merge token tiles, which keep one staging slot per epilogue warp instead of two)
 
 struct __align__(8) SwapBarriers {
   uint64_t full[STAGES3];     // used in the even CTA: bytes of both CTAs' loads
@@ -26,9 +27,18 @@ struct __align__(8) SwapBarriers {
   uint32_t pad;
 };
 
-constexpr size_t GEMM3_SMEM_BYTES = 1024 + (size_t)STAGES3 * STAGE2_BYTES + 4 * SW_SLOTS * SW_SLOT_BYTES +
-                                    4 * SW_SCRATCH_BYTES + sizeof(SwapBarriers);
-static_assert(GEMM3_SMEM_BYTES <= 227 * 1024, "shared memory budget");
+// staging per epilogue warp: two slots of 4 KB; the operators that merge store plain 2 KB boxes and keep
+// two slots of 2 KB (their operand stages need the room)
+template <int MODE>
+__host__ __device__ constexpr int staging_slot_bytes3() { return swap_merges<MODE>() ? SW_SLOT_BYTES / 2 : SW_SLOT_BYTES; }
+template <int MODE>
+__host__ __device__ constexpr size_t gemm3_smem_bytes() {
+  return 1024 + (size_t)STAGES3 * (W_STAGE_BYTES + tok_stage_bytes<MODE>()) + 4 * SW_SLOTS * staging_slot_bytes3<MODE>() +
+         (MODE == GEMM_ACT_GRAD ? 4 * SW_SCRATCH_BYTES : 0) + sizeof(SwapBarriers);
+}
+static_assert(gemm3_smem_bytes<GEMM_GATE_UP>() <= 227 * 1024 && gemm3_smem_bytes<GEMM_DOWN>() <= 227 * 1024 &&
+                  gemm3_smem_bytes<GEMM_ACT_GRAD>() <= 227 * 1024 && gemm3_smem_bytes<GEMM_GATE_GRAD>() <= 227 * 1024,
+              "shared memory budget");
 
 #ifdef MOE_STATS3
 __device__ long long g_stats3[5][160][8];
@@ -47,11 +57,13 @@ template <int MODE>
 __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(const __grid_constant__ GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  constexpr int TOKB = tok_stage_bytes<MODE>();
+  constexpr int SLOTB = staging_slot_bytes3<MODE>();
   uint8_t* sW = smem;                                   // [STAGES3][16 KB] weights
-  uint8_t* sT = smem + STAGES3 * W_STAGE_BYTES;         // [STAGES3][16 KB] tokens (this CTA's half)
-  uint8_t* sOut = smem + STAGES3 * STAGE2_BYTES;
-  uint8_t* sScr = sOut + 4 * SW_SLOTS * SW_SLOT_BYTES;  // act_grad: per epilogue warp 4 KB for the saved pre-activations
-  SwapBarriers* bars = reinterpret_cast<SwapBarriers*>(sScr + 4 * SW_SCRATCH_BYTES);
+  uint8_t* sT = smem + STAGES3 * W_STAGE_BYTES;         // [STAGES3][TOKB] tokens (this CTA's half)
+  uint8_t* sOut = smem + STAGES3 * (W_STAGE_BYTES + TOKB);
+  uint8_t* sScr = sOut + 4 * SW_SLOTS * SLOTB;          // act_grad: per epilogue warp 4 KB for the saved pre-activations
+  SwapBarriers* bars = reinterpret_cast<SwapBarriers*>(sScr + (MODE == GEMM_ACT_GRAD ? 4 * SW_SCRATCH_BYTES : 0));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int rank = (int)cluster_ctarank();
@@ -84,7 +96,7 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
   cluster_sync_all();  // both CTAs' barriers exist before anyone signals across the pair
   tc_fence_after_sync();
   const uint32_t tmem_base = bars->tmem_base;
-  const int total = a.meta[3] * a.n_tiles_n;
+  const int total = total_swap_work<MODE>(a);
 
   if (warp == 0 || warp == 6) {
     // ------------------------------------------------ TMA producers (both CTAs, one box per lane)
@@ -92,7 +104,8 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
     bool ok = true;
     S3_DECL;
     for (int t = pair; t < total && ok; t += npairs) {
-      const SwapTile st = decode_swap_tile<MODE>(a, t);
+      const SwapWork wk = decode_swap_work<MODE>(a, t);
+      const SwapTile& st = wk.a;
       for (int kb = 0; kb < st.nkb; ++kb) {
         int go = 1;
         S3_LAP(1);
@@ -100,8 +113,13 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
         go = __shfl_sync(0xffffffffu, go, 0);
         S3_LAP(0);
         if (!go) { ok = false; break; }
-        if (warp == 0) load_weights_swap<MODE>(a, st, kb, rank, sW + s * W_STAGE_BYTES, &bars->full[s], lane);
-        else load_tokens_swap(a, st, kb, rank, sT + s * HALF_B_BYTES, &bars->full[s], lane);
+        if (warp == 0) {
+          load_weights_swap<MODE>(a, st, kb, rank, sW + s * W_STAGE_BYTES, &bars->full[s], lane, wk.a.ntok + wk.b.ntok);
+        } else {
+          load_tokens_swap(a, wk.a, kb, rank, sT + s * TOKB, &bars->full[s], lane);
+          if (wk.merged)   // lanes 4..7: the second token tile, behind the first in the stage
+            load_tokens_swap(a, wk.b, kb, rank, sT + s * TOKB + (wk.a.ntok >> 1) * (BK * 2), &bars->full[s], lane - 4);
+        }
         if (++s == STAGES3) { s = 0; ph ^= 1; }
       }
     }
@@ -119,30 +137,38 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
       bool ok = true;
       S3_DECL;
       for (int t = pair; t < total && ok; t += npairs) {
-        const SwapTile st = decode_swap_tile<MODE>(a, t);
+        const SwapWork wk = decode_swap_work<MODE>(a, t);
         const int as = acc_it & 1;
         S3_LAP(2);
         if (!mbar_wait(&bars->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, t)) { ok = false; break; }
+        if (wk.merged &&   // the second token tile accumulates in the other buffer
+            !mbar_wait(&bars->tmem_empty[as ^ 1], (((acc_it + 1) >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, t)) { ok = false; break; }
         S3_LAP(0);
         tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + as * BN;
-        const uint32_t idesc = swap_idesc<MODE>(st.ntok);
-        for (int kb = 0; kb < st.nkb; ++kb) {
+        const uint32_t d_tmem = tmem_base + as * BN, d_tmem_b = tmem_base + (as ^ 1) * BN;
+        const uint32_t idesc = swap_idesc<MODE>(wk.a.ntok), idesc_b = swap_idesc<MODE>(wk.merged ? wk.b.ntok : TOK_GRAIN);
+        const uint32_t t_off_b = (uint32_t)((wk.a.ntok >> 1) * (BK * 2)) >> 4;
+        for (int kb = 0; kb < wk.a.nkb; ++kb) {
           S3_LAP(2);
           if (!mbar_wait(&bars->full[s], ph, wc, SITE_FULL, t)) { ok = false; break; }
           S3_LAP(1);
           tc_fence_after_sync();
           mma_kblock_swap<MODE>(d_tmem, w_lo, t_lo, idesc, kb == 0);
+          if (wk.merged) mma_kblock_swap<MODE>(d_tmem_b, w_lo, t_lo + t_off_b, idesc_b, kb == 0);
           tc_commit_pair(&bars->empty[s]);   // frees the stage in both CTAs
           if (++s == STAGES3) {
             s = 0; ph ^= 1; w_lo = w_lo0; t_lo = t_lo0;
           } else {
-            w_lo += W_STAGE_BYTES >> 4; t_lo += HALF_B_BYTES >> 4;
+            w_lo += W_STAGE_BYTES >> 4; t_lo += TOKB >> 4;
           }
         }
         if (!ok) break;
         tc_commit_pair(&bars->tmem_full[as]);  // accumulator slices ready in both CTAs
         ++acc_it;
+        if (wk.merged) {
+          tc_commit_pair(&bars->tmem_full[as ^ 1]);
+          ++acc_it;
+        }
       }
       S3_LAP(2);
       S3_FLUSH(0);   // [0] wait tmem_empty, [1] wait operands, [2] issue
@@ -155,18 +181,21 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
   } else if (warp < 6) {
     // ------------------------------------------------ epilogue warps (both CTAs, own features)
     const int quad = warp & 3;
-    SwStaging sg{sOut + quad * SW_SLOTS * SW_SLOT_BYTES, 0, sScr + quad * SW_SCRATCH_BYTES};
+    SwStaging sg{sOut + quad * SW_SLOTS * SLOTB, 0, sScr + quad * SW_SCRATCH_BYTES, SW_SLOTS, (uint32_t)SLOTB};
     uint32_t acc_it = 0;
-    for (int t = pair; t < total; t += npairs) {
-      const SwapTile st = decode_swap_tile<MODE>(a, t);
-      const int as = acc_it & 1;
-      if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, t, 200)) break;
-      tc_fence_after_sync();
-      epilogue_swap<MODE>(a, st, tmem_base + as * BN, rank, quad, lane, sg);
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_leader(&bars->tmem_empty[as]);
-      ++acc_it;
+    bool ok = true;
+    for (int t = pair; t < total && ok; t += npairs) {
+      const SwapWork wk = decode_swap_work<MODE>(a, t);
+      for (int part = 0; part < (wk.merged ? 2 : 1); ++part) {   // a merged item is two consecutive tiles here
+        const int as = acc_it & 1;
+        if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, t, 200)) { ok = false; break; }
+        tc_fence_after_sync();
+        epilogue_swap<MODE>(a, part ? wk.b : wk.a, tmem_base + as * BN, rank, quad, lane, sg);
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_leader(&bars->tmem_empty[as]);
+        ++acc_it;
+      }
     }
     if (lane == 0) tma_store_wait_all();
   }
@@ -187,7 +216,7 @@ static cudaError_t launch_swap_mode(const GemmArgs& a, int num_sms, cudaStream_t
   static bool attr_set = false;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(grouped_gemm_swap_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)GEMM3_SMEM_BYTES);
+                                         (int)gemm3_smem_bytes<MODE>());
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -196,7 +225,7 @@ static cudaError_t launch_swap_mode(const GemmArgs& a, int num_sms, cudaStream_t
   memset(&cfg, 0, sizeof cfg);
   cfg.gridDim = dim3((num_sms / 2) * 2);
   cfg.blockDim = dim3(GEMM3_THREADS);
-  cfg.dynamicSmemBytes = GEMM3_SMEM_BYTES;
+  cfg.dynamicSmemBytes = gemm3_smem_bytes<MODE>();
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;

@@ -39,7 +39,10 @@ struct LayoutView {
   int* mblk_expert;  // [R_pad_max / BLOCK_M] expert of each M-block
   int* pair_start;   // [Ep+1]  first M-block pair of each expert (pairs = ceil(M-blocks / 2))
   int* pblk_expert;  // [pairs] expert of each M-block pair
-  int* meta;         // [8]     {num_mblocks, R_pad, rows, num_pairs, 0...}
+  int* work_start;   // [Ep+1]  first work item of each expert (token-column GEMMs that merge: its units, the last
+                     //         two of an odd M-block count >= 3 merged into one item)
+  int* wblk_expert;  // [items] expert of each work item
+  int* meta;         // [8]     {num_mblocks, R_pad, rows, num_pairs, num_work_items, 0...}
   int* blk_hist;     // [nblk][Ep] per-block histograms, then per-block exclusive prefixes
 };
 
@@ -85,6 +88,8 @@ struct GemmArgs {
   const int* meta;
   const int* pair_start;   // CTA-pair kernels: first M-block pair of each expert
   const int* pblk_expert;  // CTA-pair kernels: expert of each M-block pair
+  const int* work_start;   // token-column kernel: first work item of each expert
+  const int* wblk_expert;  // token-column kernel: expert of each work item
   int cap_rows;            // rows of the padded row space (a row coordinate >= cap_rows reads zeros)
   int Ep;
   int n_tiles_n;       // tiles along N per M-block (row-space modes) / per expert (WGRAD)

@@ -143,6 +143,7 @@ __global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, Lay
   int* s_counts = sm;            // [Ep]
   int* s_mbstart = sm + Ep;      // [Ep+1]
   int* s_pstart = sm + 2 * Ep + 1;  // [Ep+1]
+  int* s_wstart = sm + 3 * Ep + 2;  // [Ep+1]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   for (int e = warp; e < Ep; e += 32) {
     int carry = 0;
@@ -162,19 +163,23 @@ __global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, Lay
   }
   __syncthreads();
   if (warp == 0) {
-    int carry_rows = 0, carry_mb = 0, carry_pr = 0;
+    int carry_rows = 0, carry_mb = 0, carry_pr = 0, carry_wi = 0;
     for (int e0 = 0; e0 < Ep; e0 += 32) {
       int e = e0 + lane;
       int c = e < Ep ? s_counts[e] : 0;
       int m = (c + BLOCK_M - 1) / BLOCK_M;
       int pr = (m + 1) >> 1;  // pairs of M-blocks (the tensor-core tile of a CTA pair)
-      int ic = c, im = m, ip = pr;
+      // work items of the token-column GEMM kernels that merge: the units of the expert, except that for an
+      // odd count of three or more M-blocks the last two units (one block; two blocks) share one k-loop
+      int wi = pr - (((m & 1) && m >= 3) ? 1 : 0);
+      int ic = c, im = m, ip = pr, iw = wi;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {
         int oc = __shfl_up_sync(0xffffffffu, ic, off);
         int om = __shfl_up_sync(0xffffffffu, im, off);
         int op = __shfl_up_sync(0xffffffffu, ip, off);
-        if (lane >= off) { ic += oc; im += om; ip += op; }
+        int ow = __shfl_up_sync(0xffffffffu, iw, off);
+        if (lane >= off) { ic += oc; im += om; ip += op; iw += ow; }
       }
       if (e < Ep) {
         lv.counts[e] = c;
@@ -186,10 +191,14 @@ __global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, Lay
         const int ps = carry_pr + ip - pr;
         s_pstart[e] = ps;
         lv.pair_start[e] = ps;
+        const int ws = carry_wi + iw - wi;
+        s_wstart[e] = ws;
+        lv.work_start[e] = ws;
       }
       carry_rows += __shfl_sync(0xffffffffu, ic, 31);
       carry_mb += __shfl_sync(0xffffffffu, im, 31);
       carry_pr += __shfl_sync(0xffffffffu, ip, 31);
+      carry_wi += __shfl_sync(0xffffffffu, iw, 31);
     }
     if (lane == 0) {
       lv.offsets[Ep] = carry_rows;
@@ -202,6 +211,9 @@ __global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, Lay
       s_pstart[Ep] = carry_pr;
       lv.pair_start[Ep] = carry_pr;
       lv.meta[3] = carry_pr;
+      s_wstart[Ep] = carry_wi;
+      lv.work_start[Ep] = carry_wi;
+      lv.meta[4] = carry_wi;
     }
   }
   __syncthreads();
@@ -222,6 +234,15 @@ __global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, Lay
       if (s_pstart[mid] <= pb) lo = mid; else hi = mid - 1;
     }
     lv.pblk_expert[pb] = lo;
+  }
+  const int num_wi = s_wstart[Ep];
+  for (int wb = threadIdx.x; wb < num_wi; wb += blockDim.x) {
+    int lo = 0, hi = Ep - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (s_wstart[mid] <= wb) lo = mid; else hi = mid - 1;
+    }
+    lv.wblk_expert[wb] = lo;
   }
 }
 
@@ -274,7 +295,7 @@ cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView&
   const int nblk = n > 0 ? (n + LAYOUT_CHUNK - 1) / LAYOUT_CHUNK : 1;
   const size_t sm_hist = sizeof(int) * (size_t)LAYOUT_WARPS * Ep;
   layout_hist_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv.blk_hist);
-  layout_scan_kernel<<<1, 1024, sizeof(int) * (size_t)(3 * Ep + 2), s>>>(nblk, Ep, lv);
+  layout_scan_kernel<<<1, 1024, sizeof(int) * (size_t)(4 * Ep + 3), s>>>(nblk, Ep, lv);
   layout_rank_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv, status);
   *launches += 3;
   return cudaGetLastError();
@@ -313,6 +334,8 @@ struct NoAllocScratch {
   int mblk_expert[NA_MAX_MBLK];
   int pair_start[NA_MAX_EP + 1];
   int pblk_expert[NA_MAX_MBLK];
+  int work_start[NA_MAX_EP + 1];
+  int wblk_expert[NA_MAX_MBLK];
   int blk_hist[NA_MAX_HIST];
   int prow_of[NA_MAX_SLOTS];
 };
@@ -367,6 +390,8 @@ extern "C" int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E,
   lv.mblk_expert = sc->mblk_expert;
   lv.pair_start = sc->pair_start;
   lv.pblk_expert = sc->pblk_expert;
+  lv.work_start = sc->work_start;
+  lv.wblk_expert = sc->wblk_expert;
   lv.meta = sc->meta;
   lv.blk_hist = sc->blk_hist;
   int launches = 0;
