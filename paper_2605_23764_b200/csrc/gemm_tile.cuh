@@ -159,7 +159,7 @@ __device__ __forceinline__ void load8_bf16(const uint16_t* p, float* v) {
   v[0] = bf16lo(r.x); v[1] = bf16hi(r.x); v[2] = bf16lo(r.y); v[3] = bf16hi(r.y);
   v[4] = bf16lo(r.z); v[5] = bf16hi(r.z); v[6] = bf16lo(r.w); v[7] = bf16hi(r.w);
 }
-__device__ __forceinline__ float sigmoidf_fast(float g) { return 1.0f / (1.0f + __expf(-g)); }
+__device__ __forceinline__ float sigmoidf_fast(float g) { return __fdividef(1.0f, 1.0f + __expf(-g)); }
 
 // Before refilling the staging area: the previous stores must have finished reading it.
 // `nbuf` staging areas are used round-robin: with two, the stores of one round drain while the next
