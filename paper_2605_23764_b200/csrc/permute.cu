@@ -44,6 +44,34 @@ __global__ void __launch_bounds__(PERM_THREADS) gather_rows_kernel(const uint16_
   }
 }
 
+// Short rows (up to 4 KB): one warp per row, so a block has four rows' index chains in flight.
+__global__ void __launch_bounds__(PERM_THREADS) gather_rows_warp_kernel(const uint16_t* __restrict__ src,
+                                                                         const float* __restrict__ topk_w, int d, int k,
+                                                                         int kp, LayoutView lv,
+                                                                         uint16_t* __restrict__ dst,
+                                                                         float* __restrict__ prow_w) {
+  const int r_pad = lv.meta[1];
+  const int nvec = d >> 3;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int WPB = PERM_THREADS / 32;
+  for (int p = blockIdx.x * WPB + warp; p < r_pad; p += gridDim.x * WPB) {
+    const int e = lv.mblk_expert[p / BLOCK_M];
+    const int local = p - lv.pad_off[e];
+    const bool valid = local < lv.counts[e];
+    uint4* out = reinterpret_cast<uint4*>(dst + (size_t)p * d);
+    if (valid) {
+      const int slot = lv.src_of[lv.offsets[e] + local];
+      const int t = slot / kp, j = slot - t * kp;
+      const uint4* in = reinterpret_cast<const uint4*>(src + (size_t)t * d);
+      for (int v = lane; v < nvec; v += 32) out[v] = ld_nc_v4(in + v);
+      if (prow_w && lane == 0) prow_w[p] = j < k ? topk_w[(size_t)t * k + j] : 1.0f;
+    } else {
+      for (int v = lane; v < nvec; v += 32) out[v] = make_uint4(0, 0, 0, 0);
+      if (prow_w && lane == 0) prow_w[p] = 0.0f;
+    }
+  }
+}
+
 // The same gather with bulk copies: one warp per SM, each of up to eight lanes runs its own
 // two-slot pipeline (row i+1 arrives in one shared-memory slot while row i leaves from the other):
 // whole rows move as single global -> shared and shared -> global bulk copies, up to 200 KB in
@@ -148,7 +176,10 @@ cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& 
   }
   int grid = rows_cap < 148 * 16 ? rows_cap : 148 * 16;
   if (grid < 1) grid = 1;
-  gather_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w);
+  if (row_bytes <= 4096)
+    gather_rows_warp_kernel<<<grid, PERM_THREADS, 0, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w);
+  else
+    gather_rows_kernel<<<grid, PERM_THREADS, 0, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w);
   return cudaGetLastError();
 }
 
