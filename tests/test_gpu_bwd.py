@@ -108,41 +108,54 @@ def test_training_config_full_size_sampled():
     torch.cuda.synchronize()
     assert layer.status() == (0, 0)
     ids_c, w_c = ids.cpu(), w.cpu()
-    # the operator-by-operator launches give the same bits (checksums: the gradients are 45 GB)
+
+    def check_against_oracle(out, dx, dW1, dW2, dw, what):
+        # sampled tokens: out, dx and d_topk_w need only the token's own k experts
+        g = torch.Generator().manual_seed(cfg.seed)
+        toks = sorted(set(torch.randint(0, cfg.T, (10,), generator=g).tolist()) | {0, cfg.T - 1})
+        got_o, want_o, got_dx, want_dx, got_dw, want_dw = [], [], [], [], [], []
+        sub_ids = torch.arange(cfg.k, dtype=torch.int32)[None]
+        for t in toks:
+            es = ids_c[t].long().tolist()
+            W1s, W2s = W1[es].cpu(), W2[es].cpu()
+            want_o.append(oracle.fwd(x[t:t + 1].cpu(), sub_ids, w_c[t:t + 1], W1s, W2s)[0])
+            rdx, _, _, rdw = oracle.bwd(dout[t:t + 1].cpu(), x[t:t + 1].cpu(), sub_ids, w_c[t:t + 1], W1s, W2s)
+            want_dx.append(rdx[0]); want_dw.append(rdw[0])
+            got_o.append(out[t].double().cpu().numpy()); got_dx.append(dx[t].double().cpu().numpy())
+            got_dw.append(dw[t].double().cpu().numpy())
+        assert_close_bf16(np.stack(got_o), np.stack(want_o), f"cfg4 {what} out (sampled tokens)")
+        assert_close_bf16(np.stack(got_dx), np.stack(want_dx), f"cfg4 {what} dx (sampled tokens)")
+        assert_close_bf16(np.stack(got_dw), np.stack(want_dw), f"cfg4 {what} d_topk_w (sampled tokens)")
+        # sampled experts: a weight gradient needs only the rows of its expert
+        counts = torch.bincount(ids_c.flatten().long(), minlength=cfg.E)
+        order = torch.argsort(counts)
+        for e in (int(order[0]), int(order[-1])):
+            tok, slot = torch.nonzero(ids_c == e, as_tuple=True)
+            n = tok.numel()
+            assert n > 0
+            r = oracle.bwd(dout[tok.cuda()].cpu(), x[tok.cuda()].cpu(), torch.zeros(n, 1, dtype=torch.int32),
+                           w_c[tok, slot][:, None], W1[e:e + 1].cpu(), W2[e:e + 1].cpu())
+            assert_close_bf16(dW1[e], r[1][0], f"cfg4 {what} dW_gate_up[{e}] ({n} rows)")
+            assert_close_bf16(dW2[e], r[2][0], f"cfg4 {what} dW_down[{e}] ({n} rows)")
+
+    # 1. the persistent launches against the oracle, before any other layer has written anything
+    check_against_oracle(out, dx, dW1, dW2, dw, "persistent launch")
     sums = [t.view(torch.int16).to(torch.int64).sum().item() for t in (out, dx, dW1, dW2)]
+    dw_fused = dw.clone()
+    # 2. the operator-by-operator launches into the SAME gradient tensors (45 GB: no room for a second set), zeroed
+    # first so that nothing of the persistent launches' results can pass for theirs
+    for t in (dx, dW1, dW2, dw):
+        t.zero_()
+    assert dx.view(torch.int16).to(torch.int64).abs().sum().item() == 0
     other = MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=True, serial=True)
     out2 = other.ffn_fwd(x, ids, w, W1, W2)
-    other.ffn_bwd(dout, x, ids, w, W1, W2, dx=dx, dW_gate_up=dW1, dW_down=dW2, d_topk_w=torch.empty_like(dw))
+    other.ffn_bwd(dout, x, ids, w, W1, W2, dx=dx, dW_gate_up=dW1, dW_down=dW2, d_topk_w=dw)
+    torch.cuda.synchronize()
     assert other.status() == (0, 0)
+    check_against_oracle(out2, dx, dW1, dW2, dw, "operator launches")
+    # 3. both launch modes give the same bits (checksums of the four large tensors, d_topk_w in full)
     sums2 = [t.view(torch.int16).to(torch.int64).sum().item() for t in (out2, dx, dW1, dW2)]
     assert sums == sums2, "fused and serial launches disagree"
+    assert torch.equal(out, out2) and torch.equal(dw, dw_fused)
     other.close()
-    del out2
-    # sampled tokens: out, dx and d_topk_w need only the token's own k experts
-    g = torch.Generator().manual_seed(cfg.seed)
-    toks = sorted(set(torch.randint(0, cfg.T, (10,), generator=g).tolist()) | {0, cfg.T - 1})
-    got_o, want_o, got_dx, want_dx, got_dw, want_dw = [], [], [], [], [], []
-    sub_ids = torch.arange(cfg.k, dtype=torch.int32)[None]
-    for t in toks:
-        es = ids_c[t].long().tolist()
-        W1s, W2s = W1[es].cpu(), W2[es].cpu()
-        want_o.append(oracle.fwd(x[t:t + 1].cpu(), sub_ids, w_c[t:t + 1], W1s, W2s)[0])
-        rdx, _, _, rdw = oracle.bwd(dout[t:t + 1].cpu(), x[t:t + 1].cpu(), sub_ids, w_c[t:t + 1], W1s, W2s)
-        want_dx.append(rdx[0]); want_dw.append(rdw[0])
-        got_o.append(out[t].double().cpu().numpy()); got_dx.append(dx[t].double().cpu().numpy())
-        got_dw.append(dw[t].double().cpu().numpy())
-    assert_close_bf16(np.stack(got_o), np.stack(want_o), "cfg4 out (sampled tokens)")
-    assert_close_bf16(np.stack(got_dx), np.stack(want_dx), "cfg4 dx (sampled tokens)")
-    assert_close_bf16(np.stack(got_dw), np.stack(want_dw), "cfg4 d_topk_w (sampled tokens)")
-    # sampled experts: a weight gradient needs only the rows of its expert
-    counts = torch.bincount(ids_c.flatten().long(), minlength=cfg.E)
-    order = torch.argsort(counts)
-    for e in (int(order[0]), int(order[-1])):
-        tok, slot = torch.nonzero(ids_c == e, as_tuple=True)
-        n = tok.numel()
-        assert n > 0
-        r = oracle.bwd(dout[tok.cuda()].cpu(), x[tok.cuda()].cpu(), torch.zeros(n, 1, dtype=torch.int32),
-                       w_c[tok, slot][:, None], W1[e:e + 1].cpu(), W2[e:e + 1].cpu())
-        assert_close_bf16(dW1[e], r[1][0], f"cfg4 dW_gate_up[{e}] ({n} rows)")
-        assert_close_bf16(dW2[e], r[2][0], f"cfg4 dW_down[{e}] ({n} rows)")
     layer.close()
