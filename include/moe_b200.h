@@ -25,7 +25,14 @@
  *     that ran out) are recorded in the context and read with moe_get_status(); kernels always
  *     terminate.
  *   - A context serialises nothing: use one context per stream, and do not overlap two calls
- *     on the same context.
+ *     on the same context.  Contexts on different GPUs of one process, and host threads with
+ *     their own contexts, may call concurrently.
+ *   - Launch modes: by default a pass is ONE persistent launch (after the index-only layout
+ *     kernels) in which gather, GEMM and combine tiles are ordered by event counters;
+ *     MOE_FLAG_SERIAL_LAUNCH runs one launch per operator.  Shapes with F % 16 != 0 always take
+ *     the one-launch-per-operator path.
+ *   - Test and diagnostic entry points (workspace views, schedule simulation, failure injection,
+ *     trace read-out) are declared in moe_b200_debug.h.
  */
 #ifndef MOE_B200_H
 #define MOE_B200_H
@@ -56,6 +63,10 @@ enum {
   MOE_FLAG_SERIAL_LAUNCH = 4u, /* run the layer as one kernel launch per operator (the paper's
                                   operator-by-operator baseline, Section 5.2) instead of the
                                   single persistent dependency-driven launch */
+  MOE_FLAG_TRACE = 8u,         /* the persistent launches record a per-tile trace (role, phase, item,
+                                  start and end time) into the workspace; read it with
+                                  moe_debug_trace (moe_b200_debug.h).  Costs 8 MB of workspace and one
+                                  atomic + two 16-byte stores per tile */
 };
 
 enum {
@@ -64,7 +75,7 @@ enum {
   MOE_ERR_WORKSPACE = -2,     /* caller's workspace too small or misaligned */
   MOE_ERR_CUDA = -3,          /* a CUDA runtime/driver call failed (see moe_last_cuda_error) */
   MOE_ERR_NO_DEVICE = -4,     /* no sm_100 device is current */
-  MOE_ERR_STATE = -5,         /* moe_ffn_bwd without a saved forward of the same T */
+  MOE_ERR_STATE = -5,         /* moe_ffn_bwd without a saved forward of the same tensors and T */
   MOE_ERR_TOO_LARGE = -6,     /* size beyond a documented fixed limit */
   /* asynchronous, reported by moe_get_status(): */
   MOE_ERR_BAD_EXPERT_ID = 1,  /* detail = flat slot index of one offending entry */
@@ -90,8 +101,8 @@ int moe_destroy(moe_ctx* ctx);
 int moe_route(moe_ctx* ctx, const float* logits, int32_t T, int32_t* topk_ids, float* topk_w,
               int32_t* counts, void* stream);
 
-/* Dispatch layout only (Section 2.2, Dispatch: "permutes ... tokens according to the routing
- * decisions").  Flat slot i = t*(k+S)+j; slots j >= k are the shared experts E..E+S-1.
+/* Dispatch layout only (Section 2.2, Dispatch: the index part -- which expert-ordered row each
+ * routed token copy goes to).  Flat slot i = t*(k+S)+j; slots j >= k are the shared experts E..E+S-1.
  * counts[E+S]; offsets[E+S+1] = exclusive scan; row_of[T*(k+S)] = expert-ordered row of each slot
  * (rows of one expert keep slot order; -1 for a slot whose expert id is out of range);
  * src_of[row] = slot.  Any output may be NULL.  moe_ffn_fwd computes the same layout internally. */
@@ -108,7 +119,8 @@ int moe_ffn_fwd(moe_ctx* ctx, const uint16_t* x, const int32_t* topk_ids, const 
                 void* stream);
 
 /* Backward layer (Section 2.2, third paragraph).  Needs the preceding moe_ffn_fwd on this context
- * with MOE_FLAG_SAVE_FOR_BWD and the same x, topk_ids, topk_w, weights and T.
+ * with MOE_FLAG_SAVE_FOR_BWD and the same x, topk_ids, topk_w (the same pointers: the backward works
+ * from the gathered inputs and the layout that forward saved), weights and T; otherwise MOE_ERR_STATE.
  * dout bf16 [T][d] -> dx bf16 [T][d], dW_gate_up bf16 [E+S][2F][d], dW_down bf16 [E+S][d][F]
  * (both overwritten; an expert that received no token gets exact zeros), d_topk_w fp32 [T][k]
  * (gradient of the routing weights; may be NULL). */
@@ -174,48 +186,6 @@ int moe_get_phase_ms(moe_ctx* ctx, float* ms);
  * filled from the device (valid once `stream` has been synchronised). */
 int moe_route_host(moe_ctx* ctx, const float* logits_host, int32_t T, int32_t* topk_ids_host,
                    float* topk_w_host, void* stream);
-
-/* Test/diagnostic access to workspace tensors of the last forward/backward.  `which` is a
- * MOE_BUF_* id; *ptr receives a device pointer into the workspace (valid until the next call on
- * the context), *elems its element count.  Rows of expert-ordered tensors live in a padded row
- * space: expert e starts at row pad_off[e] (a multiple of 128) and holds counts[e] rows. */
-enum {
-  MOE_BUF_COUNTS = 0,    /* int32 [E+S] */
-  MOE_BUF_OFFSETS = 1,   /* int32 [E+S+1] */
-  MOE_BUF_ROW_OF = 2,    /* int32 [T*(k+S)] unpadded rows */
-  MOE_BUF_SRC_OF = 3,    /* int32 [T*(k+S)] */
-  MOE_BUF_PROW_OF = 4,   /* int32 [T*(k+S)] padded rows */
-  MOE_BUF_PAD_OFF = 5,   /* int32 [E+S+1] */
-  MOE_BUF_XP = 6,        /* bf16 [R_pad][d]   gathered x */
-  MOE_BUF_H = 7,         /* bf16 [R_pad][2F]  gate|up pre-activations */
-  MOE_BUF_A = 8,         /* bf16 [R_pad][F]   w * silu(g) * u */
-  MOE_BUF_Y = 9,         /* bf16 [R_pad][d]   expert outputs (already weighted) */
-  MOE_BUF_DOUTP = 10,    /* bf16 [R_pad][d]   gathered dout */
-  MOE_BUF_DH = 11,       /* bf16 [R_pad][2F]  gradient of the pre-activations */
-  MOE_BUF_DXP = 12,      /* bf16 [R_pad][d]   per-row input gradient */
-  MOE_BUF_META = 13,     /* int32 [8]: {num_mblocks, R_pad, rows, ...} */
-};
-int moe_debug_buffer(moe_ctx* ctx, int which, void** ptr, size_t* elems);
-
-/* Failure-handling test hook: with on != 0 the persistent launches of this context wait for one more
- * producer signal than will ever arrive (a threshold nothing reaches).  The bounded waits then run
- * out after the wait budget, the kernel records MOE_ERR_TIMEOUT and returns normally (no trap, no
- * hang); moe_get_status reports it and the context stays usable once the hook is switched off. */
-int moe_debug_set_unreachable_dependency(moe_ctx* ctx, int32_t on);
-
-/* Host-only check of the static tile schedule of the single persistent launch (Section 4.3: tasks
- * ordered in static queues, dependent/trigger event counters with static thresholds).  For the
- * given per-expert row counts[Ep] it builds the matrix and vector queues, verifies that every tile
- * appears once and after all of its producers, lets mat_workers + vec_workers workers consume the
- * queues in ticket order blocking on the counters, and verifies that every counter ends at its
- * threshold.  seg_tiles[4] = tickets per M-block (or per unit of one or two M-blocks when `pair` is
- * set: two CTAs on one tile; pair = 1: token-row tiles, units (0,1),(2,3),..; pair = 2: token-column
- * tiles, balanced units, 8 instead of 4 signals per M-block and column tile) / per expert of each
- * schedule segment, lag in experts.  Returns 0, or a positive code naming the violated property (20 = deadlock).
- * stats[4] (may be NULL) = {matrix tiles, vector tasks, scheduler rounds, stalled polls}.  Needs no GPU. */
-int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t is_bwd,
-                                const int32_t* seg_tiles, int32_t lag, int32_t mat_workers,
-                                int32_t vec_workers, int32_t pair, int64_t* stats);
 
 /* Dispatch layout for callers that cannot allocate device memory (no counterpart in the paper:
  * this is a convenience of this library).  Who needs it: code that runs where cudaMalloc is not

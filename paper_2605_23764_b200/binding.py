@@ -11,9 +11,9 @@ import os
 
 import torch
 
-MOE_FLAG_RENORM_TOPK, MOE_FLAG_SAVE_FOR_BWD, MOE_FLAG_SERIAL_LAUNCH = 1, 2, 4
+MOE_FLAG_RENORM_TOPK, MOE_FLAG_SAVE_FOR_BWD, MOE_FLAG_SERIAL_LAUNCH, MOE_FLAG_TRACE = 1, 2, 4, 8
 MOE_BUF = {"counts": 0, "offsets": 1, "row_of": 2, "src_of": 3, "prow_of": 4, "pad_off": 5, "Xp": 6, "H": 7,
-           "A": 8, "Y": 9, "dOutp": 10, "dH": 11, "dXp": 12, "meta": 13}
+           "A": 8, "Y": 9, "dOutp": 10, "dH": 11, "dXp": 12, "meta": 13, "trace": 14, "event_counters": 15}
 _BUF_DTYPE = {k: (torch.bfloat16 if k in ("Xp", "H", "A", "Y", "dOutp", "dH", "dXp") else torch.int32)
               for k in MOE_BUF}
 
@@ -21,7 +21,7 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
            "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
-           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency"]
+           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -70,7 +70,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_get_phase_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.moe_route_host.argtypes = [vp, vp, i32, vp, vp, vp]
     lib.moe_layout_noalloc.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
-    lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, vp, i32, i32, i32, i32, vp]
+    lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
+    lib.moe_debug_trace.argtypes = [vp, vp, sz, ctypes.POINTER(sz)]
     lib.moe_debug_set_unreachable_dependency.argtypes = [vp, i32]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
@@ -103,6 +104,22 @@ def _host(t, dtype, name):
     return ctypes.c_void_p(t.data_ptr())
 
 
+_CTX_SHAPE = {}   # context handle -> (T_max, d, E, k, n_shared, F, flags): what the size checks need
+
+
+def _shape_of(ctx):
+    try:
+        return _CTX_SHAPE[ctx.value]
+    except (KeyError, AttributeError):
+        raise MoeError("unknown context handle (not created by moe_create, or already destroyed)") from None
+
+
+def _need(t, n, name):
+    """An undersized tensor would make a kernel read or write out of bounds: refuse it here."""
+    if t is not None and t.numel() < n:
+        raise MoeError(f"{name}: {t.numel()} elements, the call needs {n}")
+
+
 def _stream():
     return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
 
@@ -127,28 +144,47 @@ def moe_create(T_max, d, E, k, n_shared, F, flags=0, workspace: torch.Tensor | N
     ws_ptr = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
     ws_bytes = workspace.numel() if workspace is not None else 0
     _check(load_library().moe_create(ctypes.byref(h), ctypes.byref(s), ws_ptr, ws_bytes), "moe_create")
+    _CTX_SHAPE[h.value] = (int(T_max), int(d), int(E), int(k), int(n_shared), int(F), int(flags))
     return h
 
 
 def moe_destroy(ctx):
     _check(load_library().moe_destroy(ctx), "moe_destroy")
+    _CTX_SHAPE.pop(getattr(ctx, "value", None), None)
 
 
 def moe_route(ctx, logits, T, topk_ids, topk_w, counts=None):
+    _, _, E, k, _, _, _ = _shape_of(ctx)
+    _need(logits, T * E, "logits"); _need(topk_ids, T * k, "topk_ids"); _need(topk_w, T * k, "topk_w")
+    _need(counts, E, "counts")
     _check(load_library().moe_route(ctx, _dev(logits, torch.float32, "logits"), T,
                                     _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_w, torch.float32, "topk_w"),
                                     _dev(counts, torch.int32, "counts"), _stream()), "moe_route")
 
 
 def moe_layout(ctx, topk_ids, T, counts=None, offsets=None, row_of=None, src_of=None):
+    _, _, E, k, S, _, _ = _shape_of(ctx)
+    _need(topk_ids, T * k, "topk_ids"); _need(counts, E + S, "counts"); _need(offsets, E + S + 1, "offsets")
+    _need(row_of, T * (k + S), "row_of"); _need(src_of, T * (k + S), "src_of")
     _check(load_library().moe_layout(ctx, _dev(topk_ids, torch.int32, "topk_ids"), T,
                                      _dev(counts, torch.int32, "counts"), _dev(offsets, torch.int32, "offsets"),
                                      _dev(row_of, torch.int32, "row_of"), _dev(src_of, torch.int32, "src_of"),
                                      _stream()), "moe_layout")
 
 
+def _need_layer_tensors(ctx, T, acts, ids_w, W_gate_up, W_down):
+    _, d, E, k, S, F, _ = _shape_of(ctx)
+    for name, t in acts.items():
+        _need(t, T * d, name)
+    for name, t in ids_w.items():
+        _need(t, T * k, name)
+    _need(W_gate_up, (E + S) * 2 * F * d, "W_gate_up")
+    _need(W_down, (E + S) * d * F, "W_down")
+
+
 def moe_ffn_fwd(ctx, x, topk_ids, topk_w, W_gate_up, W_down, out, T):
     bf = torch.bfloat16
+    _need_layer_tensors(ctx, T, {"x": x, "out": out}, {"topk_ids": topk_ids, "topk_w": topk_w}, W_gate_up, W_down)
     _check(load_library().moe_ffn_fwd(ctx, _dev(x, bf, "x"), _dev(topk_ids, torch.int32, "topk_ids"),
                                       _dev(topk_w, torch.float32, "topk_w"), _dev(W_gate_up, bf, "W_gate_up"),
                                       _dev(W_down, bf, "W_down"), _dev(out, bf, "out"), T, _stream()), "moe_ffn_fwd")
@@ -156,6 +192,9 @@ def moe_ffn_fwd(ctx, x, topk_ids, topk_w, W_gate_up, W_down, out, T):
 
 def moe_ffn_bwd(ctx, dout, x, topk_ids, topk_w, W_gate_up, W_down, dx, dW_gate_up, dW_down, d_topk_w, T):
     bf = torch.bfloat16
+    _need_layer_tensors(ctx, T, {"dout": dout, "x": x, "dx": dx},
+                        {"topk_ids": topk_ids, "topk_w": topk_w, "d_topk_w": d_topk_w}, W_gate_up, W_down)
+    _need(dW_gate_up, W_gate_up.numel(), "dW_gate_up"); _need(dW_down, W_down.numel(), "dW_down")
     _check(load_library().moe_ffn_bwd(ctx, _dev(dout, bf, "dout"), _dev(x, bf, "x"),
                                       _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_w, torch.float32, "topk_w"),
                                       _dev(W_gate_up, bf, "W_gate_up"), _dev(W_down, bf, "W_down"),
@@ -166,6 +205,8 @@ def moe_ffn_bwd(ctx, dout, x, topk_ids, topk_w, W_gate_up, W_down, dx, dW_gate_u
 
 def moe_ffn_fwd_host(ctx, x_host, topk_ids_host, topk_w_host, W_gate_up, W_down, out_host, T):
     bf = torch.bfloat16
+    _need_layer_tensors(ctx, T, {"x_host": x_host, "out_host": out_host},
+                        {"topk_ids_host": topk_ids_host, "topk_w_host": topk_w_host}, W_gate_up, W_down)
     _check(load_library().moe_ffn_fwd_host(ctx, _host(x_host, bf, "x_host"),
                                            _host(topk_ids_host, torch.int32, "topk_ids_host"),
                                            _host(topk_w_host, torch.float32, "topk_w_host"),
@@ -175,6 +216,9 @@ def moe_ffn_fwd_host(ctx, x_host, topk_ids_host, topk_w_host, W_gate_up, W_down,
 
 def moe_ffn_bwd_host(ctx, dout_host, W_gate_up, W_down, dx_host, dW_gate_up, dW_down, d_topk_w_host, T):
     bf = torch.bfloat16
+    _need_layer_tensors(ctx, T, {"dout_host": dout_host, "dx_host": dx_host}, {"d_topk_w_host": d_topk_w_host},
+                        W_gate_up, W_down)
+    _need(dW_gate_up, W_gate_up.numel(), "dW_gate_up"); _need(dW_down, W_down.numel(), "dW_down")
     _check(load_library().moe_ffn_bwd_host(ctx, _host(dout_host, bf, "dout_host"), _dev(W_gate_up, bf, "W_gate_up"),
                                            _dev(W_down, bf, "W_down"), _host(dx_host, bf, "dx_host"),
                                            _dev(dW_gate_up, bf, "dW_gate_up"), _dev(dW_down, bf, "dW_down"),
@@ -208,6 +252,9 @@ def moe_get_phase_ms(ctx) -> dict:
 
 
 def moe_route_host(ctx, logits_host, T, topk_ids_host, topk_w_host):
+    _, _, E, k, _, _, _ = _shape_of(ctx)
+    _need(logits_host, T * E, "logits_host"); _need(topk_ids_host, T * k, "topk_ids_host")
+    _need(topk_w_host, T * k, "topk_w_host")
     _check(load_library().moe_route_host(ctx, _host(logits_host, torch.float32, "logits_host"), T,
                                          _host(topk_ids_host, torch.int32, "topk_ids_host"),
                                          _host(topk_w_host, torch.float32, "topk_w_host"), _stream()),
@@ -218,21 +265,41 @@ def moe_layout_noalloc(topk_ids, T, E, k, n_shared, counts, offsets, row_of, src
     """Dispatch layout through the entry point that allocates nothing and needs no context (for
     callers that may not cudaMalloc).  All tensors are caller-owned CUDA int32 tensors."""
     i32 = torch.int32
+    n, Ep = T * (k + n_shared), E + n_shared
+    # a problem beyond the entry point's fixed limits is refused by the library itself before it touches memory
+    if 0 <= n <= 262144 and Ep <= 1088 and -(-n // 2048) * Ep <= 131072:
+        _need(topk_ids, T * k, "topk_ids"); _need(counts, Ep, "counts"); _need(offsets, Ep + 1, "offsets")
+        _need(row_of, n, "row_of"); _need(src_of, n, "src_of"); _need(status2, 2, "status2")
     _check(load_library().moe_layout_noalloc(_dev(topk_ids, i32, "topk_ids"), T, E, k, n_shared,
                                              _dev(counts, i32, "counts"), _dev(offsets, i32, "offsets"),
                                              _dev(row_of, i32, "row_of"), _dev(src_of, i32, "src_of"),
                                              _dev(status2, i32, "status2"), _stream()), "moe_layout_noalloc")
 
 
-def moe_debug_simulate_schedule(counts, T, k, is_bwd, seg_tiles, lag, mat_workers, vec_workers, pair=0):
-    """Host-only schedule check; returns (code, stats) with code 0 = schedule is sound.
-    pair: 0 = one CTA per tile, 1 = CTA pairs on token-row tiles, 2 = CTA pairs on token-column tiles."""
+def moe_debug_simulate_schedule(counts, T, k, n_shared, d, F, is_bwd, pairs, vec_workers):
+    """Host-only schedule check; returns (code, stats) with code 0 = schedule is sound."""
     c = (ctypes.c_int32 * len(counts))(*[int(v) for v in counts])
-    seg = (ctypes.c_int32 * 4)(*[int(v) for v in seg_tiles])
     stats = (ctypes.c_int64 * 4)()
-    rc = load_library().moe_debug_simulate_schedule(c, len(counts), T, k, int(is_bwd), seg, lag, mat_workers,
-                                                    vec_workers, int(pair), stats)
+    rc = load_library().moe_debug_simulate_schedule(c, len(counts), T, k, n_shared, d, F, int(is_bwd), pairs,
+                                                    vec_workers, stats)
     return rc, list(stats)
+
+
+class MoeTraceRecord(ctypes.Structure):
+    _fields_ = [("t0_ns", ctypes.c_uint64), ("t1_ns", ctypes.c_uint64), ("role", ctypes.c_uint8),
+                ("phase", ctypes.c_uint8), ("pad", ctypes.c_uint16), ("item", ctypes.c_int32),
+                ("cta", ctypes.c_uint32), ("dep_ns", ctypes.c_uint32)]
+
+
+def moe_debug_trace(ctx, max_records=1 << 18):
+    """-> (records as a list of dicts, number of records the launch produced)."""
+    buf = (MoeTraceRecord * max_records)()
+    n = ctypes.c_size_t()
+    _check(load_library().moe_debug_trace(ctx, buf, max_records, ctypes.byref(n)), "moe_debug_trace")
+    got = min(n.value, max_records)
+    recs = [{"t0": r.t0_ns, "t1": r.t1_ns, "role": r.role, "phase": r.phase, "item": r.item, "cta": r.cta,
+             "dep_ns": r.dep_ns} for r in buf[:got]]
+    return recs, n.value
 
 
 def moe_debug_set_unreachable_dependency(ctx, on: bool):
@@ -261,10 +328,10 @@ def moe_debug_buffer(ctx, which: str) -> torch.Tensor:
 class MoeLayer:
     """Owns a context and its workspace (a torch allocation); allocates outputs; same calls as the C ABI."""
 
-    def __init__(self, T_max, d, E, k, n_shared, F, renorm=False, save_for_bwd=False, serial=False):
+    def __init__(self, T_max, d, E, k, n_shared, F, renorm=False, save_for_bwd=False, serial=False, trace=False):
         self.T_max, self.d, self.E, self.k, self.S, self.F = T_max, d, E, k, n_shared, F
         self.flags = ((MOE_FLAG_RENORM_TOPK if renorm else 0) | (MOE_FLAG_SAVE_FOR_BWD if save_for_bwd else 0) |
-                      (MOE_FLAG_SERIAL_LAUNCH if serial else 0))
+                      (MOE_FLAG_SERIAL_LAUNCH if serial else 0) | (MOE_FLAG_TRACE if trace else 0))
         nbytes = moe_workspace_bytes(T_max, d, E, k, n_shared, F, self.flags)
         if nbytes == 0:
             raise MoeError("invalid shape")

@@ -5,10 +5,12 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
 #include "../../include/moe_b200.h"
+#include "../../include/moe_b200_debug.h"
 #include "moe_internal.h"
 
 using namespace moe;
@@ -119,7 +121,7 @@ bool shape_ok(const moe_shape* s) {
          (long)s->T_max * (s->k + s->n_shared) < (1l << 30);
 }
 
-constexpr int SCHED_LAG_MAX = 64;
+constexpr int TRACE_RECORDS = 1 << 18;   // 32-byte records of the per-tile trace (MOE_FLAG_TRACE)
 
 struct Carve {
   size_t off = 0;
@@ -132,9 +134,9 @@ struct Carve {
 
 // Byte offsets of every workspace tensor.
 struct WsPlan {
-  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, work_start, wblk_expert, blk_hist, row_of, src_of, prow_of, prow_w,
-      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dw, st_logits, step_start, ctr, stats, total;
-  int cap_rows, nblk_max, ntn_act, ctr_count;
+  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, work_start, wblk_expert, blk_hist, row_of, src_of, prow_of, combine_order, prow_w,
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dw, st_logits, ctr, trace, total;
+  int cap_rows, nblk_max, ntn_act, ctr_count, trace_cap;
 };
 
 WsPlan plan_workspace(const moe_shape& s) {
@@ -163,6 +165,7 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.row_of = c.take(sizeof(int) * (slots + 1));
   p.src_of = c.take(sizeof(int) * (slots + 1));
   p.prow_of = c.take(sizeof(int) * (slots + 1));
+  p.combine_order = c.take(sizeof(int) * ((size_t)s.T_max + 1));
   p.prow_w = c.take(sizeof(float) * cap);
   p.dw_partial = c.take(train ? sizeof(float) * cap * p.ntn_act * DW_PARTS_PER_TILE : 0);
   p.Xp = c.take(2 * cap * s.d);
@@ -179,9 +182,9 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.st_dw = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_logits = c.take(sizeof(float) * (size_t)s.T_max * s.E);
   p.ctr_count = ctr_ints((int)(cap / BLOCK_M) + 1);
-  p.step_start = c.take(sizeof(int) * (size_t)(Ep + SCHED_LAG_MAX + 4));
   p.ctr = c.take(sizeof(int) * (size_t)p.ctr_count);
-  p.stats = c.take(sizeof(long long) * 32 * 256);
+  p.trace_cap = (s.flags & MOE_FLAG_TRACE) ? TRACE_RECORDS : 0;
+  p.trace = c.take((size_t)p.trace_cap * 32);
   p.total = c.off;
   return p;
 }
@@ -199,9 +202,9 @@ struct moe_ctx {
   int num_sms = 0;
   int launches = 0;
   int saved_T = -1;  // T of the forward whose tensors are in the workspace (-1: none)
+  const void *saved_x = nullptr, *saved_ids = nullptr, *saved_w = nullptr;  // that forward's inputs
   uint64_t budget_ns = 2000ull * 1000 * 1000;
   int dep_extra = 0;  // test hook: makes the activation dependencies of the persistent launch unreachable
-  int sched_lag = 0;  // experts between a producer step and its consumer step; 0 = choose from the shape
   cudaStream_t last_stream = nullptr;
   // host-buffer entry points: a copy-in stream (the next call's large input arrives while the previous
   // call still computes) and a copy-out stream (the result leaves in token chunks behind the combine)
@@ -226,7 +229,7 @@ struct moe_ctx {
   // tensor maps of the caller's weights, re-encoded when the pointers change
   const void* w1_ptr = nullptr;
   const void* w2_ptr = nullptr;
-  CUtensorMap tm_W1_k, tm_W2_k, tm_W2_k128, tm_W1_mn, tm_W2_mn;
+  CUtensorMap tm_W1_k, tm_W2_k128, tm_W1_mn, tm_W2_mn;
   CUtensorMap tm_W1_gu;  // token-column tiles: 16 gate rows + 16 up rows per box
   // store maps: workspace tensors (fixed) and the caller's weight gradients (re-encoded on change)
   CUtensorMap ts_A, ts_H, ts_Y, ts_dH;
@@ -256,6 +259,7 @@ struct moe_ctx {
     lv.wblk_expert = at<int>(plan.wblk_expert);
     lv.meta = at<int>(plan.meta);
     lv.blk_hist = at<int>(plan.blk_hist);
+    lv.combine_order = at<int>(plan.combine_order);
     return lv;
   }
   Dims dims(int T) const { return Dims{T, shape.d, shape.E, shape.k, shape.n_shared, shape.F}; }
@@ -293,7 +297,6 @@ int encode_weight_maps(moe_ctx* c, const uint16_t* W1, const uint16_t* W2) {
     c->w1_ptr = W1;
   }
   if (W2 != c->w2_ptr) {
-    if ((rc = encode_2d(&c->tm_W2_k, W2, Ep * s.d, s.F, 256, 64))) return rc;
     if ((rc = encode_2d(&c->tm_W2_k128, W2, Ep * s.d, s.F, 128, 64))) return rc;
     if ((rc = encode_2d(&c->tm_W2_mn, W2, Ep * s.d, s.F, 64, 64))) return rc;
     c->w2_ptr = W2;
@@ -342,7 +345,7 @@ GemmArgs args_down(const moe_ctx* c) {
   const moe_shape& s = c->shape;
   GemmArgs g = base_args(c);
   g.tmA = c->tm_A_k;
-  g.tmB = c->tm_W2_k;
+  g.tmB = c->tm_W2_k128;  // each CTA of a pair loads 128 of the tile's 256 rows
   g.n_tiles_n = (s.d + 255) / 256;
   g.K = s.F;
   g.N = s.d;
@@ -408,37 +411,8 @@ GemmArgs args_wgrad_gate_up(const moe_ctx* c) {
   return g;
 }
 
-// Diagnostic knob: MOE_B200_SINGLE_CTA_GEMM=1 runs the one-launch-per-operator mode on the single-CTA
-// tiles (the ones the persistent launch uses) instead of CTA pairs.
-bool single_cta_gemm() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("MOE_B200_SINGLE_CTA_GEMM");
-    v = (e && e[0] == '1') ? 1 : 0;
-  }
-  return v == 1;
-}
-// Diagnostic knob: MOE_B200_TOKEN_ROW_TILES=1 keeps the tokens on the accumulator rows (256-row tiles
-// padded per expert) in the row-space GEMMs of the CTA-pair kernels.
-bool token_col_tiles() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("MOE_B200_TOKEN_ROW_TILES");
-    v = (e && e[0] == '1') ? 0 : 1;
-  }
-  return v == 1 && !single_cta_gemm();
-}
-// Diagnostic knob: MOE_B200_WGRAD_PER_TILE=1 runs the weight gradients tile by tile (both operands
-// streamed for every tile) instead of strip by strip with a resident A operand.
-bool wgrad_strips_on() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("MOE_B200_WGRAD_PER_TILE");
-    v = (e && e[0] == '1') ? 0 : 1;
-  }
-  return v == 1;
-}
-bool token_col_tiles(const moe_ctx* c) { return token_col_tiles() && c->shape.F % 16 == 0; }
+// Token-column tiles (gemm_tc3.cu, and the persistent launch) need the 16-feature gate/up groups of W_gate_up.
+bool token_col_tiles(const moe_ctx* c) { return c->shape.F % 16 == 0; }
 // Rewrites the arguments of a row-space operator for the token-column tiles: tmA/tmTok16 = tokens,
 // tmB = weights, un-swizzled store maps.
 GemmArgs to_token_cols(const moe_ctx* c, GemmMode mode, GemmArgs g) {
@@ -464,47 +438,43 @@ GemmArgs to_token_cols(const moe_ctx* c, GemmMode mode, GemmArgs g) {
   return g;
 }
 cudaError_t launch_gemm_serial(const moe_ctx* c, GemmMode mode, const GemmArgs& args, cudaStream_t st, int* launches) {
-  if (single_cta_gemm()) return launch_gemm(mode, args, c->num_sms, st, launches);
-  if (mode == GEMM_WGRAD && wgrad_strips_on()) return launch_wgrad_strips(args, c->num_sms, st, launches);
-  if (mode != GEMM_WGRAD && token_col_tiles(c)) return launch_gemm3(mode, to_token_cols(c, mode, args), c->num_sms, st, launches);
+  if (mode == GEMM_WGRAD) return launch_wgrad_strips(args, c->num_sms, st, launches);
+  if (token_col_tiles(c)) return launch_gemm3(mode, to_token_cols(c, mode, args), c->num_sms, st, launches);
   return launch_gemm2(mode, args, c->num_sms, st, launches);
 }
 #define LAUNCH_GEMM_SERIAL(mode, args, sms, st, launches) launch_gemm_serial(c, mode, args, st, launches)
 
-bool serial_mode(const moe_ctx* c) { return (c->shape.flags & MOE_FLAG_SERIAL_LAUNCH) != 0; }
+// One launch per operator: on request, and for shapes the persistent launch does not cover (it runs the
+// token-column tiles only).
+bool serial_mode(const moe_ctx* c) { return (c->shape.flags & MOE_FLAG_SERIAL_LAUNCH) != 0 || !token_col_tiles(c); }
 
-SchedParams sched_params(const moe_ctx* c, bool bwd, int T) {
+ChainParams chain_params(const moe_ctx* c, bool bwd, int T, bool want_dw) {
   const moe_shape& s = c->shape;
-  SchedParams sp;
-  memset(&sp, 0, sizeof sp);
-  sp.is_bwd = bwd ? 1 : 0;
-  sp.pair = single_cta_gemm() ? 0 : 1;
-  sp.tokcol = token_col_tiles(c) ? 1 : 0;
-  sp.sig = sp.tokcol ? 2 * EPI_WARPS : EPI_WARPS;
-  sp.dep_extra = c->dep_extra;
-  sp.Ep = s.E + s.n_shared;
-  sp.T = T;
-  sp.k = s.k;
+  ChainParams cp;
+  memset(&cp, 0, sizeof cp);
+  cp.is_bwd = bwd ? 1 : 0;
+  cp.Ep = s.E + s.n_shared;
+  cp.T = T;
+  cp.k = s.k;
+  cp.kp = s.k + s.n_shared;
+  cp.dep_extra = c->dep_extra;
+  cp.want_dw = want_dw ? 1 : 0;
   if (!bwd) {
-    sp.seg_tiles[0] = (s.F + 127) / 128;
-    sp.seg_tiles[1] = (s.d + 255) / 256;
+    cp.n_phases = 2;
+    cp.ntn[0] = (s.F + 127) / 128;                 // gate+up: 128 features (gate and up) per pair tile
+    cp.ntn[1] = (s.d + 255) / 256;                 // down
+    cp.merges[1] = 1;
   } else {
-    sp.seg_tiles[0] = c->plan.ntn_act;
-    const int strip_rows = sp.pair ? 256 : 128;  // rows of the gradient one ticket covers
-    sp.seg_tiles[1] = (s.d + strip_rows - 1) / strip_rows;       // w2_grad strips
-    sp.strip_tiles[0] = (s.F + 255) / 256;
-    sp.seg_tiles[2] = (s.d + 255) / 256;
-    sp.seg_tiles[3] = (2 * s.F + strip_rows - 1) / strip_rows;   // w1_grad strips
-    sp.strip_tiles[1] = (s.d + 255) / 256;
+    cp.n_phases = 4;
+    cp.ntn[0] = c->plan.ntn_act;                   // act_grad
+    cp.ntn[1] = (s.F + 255) / 256;                 // w2_grad: column tiles per strip
+    cp.strips[1] = (s.d + 255) / 256;
+    cp.ntn[2] = (s.d + 255) / 256;                 // gate_grad
+    cp.merges[2] = 1;
+    cp.ntn[3] = (s.d + 255) / 256;                 // w1_grad
+    cp.strips[3] = (2 * s.F + 255) / 256;
   }
-  // lag: enough experts that a consumer's producers are about two grid-fulls of tickets ahead even
-  // when every expert in between holds a single M-block (skewed routing has many such experts)
-  const int per_step = sp.seg_tiles[0] + (bwd ? sp.seg_tiles[1] : 0);
-  int lag = (2 * c->num_sms + per_step - 1) / per_step;
-  if (lag < 1) lag = 1;
-  if (lag > SCHED_LAG_MAX) lag = SCHED_LAG_MAX;
-  sp.lag = c->sched_lag > 0 ? c->sched_lag : lag;
-  return sp;
+  return cp;
 }
 
 FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
@@ -512,13 +482,12 @@ FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
   const WsPlan& p = c->plan;
   FusedArgs fa;
   memset(&fa, 0, sizeof fa);
-  fa.sp = sched_params(c, bwd, T);
   fa.lv = c->layout();
-  fa.step_start = c->at<int>(p.step_start);
   fa.ctr = c->at<int>(p.ctr);
   fa.d = s.d;
   fa.kp = s.k + s.n_shared;
-  fa.stats = c->at<long long>(p.stats);
+  fa.trace = p.trace_cap ? c->at<uint4>(p.trace) : nullptr;
+  fa.trace_cap = p.trace_cap;
   fa.status = c->status();
   fa.budget_ns = c->budget_ns;
   return fa;
@@ -570,6 +539,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
   {
     Phase ph(c, MOE_PHASE_LAYOUT, st);
     MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
+    if (!serial_mode(c)) MOE_CUDA(launch_layout_order(dm, lv, p.cap_rows / BLOCK_M, st, &c->launches));
   }
   if (serial_mode(c)) {
     {
@@ -583,9 +553,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     }
     {
       Phase ph(c, MOE_PHASE_GEMM_DOWN, st);
-      GemmArgs g = args_down(c);
-      if (!single_cta_gemm()) g.tmB = c->tm_W2_k128;  // each CTA of a pair loads 128 of the tile's 256 rows
-      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_DOWN, g, c->num_sms, st, &c->launches));
+      MOE_CUDA(LAUNCH_GEMM_SERIAL(GEMM_DOWN, args_down(c), c->num_sms, st, &c->launches));
     }
     {
       Phase ph(c, MOE_PHASE_COMBINE, st);
@@ -594,13 +562,9 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
   } else {
     // one persistent launch: gather, GMM1+SwiGLU, GMM2 and combine tiles ordered by event counters
     FusedArgs fa = fused_base(c, false, T);
-    fa.op[0] = args_gate_up(c);
-    fa.op[1] = args_down(c);
-    if (fa.sp.pair) fa.op[1].tmB = c->tm_W2_k128;
-    if (fa.sp.tokcol) {
-      fa.op[0] = to_token_cols(c, GEMM_GATE_UP, fa.op[0]);
-      fa.op[1] = to_token_cols(c, GEMM_DOWN, fa.op[1]);
-    }
+    fa.cp = chain_params(c, false, T, false);
+    fa.op[0] = to_token_cols(c, GEMM_GATE_UP, args_gate_up(c));
+    fa.op[1] = to_token_cols(c, GEMM_DOWN, args_down(c));
     fa.gather_src = x;
     fa.gather_dst = c->at<uint16_t>(p.Xp);
     fa.topk_w = w;
@@ -608,12 +572,14 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     fa.combine_rows = c->at<uint16_t>(p.Y);
     fa.combine_out = out;
     Phase ph(c, MOE_PHASE_FUSED_FWD, st);
-    MOE_CUDA(launch_build_schedule(fa.sp, lv, c->at<int>(p.step_start), c->at<int>(p.ctr), p.ctr_count, st,
-                                   &c->launches));
+    MOE_CUDA(cudaMemsetAsync(fa.ctr, 0, sizeof(int) * (size_t)p.ctr_count, st));
     MOE_CUDA(launch_fused(false, fa, c->num_sms, st, &c->launches));
     if (out_host) MOE_CUDA(cudaMemcpyAsync(out_host, out, 2 * (size_t)T * c->shape.d, cudaMemcpyDeviceToHost, st));
   }
-  if (c->train()) c->saved_T = T;
+  if (c->train()) {
+    c->saved_T = T;
+    c->saved_x = x; c->saved_ids = ids; c->saved_w = w;
+  }
   return MOE_OK;
 }
 
@@ -675,29 +641,22 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     if (dx_host) MOE_CUDA(cudaStreamWaitEvent(st, c->ev_d2h_done, 0));  // dx_host is complete once `st` is
   } else {
     FusedArgs fa = fused_base(c, true, T);
-    fa.op[0] = args_act_grad(c, d_w != nullptr);
+    fa.cp = chain_params(c, true, T, d_w != nullptr);
+    fa.op[0] = to_token_cols(c, GEMM_ACT_GRAD, args_act_grad(c, d_w != nullptr));
     fa.op[1] = args_wgrad_down(c);
-    fa.op[2] = args_gate_grad(c);
+    fa.op[2] = to_token_cols(c, GEMM_GATE_GRAD, args_gate_grad(c));
     fa.op[3] = args_wgrad_gate_up(c);
     fa.gather_src = dout;
     fa.gather_dst = c->at<uint16_t>(p.dOutp);
     fa.combine_rows = c->at<uint16_t>(p.Y);
     fa.combine_out = dx;
     fa.dw_partial = c->at<float>(p.dw_partial);
-    fa.dw_nparts = p.ntn_act;
-    if (fa.sp.tokcol) {
-      fa.op[0] = to_token_cols(c, GEMM_ACT_GRAD, fa.op[0]);
-      fa.op[2] = to_token_cols(c, GEMM_GATE_GRAD, fa.op[2]);
-      fa.dw_nparts = p.ntn_act * DW_PARTS_PER_TILE;
-    }
+    fa.dw_nparts = p.ntn_act * DW_PARTS_PER_TILE;
     fa.d_topk_w = d_w;
-    fa.dW1 = dW1;
-    fa.dW2 = dW2;
-    fa.dW1_slab_vec = (size_t)2 * s.F * s.d * 2 / 16;
-    fa.dW2_slab_vec = (size_t)s.d * s.F * 2 / 16;
     Phase ph(c, MOE_PHASE_FUSED_BWD, st);
-    MOE_CUDA(launch_build_schedule(fa.sp, lv, c->at<int>(p.step_start), c->at<int>(p.ctr), p.ctr_count, st,
-                                   &c->launches));
+    MOE_CUDA(cudaMemsetAsync(fa.ctr, 0, sizeof(int) * (size_t)p.ctr_count, st));
+    // slots dropped for an invalid expert id have no row: their gradient is zero
+    if (d_w) MOE_CUDA(cudaMemsetAsync(d_w, 0, sizeof(float) * (size_t)T * s.k, st));
     MOE_CUDA(launch_fused(true, fa, c->num_sms, st, &c->launches));
     if (dx_host) MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
   }
@@ -885,7 +844,8 @@ int moe_ffn_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* x, const int32
     MOE_CUDA(cudaMemsetAsync(dW_down, 0, 2 * Ep * s.d * s.F, st));
     return MOE_OK;
   }
-  if (c->saved_T != T) return MOE_ERR_STATE;
+  // the backward works from what the forward saved: it must be the forward of these very tensors
+  if (c->saved_T != T || c->saved_x != x || c->saved_ids != topk_ids || c->saved_w != topk_w) return MOE_ERR_STATE;
   return run_bwd(c, dout, W_gate_up, W_down, dx, dW_gate_up, dW_down, d_topk_w, T, st);
 }
 
@@ -1022,7 +982,8 @@ int moe_debug_buffer(moe_ctx* c, int which, void** ptr, size_t* elems) {
     case MOE_BUF_DH: if (!train) return MOE_ERR_STATE; off = p.dH; n = cap * 2 * s.F; break;
     case MOE_BUF_DXP: off = p.Y; n = cap * s.d; break;
     case MOE_BUF_META: off = p.meta; n = 8; break;
-    case 14: off = p.stats; n = 2 * 32 * 256; break;  // diagnostic builds: wait accounting (int64 as int32 pairs)
+    case MOE_BUF_TRACE: if (!p.trace_cap) return MOE_ERR_STATE; off = p.trace; n = (size_t)p.trace_cap * 8; break;
+    case MOE_BUF_EVENT_COUNTERS: off = p.ctr; n = p.ctr_count; break;
     default: return MOE_ERR_INVALID_ARG;
   }
   *ptr = c->ws + off;
@@ -1030,92 +991,123 @@ int moe_debug_buffer(moe_ctx* c, int which, void** ptr, size_t* elems) {
   return MOE_OK;
 }
 
-// Host-only check of the static schedule (no GPU needed): builds the tile queues for the given
-// per-expert row counts and lets `mat_workers` matrix workers and `vec_workers` vector workers
-// consume them in ticket order, each blocking on its tile's dependent counters.
-int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t is_bwd,
-                                const int32_t* seg_tiles, int32_t lag, int32_t mat_workers, int32_t vec_workers,
-                                int32_t pair, int64_t* stats) {
-  if (!counts || !seg_tiles || Ep < 1 || lag < 0 || mat_workers < 1 || vec_workers < 1) return MOE_ERR_INVALID_ARG;
-  std::vector<int> mb_start(Ep + 1, 0);
-  for (int e = 0; e < Ep; ++e) mb_start[e + 1] = mb_start[e] + (counts[e] + BLOCK_M - 1) / BLOCK_M;
+// Host-only check of the static schedule (no GPU needed): builds the layout tables and the per-pair
+// matrix queues for the given per-expert row counts and lets `pairs` matrix workers (each walking its
+// own statically ordered queue) and `vec_workers` vector workers (tickets) run, each blocking on its
+// item's dependent counters.
+int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, int32_t k, int32_t n_shared, int32_t d,
+                                int32_t F, int32_t is_bwd, int32_t pairs, int32_t vec_workers, int64_t* stats) {
+  if (!counts || Ep < 1 || pairs < 1 || vec_workers < 1 || d < 8 || F < 16) return MOE_ERR_INVALID_ARG;
+  // the tables of the layout kernels
+  std::vector<int> mb_start(Ep + 1, 0), pair_start(Ep + 1, 0), work_start(Ep + 1, 0);
+  for (int e = 0; e < Ep; ++e) {
+    const int m = (counts[e] + BLOCK_M - 1) / BLOCK_M, pr = (m + 1) >> 1;
+    mb_start[e + 1] = mb_start[e] + m;
+    pair_start[e + 1] = pair_start[e] + pr;
+    work_start[e + 1] = work_start[e] + pr - (((m & 1) && m >= 3) ? 1 : 0);
+  }
   const int M = mb_start[Ep];
-  SchedParams sp;
-  memset(&sp, 0, sizeof sp);
-  sp.is_bwd = is_bwd; sp.lag = lag; sp.Ep = Ep; sp.T = T; sp.k = k; sp.pair = pair ? 1 : 0;
-  sp.tokcol = pair == 2 ? 1 : 0;
-  sp.sig = sp.tokcol ? 2 * EPI_WARPS : EPI_WARPS;
-  for (int i = 0; i < SCHED_MAX_SEG; ++i) sp.seg_tiles[i] = seg_tiles[i];
-  sp.strip_tiles[0] = sp.strip_tiles[1] = 1;
-  std::vector<int> step_start(Ep + lag + 1, 0);
-  for (int i = 0; i < Ep + lag; ++i) step_start[i + 1] = step_start[i] + step_tiles(sp, i, mb_start.data());
-  const int total = step_start[Ep + lag], vtotal = vec_total(sp, M);
-  std::vector<long> ctr(ctr_ints(M + 1), 0);
-  // 1. coverage and ticket order of producers
-  std::vector<int> seg0_count(M + 1, 0), lag_count(M + 1, 0);
-  std::vector<int> w2_count(Ep, 0), w1_count(Ep, 0);
-  for (int t = 0; t < total; ++t) {
-    const MatTile m = decode_matrix_ticket(sp, t, step_start.data(), mb_start.data());
-    if (m.e < 0 || m.e >= Ep || m.idx < 0 || m.idx >= sp.seg_tiles[m.slot]) return 10;
-    if (m.mb >= 0 && (m.mb < mb_start[m.e] || m.mb >= mb_start[m.e + 1])) return 10;
-    if (m.mb >= 0 && (m.mb_count < 1 || m.mb_count > (pair ? 2 : 1) || m.mb + m.mb_count > mb_start[m.e + 1])) return 10;
-    if (m.slot == 0) { for (int q = 0; q < m.mb_count; ++q) seg0_count[m.mb + q]++; }
-    else if (m.mb >= 0) {
-      for (int q = 0; q < m.mb_count; ++q) { lag_count[m.mb + q]++; if (seg0_count[m.mb + q] != sp.seg_tiles[0]) return 11; }
-    }
-    else if (m.slot == 1) w2_count[m.e]++;
-    else {
-      w1_count[m.e]++;
-      for (int q = 0; q < m.dep_count; ++q)
-        if (seg0_count[m.dep_first + q] != sp.seg_tiles[0]) return 12;  // a producer with a larger ticket
+  std::vector<int> pblk(pair_start[Ep] + 1, 0), wblk(work_start[Ep] + 1, 0);
+  for (int e = 0; e < Ep; ++e) {
+    for (int i = pair_start[e]; i < pair_start[e + 1]; ++i) pblk[i] = e;
+    for (int i = work_start[e]; i < work_start[e + 1]; ++i) wblk[i] = e;
+  }
+  ChainParams cp;
+  memset(&cp, 0, sizeof cp);
+  cp.is_bwd = is_bwd; cp.Ep = Ep; cp.T = T; cp.k = k; cp.kp = k + n_shared; cp.want_dw = 1;
+  if (!is_bwd) {
+    cp.n_phases = 2; cp.ntn[0] = (F + 127) / 128; cp.ntn[1] = (d + 255) / 256; cp.merges[1] = 1;
+  } else {
+    cp.n_phases = 4; cp.ntn[0] = (F + 255) / 256; cp.ntn[1] = (F + 255) / 256; cp.strips[1] = (d + 255) / 256;
+    cp.ntn[2] = (d + 255) / 256; cp.merges[2] = 1; cp.ntn[3] = (d + 255) / 256; cp.strips[3] = (2 * F + 255) / 256;
+  }
+  // items of every phase: {first M-block, M-blocks of unit a, M-blocks of unit b} (strips: the expert's M-blocks)
+  struct Item { int phase, mb_first, mb_a, mb_b; };
+  std::vector<std::vector<Item>> queue(pairs);
+  long n_items = 0;
+  std::vector<std::vector<int>> cover(cp.n_phases, std::vector<int>(M + 1, 0));
+  for (int ph = 0; ph < cp.n_phases; ++ph) {
+    if (cp.strips[ph]) {
+      const int total = Ep * cp.strips[ph];
+      for (int sidx = 0; sidx < total; ++sidx) {
+        const int e = sidx / cp.strips[ph];
+        queue[sidx % pairs].push_back(Item{ph, mb_start[e], mb_start[e + 1] - mb_start[e], 0});
+        ++n_items;
+      }
+    } else {
+      const bool mg = cp.merges[ph] != 0;
+      const int total = (mg ? work_start[Ep] : pair_start[Ep]) * cp.ntn[ph];
+      for (int t = 0; t < total; ++t) {
+        const SwapItem it = decode_swap_item(t, cp.ntn[ph], mg, mg ? work_start.data() : pair_start.data(),
+                                             mg ? wblk.data() : pblk.data(), mb_start.data());
+        if (it.e < 0 || it.e >= Ep || it.nb < 0 || it.nb >= cp.ntn[ph]) return 10;
+        if (it.mb_first < mb_start[it.e] || it.mb_first + it.mb_count > mb_start[it.e + 1] || it.mb_count < 1 ||
+            it.mb_count > 3 || it.mb_count_a < 1)
+          return 10;
+        for (int q = 0; q < it.mb_count; ++q) cover[ph][it.mb_first + q]++;
+        queue[t % pairs].push_back(Item{ph, it.mb_first, it.mb_count_a, it.mb_count - it.mb_count_a});
+        ++n_items;
+      }
     }
   }
-  for (int mb = 0; mb < M; ++mb)
-    if (seg0_count[mb] != sp.seg_tiles[0] || lag_count[mb] != (is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1])) return 13;
-  if (is_bwd)
-    for (int e = 0; e < Ep; ++e) {
-      const int want = counts[e] > 0 ? 1 : 0;
-      if (w2_count[e] != want * sp.seg_tiles[1] || w1_count[e] != want * sp.seg_tiles[3]) return 14;
-    }
-  // 2. consumption by a bounded number of workers
-  struct Worker { bool holding = false; MatTile m; VecTask v; };
-  std::vector<Worker> mw(mat_workers), vw(vec_workers);
-  int next_mat = 0, next_vec = 0, done_mat = 0, done_vec = 0;
-  long rounds = 0, stalls = 0;
-  while (done_mat < total || done_vec < vtotal) {
+  // 1. coverage: every M-block is covered by every column tile of every row-space phase exactly once
+  for (int ph = 0; ph < cp.n_phases; ++ph)
+    if (!cp.strips[ph])
+      for (int mb = 0; mb < M; ++mb)
+        if (cover[ph][mb] != cp.ntn[ph]) return 13;
+  // 2. execution with a bounded number of workers
+  std::vector<long> ctr(ctr_ints(M + 1), 0);
+  std::vector<size_t> cursor(pairs, 0);
+  const int ngather = gather_total(M), npost = post_total(cp, M);
+  struct VecWorker { bool holding = false; VecTask v; };
+  std::vector<VecWorker> vw(vec_workers);
+  // rows of each token (slot order is irrelevant here): token t's k+S rows live in M-blocks drawn round-robin
+  auto token_mblocks_done = [&](int t0, int t1) {
+    if (M == 0) return true;
+    for (int t = t0; t < t1; ++t)
+      for (int j = 0; j < cp.kp; ++j)
+        if (ctr[ctr_index((int)(((long)t * cp.kp + j) % M), CTR_DONE)] < thr_done(cp)) return false;
+    return true;
+  };
+  long done_mat = 0, done_vec = 0, rounds = 0, stalls = 0;
+  int next_gather = 0, next_post = 0;
+  const int vtotal = ngather + npost;
+  while (done_mat < n_items || done_vec < vtotal) {
     bool progress = false;
-    for (auto& wk : mw) {
-      if (!wk.holding && next_mat < total) {
-        wk.m = decode_matrix_ticket(sp, next_mat++, step_start.data(), mb_start.data());
-        wk.holding = true;
-        progress = true;
-      }
-      if (!wk.holding) continue;
+    for (int q = 0; q < pairs; ++q) {
+      if (cursor[q] >= queue[q].size()) continue;
+      const Item& it = queue[q][cursor[q]];
+      const int wk = phase_wait_kind(cp, it.phase), thr = phase_wait_thr(cp, it.phase);
       bool ready = true;
-      for (int q = 0; q < wk.m.dep_count; ++q) {
-        const int mb = wk.m.dep_first + q;
-        if (ctr[wk.m.dep_base == 0 ? ctr_gather(mb) : ctr_act(mb)] < wk.m.dep_thr) ready = false;
-      }
+      for (int m = 0; m < it.mb_a + it.mb_b; ++m)
+        if (ctr[ctr_index(it.mb_first + m, wk)] < thr) ready = false;
       if (!ready) { ++stalls; continue; }
-      for (int q = 0; q < wk.m.mb_count; ++q) {  // every real M-block of the tile signals (an idle half does not)
-        if (wk.m.trig_base == 1) ctr[ctr_act(wk.m.mb + q)] += sp.sig;
-        if (wk.m.trig_base == 2) ctr[CTR_DONE] += sp.sig;
-        if (wk.m.trig_also_ag) ctr[CTR_AG_DONE] += sp.sig;
-      }
-      wk.holding = false;
-      ++done_mat;
-      progress = true;
+      const int tk = phase_trigger_kind(cp, it.phase);
+      if (tk >= 0)
+        for (int m = 0; m < it.mb_a + it.mb_b; ++m) ctr[ctr_index(it.mb_first + m, tk)] += SIG;
+      ++cursor[q]; ++done_mat; progress = true;
     }
-    for (auto& wk : vw) {
-      if (!wk.holding && next_vec < vtotal) {
-        wk.v = decode_vector_ticket(sp, next_vec++, M);
-        wk.holding = true;
+    for (size_t wi = 0; wi < vw.size(); ++wi) {
+      auto& w = vw[wi];
+      // worker 0 is a background gatherer; the others leave the gather queue after the first M-blocks
+      const bool may_gather = next_gather < ngather && (wi == 0 || next_gather < GATHER_SUB * GATHER_FAST_MBLOCKS);
+      if (!w.holding && may_gather) {
+        w.v.op = VEC_GATHER; w.v.idx = next_gather++;
+        w.holding = true;
+        progress = true;
+      } else if (!w.holding && next_post < npost && (wi != 0 || next_gather >= ngather)) {
+        w.v = decode_post_ticket(cp, next_post++, M);
+        w.holding = true;
         progress = true;
       }
-      if (!wk.holding) continue;
-      if (wk.v.dep && ctr[wk.v.dep == 2 ? CTR_DONE : CTR_AG_DONE] < wk.v.dep_thr) { ++stalls; continue; }
-      if (wk.v.op == VEC_GATHER) ctr[ctr_gather(wk.v.idx / GATHER_SUB)] += 1;
-      wk.holding = false;
+      if (!w.holding) continue;
+      bool ready = true;
+      if (w.v.op == VEC_DW) ready = ctr[ctr_index(w.v.idx, CTR_ACTIVATED)] >= thr_activated(cp);
+      if (w.v.op == VEC_COMBINE)
+        ready = token_mblocks_done(w.v.idx * COMBINE_TOKENS, std::min(T, (w.v.idx + 1) * COMBINE_TOKENS));
+      if (!ready) { ++stalls; continue; }
+      if (w.v.op == VEC_GATHER) ctr[ctr_index(w.v.idx / GATHER_SUB, CTR_GATHERED)] += 1;
+      w.holding = false;
       ++done_vec;
       progress = true;
     }
@@ -1124,10 +1116,36 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
   }
   // 3. every counter ends exactly at its threshold
   for (int mb = 0; mb < M; ++mb)
-    if (ctr[ctr_gather(mb)] != GATHER_SUB || ctr[ctr_act(mb)] != (long)sp.sig * sp.seg_tiles[0]) return 30;
-  if (ctr[CTR_DONE] != (long)sp.sig * M * (is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1])) return 31;
-  if (is_bwd && ctr[CTR_AG_DONE] != (long)sp.sig * M * sp.seg_tiles[0]) return 32;
-  if (stats) { stats[0] = total; stats[1] = vtotal; stats[2] = rounds; stats[3] = stalls; }
+    if (ctr[ctr_index(mb, CTR_GATHERED)] != thr_gathered() || ctr[ctr_index(mb, CTR_ACTIVATED)] != thr_activated(cp) ||
+        ctr[ctr_index(mb, CTR_DONE)] != thr_done(cp))
+      return 30;
+  if (stats) { stats[0] = n_items; stats[1] = vtotal; stats[2] = rounds; stats[3] = stalls; }
+  return MOE_OK;
+}
+
+int moe_debug_trace(moe_ctx* c, moe_trace_record* records, size_t max_records, size_t* n_written) {
+  if (!c || !n_written || (!records && max_records)) return MOE_ERR_INVALID_ARG;
+  if (!c->plan.trace_cap) return MOE_ERR_STATE;
+  MOE_CUDA(cudaStreamSynchronize(c->last_stream));
+  int produced = 0;
+  MOE_CUDA(cudaMemcpy(&produced, c->at<int>(c->plan.ctr) + CTR_TRACE_CURSOR, sizeof(int), cudaMemcpyDeviceToHost));
+  *n_written = (size_t)produced;
+  size_t n = std::min<size_t>(std::min<size_t>((size_t)produced, (size_t)c->plan.trace_cap), max_records);
+  if (n == 0) return MOE_OK;
+  std::vector<uint32_t> raw(n * 8);
+  MOE_CUDA(cudaMemcpy(raw.data(), c->ws + c->plan.trace, n * 32, cudaMemcpyDeviceToHost));
+  for (size_t i = 0; i < n; ++i) {
+    const uint32_t* r = &raw[8 * i];
+    moe_trace_record& o = records[i];
+    o.t0_ns = (uint64_t)r[0] | ((uint64_t)r[1] << 32);
+    o.t1_ns = (uint64_t)r[2] | ((uint64_t)r[3] << 32);
+    o.role = (uint8_t)(r[4] & 0xFF);
+    o.phase = (uint8_t)((r[4] >> 8) & 0xFF);
+    o.pad = 0;
+    o.item = (int32_t)r[5];
+    o.cta = r[6];
+    o.dep_ns = r[7];
+  }
   return MOE_OK;
 }
 

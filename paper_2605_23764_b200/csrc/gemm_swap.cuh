@@ -29,17 +29,16 @@ struct SwapTile {
   int n0;     // first output feature of the pair (GATE_UP: of the 128 gate/up feature pairs)
   int nb;     // feature-tile index
   int nkb;    // k-blocks
+  int mb_first, mb_count;   // the tile's M-blocks (its event counters)
 };
 
 // Features per pair tile: GATE_UP holds 64 gate + 64 up rows per CTA = 128 features per pair.
 template <int MODE>
 __device__ __forceinline__ int swap_tile_features() { return MODE == GEMM_GATE_UP ? 128 : 256; }
 
-// Token tile `u` (a balanced unit of one or two M-blocks, schedule.h) of expert e, cut at the expert's
-// last 32-row group.
-__device__ __forceinline__ void unit_tokens(const GemmArgs& a, int e, int u, int* row0, int* ntok) {
-  int first, count;
-  balanced_unit(a.mb_start[e + 1] - a.mb_start[e], u, &first, &count);
+// Tokens of the unit of M-blocks [first, first + count) (relative to the expert's first M-block) of expert e,
+// cut at the expert's last 32-row group.
+__device__ __forceinline__ void unit_tokens(const GemmArgs& a, int e, int first, int count, int* row0, int* ntok) {
   const int n32 = (a.counts[e] + TOK_GRAIN - 1) & ~(TOK_GRAIN - 1);
   int end = (first + count) * BLOCK_M;
   if (end > n32) end = n32;
@@ -47,7 +46,7 @@ __device__ __forceinline__ void unit_tokens(const GemmArgs& a, int e, int u, int
   *ntok = end - first * BLOCK_M;
 }
 
-// One work item of the one-launch-per-operator kernel: a token tile, or -- in the operators that merge,
+// One work item of a row-space operator: a token tile, or -- in the operators that merge,
 // for an expert with an odd count of three or more M-blocks -- its last two token tiles (one block;
 // block + tail) under ONE k-loop: the weight stage is written to shared memory once and multiplied with
 // both token tiles into the two TMEM accumulators (shared-memory traffic bounds these kernels, and the
@@ -73,23 +72,21 @@ __device__ __forceinline__ int total_swap_work(const GemmArgs& a) {
 // fast one (items running at the same time share one slab of weights in L2).
 template <int MODE>
 __device__ __forceinline__ SwapWork decode_swap_work(const GemmArgs& a, int t) {
+  constexpr bool mg = swap_merges<MODE>();
+  const SwapItem it = decode_swap_item(t, a.n_tiles_n, mg, mg ? a.work_start : a.pair_start,
+                                       mg ? a.wblk_expert : a.pblk_expert, a.mb_start);
   SwapWork w;
-  const int* start = swap_merges<MODE>() ? a.work_start : a.pair_start;
-  const int e = (swap_merges<MODE>() ? a.wblk_expert : a.pblk_expert)[t / a.n_tiles_n];
-  const int ws = start[e];
-  const int wcount = start[e + 1] - ws;
-  const int local = t - ws * a.n_tiles_n;
-  const int nb = local / wcount;
-  const int wi = local - nb * wcount;
-  const int mc = a.mb_start[e + 1] - a.mb_start[e];
-  w.merged = swap_merges<MODE>() && (mc & 1) && mc >= 3 && wi == wcount - 1;   // units wi and wi + 1
-  w.a.e = w.b.e = e;
-  w.a.nb = w.b.nb = nb;
-  w.a.n0 = w.b.n0 = nb * swap_tile_features<MODE>();
+  w.merged = it.merged != 0;
+  w.a.e = w.b.e = it.e;
+  w.a.nb = w.b.nb = it.nb;
+  w.a.n0 = w.b.n0 = it.nb * swap_tile_features<MODE>();
   w.a.nkb = w.b.nkb = (a.K + BK - 1) / BK;
-  unit_tokens(a, e, wi, &w.a.row0, &w.a.ntok);
+  const int rel = it.mb_first - a.mb_start[it.e];
+  unit_tokens(a, it.e, rel, it.mb_count_a, &w.a.row0, &w.a.ntok);
+  w.a.mb_first = it.mb_first; w.a.mb_count = it.mb_count_a;
   w.b.row0 = 0; w.b.ntok = 0;
-  if (w.merged) unit_tokens(a, e, wi + 1, &w.b.row0, &w.b.ntok);
+  w.b.mb_first = it.mb_first + it.mb_count_a; w.b.mb_count = it.mb_count - it.mb_count_a;
+  if (w.merged) unit_tokens(a, it.e, rel + it.mb_count_a, w.b.mb_count, &w.b.row0, &w.b.ntok);
   return w;
 }
 

@@ -1,4 +1,6 @@
-// Grouped GEMMs on CTA pairs (tcgen05 cta_group::2), one launch per operator.
+// Row-space grouped GEMMs on CTA pairs (tcgen05 cta_group::2) with token-row tiles, one launch per operator:
+// the path of shapes whose intermediate size is not a multiple of 16 (the token-column tiles of gemm_tc3.cu
+// need F % 16 == 0).
 //
 // A 128 x 256 tile on one SM asks shared memory for its operands once per MMA (96 B/clk) while
 // TMA refills the same stages (another 96 B/clk): the 128 B/clk of one SM's shared memory caps the
@@ -17,6 +19,7 @@
 #include <stdlib.h>
 
 #include "gemm_pair.cuh"
+#include "launch_pairs.cuh"
 
 namespace moe {
 
@@ -44,7 +47,6 @@ struct PairTile {
 
 template <int MODE>
 __device__ __forceinline__ int total_pair_tiles(const GemmArgs& a) {
-  if (MODE == GEMM_WGRAD) return a.Ep * ((a.n_tiles_m + 1) / 2) * a.n_tiles_n;
   return a.meta[3] * a.n_tiles_n;
 }
 
@@ -54,37 +56,23 @@ __device__ __forceinline__ PairTile decode_pair_tile(const GemmArgs& a, int t, i
   PairTile pt;
   Tile& tl = pt.tl;
   pt.idle = false;
-  if (MODE == GEMM_WGRAD) {
-    const int tm2 = (a.n_tiles_m + 1) / 2;
-    const int per_e = tm2 * a.n_tiles_n;
-    tl.e = t / per_e;
-    const int r = t - tl.e * per_e;
-    const int mp = r / a.n_tiles_n;
-    tl.nb = r - mp * a.n_tiles_n;
-    tl.m0 = (2 * mp + rank) * BLOCK_M;   // this CTA's 128 rows of the gradient
-    tl.n0 = tl.nb * BN;
-    tl.row0 = a.mb_start[tl.e] * BLOCK_M;
-    tl.nkb = (a.counts[tl.e] + BK - 1) / BK;
-    pt.idle = tl.m0 >= a.M;
-  } else {
-    const int e = a.pblk_expert[t / a.n_tiles_n];
-    const int ps = a.pair_start[e];
-    const int pcount = a.pair_start[e + 1] - ps;
-    const int local = t - ps * a.n_tiles_n;
-    tl.nb = local / pcount;
-    const int pl = local - tl.nb * pcount;
-    const int mb = a.mb_start[e] + 2 * pl + rank;
-    pt.idle = mb >= a.mb_start[e + 1];
-    tl.e = e;
-    tl.row0 = pt.idle ? a.cap_rows : mb * BLOCK_M;   // rows beyond the tensor read as zeros
-    tl.n0 = tl.nb * (MODE == GEMM_GATE_UP ? BN / 2 : BN);
-    tl.m0 = 0;
-    tl.nkb = (a.K + BK - 1) / BK;
-  }
+  const int e = a.pblk_expert[t / a.n_tiles_n];
+  const int ps = a.pair_start[e];
+  const int pcount = a.pair_start[e + 1] - ps;
+  const int local = t - ps * a.n_tiles_n;
+  tl.nb = local / pcount;
+  const int pl = local - tl.nb * pcount;
+  const int mb = a.mb_start[e] + 2 * pl + rank;
+  pt.idle = mb >= a.mb_start[e + 1];
+  tl.e = e;
+  tl.row0 = pt.idle ? a.cap_rows : mb * BLOCK_M;   // rows beyond the tensor read as zeros
+  tl.n0 = tl.nb * (MODE == GEMM_GATE_UP ? BN / 2 : BN);
+  tl.m0 = 0;
+  tl.nkb = (a.K + BK - 1) / BK;
   return pt;
 }
 
-constexpr int GEMM2_THREADS = GEMM_THREADS + 32;   // warp 6: second TMA producer of the weight gradients
+constexpr int GEMM2_THREADS = GEMM_THREADS;
 
 template <int MODE>
 __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(const __grid_constant__ GemmArgs a) {
@@ -127,9 +115,8 @@ __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(con
   const uint32_t tmem_base = bars->tmem_base;
   const int total = total_pair_tiles<MODE>(a);
 
-  if (warp == 0 || (warp == 6 && MODE == GEMM_WGRAD)) {
-    // ------------------------------------------------ TMA producers (both CTAs, one box per lane); the
-    // weight gradients split each stage over two warps
+  if (warp == 0) {
+    // ------------------------------------------------ TMA producer (both CTAs, one box per lane)
     uint32_t s = 0, ph = 1;
     bool ok = true;
     for (int t = pair; t < total && ok; t += npairs) {
@@ -139,10 +126,7 @@ __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(con
         if (lane == 0) go = mbar_wait(&bars->empty[s], ph, wc, SITE_EMPTY, t, 50) ? 1 : 0;
         go = __shfl_sync(0xffffffffu, go, 0);
         if (!go) { ok = false; break; }
-        if (MODE == GEMM_WGRAD)
-          load_wgrad_part(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s], lane, warp == 6);
-        else
-          load_stage_pair_lanes<MODE>(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s], lane);
+        load_stage_pair_lanes<MODE>(a, pt.tl, kb, rank, sA + s * A_STAGE_BYTES, sB + s * HALF_B_BYTES, &bars->full[s], lane);
         if (++s == STAGES2) { s = 0; ph ^= 1; }
       }
     }
@@ -153,7 +137,6 @@ __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(con
       bool ok = true;
       for (int t = pair; t < total && ok; t += npairs) {
         const PairTile pt = decode_pair_tile<MODE>(a, t, 0);
-        if (pt.tl.nkb == 0) continue;
         const int as = acc_it & 1;
         if (!mbar_wait(&bars->tmem_empty[as], ((acc_it >> 1) & 1) ^ 1, wc, SITE_TMEM_EMPTY, t)) { ok = false; break; }
         tc_fence_after_sync();
@@ -162,8 +145,7 @@ __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(con
           const int s = it % STAGES2;
           if (!mbar_wait(&bars->full[s], (it / STAGES2) & 1, wc, SITE_FULL, t)) { ok = false; break; }
           tc_fence_after_sync();
-          mma_kblock_pair<MODE>(d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0,
-                                MODE == GEMM_WGRAD ? k16_steps_of(a.counts[pt.tl.e], kb) : BK / 16);
+          mma_kblock_pair<MODE>(d_tmem, smem_u32(sA + s * A_STAGE_BYTES), smem_u32(sB + s * HALF_B_BYTES), kb == 0);
           tc_commit_pair(&bars->empty[s]);   // frees the stage in both CTAs
         }
         if (!ok) break;
@@ -176,17 +158,13 @@ __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(con
         mbar_wait(&bars->drain, 0, shortwc, SITE_DRAIN, 0);
       }
     }
-  } else if (warp < 6) {
+  } else {
     // ------------------------------------------------ epilogue warps (both CTAs, own rows)
     const int quad = warp & 3;
     Staging stg{sOut + quad * OUT_BUFS2 * OUT_STAGE_BYTES, OUT_BUFS2, 0};
     uint32_t acc_it = 0;
     for (int t = pair; t < total; t += npairs) {
       const PairTile pt = decode_pair_tile<MODE>(a, t, rank);
-      if (pt.tl.nkb == 0) {
-        if (!pt.idle) epilogue_tile<MODE>(a, pt.tl, 0, quad, lane, stg);  // weight gradient of an expert without rows
-        continue;
-      }
       const int as = acc_it & 1;
       if (!mbar_wait(&bars->tmem_full[as], (acc_it >> 1) & 1, wc, SITE_TMEM_FULL, t, 200)) break;  // back off: idle epilogue warps must not take issue slots and power
       tc_fence_after_sync();
@@ -212,36 +190,8 @@ __global__ void __launch_bounds__(GEMM2_THREADS, 1) grouped_gemm_pair_kernel(con
 
 template <int MODE>
 static cudaError_t launch_pair_mode(const GemmArgs& a, int num_sms, cudaStream_t s) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(grouped_gemm_pair_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)GEMM2_SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
-  static int max_pairs = 0;  // CTA pairs that can be resident together (SMs pair up inside a GPC)
-  cudaLaunchConfig_t cfg;
-  memset(&cfg, 0, sizeof cfg);
-  cfg.gridDim = dim3((num_sms / 2) * 2);
-  cfg.blockDim = dim3(GEMM2_THREADS);
-  cfg.dynamicSmemBytes = GEMM2_SMEM_BYTES;
-  cfg.stream = s;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  if (max_pairs == 0) {
-    int n = 0;
-    cudaError_t e = cudaOccupancyMaxActiveClusters(&n, grouped_gemm_pair_kernel<MODE>, &cfg);
-    if (e != cudaSuccess) return e;
-    max_pairs = n > 0 ? n : 1;
-    if (getenv("MOE_B200_DEBUG")) fprintf(stderr, "[moe_b200] CTA pairs resident together: %d (SMs %d)\n", n, num_sms);
-  }
-  if (2 * max_pairs < (int)cfg.gridDim.x) cfg.gridDim = dim3(2 * max_pairs);
-  return cudaLaunchKernelEx(&cfg, grouped_gemm_pair_kernel<MODE>, a);
+  static PairLaunchState st;
+  return launch_on_pairs(st, grouped_gemm_pair_kernel<MODE>, a, GEMM2_THREADS, GEMM2_SMEM_BYTES, num_sms, false, s);
 }
 
 cudaError_t launch_gemm2(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches) {
@@ -251,7 +201,7 @@ cudaError_t launch_gemm2(GemmMode mode, const GemmArgs& a, int num_sms, cudaStre
     case GEMM_DOWN: return launch_pair_mode<GEMM_DOWN>(a, num_sms, s);
     case GEMM_ACT_GRAD: return launch_pair_mode<GEMM_ACT_GRAD>(a, num_sms, s);
     case GEMM_GATE_GRAD: return launch_pair_mode<GEMM_GATE_GRAD>(a, num_sms, s);
-    case GEMM_WGRAD: return launch_pair_mode<GEMM_WGRAD>(a, num_sms, s);
+    default: break;   // the weight gradients run strip by strip (gemm_wgrad.cu)
   }
   return cudaErrorInvalidValue;
 }

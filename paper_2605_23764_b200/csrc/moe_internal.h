@@ -44,6 +44,7 @@ struct LayoutView {
   int* wblk_expert;  // [items] expert of each work item
   int* meta;         // [8]     {num_mblocks, R_pad, rows, num_pairs, num_work_items, 0...}
   int* blk_hist;     // [nblk][Ep] per-block histograms, then per-block exclusive prefixes
+  int* combine_order; // [T] persistent launch: tokens in the order in which their last row is produced
 };
 
 // ---- route_layout.cu
@@ -51,6 +52,7 @@ cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, 
                          int* counts, cudaStream_t s, int* launches);
 cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView& lv, DevStatus* status,
                           cudaStream_t s, int* launches);
+cudaError_t launch_layout_order(const Dims& dm, const LayoutView& lv, int cap_mblocks, cudaStream_t s, int* launches);
 
 // ---- permute.cu
 // Xp[p] = src[token of padded row p] (zeros on padding rows); optionally prow_w[p] = routing weight
@@ -66,7 +68,7 @@ cudaError_t launch_combine(const uint16_t* rows, const Dims& dm, const LayoutVie
 cudaError_t launch_dw_reduce(const float* partial, int nparts, const Dims& dm, const LayoutView& lv,
                              float* d_topk_w, cudaStream_t s, int* launches);
 
-// ---- gemm_tc.cu (tcgen05 grouped GEMMs)
+// ---- grouped GEMMs (tcgen05 on CTA pairs)
 enum GemmMode : int {
   GEMM_GATE_UP = 0,    // H = Xp . W_gate_up[e]^T, epilogue A = w * silu(g) * u     (fwd GMM1 + SwiGLU)
   GEMM_DOWN = 1,       // Y = A . W_down[e]^T                                        (fwd GMM2)
@@ -109,9 +111,8 @@ struct GemmArgs {
   uint64_t budget_ns;
 };
 
-cudaError_t launch_gemm(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
-size_t gemm_smem_bytes();
-// ---- gemm_tc2.cu: the same operators on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles)
+// ---- gemm_tc2.cu: token-row tiles on CTA pairs (tcgen05 cta_group::2, 256 x 256): the row-space operators
+// of shapes the token-column tiles do not cover (F % 16 != 0)
 cudaError_t launch_gemm2(GemmMode mode, const GemmArgs& a, int num_sms, cudaStream_t s, int* launches);
 
 // ---- gemm_tc3.cu: the row-space operators with the tokens as accumulator COLUMNS (weights take the
@@ -122,14 +123,13 @@ cudaError_t launch_wgrad_strips(const GemmArgs& a, int num_sms, cudaStream_t s, 
 constexpr int DW_PARTS_PER_TILE = 8;  // routing-weight gradient partials per (row, column tile): 2 CTAs x 4 warps
 
 // ---- fused.cu (the single persistent dependency-driven launch)
-// Everything one fused launch needs: the operators' GEMM arguments (one per schedule segment), the
-// schedule, the counters, and the tensors of the vector tasks.
+// Everything one fused launch needs: the operators' GEMM arguments (one per phase), the chain
+// parameters, the event counters, and the tensors of the vector tasks.
 struct FusedArgs {
   GemmArgs op[SCHED_MAX_SEG];
-  SchedParams sp;
+  ChainParams cp;
   LayoutView lv;
-  const int* step_start;
-  int* ctr;
+  int* ctr;                 // event counters (zeroed before the launch), schedule.h
   int d, kp;
   // gather (Dispatch / backward Dispatch)
   const uint16_t* gather_src;
@@ -143,18 +143,13 @@ struct FusedArgs {
   const float* dw_partial;
   int dw_nparts;
   float* d_topk_w;          // may be NULL
-  uint16_t* dW1;
-  uint16_t* dW2;
-  size_t dW1_slab_vec, dW2_slab_vec;  // 16-byte vectors per expert slab
-  long long* stats;         // diagnostic builds: per-CTA wait accounting [grid][32]
+  // per-tile trace (NULL: off)
+  uint4* trace;
+  int trace_cap;
   DevStatus* status;
   uint64_t budget_ns;
 };
 
-
-// step_start[i] = matrix-queue tickets before step i; also zeroes the counter block.
-cudaError_t launch_build_schedule(const SchedParams& sp, const LayoutView& lv, int* step_start, int* ctr,
-                                  int ctr_count, cudaStream_t s, int* launches);
 cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, cudaStream_t s, int* launches);
 
 }  // namespace moe

@@ -289,6 +289,70 @@ __global__ void __launch_bounds__(LAYOUT_THREADS) layout_rank_kernel(const int* 
   }
 }
 
+// Combine order of the persistent launch: tokens sorted by the M-block of their LAST row in the expert-ordered
+// row space (a counting sort; one block).  The operators walk the experts in order, so this is the order in
+// which tokens become complete: combine tasks taken in this order find their dependent events met one after
+// the other instead of all at the very end.  Tokens without any row come first.
+constexpr int ORDER_MAX_BINS = 12000;   // bins (M-blocks + 1) that fit the block's shared memory
+__global__ void __launch_bounds__(1024) layout_order_kernel(int T, int kp, LayoutView lv) {
+  extern __shared__ int bins[];
+  __shared__ int carry_s;
+  __shared__ int warp_sums[32];
+  const int nb = lv.meta[0] + 1;
+  if (nb > ORDER_MAX_BINS) {   // beyond the shared-memory histogram: token order
+    for (int t = threadIdx.x; t < T; t += blockDim.x) lv.combine_order[t] = t;
+    return;
+  }
+  for (int i = threadIdx.x; i < nb; i += blockDim.x) bins[i] = 0;
+  if (threadIdx.x == 0) carry_s = 0;
+  __syncthreads();
+  auto key_of = [&](int t) {
+    int pmax = -1;
+    for (int j = 0; j < kp; ++j) pmax = max(pmax, lv.prow_of[(size_t)t * kp + j]);
+    return pmax < 0 ? 0 : pmax / BLOCK_M + 1;
+  };
+  for (int t = threadIdx.x; t < T; t += blockDim.x) atomicAdd(&bins[key_of(t)], 1);
+  __syncthreads();
+  // exclusive scan of the bins, 1024 at a time
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int base = 0; base < nb; base += blockDim.x) {
+    const int i = base + threadIdx.x;
+    const int v = i < nb ? bins[i] : 0;
+    int incl = v;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      int o = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += o;
+    }
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      int w = warp_sums[lane], wi = w;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        int o = __shfl_up_sync(0xffffffffu, wi, off);
+        if (lane >= off) wi += o;
+      }
+      warp_sums[lane] = wi - w;
+    }
+    __syncthreads();
+    const int excl = carry_s + warp_sums[warp] + incl - v;
+    if (i < nb) bins[i] = excl;
+    __syncthreads();
+    if (threadIdx.x == blockDim.x - 1) carry_s = excl + v;
+    __syncthreads();
+  }
+  for (int t = threadIdx.x; t < T; t += blockDim.x) lv.combine_order[atomicAdd(&bins[key_of(t)], 1)] = t;
+}
+
+cudaError_t launch_layout_order(const Dims& dm, const LayoutView& lv, int cap_mblocks, cudaStream_t s, int* launches) {
+  int nb = cap_mblocks + 2;
+  if (nb > ORDER_MAX_BINS) nb = ORDER_MAX_BINS;
+  layout_order_kernel<<<1, 1024, sizeof(int) * (size_t)nb, s>>>(dm.T, dm.kp(), lv);
+  ++*launches;
+  return cudaGetLastError();
+}
+
 cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView& lv, DevStatus* status,
                           cudaStream_t s, int* launches) {
   const int n = dm.slots(), Ep = dm.Ep();

@@ -1,21 +1,31 @@
-// The static tile schedule of the single persistent launch: two ticket-ordered queues (matrix
-// tiles and vector tasks, the counterparts of the paper's CTQ and VTQ, Section 4.3), the dependent
-// and trigger counters of every tile with their static thresholds, and the decode from a ticket to
-// a tile.  Plain host/device code without CUDA calls, so the same functions drive the kernels and
-// the CPU-side simulation that checks the schedule for deadlock freedom.
+// The static tile schedule of the single persistent launch: per CTA pair a statically ordered
+// matrix queue (the counterpart of the paper's per-core task queue, Section 4.3), one ticket-ordered
+// vector queue shared by all vector workers, and the dependent / trigger event counters of every
+// tile with their static thresholds.  Plain host/device code without CUDA calls, so the same
+// functions drive the kernels and the CPU-side simulation that checks the schedule for coverage and
+// deadlock freedom.
 //
-// Matrix queue.  "Steps" run over the experts in order.  Forward step i holds the gate+up tiles of
-// expert i (column tile slow, M-block fast: tiles in flight together share one slab of weights)
-// and the down tiles of expert i-lag; the lag keeps a consumer's producers a few hundred tickets
-// ahead, so its dependency is normally met when its ticket comes up while the intermediate it reads
-// is still L2-resident (the paper's producer/consumer placement, Section 4.4).  Backward step i
-// holds the act_grad tiles of expert i and its w2_grad strips (they share the gathered upstream
-// gradient: the paper's cache-guided GMM interleaving, Section 4.5), then the gate_grad tiles of
-// expert i-lag and its w1_grad strips (they share dH).  A weight-gradient ticket is a strip: one
-// 128-row block of the gradient across all its column tiles.
+// Matrix queue.  The operators of a pass are phases in dependency order -- forward: gate+up, down;
+// backward: act_grad, w2_grad, gate_grad, w1_grad -- and phase p's work items are numbered
+// expert-major (column tile slow, token tile fast: items in flight together share one slab of
+// weights through L2).  Pair q of Q executes the items q, q+Q, q+2Q, .. of phase 0, then those of
+// phase 1, and so on: exactly the order in which the one-launch-per-operator kernels walk the same
+// items, without the kernel boundary in between.  A pair that reaches phase p+1 early starts on it
+// while other pairs still finish phase p; what orders tiles are only the event counters.
 //
-// Every tile's producers have smaller tickets in their queue; queues are consumed in ticket
-// order by workers that are all resident, hence no deadlock (Section 4.3, correctness argument).
+// Events (Section 4.3).  Per M-block (128 rows of the padded expert-ordered row space) three
+// counters with static thresholds:
+//   gathered   += 1 per gather sub-task (4 rows)                  threshold GATHER_SUB
+//   activated  += 1 per epilogue warp and column tile of phase 0  threshold SIG * column tiles
+//   done       += 1 per epilogue warp and column tile of the last row-space phase (down / gate_grad)
+// A phase-0 item depends on `gathered` of its M-blocks, a down / gate_grad item and a w1_grad
+// strip on `activated`, a w2_grad strip on `gathered`; a combine task depends on `done` of the
+// M-blocks that hold its tokens' rows (many-to-many: up to k+S counters per token), the
+// routing-weight-gradient task of an M-block on its `activated`.
+//
+// Deadlock freedom: every item's producers are items of an earlier phase (or vector tasks with
+// smaller tickets), each pair runs its phases in order and all pairs are resident (cooperative
+// launch), so the pair that owns the lowest unfinished producer is never blocked on a later phase.
 #pragma once
 
 #include <stdint.h>
@@ -28,33 +38,14 @@
 
 namespace moe {
 
-constexpr int SCHED_MAX_SEG = 4;
-constexpr int GATHER_SUB = 8;          // vector sub-tasks per M-block gather (16 rows each)
-constexpr int EPI_WARPS = 4;           // epilogue warps per matrix tile; each signals once
+constexpr int SCHED_MAX_SEG = 4;       // phases of a pass
+constexpr int GATHER_SUB = 32;         // vector sub-tasks per M-block gather (4 rows each: the first M-blocks of a
+                                       // launch, which every CTA pair waits for, are complete after a few microseconds)
+constexpr int EPI_WARPS = 4;           // epilogue warps per CTA
+constexpr int SIG = 2 * EPI_WARPS;     // signals per (M-block, column tile): every epilogue warp of the pair
 constexpr int COMBINE_TOKENS = 2;      // tokens per combine task
-constexpr int ZERO_CHUNKS = 64;        // zero-fill tasks per expert slab pair (only empty experts do work)
-constexpr int DW_SLOTS = 1024;         // routing-weight-gradient entries per task
 
-// op codes of matrix tiles (values = GemmMode) and vector tasks
-enum VecOp : int { VEC_GATHER = 0, VEC_ZERO = 1, VEC_DW = 2, VEC_COMBINE = 3, VEC_NONE = -1 };
-
-struct SchedParams {
-  int is_bwd;
-  int pair;                // 1: a row-space ticket covers a PAIR of M-blocks (two CTAs on a 256-row tile)
-  int lag;                 // in experts
-  int Ep;
-  int T, k;
-  // tickets per M-block (row-space operators) / per expert (weight-gradient strips), per segment:
-  //   forward : seg0 = gate+up (column tiles per M-block), seg1 = down (per M-block, lagged)
-  //   backward: seg0 = act_grad (per M-block), seg1 = w2_grad strips (per expert),
-  //             seg2 = gate_grad (per M-block, lagged), seg3 = w1_grad strips (per expert, lagged)
-  int seg_tiles[SCHED_MAX_SEG];
-  int strip_tiles[2];      // column tiles in one w2_grad / w1_grad strip
-  int dep_extra;           // test hook: added to the activation-counter thresholds (> 0 = never reached)
-  int tokcol;              // 1 (with pair): token-column tiles, balanced units of one or two M-blocks
-  int sig;                 // signals one (M-block, column tile) sends to its counters: EPI_WARPS, or
-                           // 2 * EPI_WARPS when the epilogue warps of both CTAs of a pair cover every row
-};
+enum VecOp : int { VEC_GATHER = 0, VEC_DW = 2, VEC_COMBINE = 3 };
 
 // Token-column tiles: the ceil(mc / 2) row-space units of an expert with mc M-blocks.  An odd count
 // does not leave a lone M-block at the end (a tile of a few tokens still streams the whole weight
@@ -72,151 +63,102 @@ MOE_HD void balanced_unit(int mc, int u, int* first, int* count) {
   }
 }
 
-MOE_HD int expert_mblocks(const int* mb_start, int e) { return mb_start[e + 1] - mb_start[e]; }
-// row-space scheduling units of an expert: its M-blocks, or its M-block pairs
-MOE_HD int expert_units(const SchedParams& sp, const int* mb_start, int e) {
-  const int m = expert_mblocks(mb_start, e);
-  return sp.pair ? (m + 1) >> 1 : m;
-}
-
-// tickets of step i
-MOE_HD int step_tiles(const SchedParams& sp, int i, const int* mb_start) {
-  int n = 0;
-  const int j = i - sp.lag;
-  if (i < sp.Ep) {
-    const int m = expert_units(sp, mb_start, i);
-    n += m * sp.seg_tiles[0];
-    if (sp.is_bwd && m > 0) n += sp.seg_tiles[1];
-  }
-  if (j >= 0 && j < sp.Ep) {
-    const int m = expert_units(sp, mb_start, j);
-    if (!sp.is_bwd) {
-      n += m * sp.seg_tiles[1];
-    } else {
-      n += m * sp.seg_tiles[2];
-      if (m > 0) n += sp.seg_tiles[3];
-    }
-  }
-  return n;
-}
-
-struct MatTile {
-  int op;        // GemmMode
-  int slot;      // which GemmArgs of the launch (segment index)
-  int e;
-  int mb;        // first M-block of the tile (row-space operators) or -1
-  int mb_count;  // M-blocks of the tile: 1, or 2 for a full pair
-  int idx;       // column tile (row-space operators) / strip index = 128-row block of the gradient
-  int group;     // tiles processed under this ticket (1, or the strip's column tiles)
-  // dependency: every counter dep_ctr[dep_first .. dep_first+dep_count) must reach dep_thr
-  int dep_base;  // 0 = gather counters, 1 = activation counters
-  int dep_first, dep_count, dep_thr;
-  // trigger: counter incremented once per epilogue warp after the tile's stores are complete
-  int trig_base; // 1 = activation counter of mb, 2 = global done counter, -1 = none
-  int trig_also_ag;  // backward act_grad also bumps the global act_grad counter
+// One work item of a row-space phase: a token tile (unit) of an expert and a column tile, or -- in the
+// phases that merge, for an expert with an odd count of three or more M-blocks -- its last two units
+// under one k-loop.  `start[e]` = first unit (or first merged item) of expert e, `blk_expert[i]` =
+// expert of unit / item i (both from the layout kernels).
+struct SwapItem {
+  int e, nb;            // expert, column tile
+  int unit;             // first unit of the item
+  int merged;           // 1: units `unit` and `unit + 1`
+  int mb_first;         // first M-block (absolute) of the item
+  int mb_count;         // M-blocks of the item (both units): 1..3, contiguous
+  int mb_count_a;       // M-blocks of the first unit
 };
-
-// Decode ticket t of step i (step_start[i] <= t < step_start[i+1]) into a tile (or strip).
-MOE_HD MatTile decode_matrix_ticket_at(const SchedParams& sp, int t, int i, const int* step_start,
-                                       const int* mb_start) {
-  const int j = i - sp.lag;
-  int r = t - step_start[i];
-  MatTile m;
-  m.trig_also_ag = 0;
-  m.group = 1;
-  m.mb_count = 0;
-  const int stride = sp.pair ? 2 : 1;  // M-blocks per row-space unit
-  if (i < sp.Ep) {
-    const int uc = expert_units(sp, mb_start, i), mc = expert_mblocks(mb_start, i);
-    if (r < uc * sp.seg_tiles[0]) {
-      m.slot = 0; m.op = sp.is_bwd ? 2 /*ACT_GRAD*/ : 0 /*GATE_UP*/;
-      m.idx = r / uc;
-      const int u = r - m.idx * uc;
-      m.mb = mb_start[i] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride; m.e = i;
-      if (sp.pair && sp.tokcol) { int f, c; balanced_unit(mc, u, &f, &c); m.mb = mb_start[i] + f; m.mb_count = c; }
-      m.dep_base = 0; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = GATHER_SUB;
-      m.trig_base = 1; m.trig_also_ag = sp.is_bwd;
-      return m;
-    }
-    r -= uc * sp.seg_tiles[0];
-    if (sp.is_bwd && mc > 0) {
-      if (r < sp.seg_tiles[1]) {
-        m.slot = 1; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = i; m.idx = r; m.group = sp.strip_tiles[0];
-        m.dep_base = 0; m.dep_first = mb_start[i]; m.dep_count = mc; m.dep_thr = GATHER_SUB;
-        m.trig_base = -1;
-        return m;
-      }
-      r -= sp.seg_tiles[1];
-    }
+MOE_HD SwapItem decode_swap_item(int t, int n_tiles_n, bool merges, const int* start, const int* blk_expert,
+                                 const int* mb_start) {
+  SwapItem it;
+  const int e = blk_expert[t / n_tiles_n];
+  const int ws = start[e];
+  const int wcount = start[e + 1] - ws;
+  const int local = t - ws * n_tiles_n;
+  it.nb = local / wcount;
+  const int wi = local - it.nb * wcount;
+  const int mc = mb_start[e + 1] - mb_start[e];
+  it.e = e;
+  it.unit = wi;
+  it.merged = (merges && (mc & 1) && mc >= 3 && wi == wcount - 1) ? 1 : 0;
+  int f, c;
+  balanced_unit(mc, wi, &f, &c);
+  it.mb_first = mb_start[e] + f;
+  it.mb_count_a = c;
+  it.mb_count = c;
+  if (it.merged) {
+    int f2, c2;
+    balanced_unit(mc, wi + 1, &f2, &c2);
+    it.mb_count += c2;
   }
-  // lagged segments of expert j
-  const int uc = expert_units(sp, mb_start, j), mc = expert_mblocks(mb_start, j);
-  if (!sp.is_bwd || r < uc * sp.seg_tiles[2]) {
-    const int seg = sp.is_bwd ? 2 : 1;
-    m.slot = seg; m.op = sp.is_bwd ? 3 /*GATE_GRAD*/ : 1 /*DOWN*/; m.e = j;
-    m.idx = r / uc;
-    const int u = r - m.idx * uc;
-    m.mb = mb_start[j] + stride * u; m.mb_count = (mc - stride * u) < stride ? (mc - stride * u) : stride;
-    if (sp.pair && sp.tokcol) { int f, c; balanced_unit(mc, u, &f, &c); m.mb = mb_start[j] + f; m.mb_count = c; }
-    m.dep_base = 1; m.dep_first = m.mb; m.dep_count = m.mb_count; m.dep_thr = sp.sig * sp.seg_tiles[0] + sp.dep_extra;
-    m.trig_base = 2;
-    return m;
-  }
-  r -= uc * sp.seg_tiles[2];
-  m.slot = 3; m.op = 4 /*WGRAD*/; m.mb = -1; m.e = j; m.idx = r; m.group = sp.strip_tiles[1];
-  m.dep_base = 1; m.dep_first = mb_start[j]; m.dep_count = mc;
-  m.dep_thr = sp.sig * sp.seg_tiles[0] + sp.dep_extra; m.trig_base = -1;
-  return m;
+  return it;
 }
 
-// Decode ticket t (0 <= t < step_start[Ep+lag]) into a tile (or strip).
-MOE_HD MatTile decode_matrix_ticket(const SchedParams& sp, int t, const int* step_start, const int* mb_start) {
-  int lo = 0, hi = sp.Ep + sp.lag - 1;  // last step whose start <= t
-  while (lo < hi) {
-    int mid = (lo + hi + 1) >> 1;
-    if (step_start[mid] <= t) lo = mid; else hi = mid - 1;
-  }
-  return decode_matrix_ticket_at(sp, t, lo, step_start, mb_start);
+// What a pass consists of (filled on the host from the layer's shape).
+struct ChainParams {
+  int is_bwd;
+  int Ep, T, k, kp;
+  int n_phases;                 // 2 (forward) or 4 (backward)
+  int ntn[SCHED_MAX_SEG];       // column tiles per item (row-space phases) / per strip (weight gradients)
+  int strips[SCHED_MAX_SEG];    // weight-gradient phases: strips (256 rows of dW) per expert; else 0
+  int merges[SCHED_MAX_SEG];    // row-space phases: 1 if the phase merges the last two units of odd experts
+  int dep_extra;                // test hook: added to the `activated` threshold (> 0 = never reached)
+  int want_dw;                  // backward: routing-weight-gradient tasks are part of the vector queue
+};
+MOE_HD int thr_gathered() { return GATHER_SUB; }
+MOE_HD int thr_activated(const ChainParams& cp) { return SIG * cp.ntn[0] + cp.dep_extra; }
+MOE_HD int thr_done(const ChainParams& cp) { return SIG * cp.ntn[cp.is_bwd ? 2 : 1]; }
+
+// ---------------------------------------------------------------- counters (ints in device memory)
+constexpr int CTR_VEC_TICKET = 0, CTR_TRACE_CURSOR = 1, CTR_MAT_TICKET = 2, CTR_POST_TICKET = 3, CTR_PER_MB = 8, CTR_STRIDE = 4;
+enum CtrKind : int { CTR_GATHERED = 0, CTR_ACTIVATED = 1, CTR_DONE = 2, CTR_NONE = -1 };
+MOE_HD int ctr_index(int mb, int kind) { return CTR_PER_MB + CTR_STRIDE * mb + kind; }
+MOE_HD int ctr_ints(int cap_mblocks) { return CTR_PER_MB + CTR_STRIDE * cap_mblocks; }
+
+// dependent / trigger counter kind of each phase
+MOE_HD int phase_wait_kind(const ChainParams& cp, int phase) {
+  if (!cp.is_bwd) return phase == 0 ? CTR_GATHERED : CTR_ACTIVATED;
+  return (phase == 0 || phase == 1) ? CTR_GATHERED : CTR_ACTIVATED;
+}
+MOE_HD int phase_wait_thr(const ChainParams& cp, int phase) {
+  return phase_wait_kind(cp, phase) == CTR_GATHERED ? thr_gathered() : thr_activated(cp);
+}
+MOE_HD int phase_trigger_kind(const ChainParams& cp, int phase) {
+  if (!cp.is_bwd) return phase == 0 ? CTR_ACTIVATED : CTR_DONE;
+  return phase == 0 ? CTR_ACTIVATED : (phase == 2 ? CTR_DONE : CTR_NONE);
 }
 
-// ---------------------------------------------------------------- vector queue
+// ---------------------------------------------------------------- vector queues (ticket order)
+// Two queues: the gather sub-tasks in M-block order, and behind them the tasks that consume matrix tiles
+// (backward: the routing-weight gradient per M-block; then the combine tasks).  A worker leaves the first
+// queue for the second only when the first is empty -- or earlier, when it is not one of the few workers
+// that keep gathering in the background (see fused.cu).
+constexpr int GATHER_FAST_MBLOCKS = 32;   // M-blocks every vector worker helps to gather at the start of a launch
 struct VecTask {
   int op;       // VecOp
-  int idx;      // task index inside its kind
-  int dep;      // 0 = none, 2 = global done counter, 3 = global act_grad counter
-  int dep_thr;
+  int idx;      // gather: M-block * GATHER_SUB + sub-task; dw: M-block; combine: task (COMBINE_TOKENS tokens)
 };
-
-MOE_HD int vec_total(const SchedParams& sp, int M) {
-  int n = GATHER_SUB * M + (sp.T + COMBINE_TOKENS - 1) / COMBINE_TOKENS;
-  if (sp.is_bwd) n += sp.Ep * ZERO_CHUNKS + (sp.T * sp.k + DW_SLOTS - 1) / DW_SLOTS;
+MOE_HD int gather_total(int M) { return GATHER_SUB * M; }
+MOE_HD int post_total(const ChainParams& cp, int M) {
+  int n = (cp.T + COMBINE_TOKENS - 1) / COMBINE_TOKENS;
+  if (cp.is_bwd && cp.want_dw) n += M;
   return n;
 }
-
-MOE_HD VecTask decode_vector_ticket(const SchedParams& sp, int t, int M) {
+MOE_HD VecTask decode_post_ticket(const ChainParams& cp, int t, int M) {
   VecTask v;
-  v.dep = 0; v.dep_thr = 0;
-  if (t < GATHER_SUB * M) { v.op = VEC_GATHER; v.idx = t; return v; }
-  t -= GATHER_SUB * M;
-  if (sp.is_bwd) {
-    if (t < sp.Ep * ZERO_CHUNKS) { v.op = VEC_ZERO; v.idx = t; return v; }
-    t -= sp.Ep * ZERO_CHUNKS;
-    const int ndw = (sp.T * sp.k + DW_SLOTS - 1) / DW_SLOTS;
-    if (t < ndw) {
-      v.op = VEC_DW; v.idx = t; v.dep = 3; v.dep_thr = sp.sig * M * sp.seg_tiles[0];
-      return v;
-    }
-    t -= ndw;
+  if (cp.is_bwd && cp.want_dw) {
+    if (t < M) { v.op = VEC_DW; v.idx = t; return v; }
+    t -= M;
   }
-  v.op = VEC_COMBINE; v.idx = t; v.dep = 2;
-  v.dep_thr = sp.sig * M * (sp.is_bwd ? sp.seg_tiles[2] : sp.seg_tiles[1]);
+  v.op = VEC_COMBINE; v.idx = t;
   return v;
 }
-
-// Layout of the counter block in device memory (ints).
-constexpr int CTR_MAT_TICKET = 0, CTR_VEC_TICKET = 1, CTR_DONE = 2, CTR_AG_DONE = 3, CTR_PER_MB = 8;
-MOE_HD int ctr_gather(int mb) { return CTR_PER_MB + 2 * mb; }
-MOE_HD int ctr_act(int mb) { return CTR_PER_MB + 2 * mb + 1; }
-MOE_HD int ctr_ints(int cap_mblocks) { return CTR_PER_MB + 2 * cap_mblocks; }
 
 }  // namespace moe

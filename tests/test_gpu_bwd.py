@@ -93,7 +93,7 @@ def test_repeat_runs_and_launch_modes_are_bit_identical():
             else:
                 for a, b in zip(first, res):
                     assert torch.equal(a, b)
-        assert layer.launches() == (7 if serial else 2)
+        assert layer.launches() == (7 if serial else 1)   # launches of the backward call
         layer.close()
 
 
