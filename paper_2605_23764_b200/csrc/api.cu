@@ -134,7 +134,7 @@ struct Carve {
 
 // Byte offsets of every workspace tensor.
 struct WsPlan {
-  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, work_start, wblk_expert, blk_hist, row_of, src_of, prow_of, combine_order, prow_w,
+  size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, work_start, wblk_expert, blk_hist, row_of, src_of, prow_of, combine_order, tok_last, prow_w,
       dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dw, st_logits, ctr, trace, total;
   int cap_rows, nblk_max, ntn_act, ctr_count, trace_cap;
 };
@@ -166,6 +166,7 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.src_of = c.take(sizeof(int) * (slots + 1));
   p.prow_of = c.take(sizeof(int) * (slots + 1));
   p.combine_order = c.take(sizeof(int) * ((size_t)s.T_max + 1));
+  p.tok_last = c.take(sizeof(int) * ((size_t)s.T_max + 1));
   p.prow_w = c.take(sizeof(float) * cap);
   p.dw_partial = c.take(train ? sizeof(float) * cap * p.ntn_act * DW_PARTS_PER_TILE : 0);
   p.Xp = c.take(2 * cap * s.d);
@@ -244,7 +245,7 @@ struct moe_ctx {
   T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
   DevStatus* status() const { return at<DevStatus>(plan.status); }
   LayoutView layout() const {
-    LayoutView lv;
+    LayoutView lv{};
     lv.counts = at<int>(plan.counts);
     lv.offsets = at<int>(plan.offsets);
     lv.row_of = at<int>(plan.row_of);
@@ -260,6 +261,7 @@ struct moe_ctx {
     lv.meta = at<int>(plan.meta);
     lv.blk_hist = at<int>(plan.blk_hist);
     lv.combine_order = at<int>(plan.combine_order);
+    lv.tok_last = (shape.n_shared == 0 && !(shape.flags & MOE_FLAG_SERIAL_LAUNCH) && shape.F % 16 == 0) ? at<int>(plan.tok_last) : nullptr;
     return lv;
   }
   Dims dims(int T) const { return Dims{T, shape.d, shape.E, shape.k, shape.n_shared, shape.F}; }
@@ -483,6 +485,7 @@ FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
   FusedArgs fa;
   memset(&fa, 0, sizeof fa);
   fa.lv = c->layout();
+  if (s.n_shared != 0) fa.lv.combine_order = nullptr;   // token order
   fa.ctr = c->at<int>(p.ctr);
   fa.d = s.d;
   fa.kp = s.k + s.n_shared;
@@ -539,7 +542,8 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
   {
     Phase ph(c, MOE_PHASE_LAYOUT, st);
     MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
-    if (!serial_mode(c)) MOE_CUDA(launch_layout_order(dm, lv, p.cap_rows / BLOCK_M, st, &c->launches));
+    // with shared experts every token's last row belongs to the last expert: token order is as good as any
+    if (!serial_mode(c) && c->shape.n_shared == 0) MOE_CUDA(launch_layout_order(dm, lv, p.cap_rows / BLOCK_M, st, &c->launches));
   }
   if (serial_mode(c)) {
     {

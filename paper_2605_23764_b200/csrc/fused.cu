@@ -98,7 +98,7 @@ __device__ __forceinline__ bool vec_combine(const FusedArgs& fa, int task, int l
   const int i0 = task * COMBINE_TOKENS, i1 = min(T, i0 + COMBINE_TOKENS);
   const int thr = thr_done(fa.cp);
   for (int i = i0; i < i1; ++i) {
-    const int t = fa.lv.combine_order[i];   // tokens in the order in which their last row is produced
+    const int t = fa.lv.combine_order ? fa.lv.combine_order[i] : i;   // tokens in the order in which their last row is produced
     const int* prow = fa.lv.prow_of + (size_t)t * kp;
     // dependent events: `done` of every M-block that holds one of the token's rows
     int ok = 1;

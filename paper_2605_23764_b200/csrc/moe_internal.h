@@ -44,7 +44,8 @@ struct LayoutView {
   int* wblk_expert;  // [items] expert of each work item
   int* meta;         // [8]     {num_mblocks, R_pad, rows, num_pairs, num_work_items, 0...}
   int* blk_hist;     // [nblk][Ep] per-block histograms, then per-block exclusive prefixes
-  int* combine_order; // [T] persistent launch: tokens in the order in which their last row is produced
+  int* combine_order; // [T] persistent launch: tokens in the order in which their last row is produced (NULL: token order)
+  int* tok_last;      // [T] 1 + largest padded row of each token (0: none); NULL when the combine order is not wanted
 };
 
 // ---- route_layout.cu

@@ -125,8 +125,11 @@ __device__ __forceinline__ void chunk_histogram(const int* __restrict__ ids, int
 
 __global__ void __launch_bounds__(LAYOUT_THREADS) layout_hist_kernel(const int* __restrict__ ids, int n, int k,
                                                                       int kp, int E, int Ep,
-                                                                      int* __restrict__ blk_hist) {
+                                                                      int* __restrict__ blk_hist, int* __restrict__ tok_last) {
   extern __shared__ int whist[];
+  if (tok_last)   // the tokens whose first slot lies in this block's chunk
+    for (int i = blockIdx.x * LAYOUT_CHUNK + threadIdx.x; i < min(n, (blockIdx.x + 1) * LAYOUT_CHUNK); i += LAYOUT_THREADS)
+      if (i % kp == 0) tok_last[i / kp] = 0;
   chunk_histogram(ids, n, k, kp, E, Ep, whist);
   for (int e = threadIdx.x; e < Ep; e += LAYOUT_THREADS) {
     int tot = 0;
@@ -280,6 +283,7 @@ __global__ void __launch_bounds__(LAYOUT_THREADS) layout_rank_kernel(const int* 
         lv.row_of[i] = row;
         lv.prow_of[i] = lv.pad_off[e] + r;
         lv.src_of[row] = i;
+        if (lv.tok_last) atomicMax(&lv.tok_last[i / kp], lv.pad_off[e] + r + 1);
       } else {
         lv.row_of[i] = -1;
         lv.prow_of[i] = -1;
@@ -306,10 +310,9 @@ __global__ void __launch_bounds__(1024) layout_order_kernel(int T, int kp, Layou
   for (int i = threadIdx.x; i < nb; i += blockDim.x) bins[i] = 0;
   if (threadIdx.x == 0) carry_s = 0;
   __syncthreads();
-  auto key_of = [&](int t) {
-    int pmax = -1;
-    for (int j = 0; j < kp; ++j) pmax = max(pmax, lv.prow_of[(size_t)t * kp + j]);
-    return pmax < 0 ? 0 : pmax / BLOCK_M + 1;
+  auto key_of = [&](int t) {   // tok_last[t] = 1 + the token's largest padded row (0: no row), from the rank kernel
+    const int last = lv.tok_last[t];
+    return last == 0 ? 0 : (last - 1) / BLOCK_M + 1;
   };
   for (int t = threadIdx.x; t < T; t += blockDim.x) atomicAdd(&bins[key_of(t)], 1);
   __syncthreads();
@@ -358,7 +361,7 @@ cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView&
   const int n = dm.slots(), Ep = dm.Ep();
   const int nblk = n > 0 ? (n + LAYOUT_CHUNK - 1) / LAYOUT_CHUNK : 1;
   const size_t sm_hist = sizeof(int) * (size_t)LAYOUT_WARPS * Ep;
-  layout_hist_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv.blk_hist);
+  layout_hist_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv.blk_hist, lv.tok_last);
   layout_scan_kernel<<<1, 1024, sizeof(int) * (size_t)(4 * Ep + 3), s>>>(nblk, Ep, lv);
   layout_rank_kernel<<<nblk, LAYOUT_THREADS, sm_hist, s>>>(topk_ids, n, dm.k, dm.kp(), dm.E, Ep, lv, status);
   *launches += 3;
@@ -443,7 +446,7 @@ extern "C" int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E,
   // the array keeps the previous call's contents: the status word must start at zero
   if (cudaMemsetAsync(&sc->status, 0, sizeof(moe::DevStatus), st) != cudaSuccess) return MOE_ERR_CUDA;
   moe::Dims dm{T, 8, E, k, n_shared, 8};
-  moe::LayoutView lv;
+  moe::LayoutView lv{};   // (fields not set below stay NULL: no combine order here)
   lv.counts = counts;
   lv.offsets = offsets;
   lv.row_of = row_of;
