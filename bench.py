@@ -1,18 +1,25 @@
 #!/usr/bin/env python
 """Benchmark of the Dispatch->Combine MoE-FFN layer on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--launch auto|fused|serial] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
 
 One step = one pass of the whole hot path on one batch of seeded synthetic input: routing,
 forward (dispatch layout, permute-gather, grouped GEMM gate+up with SwiGLU, grouped GEMM down,
-combine) and, for the training workloads, backward (the seven backward operators).  Rank 0
+combine) and, for the training workload, backward (the seven backward operators).  Rank 0
 prints ONE JSON line.  Throughput counts 6*R*d*F FLOP per forward and 12*R*d*F per backward
-(R = tokens x experts per token).  With N > 1 every rank runs an independent replica on its
-own GPU (the layer is not sharded; there is no data-path collective).
+(R = tokens x experts per token).
+
+The headline `value` is the library's default launch mode: one persistent dependency-driven
+launch per pass.  The one-launch-per-operator mode is timed in the same run and reported as
+`other_launch_mode`; `all_configs` holds both modes for the forward-only workloads.
+With N > 1 every rank runs an independent replica on its own GPU (the layer is not sharded;
+there is no data-path collective); `python bench.py --gpus N` without a launcher starts the N
+ranks itself.
 """
 from __future__ import annotations
 
 import argparse
+import gc
 import json
 import os
 import statistics
@@ -29,6 +36,10 @@ sys.path.insert(0, ROOT)
 from workloads import configs  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+METRIC = "moe_ffn_dispatch_to_combine_tflops"
+LAUNCH_NAMES = {"serial": "serial kernels (one launch per operator)",
+                "fused": "fused persistent (one launch each for forward and backward, after the index-only "
+                         "layout kernels)"}
 
 
 def load_peaks():
@@ -98,7 +109,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
             self.proc = None
@@ -110,7 +121,7 @@ class ClockSampler:
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.12)
         self.proc.terminate()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
@@ -129,7 +140,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def dist_setup(n_gpus):
+def dist_setup():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -167,74 +178,74 @@ def replica_throughput(local_ms_per_step, flops_per_replica_step, world, device=
 # ----------------------------------------------------------------------------------------------
 # CPU oracle legs (rank 0 only): a bounded sample of the same workload
 # ----------------------------------------------------------------------------------------------
-def oracle_sample(cfg, train, n_experts, inputs=None, max_rows=None):
-    """Times the oracle on the rows of `n_experts` experts (forward, and backward if `train`).
+def oracle_sample(cfg, train, n_experts, rows_per_expert, inputs=None):
+    """Times the oracle on an exact sub-problem of the workload: up to `rows_per_expert` rows of each
+    of `n_experts` median-loaded experts, ONE oracle call over all of them (forward, and backward if
+    `train`), so that its loops over tokens and over experts have work for every thread.
 
-    Returns (seconds, flops, description).  A weight gradient and an expert's rows need only that
-    expert's slabs, so the sample is an exact sub-problem of the workload."""
+    Returns (seconds, flops, description).  An expert's rows and weight gradient need only that
+    expert's slabs, which is what makes the sample exact."""
     import oracle
     dev = "cpu"
     x = inputs["x"].cpu() if inputs else configs.make_x(cfg, dev)
     logits = inputs["logits"].cpu() if inputs else configs.make_logits(cfg, x)
     ids, w = oracle.route(logits, cfg.k, cfg.renorm)
-    ids_t = torch.from_numpy(ids)
+    ids_t, w_t = torch.from_numpy(ids), torch.from_numpy(w)
     dout = (inputs["dout"].cpu() if inputs else configs.make_dout(cfg, dev)) if train else None
     counts = torch.bincount(ids_t.flatten().long(), minlength=cfg.E)
     order = torch.argsort(counts, descending=True)
-    picked = [int(e) for e in order[len(order) // 2: len(order) // 2 + n_experts]]  # median-loaded experts
-    secs, flops, rows = 0.0, 0.0, 0
-    for e in picked:
+    lo = max(0, len(order) // 2 - n_experts // 2)
+    picked = [int(e) for e in order[lo: lo + n_experts] if counts[int(e)] > 0]
+    toks, sub_ids, sub_w = [], [], []
+    for i, e in enumerate(picked):
         tok, slot = torch.nonzero(ids_t == e, as_tuple=True)
-        if max_rows is not None:
-            tok, slot = tok[:max_rows], slot[:max_rows]
-        n = tok.numel()
-        if n == 0:
-            continue
-        W1 = configs.w_gate_up_slab(cfg, e)[None]
-        W2 = configs.w_down_slab(cfg, e)[None]
-        sub_ids = torch.zeros(n, 1, dtype=torch.int32)
-        sub_w = torch.from_numpy(w)[tok, slot][:, None]
-        xs = x[tok]
-        t0 = time.perf_counter()
-        oracle.fwd(xs, sub_ids, sub_w, W1, W2)
-        if train:
-            oracle.bwd(dout[tok], xs, sub_ids, sub_w, W1, W2)
-        secs += time.perf_counter() - t0
-        flops += 6.0 * n * cfg.d * cfg.F * (3.0 if train else 1.0)
-        rows += n
-    desc = (f"{'fwd+bwd' if train else 'fwd'} of {rows} rows of {len(picked)} median-loaded experts "
-            f"(of {cfg.R} rows, {cfg.Ep} experts)")
+        tok, slot = tok[:rows_per_expert], slot[:rows_per_expert]
+        toks.append(tok)
+        sub_ids.append(torch.full((tok.numel(), 1), i, dtype=torch.int32))
+        sub_w.append(w_t[tok, slot][:, None])
+    tok = torch.cat(toks)
+    sub_ids, sub_w = torch.cat(sub_ids), torch.cat(sub_w)
+    W1 = torch.stack([configs.w_gate_up_slab(cfg, e) for e in picked])
+    W2 = torch.stack([configs.w_down_slab(cfg, e) for e in picked])
+    xs = x[tok]
+    rows = tok.numel()
+    t0 = time.perf_counter()
+    oracle.fwd(xs, sub_ids, sub_w, W1, W2)
+    if train:
+        oracle.bwd(dout[tok], xs, sub_ids, sub_w, W1, W2)
+    secs = time.perf_counter() - t0
+    flops = 6.0 * rows * cfg.d * cfg.F * (3.0 if train else 1.0)
+    desc = (f"{'fwd+bwd' if train else 'fwd'} of {rows} rows of {len(picked)} median-loaded experts in one oracle "
+            f"call (of {cfg.R} rows, {cfg.Ep} experts)")
     return secs, flops, desc
 
 
-def calibrate_sample(cfg, train, target_s=15.0):
-    """(experts, rows per expert) giving roughly `target_s` seconds of oracle work.  The rate is a
-    fixed estimate of the plain-loop fp64 oracle (its weight-gradient loop of a one-expert
-    sub-problem runs on one thread), not a measurement."""
-    rows_per_expert = max(1, int(cfg.T * cfg.k / cfg.E))
+def calibrate_sample(cfg, train, threads, target_s=15.0):
+    """(experts, rows per expert) giving roughly `target_s` seconds of oracle work with every thread
+    busy: at least `threads` experts, as many rows each as the time allows.  The rate is a fixed estimate
+    of the plain-loop fp64 oracle per thread, not a measurement."""
+    n_exp = int(min(cfg.E, max(threads, 1)))
     flop_per_row = 6.0 * cfg.d * cfg.F * (3.0 if train else 1.0)
-    est_rate = 3.0e9 if train else 1.0e10
-    rows = max(1, int(target_s * est_rate / flop_per_row))
-    if rows <= rows_per_expert:
-        return 1, rows
-    return int(min(cfg.E, max(1, round(rows / rows_per_expert)))), None
+    est_rate_per_thread = 0.15e9 if train else 0.5e9
+    rows = max(1, int(target_s * est_rate_per_thread * min(threads, n_exp) / flop_per_row))
+    return n_exp, max(1, rows // n_exp)
 
 
 def run_reference(args, cfg, train):
     import oracle
-    n_exp, max_rows = calibrate_sample(cfg, train, target_s=4.0)
+    n_exp, rows = calibrate_sample(cfg, train, oracle.threads(), target_s=4.0)
     times, flops, desc = [], 0.0, ""
     for i in range(args.warmup + args.steps):
-        secs, flops, desc = oracle_sample(cfg, train, n_exp, max_rows=max_rows)
+        secs, flops, desc = oracle_sample(cfg, train, n_exp, rows)
         if i >= args.warmup:
             times.append(secs)
     ms = 1e3 * sum(times) / len(times)
     val = flops / (ms * 1e-3) / 1e12
-    cfg_desc = workload_desc(cfg, train, args)
+    cfg_desc = workload_desc(cfg, train)
     cfg_desc["launch"] = "none (CPU oracle on host cores)"
     line = {
-        "impl": "reference", "metric": "moe_ffn_dispatch_to_combine_tflops", "value": val, "unit": "TFLOP/s",
-        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s",
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": cfg_desc, "gpu_launches": 0,
         "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle", "sample": desc},
@@ -243,262 +254,139 @@ def run_reference(args, cfg, train):
     print(json.dumps(line), flush=True)
 
 
-def workload_desc(cfg, train, args):
+def workload_desc(cfg, train):
     return {"workload": cfg.name, "T": cfg.T, "d": cfg.d, "E": cfg.E, "top_k": cfg.k, "shared": cfg.S, "F": cfg.F,
             "pass": "route+fwd+bwd" if train else "route+fwd",
-            "launch": "serial kernels" if getattr(args, "launch", "") == "serial" else "fused persistent",
             "l2": "weights and expert-ordered activations exceed the 126 MB L2 (no flush needed)"
             if cfg.weight_bytes() > 4e8 else "L2 flushed between timed steps"}
 
 
 # ----------------------------------------------------------------------------------------------
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=4, help="index into BASELINE.json configs (default: the training step)")
-    ap.add_argument("--launch", default="auto", choices=["auto", "fused", "serial"],
-                    help="fused: one persistent launch per pass; serial: one launch per operator; auto (default): "
-                         "time both, report the faster as the headline and the other beside it")
-    ap.add_argument("--serial", action="store_true", help="same as --launch serial")
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--fwd-only", action="store_true")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-compare", action="store_true", help="skip timing the other launch mode")
-    ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
-    args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.serial:
-        args.launch = "serial"
-    if args.launch == "auto" and args.no_compare:
-        args.launch = "serial"
+# one workload resident on the GPU, timed in one or both launch modes
+# ----------------------------------------------------------------------------------------------
+class Workload:
+    def __init__(self, cfg, train):
+        self.cfg, self.train = cfg, train
+        self.inp = configs.make_inputs(cfg, "cuda")
+        T = cfg.T
+        self.ids = torch.empty(T, cfg.k, dtype=torch.int32, device="cuda")
+        self.w = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
+        self.out = torch.empty_like(self.inp["x"])
+        if train:
+            self.dx = torch.empty_like(self.inp["x"])
+            self.dW1, self.dW2 = torch.empty_like(self.inp["W_gate_up"]), torch.empty_like(self.inp["W_down"])
+            self.dw = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
+        # weights that fit L2 would stay there from step to step: flush between timed steps
+        self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if cfg.weight_bytes() <= 4e8 else None
 
-    cfg = configs.CONFIGS[args.config]
-    if args.small:
-        v = [int(q) for q in args.small.split(",")]
-        cfg = configs.small_variant(cfg, v[0], v[1], v[2], v[3] if len(v) > 3 else None)
-    train = cfg.bwd and not args.fwd_only
+    def make_layer(self, mode):
+        from paper_2605_23764_b200 import MoeLayer
+        c = self.cfg
+        return MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=self.train, serial=(mode == "serial"))
 
-    if args.impl == "reference":
-        if int(os.environ.get("RANK", "0")) == 0:
-            run_reference(args, cfg, train)
-        return
+    def step(self, lay, phases=None):
+        """One pass of the hot path through the C ABI (device buffers).  -> kernels launched"""
+        from paper_2605_23764_b200 import binding as B
+        i, T, n = self.inp, self.cfg.T, 0
+        B.moe_route(lay.ctx, i["logits"], T, self.ids, self.w)
+        n += lay.launches()
+        if phases is not None:
+            phases.update(B.moe_get_phase_ms(lay.ctx))
+        B.moe_ffn_fwd(lay.ctx, i["x"], self.ids, self.w, i["W_gate_up"], i["W_down"], self.out, T)
+        n += lay.launches()
+        if phases is not None:
+            phases.update(B.moe_get_phase_ms(lay.ctx))
+        if self.train:
+            B.moe_ffn_bwd(lay.ctx, i["dout"], i["x"], self.ids, self.w, i["W_gate_up"], i["W_down"], self.dx, self.dW1,
+                          self.dW2, self.dw, T)
+            n += lay.launches()
+            if phases is not None:
+                phases.update(B.moe_get_phase_ms(lay.ctx))
+        return n
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (the layer has no CPU path)")
-    from paper_2605_23764_b200 import MoeLayer, binding as B
-
-    world, rank, local = dist_setup(args.gpus)
-    torch.cuda.set_device(local)
-    peaks = load_peaks()
-
-    inp = configs.make_inputs(cfg, "cuda")
-    x, W1, W2, logits = inp["x"], inp["W_gate_up"], inp["W_down"], inp["logits"]
-    dout = inp.get("dout")
-    def make_layer(mode):
-        return MoeLayer(cfg.T, cfg.d, cfg.E, cfg.k, cfg.S, cfg.F, renorm=cfg.renorm, save_for_bwd=train,
-                        serial=(mode == "serial"))
-    T = cfg.T
-    ids = torch.empty(T, cfg.k, dtype=torch.int32, device="cuda")
-    w = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
-    out = torch.empty_like(x)
-    if train:
-        dx, dW1, dW2 = torch.empty_like(x), torch.empty_like(W1), torch.empty_like(W2)
-        dw = torch.empty(T, cfg.k, dtype=torch.float32, device="cuda")
-    flush = None
-    if cfg.weight_bytes() <= 4e8:
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-
-    def measure(lay):
+    def measure(self, lay, steps, warmup, world, local):
         """W warm-up steps, then K timed steps back to back (CUDA events on the launching stream; the
         per-operator events inside the library are read after each call).  -> dict"""
-        def step(count=False, phases=None):
-            n = 0
-            B.moe_route(lay.ctx, logits, T, ids, w)
-            n += lay.launches()
-            if phases is not None:
-                phases.update(B.moe_get_phase_ms(lay.ctx))
-            B.moe_ffn_fwd(lay.ctx, x, ids, w, W1, W2, out, T)
-            n += lay.launches()
-            if phases is not None:
-                phases.update(B.moe_get_phase_ms(lay.ctx))
-            if train:
-                B.moe_ffn_bwd(lay.ctx, dout, x, ids, w, W1, W2, dx, dW1, dW2, dw, T)
-                n += lay.launches()
-                if phases is not None:
-                    phases.update(B.moe_get_phase_ms(lay.ctx))
-            return n
-
-        for _ in range(args.warmup - 1):
-            step()
+        from paper_2605_23764_b200 import binding as B
+        for _ in range(warmup - 1):
+            self.step(lay)
         w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        w0.record(); step(); w1.record()
+        w0.record(); self.step(lay); w1.record()
         torch.cuda.synchronize()
         assert lay.status() == (0, 0), "device-side error during warm-up"
         # The per-operator events are recorded in every timed step; READING them synchronises the stream, which
         # a sub-millisecond step would feel: short steps are read every few steps only (about one read per 5 ms).
-        read_every = max(1, min(args.steps, int(5.0 / max(w0.elapsed_time(w1), 1e-3))))
+        read_every = max(1, min(steps, int(5.0 / max(w0.elapsed_time(w1), 1e-3))))
         B.moe_set_profiling(lay.ctx, True)
         phase_sum, n_launch, n_reads = {}, 0, 0
         sampler = ClockSampler(local)
         sampler.start()
         barrier(world)
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        flush_ms = 0.0
+        flush_ms, flush_events = 0.0, []
         ev0.record()
-        for i in range(args.steps):
-            if flush is not None:
+        for i in range(steps):
+            if self.flush is not None:
                 f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                f0.record(); flush.zero_(); f1.record()
+                f0.record(); self.flush.zero_(); f1.record()
+                flush_events.append((f0, f1))
             read = (i % read_every) == read_every - 1
             ph = {} if read else None
-            n_launch += step(phases=ph)
+            n_launch += self.step(lay, phases=ph)
             if read:
                 n_reads += 1
                 for kname, v in ph.items():
                     phase_sum[kname] = phase_sum.get(kname, 0.0) + v
-            if flush is not None:
-                f1.synchronize()
-                flush_ms += f0.elapsed_time(f1)
         ev1.record()
         barrier(world)
         clk = sampler.stop()
-        local_ms = (ev0.elapsed_time(ev1) - flush_ms) / args.steps
-        value_all, ms = replica_throughput(local_ms, step_flops(cfg, train), world)
-        elapsed = ms * args.steps
+        for f0, f1 in flush_events:
+            flush_ms += f0.elapsed_time(f1)
+        local_ms = (ev0.elapsed_time(ev1) - flush_ms) / steps
+        value_all, ms = replica_throughput(local_ms, step_flops(self.cfg, self.train), world)
         B.moe_set_profiling(lay.ctx, False)
         code, detail = lay.status()
         assert code == 0, f"device-side error {code} detail {detail:#x}"
         return {"ms_per_step": ms, "value": value_all,
-                "phases_ms": {k: v / max(1, n_reads) for k, v in phase_sum.items()}, "launches": n_launch, "clocks": clk,
-                "timed_ms": elapsed}
+                "phases_ms": {k: v / max(1, n_reads) for k, v in phase_sum.items()}, "launches": n_launch,
+                "clocks": clk, "timed_ms": ms * steps}
 
-    def rooflines(res):
-        """Roofline of the operator with the largest time, and of the whole step."""
-        work = phase_work(cfg, train)
-        phases_ms = res["phases_ms"]
-        # sustained peak for work timed inside a long, power-capped region (the clocks sampled during the timed
-        # steps say which): more than 0.5 s of timed work, or the power cap active with SM clocks a fifth or
-        # more below their maximum; burst peak otherwise
-        clk = res.get("clocks") or {}
-        capped = ("sw_power_cap" in (clk.get("reasons") or []) and clk.get("sm_mhz") and clk.get("sm_max_mhz")
-                  and clk["sm_mhz"] < 0.8 * clk["sm_max_mhz"])
-        peak_tf = peaks["bf16_tflops_sustained"] if (res["timed_ms"] > 500 or capped) else peaks["bf16_tflops"]
-        peak_gb = peaks["hbm_gbs"]
-        dom = max((k for k in phases_ms if k in work), key=lambda k: phases_ms[k], default=None)
-        roof = None
-        if dom:
-            fl, by = work[dom]
-            t_s = phases_ms[dom] * 1e-3
-            tensor_bound = fl / (peak_tf * 1e12) >= by / (peak_gb * 1e9)
-            if tensor_bound:
-                roof = {"kernel": dom, "bound": "tensor", "achieved": fl / t_s / 1e12, "peak": peak_tf, "unit": "TFLOP/s"}
-            else:
-                roof = {"kernel": dom, "bound": "hbm", "achieved": by / t_s / 1e9, "peak": peak_gb, "unit": "GB/s"}
-            roof["frac"] = roof["achieved"] / roof["peak"]
-            roof["peak_source"] = peaks["source"] + ((" sustained" if peak_tf == peaks.get("bf16_tflops_sustained")
-                                                      else " burst") if tensor_bound else "")
-            roof["traffic"] = ncu_traffic(dom, cfg)
-            roof["launch_ms"] = phases_ms[dom]
-        flops = step_flops(cfg, train)
-        t_roof = max(flops / (peak_tf * 1e12), step_min_bytes(cfg, train) / (peak_gb * 1e9))
-        step_roof = {"roofline_ms": t_roof * 1e3, "frac": t_roof * 1e3 / res["ms_per_step"],
-                     "flop_ms": flops / (peak_tf * 1e12) * 1e3,
-                     "hbm_ms": step_min_bytes(cfg, train) / (peak_gb * 1e9) * 1e3}
-        return roof, step_roof
 
-    # ---- device-resident timing of the launch modes (max over ranks: every rank sees the same numbers) ----
-    launch_names = {"serial": "serial kernels (one launch per operator)",
-                    "fused": "fused persistent (one launch each for forward and backward, after the index-only "
-                             "layout and schedule kernels)"}
-    modes = ["fused", "serial"] if args.launch == "auto" else (
-        [args.launch] if args.no_compare else [args.launch, "serial" if args.launch == "fused" else "fused"])
-    layers = {m: make_layer(m) for m in modes}
-    results = {m: measure(layers[m]) for m in modes}
-    head = min(modes, key=lambda m: results[m]["ms_per_step"]) if args.launch == "auto" else args.launch
-    layer, res = layers[head], results[head]
-    ms_per_step, value, launches, clocks, phases_ms = (res["ms_per_step"], res["value"], res["launches"],
-                                                       res["clocks"], res["phases_ms"])
+def rooflines(cfg, train, res, peaks):
+    """Roofline of the operator with the largest time, and of the whole step."""
+    work = phase_work(cfg, train)
+    phases_ms = res["phases_ms"]
+    # sustained peak for work timed inside a long, power-capped region (the clocks sampled during the timed
+    # steps say which): more than 0.5 s of timed work, or the power cap active with SM clocks a fifth or
+    # more below their maximum; burst peak otherwise
+    clk = res.get("clocks") or {}
+    capped = ("sw_power_cap" in (clk.get("reasons") or []) and clk.get("sm_mhz") and clk.get("sm_max_mhz")
+              and clk["sm_mhz"] < 0.8 * clk["sm_max_mhz"])
+    sustained = res["timed_ms"] > 500 or capped
+    peak_tf = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    peak_gb = peaks["hbm_gbs"]
+    dom = max((k for k in phases_ms if k in work), key=lambda k: phases_ms[k], default=None)
+    roof = None
+    if dom:
+        fl, by = work[dom]
+        t_s = phases_ms[dom] * 1e-3
+        tensor_bound = fl / (peak_tf * 1e12) >= by / (peak_gb * 1e9)
+        if tensor_bound:
+            roof = {"kernel": dom, "bound": "tensor", "achieved": fl / t_s / 1e12, "peak": peak_tf, "unit": "TFLOP/s"}
+        else:
+            roof = {"kernel": dom, "bound": "hbm", "achieved": by / t_s / 1e9, "peak": peak_gb, "unit": "GB/s"}
+        roof["frac"] = roof["achieved"] / roof["peak"]
+        roof["peak_source"] = peaks["source"] + ((" sustained" if sustained else " burst") if tensor_bound else "")
+        roof["traffic"] = ncu_traffic(dom, cfg)
+        roof["launch_ms"] = phases_ms[dom]
     flops = step_flops(cfg, train)
-    roofline, step_roofline = rooflines(res)
-    other = None
-    for m in modes:
-        if m == head:
-            continue
-        r2 = results[m]
-        roof2, step2 = rooflines(r2)
-        other = {"launch": launch_names[m], "ms_per_step": r2["ms_per_step"], "value": r2["value"],
-                 "phases_ms": r2["phases_ms"], "roofline": roof2, "step_roofline": step2, "clocks": r2["clocks"]}
-        layers[m].close()
-
-    # ---- end to end through the host-buffer entry points ------------------------------------------
-    e2e = None
-    if not args.no_e2e:
-        pin = dict(pin_memory=True)
-        xh, lh = x.cpu().pin_memory(), logits.cpu().pin_memory()
-        idh = torch.empty(T, cfg.k, dtype=torch.int32, **pin)
-        wh = torch.empty(T, cfg.k, dtype=torch.float32, **pin)
-        oh = torch.empty(T, cfg.d, dtype=torch.bfloat16, **pin)
-        h2d = lh.numel() * 4 + xh.numel() * 2 + idh.numel() * 4 + wh.numel() * 4
-        d2h = idh.numel() * 4 + wh.numel() * 4 + oh.numel() * 2
-        if train:
-            doh = dout.cpu().pin_memory()
-            dxh = torch.empty(T, cfg.d, dtype=torch.bfloat16, **pin)
-            dwh = torch.empty(T, cfg.k, dtype=torch.float32, **pin)
-            h2d += doh.numel() * 2
-            d2h += dxh.numel() * 2 + dwh.numel() * 4
-
-        def e2e_step():
-            B.moe_route_host(layer.ctx, lh, T, idh, wh)
-            B.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, W1, W2, oh, T)
-            if train:
-                B.moe_ffn_bwd_host(layer.ctx, doh, W1, W2, dxh, dW1, dW2, dwh, T)
-
-        for _ in range(2):
-            e2e_step()
-        barrier(world)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            e2e_step()
-        e1.record()
-        barrier(world)
-        e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / args.steps
-        assert layer.status()[0] == 0
-        assert torch.equal(oh.cuda(), out), "host-buffer path disagrees with the device-buffer path"
-        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
-
-    # ---- CPU oracle baseline (rank 0, single-GPU run only) ----------------------------------------
-    cpu_baseline = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        n_exp, max_rows = calibrate_sample(cfg, train)
-        secs, fl, desc = oracle_sample(cfg, train, n_exp, inputs=inp, max_rows=max_rows)
-        cpu_baseline = {"value": fl / secs / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
-                        "sample": desc, "seconds": secs}
-
-    if rank == 0:
-        line = {
-            "metric": "moe_ffn_dispatch_to_combine_tflops", "value": value, "unit": "TFLOP/s", "n_gpus": world,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": workload_desc(cfg, train, args), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "step_roofline": step_roofline, "phases_ms": phases_ms,
-            "other_launch_mode": other, "cpu_baseline": cpu_baseline,
-        }
-        per_step = launches / max(1, args.steps)
-        line["config"]["launch"] = launch_names[head]
-        line["config"]["launch_choice"] = ("faster of the two launch modes, both timed" if args.launch == "auto"
-                                           else "requested")
-        line["config"]["launches_per_step"] = per_step
-        print(json.dumps(line), flush=True)
-    layer.close()
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    flop_ms = flops / (peak_tf * 1e12) * 1e3
+    hbm_ms = step_min_bytes(cfg, train) / (peak_gb * 1e9) * 1e3
+    t_roof = max(flop_ms, hbm_ms)
+    step_roof = {"roofline_ms": t_roof, "frac": t_roof / res["ms_per_step"], "flop_ms": flop_ms, "hbm_ms": hbm_ms,
+                 "bound": "tensor" if flop_ms >= hbm_ms else "hbm",
+                 "tensor_peak": "sustained" if sustained else "burst"}
+    return roof, step_roof
 
 
 def ncu_traffic(phase, cfg):
@@ -511,6 +399,180 @@ def ncu_traffic(phase, cfg):
         if len(parts) >= 3 and not ln.startswith("#") and parts[0] == phase and parts[1] == cfg.name:
             return float(parts[2])
     return None
+
+
+def run_e2e(wl, layer, steps, world):
+    """The same step through the host-buffer entry points: pinned host inputs in, results out, copies timed."""
+    from paper_2605_23764_b200 import binding as B
+    cfg, train, inp = wl.cfg, wl.train, wl.inp
+    T = cfg.T
+    pin = dict(pin_memory=True)
+    xh, lh = inp["x"].cpu().pin_memory(), inp["logits"].cpu().pin_memory()
+    idh = torch.empty(T, cfg.k, dtype=torch.int32, **pin)
+    wh = torch.empty(T, cfg.k, dtype=torch.float32, **pin)
+    oh = torch.empty(T, cfg.d, dtype=torch.bfloat16, **pin)
+    h2d = lh.numel() * 4 + xh.numel() * 2 + idh.numel() * 4 + wh.numel() * 4
+    d2h = idh.numel() * 4 + wh.numel() * 4 + oh.numel() * 2
+    if train:
+        doh = inp["dout"].cpu().pin_memory()
+        dxh = torch.empty(T, cfg.d, dtype=torch.bfloat16, **pin)
+        dwh = torch.empty(T, cfg.k, dtype=torch.float32, **pin)
+        h2d += doh.numel() * 2
+        d2h += dxh.numel() * 2 + dwh.numel() * 4
+
+    def e2e_step():
+        B.moe_route_host(layer.ctx, lh, T, idh, wh)
+        B.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, inp["W_gate_up"], inp["W_down"], oh, T)
+        if train:
+            B.moe_ffn_bwd_host(layer.ctx, doh, inp["W_gate_up"], inp["W_down"], dxh, wl.dW1, wl.dW2, dwh, T)
+
+    for _ in range(2):
+        e2e_step()
+    barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        e2e_step()
+    e1.record()
+    barrier(world)
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world) / steps
+    assert layer.status()[0] == 0
+    assert torch.equal(oh.cuda(), wl.out), "host-buffer path disagrees with the device-buffer path"
+    return {"value": world * step_flops(cfg, train) / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+
+def respawn_under_launcher(n):
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU) and pass their output on."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
+# ----------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, help="index of the headline workload (default: the training step)")
+    ap.add_argument("--launch", default="fused", choices=["fused", "serial"],
+                    help="launch mode of the headline value (default: the library's default, the persistent launch); "
+                         "the other mode is timed too and reported beside it")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--fwd-only", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-compare", action="store_true", help="skip timing the other launch mode")
+    ap.add_argument("--no-all-configs", action="store_true", help="skip the other workloads")
+    ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    cfg = configs.CONFIGS[args.config]
+    if args.small:
+        v = [int(q) for q in args.small.split(",")]
+        cfg = configs.small_variant(cfg, v[0], v[1], v[2], v[3] if len(v) > 3 else None)
+    train = cfg.bwd and not args.fwd_only
+
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_reference(args, cfg, train)
+        return
+
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        respawn_under_launcher(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the layer has no CPU path)")
+
+    world, rank, local = dist_setup()
+    if args.gpus != world and rank == 0:
+        print(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s); reporting n_gpus={world}",
+              file=sys.stderr)
+    torch.cuda.set_device(local)
+    peaks = load_peaks()
+    other_mode = "serial" if args.launch == "fused" else "fused"
+    modes = [args.launch] if args.no_compare else [args.launch, other_mode]
+
+    # ---- headline workload: device-resident timing of the launch modes (max over ranks) ----------
+    wl = Workload(cfg, train)
+    layers = {m: wl.make_layer(m) for m in modes}
+    results = {m: wl.measure(layers[m], args.steps, args.warmup, world, local) for m in modes}
+    head = args.launch
+    layer, res = layers[head], results[head]
+    roofline, step_roofline = rooflines(cfg, train, res, peaks)
+    other = None
+    if other_mode in results:
+        r2 = results[other_mode]
+        roof2, step2 = rooflines(cfg, train, r2, peaks)
+        other = {"launch": LAUNCH_NAMES[other_mode], "ms_per_step": r2["ms_per_step"], "value": r2["value"],
+                 "phases_ms": r2["phases_ms"], "roofline": roof2, "step_roofline": step2, "clocks": r2["clocks"]}
+        layers[other_mode].close()
+
+    # ---- end to end through the host-buffer entry points (headline launch mode) -------------------
+    e2e = None if args.no_e2e else run_e2e(wl, layer, args.steps, world)
+
+    # ---- CPU oracle baseline (rank 0, single-GPU run only) ----------------------------------------
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n_exp, rows = calibrate_sample(cfg, train, oracle.threads())
+        secs, fl, desc = oracle_sample(cfg, train, n_exp, rows, inputs=wl.inp)
+        cpu_baseline = {"value": fl / secs / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                        "sample": desc, "seconds": secs}
+    layer.close()
+
+    # ---- the other workloads, both launch modes (forward-only configurations) ---------------------
+    all_configs = None
+    if not args.no_all_configs and not args.small:
+        del wl, layers, layer
+        gc.collect(); torch.cuda.empty_cache()
+        all_configs = [{"workload": cfg.name, "launch_fused_ms": results.get("fused", {}).get("ms_per_step"),
+                        "launch_serial_ms": results.get("serial", {}).get("ms_per_step"),
+                        "fused": {"step_roofline": rooflines(cfg, train, results["fused"], peaks)[1],
+                                  "clocks": results["fused"]["clocks"]} if "fused" in results else None,
+                        "serial": {"step_roofline": rooflines(cfg, train, results["serial"], peaks)[1],
+                                   "clocks": results["serial"]["clocks"]} if "serial" in results else None}]
+        for ci in (1, 2, 3):
+            if ci == args.config:
+                continue
+            c2 = configs.CONFIGS[ci]
+            w2 = Workload(c2, False)
+            entry = {"workload": c2.name}
+            for m in ("fused", "serial"):
+                lay = w2.make_layer(m)
+                r = w2.measure(lay, args.steps, args.warmup, world, local)
+                lay.close()
+                roof_m, step_m = rooflines(c2, False, r, peaks)
+                entry[f"launch_{m}_ms"] = r["ms_per_step"]
+                entry[m] = {"value": r["value"], "step_roofline": step_m, "roofline": roof_m, "clocks": r["clocks"],
+                            "phases_ms": r["phases_ms"]}
+            all_configs.append(entry)
+            del w2
+            gc.collect(); torch.cuda.empty_cache()
+
+    if rank == 0:
+        desc = workload_desc(cfg, train)
+        desc["launch"] = LAUNCH_NAMES[head]
+        desc["launch_choice"] = "the library's default mode" if head == "fused" else "requested"
+        desc["launches_per_step"] = res["launches"] / max(1, args.steps)
+        line = {
+            "metric": METRIC, "value": res["value"], "unit": "TFLOP/s", "n_gpus": world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"],
+            "us_per_layer": res["ms_per_step"] * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": desc, "clocks": res["clocks"], "e2e": e2e, "gpu_launches": res["launches"],
+            "roofline": roofline, "step_roofline": step_roofline, "phases_ms": res["phases_ms"],
+            "other_launch_mode": other, "all_configs": all_configs, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":
