@@ -17,7 +17,7 @@
  * Every function below is pinned by tests/test_oracle_*.py (brute force, library
  * routines, closed-form special cases, finite differences, autograd).
  *
- * Readings where the paper is silent (listed with reasons in the design notes):
+ * Readings where the paper is silent:
  *   - scores = softmax over all E logits; the k experts are the k largest raw
  *     logits, ties to the lower expert id, slots ordered by descending logit;
  *   - optional renormalisation of the k scores to sum 1;
@@ -45,7 +45,7 @@ int moe_oracle_threads(void) {
 #endif
 }
 
-/* ---- routing (Section 2.2: "the router selects a small subset of experts ... top-k") ---- */
+/* ---- routing (Section 2.2, first paragraph: the router keeps the k best-scoring experts of each token) ---- */
 int moe_oracle_route(const float* logits, int T, int E, int k, int renorm,
                      int32_t* topk_ids, double* topk_w) {
   if (k < 1 || k > E) return -1;
@@ -83,7 +83,7 @@ static inline int slot_expert(const int32_t* ids, int k, int S, int E, int t, in
   return j < k ? ids[(size_t)t * k + j] : E + (j - k);
 }
 
-/* ---- dispatch layout (Section 2.2: Dispatch "permutes ... tokens according to the routing decisions") ---- */
+/* ---- dispatch layout (Section 2.2, Dispatch: the expert-ordered row of every routed token copy) ---- */
 int moe_oracle_layout(const int32_t* ids, int T, int E, int k, int S,
                       int32_t* counts, int32_t* offsets, int32_t* row_of, int32_t* src_of) {
   const int Ep = E + S, kp = k + S;
@@ -267,4 +267,20 @@ int moe_oracle_bwd(const double* dout, const double* x, const int32_t* ids, cons
   }
   free(a_all); free(dh_all); free(dxrow);
   return bad ? -1 : 0;
+}
+
+/* ---- SwiGLU + Add operator pair (Section 6, microbenchmarks): the producer/consumer pair the paper
+ * uses to study tile interleaving and scheduling cost.  x[M][2C] holds the gate half (columns 0..C-1)
+ * and the up half (columns C..2C-1); s = silu(gate) * up; z = s + r.  fp64, no intermediate rounding. */
+int moe_oracle_swiglu_add(const double* x, const double* r, int M, int C, double* s_out, double* z) {
+  if (M < 0 || C < 1) return -1;
+#pragma omp parallel for schedule(static)
+  for (long m = 0; m < (long)M; ++m)
+    for (int c = 0; c < C; ++c) {
+      const double g = x[(size_t)m * 2 * C + c], u = x[(size_t)m * 2 * C + C + c];
+      const double s = g / (1.0 + exp(-g)) * u;
+      if (s_out) s_out[(size_t)m * C + c] = s;
+      z[(size_t)m * C + c] = s + r[(size_t)m * C + c];
+    }
+  return 0;
 }

@@ -39,6 +39,7 @@ def _load():
         lib.moe_oracle_fwd.argtypes = [f64p, i32p, f64p, f64p, f64p, ci, ci, ci, ci, ci, ci, f64p, f64p, f64p, f64p]
         lib.moe_oracle_bwd.argtypes = [f64p, f64p, i32p, f64p, f64p, f64p, ci, ci, ci, ci, ci, ci,
                                        f64p, f64p, f64p, f64p]
+        lib.moe_oracle_swiglu_add.argtypes = [f64p, f64p, ci, ci, f64p, f64p]
         _lib = lib
     return _lib
 
@@ -144,3 +145,20 @@ def bwd(dout, x, ids, w, W_gate_up, W_down, S: int = 0):
     if rc:
         raise ValueError(f"moe_oracle_bwd failed ({rc})")
     return dx, dWgu, dWd, dw
+
+
+def swiglu_add(x, r):
+    """SwiGLU + Add operator pair of the scheduling microbenchmarks (Section 6): x [M,2C] = gate | up halves,
+    r [M,C].  -> s = silu(gate) * up [M,C], z = s + r [M,C] (float64)."""
+    x = _np(x, np.float64)
+    r = _np(r, np.float64)
+    M, C2 = x.shape
+    C = C2 // 2
+    assert C2 == 2 * C and r.shape == (M, C)
+    s = np.empty((M, C), np.float64)
+    z = np.empty((M, C), np.float64)
+    dp = ctypes.c_double
+    rc = _load().moe_oracle_swiglu_add(_p(x, dp), _p(r, dp), M, C, _p(s, dp), _p(z, dp))
+    if rc:
+        raise ValueError(f"moe_oracle_swiglu_add failed ({rc})")
+    return s, z
