@@ -44,6 +44,12 @@ int moe_debug_buffer(moe_ctx* ctx, int which, void** ptr, size_t* elems);
  * hang); moe_get_status reports it and the context stays usable once the hook is switched off. */
 int moe_debug_set_unreachable_dependency(moe_ctx* ctx, int32_t on);
 
+/* Profiling aid: with on != 0 the persistent launches of this context are made without the cooperative
+ * launch attribute (some profilers reject cooperative launches of thread-block clusters).  The grid is
+ * sized to what can be resident either way; what is lost is the driver's guarantee of co-residency when
+ * other work shares the GPU -- every device-side wait stays bounded. */
+int moe_debug_set_plain_launch(moe_ctx* ctx, int32_t on);
+
 /* Host-only check of the static tile schedule of the single persistent launch (Section 4.3: tasks
  * in statically ordered queues, dependent/trigger event counters with static thresholds).  For the
  * given per-expert row counts[Ep] and layer shape it builds the layout tables, the matrix queue of

@@ -21,7 +21,7 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
            "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
-           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace"]
+           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace", "moe_debug_set_plain_launch"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -73,6 +73,7 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_simulate_schedule.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp]
     lib.moe_debug_trace.argtypes = [vp, vp, sz, ctypes.POINTER(sz)]
     lib.moe_debug_set_unreachable_dependency.argtypes = [vp, i32]
+    lib.moe_debug_set_plain_launch.argtypes = [vp, i32]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -305,6 +306,10 @@ def moe_debug_trace(ctx, max_records=1 << 18):
 def moe_debug_set_unreachable_dependency(ctx, on: bool):
     _check(load_library().moe_debug_set_unreachable_dependency(ctx, 1 if on else 0),
            "moe_debug_set_unreachable_dependency")
+
+
+def moe_debug_set_plain_launch(ctx, on: bool):
+    _check(load_library().moe_debug_set_plain_launch(ctx, 1 if on else 0), "moe_debug_set_plain_launch")
 
 
 class _DevView:

@@ -1,6 +1,7 @@
 // C ABI of libmoe_b200: context, workspace carving, tensor-map encoding and the launch
 // sequences of the forward and backward layer.  Argument marshalling and planning only; every
-// step of the layer runs in the kernels of route_layout.cu, permute.cu and gemm_tc.cu.
+// step of the layer runs in the kernels of route_layout.cu, permute.cu, gemm_tc3.cu, gemm_wgrad.cu,
+// gemm_tc2.cu and fused.cu.
 #include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
@@ -206,6 +207,7 @@ struct moe_ctx {
   const void *saved_x = nullptr, *saved_ids = nullptr, *saved_w = nullptr;  // that forward's inputs
   uint64_t budget_ns = 2000ull * 1000 * 1000;
   int dep_extra = 0;  // test hook: makes the activation dependencies of the persistent launch unreachable
+  bool plain_launch = false;  // diagnostic: persistent launches without the cooperative attribute
   cudaStream_t last_stream = nullptr;
   // host-buffer entry points: a copy-in stream (the next call's large input arrives while the previous
   // call still computes) and a copy-out stream (the result leaves in token chunks behind the combine)
@@ -235,7 +237,7 @@ struct moe_ctx {
   // store maps: workspace tensors (fixed) and the caller's weight gradients (re-encoded on change)
   CUtensorMap ts_A, ts_H, ts_Y, ts_dH;
   // token-column tiles: token operands with 64-row and 16-row boxes, un-swizzled store maps
-  CUtensorMap tk_Xp[3], tk_A[3], tk_dOutp[3], tk_dH[3];
+  CUtensorMap tk_Xp[8], tk_A[8], tk_dOutp[8], tk_dH[8];
   CUtensorMap tp_A, tp_H, tp_Y, tp_dH;
   const void* dw1_ptr = nullptr;
   const void* dw2_ptr = nullptr;
@@ -577,7 +579,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     fa.combine_out = out;
     Phase ph(c, MOE_PHASE_FUSED_FWD, st);
     MOE_CUDA(cudaMemsetAsync(fa.ctr, 0, sizeof(int) * (size_t)p.ctr_count, st));
-    MOE_CUDA(launch_fused(false, fa, c->num_sms, st, &c->launches));
+    MOE_CUDA(launch_fused(false, fa, c->num_sms, !c->plain_launch, st, &c->launches));
     if (out_host) MOE_CUDA(cudaMemcpyAsync(out_host, out, 2 * (size_t)T * c->shape.d, cudaMemcpyDeviceToHost, st));
   }
   if (c->train()) {
@@ -661,7 +663,7 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     MOE_CUDA(cudaMemsetAsync(fa.ctr, 0, sizeof(int) * (size_t)p.ctr_count, st));
     // slots dropped for an invalid expert id have no row: their gradient is zero
     if (d_w) MOE_CUDA(cudaMemsetAsync(d_w, 0, sizeof(float) * (size_t)T * s.k, st));
-    MOE_CUDA(launch_fused(true, fa, c->num_sms, st, &c->launches));
+    MOE_CUDA(launch_fused(true, fa, c->num_sms, !c->plain_launch, st, &c->launches));
     if (dx_host) MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
   }
   return MOE_OK;
@@ -726,8 +728,8 @@ int moe_create(moe_ctx** out, const moe_shape* shape, void* workspace, size_t wo
   if (!rc && train) rc = encode_2d(&c->tm_A_mn, c->ws + p.A, cap, s.F, 64, 64);
   if (!rc && train) rc = encode_2d(&c->tm_dH_mn, c->ws + p.dH, cap, 2 * s.F, 64, 64);
   if (!rc && train) rc = encode_2d(&c->tm_Xp_mn, c->ws + p.Xp, cap, s.d, 64, 64);
-  for (int i = 0; i < 3 && !rc; ++i) {
-    const uint32_t br = 64u >> i;
+  for (int i = 0; i < 8 && !rc; ++i) {
+    const uint32_t br = 16u * (i + 1);
     rc = encode_2d(&c->tk_Xp[i], c->ws + p.Xp, cap, s.d, br, 64);
     if (!rc) rc = encode_2d(&c->tk_A[i], c->ws + p.A, cap, s.F, br, 64);
     if (!rc && train) rc = encode_2d(&c->tk_dOutp[i], c->ws + p.dOutp, cap, s.d, br, 64);
@@ -961,6 +963,12 @@ int moe_get_phase_ms(moe_ctx* c, float* ms) {
 int moe_debug_set_unreachable_dependency(moe_ctx* c, int32_t on) {
   if (!c) return MOE_ERR_INVALID_ARG;
   c->dep_extra = on ? 1 : 0;
+  return MOE_OK;
+}
+
+int moe_debug_set_plain_launch(moe_ctx* c, int32_t on) {
+  if (!c) return MOE_ERR_INVALID_ARG;
+  c->plain_launch = on != 0;
   return MOE_OK;
 }
 

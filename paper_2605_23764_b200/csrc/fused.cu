@@ -10,11 +10,11 @@
 //   warps 8-14  vector workers: tickets of the vector queue (permute-gather, routing-weight
 //               gradient, combine); the matrix-role warps join them once the matrix queue is empty.
 // The matrix roles are the ones of the one-launch-per-operator kernels (gemm_roles.cuh); here they
-// run the operators of the pass as consecutive phases of a statically ordered queue per CTA pair
-// (schedule.h) with the pipeline state carried across, so that no SM drains at an operator
-// boundary, the permutes overlap the GEMMs, and what orders tiles are event counters with static
-// thresholds -- the paper's unified runtime (Sections 4.3, 4.4) restated for one SM, where "matrix
-// core" and "vector core" are warp roles of the same CTA.
+// take the items of all operators of the pass from one ticket queue (schedule.h) with the pipeline
+// state carried from item to item, so that no SM waits at an operator boundary for the others, the
+// permutes run beside the GEMMs, and what orders tiles are event counters with static thresholds --
+// the paper's unified runtime (Sections 4.3, 4.4) restated for one SM, where "matrix core" and
+// "vector core" are warp roles of the same CTA.
 #include "gemm_roles.cuh"
 #include "launch_pairs.cuh"
 #include "schedule.h"
@@ -517,11 +517,12 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_chain_kernel(const __g
   }
 }
 
-cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, cudaStream_t s, int* launches) {
+cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, bool cooperative, cudaStream_t s, int* launches) {
   ++*launches;
   static PairLaunchState st_fwd, st_bwd;
-  if (bwd) return launch_on_pairs(st_bwd, fused_chain_kernel<true>, fa, FUSED_THREADS, FUSED_SMEM_BYTES, num_sms, true, s);
-  return launch_on_pairs(st_fwd, fused_chain_kernel<false>, fa, FUSED_THREADS, FUSED_SMEM_BYTES, num_sms, true, s);
+  if (bwd)
+    return launch_on_pairs(st_bwd, fused_chain_kernel<true>, fa, FUSED_THREADS, FUSED_SMEM_BYTES, num_sms, cooperative, s);
+  return launch_on_pairs(st_fwd, fused_chain_kernel<false>, fa, FUSED_THREADS, FUSED_SMEM_BYTES, num_sms, cooperative, s);
 }
 
 }  // namespace moe

@@ -1,6 +1,6 @@
 // Tile-level pieces of the CTA-pair (tcgen05 cta_group::2) grouped GEMMs shared by the
-// one-launch-per-operator kernel (gemm_tc2.cu) and the persistent launch (fused.cu): each CTA of a
-// pair loads its own 128 rows of A and its half of the B tile; the even CTA issues 256 x 256 MMAs.
+// token-row kernel (gemm_tc2.cu) and the weight gradients (gemm_roles.cuh): each CTA of a pair loads its
+// own 128 rows of A and its half of the B tile; the even CTA issues 256 x 256 MMAs.
 #pragma once
 
 #include "gemm_tile.cuh"
@@ -9,34 +9,6 @@ namespace moe {
 
 constexpr int HALF_B_BYTES = B_STAGE_BYTES / 2;                 // 16 KB: this CTA's half of the B tile
 constexpr int STAGE2_BYTES = A_STAGE_BYTES + HALF_B_BYTES;      // 32 KB per stage and CTA
-
-// This CTA's loads of one k-block: its 128 rows of A and its half of B.  Completion bytes go to the
-// even CTA's barrier.
-template <int MODE>
-__device__ __forceinline__ void load_stage_pair(const GemmArgs& a, const Tile& tl, int kb, int rank, uint8_t* sA,
-                                                uint8_t* sB, uint64_t* bar) {
-  const int k0 = kb * BK;
-  if (MODE == GEMM_WGRAD) {
-#pragma unroll
-    for (int j = 0; j < 2; ++j) tma_load_2d_pair(sA + j * MN_BOX_BYTES, &a.tmA, tl.m0 + j * 64, tl.row0 + k0, bar);
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-      tma_load_2d_pair(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + (2 * rank + j) * 64, tl.row0 + k0, bar);
-    return;
-  }
-  tma_load_2d_pair(sA, &a.tmA, k0, tl.row0, bar);
-  const int brow = tl.e * a.b_rows_per_expert;
-  if (MODE == GEMM_GATE_UP) {
-    // accumulator columns 0..127 = gate (even CTA's half of B), 128..255 = up (odd CTA's half)
-    tma_load_2d_pair(sB, &a.tmB, k0, brow + rank * a.F + tl.n0, bar);
-  } else if (MODE == GEMM_DOWN) {
-    tma_load_2d_pair(sB, &a.tmB, k0, brow + tl.n0 + rank * (BN / 2), bar);
-  } else {
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-      tma_load_2d_pair(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + (2 * rank + j) * 64, brow + k0, bar);
-  }
-}
 
 // 16-row MMA steps needed in k-block kb of a reduction over `rows` rows
 __device__ __forceinline__ int k16_steps_of(int rows, int kb) {
@@ -71,12 +43,6 @@ __device__ __forceinline__ void load_stage_pair_lanes(const GemmArgs& a, const T
   const int k0 = kb * BK;
   if (lane == 0 && rank == 0) mbar_expect_tx(bar, 2 * STAGE2_BYTES);
   __syncwarp();
-  if (MODE == GEMM_WGRAD) {
-    if (lane < 2) tma_load_2d_pair(sA + lane * MN_BOX_BYTES, &a.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
-    else if (lane < 4)
-      tma_load_2d_pair(sB + (lane - 2) * MN_BOX_BYTES, &a.tmB, tl.n0 + (2 * rank + lane - 2) * 64, tl.row0 + k0, bar);
-    return;
-  }
   const int brow = tl.e * a.b_rows_per_expert;
   if (lane == 0) {
     tma_load_2d_pair(sA, &a.tmA, k0, tl.row0, bar);
@@ -87,23 +53,6 @@ __device__ __forceinline__ void load_stage_pair_lanes(const GemmArgs& a, const T
   } else {
     if (lane < 3)
       tma_load_2d_pair(sB + (lane - 1) * MN_BOX_BYTES, &a.tmB, tl.n0 + (2 * rank + lane - 1) * 64, brow + k0, bar);
-  }
-}
-
-// A weight-gradient stage split over two loader warps (the first: this CTA's A boxes and the byte
-// count; the second: its B boxes): issuing a TMA box costs the issuing warp on the order of a hundred
-// cycles, and four boxes in one warp take about as long as the k-block's MMAs.  Both warps take part
-// in every stage, so neither can fall two phases behind a stage's barrier (where a parity wait is no
-// longer meaningful).
-__device__ __forceinline__ void load_wgrad_part(const GemmArgs& g, const Tile& tl, int kb, int rank, uint8_t* sA,
-                                                uint8_t* sB, uint64_t* bar, int lane, bool second_warp) {
-  const int k0 = kb * BK;
-  if (!second_warp) {
-    if (lane == 0 && rank == 0) mbar_expect_tx(bar, 2 * STAGE2_BYTES);
-    __syncwarp();
-    if (lane < 2) tma_load_2d_pair(sA + lane * MN_BOX_BYTES, &g.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
-  } else {
-    if (lane < 2) tma_load_2d_pair(sB + lane * MN_BOX_BYTES, &g.tmB, tl.n0 + (2 * rank + lane) * 64, tl.row0 + k0, bar);
   }
 }
 

@@ -173,8 +173,8 @@ __device__ __forceinline__ bool swap_load_item(const GemmArgs& a, uint8_t* smem,
       load_weights_swap<MODE>(a, wk.a, kb, rank, sW + ls.s * W_STAGE_BYTES, &bars->full[ls.s], lane, wk.a.ntok + wk.b.ntok);
     } else {
       load_tokens_swap(a, wk.a, kb, rank, sT + ls.s * TOKB, &bars->full[ls.s], lane);
-      if (wk.merged)   // lanes 4..7: the second token tile, behind the first in the stage
-        load_tokens_swap(a, wk.b, kb, rank, sT + ls.s * TOKB + (wk.a.ntok >> 1) * (BK * 2), &bars->full[ls.s], lane - 4);
+      if (wk.merged)   // lane 1: the second token tile, behind the first in the stage
+        load_tokens_swap(a, wk.b, kb, rank, sT + ls.s * TOKB + (wk.a.ntok >> 1) * (BK * 2), &bars->full[ls.s], lane - 1);
     }
     if (++ls.s == PIPE_STAGES) ls.s = 0;
   }

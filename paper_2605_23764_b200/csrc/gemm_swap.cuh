@@ -96,17 +96,12 @@ __device__ __forceinline__ uint32_t swap_stage_tx_bytes(int ntok) {
 
 // This CTA's loads of one k-block are split over two producer warps, one box per lane (issuing a TMA
 // box costs its thread on the order of a hundred cycles, and a k-block of a short tile only lasts a
-// few hundred).  Tokens: rows [row0 + rank * ntok/2, + ntok/2) as one box per set bit of ntok/2
-// (128, 64, 32, 16 rows).  The even CTA's weight producer arms the barrier for both CTAs' bytes.
+// few hundred).  Tokens: rows [row0 + rank * ntok/2, + ntok/2) as ONE box (a tensor map per box height).  The even CTA's weight producer arms the barrier for both CTAs' bytes.
 __device__ __forceinline__ void load_tokens_swap(const GemmArgs& a, const SwapTile& st, int kb, int rank, uint8_t* sT,
                                                  uint64_t* bar, int lane) {
-  if (lane < 0 || lane >= 4) return;
-  const int half = st.ntok >> 1;
-  const int size = 128 >> lane;                 // lane 0: 128-row box ... lane 3: 16-row box
-  if (!(half & size)) return;
-  const int before = half & ~(2 * size - 1);    // rows covered by the larger boxes
-  const CUtensorMap* m = lane == 0 ? &a.tmA : &a.tmTok[lane - 1];
-  tma_load_2d_pair(sT + before * (BK * 2), m, kb * BK, st.row0 + rank * half + before, bar);
+  if (lane != 0) return;
+  const int half = st.ntok >> 1;   // a multiple of 16, at most 128: one box of exactly that many rows
+  tma_load_2d_pair(sT, &a.tmTok[(half >> 4) - 1], kb * BK, st.row0 + rank * half, bar);
 }
 template <int MODE>
 __device__ __forceinline__ void load_weights_swap(const GemmArgs& a, const SwapTile& st, int kb, int rank, uint8_t* sW,

@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(GEMM3_THREADS, 1) grouped_gemm_swap_kernel(con
     mbar_fence_init();
     fence_proxy_async();
     tma_prefetch_desc(&a.tmA);
-    for (int i = 0; i < 3; ++i) tma_prefetch_desc(&a.tmTok[i]);
+    for (int i = 0; i < 8; ++i) tma_prefetch_desc(&a.tmTok[i]);
     tma_prefetch_desc(&a.tmB);
     tma_prefetch_desc(&a.tmOut0);
   }

@@ -1,7 +1,6 @@
-// Tile-level building blocks of the grouped GEMMs on the sm_100a tensor cores, shared by the
-// one-launch-per-operator kernel (gemm_tc.cu) and the single persistent dependency-driven kernel
-// (fused.cu): tile geometry, TMA loads of one k-block, tcgen05.mma issue of one k-block, and the
-// fused epilogues (TMEM -> registers -> element-wise math -> swizzled shared staging -> TMA store).
+// Tile-level building blocks of the grouped GEMMs on the sm_100a tensor cores: tile geometry and the
+// fused epilogues of the token-row tiles (TMEM -> registers -> element-wise math -> swizzled shared
+// staging -> TMA store).
 //
 // Tiles never straddle experts: rows live in a padded row space where every expert segment starts
 // on a multiple of 128 (the paper's rule that vector tiles align with GMM row partitions and that
@@ -15,10 +14,6 @@ namespace moe {
 
 constexpr int BN = 256;                       // accumulator columns per tile
 constexpr int BK = 64;                        // reduction elements per stage (one 128-byte swizzle row)
-#ifndef MOE_STAGES
-#define MOE_STAGES 4
-#endif
-constexpr int STAGES = MOE_STAGES;
 constexpr int A_STAGE_BYTES = BLOCK_M * BK * 2;  // 16 KB
 constexpr int B_STAGE_BYTES = BN * BK * 2;       // 32 KB
 constexpr int MN_BOX_BYTES = 64 * BK * 2;        // one [64 k][64 mn] box of an MN-major operand
@@ -26,20 +21,6 @@ constexpr int GEMM_THREADS = 192;
 constexpr int TMEM_COLS = 512;
 constexpr int OUT_BOX_BYTES = 32 * 64 * 2;       // epilogue staging box: 32 rows x 64 bf16 columns
 constexpr int OUT_STAGE_BYTES = 2 * OUT_BOX_BYTES;  // per epilogue warp: two boxes
-
-struct __align__(8) GemmBarriers {
-  uint64_t full[STAGES];
-  uint64_t empty[STAGES];
-  uint64_t tmem_full[2];
-  uint64_t tmem_empty[2];
-  uint64_t drain;
-  uint32_t tmem_base;
-  uint32_t pad;
-};
-
-constexpr size_t GEMM_SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) +
-                                   4 * OUT_STAGE_BYTES + sizeof(GemmBarriers);
-static_assert(GEMM_SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
 struct Tile {
   int e;      // expert
@@ -49,100 +30,6 @@ struct Tile {
   int nkb;    // k-blocks of the main loop (may be 0 for an expert without rows in WGRAD)
   int nb;     // column-tile index (ACT_GRAD partials)
 };
-
-template <int MODE>
-__device__ __forceinline__ int total_tiles(const GemmArgs& a) {
-  if (MODE == GEMM_WGRAD) return a.Ep * a.n_tiles_m * a.n_tiles_n;
-  return a.meta[0] * a.n_tiles_n;
-}
-
-// Tile order.  Row-space modes: expert-major; inside an expert the column tile is the slow index
-// and the M-block the fast one, so CTAs running at the same time share one slab of weights (read
-// from HBM once, then from L2) while the expert's rows stay L2-resident.
-template <int MODE>
-__device__ __forceinline__ Tile decode_tile(const GemmArgs& a, int t) {
-  Tile tl;
-  if (MODE == GEMM_WGRAD) {
-    const int per_e = a.n_tiles_m * a.n_tiles_n;
-    tl.e = t / per_e;
-    const int r = t - tl.e * per_e;
-    const int mb = r / a.n_tiles_n;
-    tl.nb = r - mb * a.n_tiles_n;
-    tl.m0 = mb * BLOCK_M;
-    tl.n0 = tl.nb * BN;
-    tl.row0 = a.mb_start[tl.e] * BLOCK_M;
-    tl.nkb = (a.counts[tl.e] + BK - 1) / BK;
-  } else {
-    const int e = a.mblk_expert[t / a.n_tiles_n];
-    const int ms = a.mb_start[e];
-    const int mcount = a.mb_start[e + 1] - ms;
-    const int local = t - ms * a.n_tiles_n;
-    tl.nb = local / mcount;
-    const int mbl = local - tl.nb * mcount;
-    tl.e = e;
-    tl.row0 = (ms + mbl) * BLOCK_M;
-    tl.n0 = tl.nb * (MODE == GEMM_GATE_UP ? BN / 2 : BN);
-    tl.m0 = 0;
-    tl.nkb = (a.K + BK - 1) / BK;
-  }
-  return tl;
-}
-
-// ---------------------------------------------------------------- producer: TMA loads of one k-block
-template <int MODE>
-__device__ __forceinline__ void load_stage(const GemmArgs& a, const Tile& tl, int kb, uint8_t* sA, uint8_t* sB,
-                                           uint64_t* bar) {
-  const int k0 = kb * BK;
-  if (MODE == GEMM_WGRAD) {
-    // both operands MN-major: boxes of [64 rows of the expert][64 columns]
-    mbar_expect_tx(bar, 2 * MN_BOX_BYTES + 4 * MN_BOX_BYTES);
-#pragma unroll
-    for (int j = 0; j < 2; ++j) tma_load_2d(sA + j * MN_BOX_BYTES, &a.tmA, tl.m0 + j * 64, tl.row0 + k0, bar);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + j * 64, tl.row0 + k0, bar);
-    return;
-  }
-  mbar_expect_tx(bar, A_STAGE_BYTES + B_STAGE_BYTES);
-  tma_load_2d(sA, &a.tmA, k0, tl.row0, bar);  // A: [128 rows][64 k], K-major
-  const int brow = tl.e * a.b_rows_per_expert;
-  if (MODE == GEMM_GATE_UP) {
-    tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);                          // gate rows -> columns 0..127
-    tma_load_2d(sB + B_STAGE_BYTES / 2, &a.tmB, k0, brow + a.F + tl.n0, bar);  // up rows   -> columns 128..255
-  } else if (MODE == GEMM_DOWN) {
-    tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);  // [256 rows of W_down][64 k], K-major
-  } else {
-    // ACT_GRAD / GATE_GRAD: B = forward weight read along its rows (reduction) -> MN-major boxes
-#pragma unroll
-    for (int j = 0; j < 4; ++j) tma_load_2d(sB + j * MN_BOX_BYTES, &a.tmB, tl.n0 + j * 64, brow + k0, bar);
-  }
-}
-
-// The same loads issued by a whole warp, one box per lane (a single thread needs several hundred
-// cycles to issue the five or six boxes of a k-block).  All lanes call it; lane 0 arms the barrier.
-template <int MODE>
-__device__ __forceinline__ void load_stage_lanes(const GemmArgs& a, const Tile& tl, int kb, uint8_t* sA, uint8_t* sB,
-                                                 uint64_t* bar, int lane) {
-  const int k0 = kb * BK;
-  if (lane == 0)
-    mbar_expect_tx(bar, MODE == GEMM_WGRAD ? 6 * MN_BOX_BYTES : A_STAGE_BYTES + B_STAGE_BYTES);
-  __syncwarp();
-  if (MODE == GEMM_WGRAD) {
-    if (lane < 2) tma_load_2d(sA + lane * MN_BOX_BYTES, &a.tmA, tl.m0 + lane * 64, tl.row0 + k0, bar);
-    else if (lane < 6) tma_load_2d(sB + (lane - 2) * MN_BOX_BYTES, &a.tmB, tl.n0 + (lane - 2) * 64, tl.row0 + k0, bar);
-    return;
-  }
-  const int brow = tl.e * a.b_rows_per_expert;
-  if (lane == 0) {
-    tma_load_2d(sA, &a.tmA, k0, tl.row0, bar);
-  } else if (MODE == GEMM_GATE_UP) {
-    if (lane == 1) tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);
-    else if (lane == 2) tma_load_2d(sB + B_STAGE_BYTES / 2, &a.tmB, k0, brow + a.F + tl.n0, bar);
-  } else if (MODE == GEMM_DOWN) {
-    if (lane == 1) tma_load_2d(sB, &a.tmB, k0, brow + tl.n0, bar);
-  } else {
-    if (lane < 5) tma_load_2d(sB + (lane - 1) * MN_BOX_BYTES, &a.tmB, tl.n0 + (lane - 1) * 64, brow + k0, bar);
-  }
-}
 
 // ---------------------------------------------------------------- epilogues
 // Each epilogue warp owns 32 rows of the tile (its TMEM lane quadrant) and a private staging area of
@@ -282,60 +169,30 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs& a, const Tile& tl,
     }
     if (a.dw_partial) a.dw_partial[p * a.n_tiles_n + tl.nb] = part;
   } else {
-    // plain bf16 store of the accumulator: DOWN (Y), GATE_GRAD (dXp), WGRAD (dW)
-    const int y0 = (MODE == GEMM_WGRAD ? tl.m0 : tl.row0) + quad * 32;
+    // plain bf16 store of the accumulator: DOWN (Y), GATE_GRAD (dXp)
+    const int y0 = tl.row0 + quad * 32;
 #pragma unroll 1
     for (int c0 = 0; c0 < BN; c0 += 128) {
       if (tl.n0 + c0 >= a.N) break;
-      if (MODE == GEMM_WGRAD && y0 >= a.M) break;
       box0 = staging_acquire(sg, lane); box1 = box0 + OUT_BOX_BYTES;
 #pragma unroll
       for (int c = 0; c < 128; c += 64) {
-        // 64 columns per TMEM round trip (one wait per box): fewer round trips keep this epilogue
-        // shorter than the four-or-five-k-block main loop of a weight-gradient tile
+        // 64 columns per TMEM round trip (one wait per box)
         float v[64];
-        if (MODE == GEMM_WGRAD && tl.nkb == 0) {
 #pragma unroll
-          for (int i = 0; i < 64; ++i) v[i] = 0.f;
-        } else {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) tmem_ld16(trow + c0 + c + 16 * q, v + 16 * q);
-          tmem_ld_wait();
-        }
+        for (int q = 0; q < 4; ++q) tmem_ld16(trow + c0 + c + 16 * q, v + 16 * q);
+        tmem_ld_wait();
         uint8_t* box = (c < 64) ? box0 : box1;
 #pragma unroll
         for (int h = 0; h < 64; h += 8) stage8(box, lane, h >> 3, v + h);
       }
       staging_release();
       if (lane == 0) {
-        if (MODE == GEMM_WGRAD) {
-          tma_store_3d(&a.tmOut0, tl.n0 + c0, y0, tl.e, box0);
-          if (tl.n0 + c0 + 64 < a.N) tma_store_3d(&a.tmOut0, tl.n0 + c0 + 64, y0, tl.e, box1);
-        } else {
-          tma_store_2d(&a.tmOut0, tl.n0 + c0, y0, box0);
-          if (tl.n0 + c0 + 64 < a.N) tma_store_2d(&a.tmOut0, tl.n0 + c0 + 64, y0, box1);
-        }
+        tma_store_2d(&a.tmOut0, tl.n0 + c0, y0, box0);
+        if (tl.n0 + c0 + 64 < a.N) tma_store_2d(&a.tmOut0, tl.n0 + c0 + 64, y0, box1);
         tma_store_commit();
       }
     }
-  }
-}
-
-
-// tcgen05.mma issue of one 64-deep k-block from shared stage (a_addr, b_addr) into accumulator d_tmem.
-template <int MODE>
-__device__ __forceinline__ void mma_kblock(uint32_t d_tmem, uint32_t a_addr, uint32_t b_addr, bool first_kblock) {
-  constexpr bool A_MN = (MODE == GEMM_WGRAD);
-  constexpr bool B_MN = (MODE == GEMM_ACT_GRAD || MODE == GEMM_GATE_GRAD || MODE == GEMM_WGRAD);
-  constexpr uint32_t idesc = make_idesc_bf16(BLOCK_M, BN, A_MN ? 1 : 0, B_MN ? 1 : 0);
-#pragma unroll
-  for (int k16 = 0; k16 < BK / 16; ++k16) {
-    // K-major: 16 k-elements = 32 bytes inside the swizzled row; MN-major: 16 k-rows of 128 bytes
-    const uint64_t da = A_MN ? make_smem_desc(a_addr + k16 * 2048, MN_BOX_BYTES, 1024)
-                             : make_smem_desc(a_addr + k16 * 32, 16, 1024);
-    const uint64_t db = B_MN ? make_smem_desc(b_addr + k16 * 2048, MN_BOX_BYTES, 1024)
-                             : make_smem_desc(b_addr + k16 * 32, 16, 1024);
-    tc_mma_bf16(d_tmem, da, db, idesc, !(first_kblock && k16 == 0));
   }
 }
 

@@ -83,7 +83,8 @@ struct GemmArgs {
   CUtensorMap tmB;     // B operand
   CUtensorMap tmOut0;  // store map of out0: [rows][N] (2-D), [rows][2][F] (dH), or [Ep][M][N] (WGRAD)
   CUtensorMap tmOut1;  // GATE_UP: store map of H as [rows][2][F]
-  CUtensorMap tmTok[3]; // token-column tiles (gemm_tc3.cu): the token operand with 64-, 32- and 16-row boxes (tmA: 128)
+  CUtensorMap tmTok[8]; // token-column tiles: the token operand with boxes of 16, 32, .., 128 rows (one TMA instruction
+                        // per k-block whatever the tile's token count)
   // tile table
   const int* mblk_expert;
   const int* mb_start;
@@ -151,6 +152,8 @@ struct FusedArgs {
   uint64_t budget_ns;
 };
 
-cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, cudaStream_t s, int* launches);
+// cooperative = false drops the co-residency guarantee of the launch (profilers that reject cooperative cluster
+// launches); the grid is sized to the resident capacity either way and every wait is bounded
+cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, bool cooperative, cudaStream_t s, int* launches);
 
 }  // namespace moe

@@ -1,17 +1,18 @@
-// The static tile schedule of the single persistent launch: per CTA pair a statically ordered
-// matrix queue (the counterpart of the paper's per-core task queue, Section 4.3), one ticket-ordered
-// vector queue shared by all vector workers, and the dependent / trigger event counters of every
-// tile with their static thresholds.  Plain host/device code without CUDA calls, so the same
-// functions drive the kernels and the CPU-side simulation that checks the schedule for coverage and
-// deadlock freedom.
+// The tile schedule of the single persistent launch: one ticket-ordered matrix queue (the counterpart
+// of the paper's matrix-core task queue, Section 4.3), two ticket-ordered vector queues, and the
+// dependent / trigger event counters of every tile with their static thresholds.  Plain host/device
+// code without CUDA calls, so the same functions drive the kernels and the CPU-side simulation that
+// checks the schedule for coverage and deadlock freedom.
 //
 // Matrix queue.  The operators of a pass are phases in dependency order -- forward: gate+up, down;
 // backward: act_grad, w2_grad, gate_grad, w1_grad -- and phase p's work items are numbered
-// expert-major (column tile slow, token tile fast: items in flight together share one slab of
-// weights through L2).  Pair q of Q executes the items q, q+Q, q+2Q, .. of phase 0, then those of
-// phase 1, and so on: exactly the order in which the one-launch-per-operator kernels walk the same
-// items, without the kernel boundary in between.  A pair that reaches phase p+1 early starts on it
-// while other pairs still finish phase p; what orders tiles are only the event counters.
+// expert-major (column tile slow, token tile fast).  The queue is the concatenation of the phases'
+// item lists, fixed before the launch; CTA pairs take its tickets in order.  The order of the queue
+// is static (the paper's statically ordered task lists); which pair runs which item is decided by
+// arrival, which keeps the items in flight a contiguous window of the queue: items that share an
+// operand (the token tiles of one expert and column tile share its weight slab, the strips of one
+// expert share its rows) start within microseconds of each other and meet in L2 however the pairs'
+// speeds differ.  A pair that reaches phase p+1 early starts on it while others still finish phase p.
 //
 // Events (Section 4.3).  Per M-block (128 rows of the padded expert-ordered row space) three
 // counters with static thresholds:
@@ -20,12 +21,13 @@
 //   done       += 1 per epilogue warp and column tile of the last row-space phase (down / gate_grad)
 // A phase-0 item depends on `gathered` of its M-blocks, a down / gate_grad item and a w1_grad
 // strip on `activated`, a w2_grad strip on `gathered`; a combine task depends on `done` of the
-// M-blocks that hold its tokens' rows (many-to-many: up to k+S counters per token), the
+// M-blocks that hold its token's rows (many-to-many: up to k+S counters per token), the
 // routing-weight-gradient task of an M-block on its `activated`.
 //
-// Deadlock freedom: every item's producers are items of an earlier phase (or vector tasks with
-// smaller tickets), each pair runs its phases in order and all pairs are resident (cooperative
-// launch), so the pair that owns the lowest unfinished producer is never blocked on a later phase.
+// Deadlock freedom: every item's producers have smaller tickets (an earlier phase) or are vector
+// tasks that never wait for matrix items of the same or a later phase; tickets are taken in order
+// by pairs that are all resident (cooperative launch), so the holder of the smallest unfinished
+// ticket always finds its dependent events met in finite time.
 #pragma once
 
 #include <stdint.h>
