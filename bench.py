@@ -11,7 +11,9 @@ prints ONE JSON line.  Throughput counts 6*R*d*F FLOP per forward and 12*R*d*F p
 
 The headline `value` is the library's default launch mode: one persistent dependency-driven
 launch per pass.  The one-launch-per-operator mode is timed in the same run and reported as
-`other_launch_mode`; `all_configs` holds both modes for the forward-only workloads.
+`other_launch_mode`; `all_configs` holds both modes for the forward-only workloads;
+`scheduling_study` holds the SwiGLU+Add scheduling microbenchmark (Section 6): serial, statically
+interleaved and dynamically dispatched, with the dispatch time per task.
 With N > 1 every rank runs an independent replica on its own GPU (the layer is not sharded;
 there is no data-path collective); `python bench.py --gpus N` without a launcher starts the N
 ranks itself.
@@ -442,6 +444,42 @@ def run_e2e(wl, layer, steps, world):
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
 
+def scheduling_study(peaks, iters=30):
+    """SwiGLU(M x 4096) + Add(M x 2048) under the three schedules (Section 6.1, 6.2): median microseconds per
+    pass with L2 flushed before each, and the workers' dispatch time per task."""
+    from paper_2605_23764_b200 import binding as B
+    dev, C, tile_rows = torch.device("cuda"), 2048, 8
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    rows = []
+    for M in (2048, 8192, 32768):
+        g = torch.Generator(device="cuda").manual_seed(1000 + M)
+        x = torch.randn(M, 2 * C, device=dev, generator=g).to(torch.bfloat16)
+        r = torch.randn(M, C, device=dev, generator=g).to(torch.bfloat16)
+        s, z = torch.empty_like(r), torch.empty_like(r)
+        ws = torch.empty(B.moe_sched_study_workspace_bytes(M, tile_rows), dtype=torch.uint8, device=dev)
+        algo_bytes = M * C * 2 * (2 + 1 + 1 + 1 + 1)   # x (2C), s written and read, r, z: per row and column 2 bytes each
+        row = {"M": M, "tile_rows": tile_rows, "tasks": 2 * (-(-M // tile_rows))}
+        for mode, name in ((0, "serial"), (1, "static"), (2, "dynamic")):
+            ts = []
+            for it in range(iters + 3):
+                flush.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); B.moe_sched_study(mode, x, r, s, z, M, C, tile_rows, ws); e1.record()
+                torch.cuda.synchronize()
+                if it >= 3:
+                    ts.append(e0.elapsed_time(e1) * 1e3)
+            status, ns, n = B.moe_sched_study_stats(ws)
+            if status != (0, 0):
+                raise SystemExit(f"scheduling study: device status {status}")
+            us = sorted(ts)[len(ts) // 2]
+            row[name] = {"us": us, "GBps": algo_bytes / us / 1e3, "frac_of_hbm_peak": algo_bytes / us / 1e3 / peaks["hbm_gbs"],
+                         "dispatch_ns_per_task": (ns / n) if n else None}
+        rows.append(row)
+    return {"operators": "SwiGLU(M x 4096) -> s(M x 2048, bf16, in global memory) -> Add(M x 2048)",
+            "timing": "CUDA events around each call (workspace clear + kernels), L2 flushed before each; median of %d" % iters,
+            "rows": rows}
+
+
 def respawn_under_launcher(n):
     """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU) and pass their output on."""
     import socket
@@ -469,6 +507,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-compare", action="store_true", help="skip timing the other launch mode")
     ap.add_argument("--no-all-configs", action="store_true", help="skip the other workloads")
+    ap.add_argument("--no-study", action="store_true", help="skip the SwiGLU+Add scheduling microbenchmark")
     ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -555,6 +594,10 @@ def main():
             del w2
             gc.collect(); torch.cuda.empty_cache()
 
+    study = None
+    if rank == 0 and world == 1 and not args.no_study and not args.small:
+        study = scheduling_study(peaks)
+
     if rank == 0:
         desc = workload_desc(cfg, train)
         desc["launch"] = LAUNCH_NAMES[head]
@@ -568,6 +611,7 @@ def main():
             "config": desc, "clocks": res["clocks"], "e2e": e2e, "gpu_launches": res["launches"],
             "roofline": roofline, "step_roofline": step_roofline, "phases_ms": res["phases_ms"],
             "other_launch_mode": other, "all_configs": all_configs, "cpu_baseline": cpu_baseline,
+            "scheduling_study": study,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -210,6 +210,37 @@ int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E, int32_t k,
                        int32_t* counts, int32_t* offsets, int32_t* row_of, int32_t* src_of,
                        int32_t* status2, void* stream);
 
+/* ---- Scheduling microbenchmark: SwiGLU + Add operator pair (Section 6.1, Section 6.2) -------------
+ * The two element-wise operators the paper uses to study scheduling in isolation, on
+ *   x[M][2C] bf16 (gate | up halves of each row), r[M][C] bf16  ->
+ *   s[M][C] = bf16(silu(gate) * up)   (the intermediate, stored in global memory in every mode)
+ *   z[M][C] = bf16(s + r)
+ * with rows split into tiles of tile_rows, one task per operator and tile, run in one of three ways:
+ *   MOE_STUDY_SERIAL   two launches, one per operator (all of SwiGLU, then all of Add);
+ *   MOE_STUDY_STATIC   one persistent launch; each worker runs a fixed alternating list of SwiGLU and Add
+ *                      tasks, an Add task waiting on the event counter its producer (another worker) raises;
+ *   MOE_STUDY_DYNAMIC  one persistent launch; the same tasks and events, dispatched from a ready queue in
+ *                      global memory (atomic head / tail; a finished SwiGLU task publishes its Add task).
+ * All pointers are device pointers, 16-byte aligned; C % 8 == 0; M >= 0 (M == 0 launches nothing and
+ * ignores x, r, s and z).
+ * workspace: moe_sched_study_workspace_bytes(M, tile_rows) bytes of device memory owned by the caller, cleared
+ * by the call; it holds the status word, the queue and the event counters, and afterwards the workers'
+ * dispatch accounting, which moe_sched_study_stats() reads back (it synchronises the stream):
+ *   status2[2] = {code, detail} ({0,0}, or MOE_ERR_TIMEOUT and the tile whose wait ran out after 2 s),
+ *   dispatch_ns = summed over workers, the time between the end of one task's work and the start of the
+ *   next one's (ticket, decode, queue and event waits); tasks = the number of tasks that ran (2 * tiles;
+ *   both are 0 in the serial mode).  Any of the three may be NULL.
+ * Returns MOE_OK or MOE_ERR_INVALID_ARG / MOE_ERR_WORKSPACE / MOE_ERR_NO_DEVICE / MOE_ERR_CUDA. */
+#define MOE_STUDY_SERIAL 0
+#define MOE_STUDY_STATIC 1
+#define MOE_STUDY_DYNAMIC 2
+size_t moe_sched_study_workspace_bytes(int32_t M, int32_t tile_rows);
+int moe_sched_study(int32_t mode, const uint16_t* x, const uint16_t* r, uint16_t* s, uint16_t* z,
+                    int32_t M, int32_t C, int32_t tile_rows, void* workspace, size_t workspace_bytes,
+                    void* stream);
+int moe_sched_study_stats(const void* workspace, int32_t* status2, uint64_t* dispatch_ns,
+                          uint64_t* tasks, void* stream);
+
 const char* moe_strerror(int code);
 /* Text of the last CUDA error a call on this thread ran into ("" if none). */
 const char* moe_last_cuda_error(void);

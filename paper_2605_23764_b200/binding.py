@@ -21,7 +21,8 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_ffn_bwd", "moe_ffn_fwd_host", "moe_ffn_bwd_host", "moe_get_status", "moe_last_launch_count",
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
            "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
-           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace", "moe_debug_set_plain_launch"]
+           "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace", "moe_debug_set_plain_launch",
+           "moe_sched_study_workspace_bytes", "moe_sched_study", "moe_sched_study_stats"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -74,6 +75,11 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_trace.argtypes = [vp, vp, sz, ctypes.POINTER(sz)]
     lib.moe_debug_set_unreachable_dependency.argtypes = [vp, i32]
     lib.moe_debug_set_plain_launch.argtypes = [vp, i32]
+    lib.moe_sched_study_workspace_bytes.restype = sz
+    lib.moe_sched_study_workspace_bytes.argtypes = [i32, i32]
+    lib.moe_sched_study.argtypes = [i32, vp, vp, vp, vp, i32, i32, i32, vp, sz, vp]
+    lib.moe_sched_study_stats.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_uint64),
+                                          ctypes.POINTER(ctypes.c_uint64), vp]
     lib.moe_strerror.restype = ctypes.c_char_p
     lib.moe_strerror.argtypes = [ctypes.c_int]
     lib.moe_last_cuda_error.restype = ctypes.c_char_p
@@ -275,6 +281,35 @@ def moe_layout_noalloc(topk_ids, T, E, k, n_shared, counts, offsets, row_of, src
                                              _dev(counts, i32, "counts"), _dev(offsets, i32, "offsets"),
                                              _dev(row_of, i32, "row_of"), _dev(src_of, i32, "src_of"),
                                              _dev(status2, i32, "status2"), _stream()), "moe_layout_noalloc")
+
+
+MOE_STUDY_SERIAL, MOE_STUDY_STATIC, MOE_STUDY_DYNAMIC = 0, 1, 2
+
+
+def moe_sched_study_workspace_bytes(M, tile_rows) -> int:
+    return int(load_library().moe_sched_study_workspace_bytes(int(M), int(tile_rows)))
+
+
+def moe_sched_study(mode, x, r, s, z, M, C, tile_rows, workspace):
+    """SwiGLU + Add operator pair under one of the three schedules; all tensors are CUDA tensors
+    (bf16 x[M][2C], r/s/z[M][C]; workspace: any dtype, at least moe_sched_study_workspace_bytes)."""
+    bf = torch.bfloat16
+    _need(x, M * 2 * C, "x"); _need(r, M * C, "r"); _need(s, M * C, "s"); _need(z, M * C, "z")
+    if workspace is None or not workspace.is_cuda or not workspace.is_contiguous():
+        raise MoeError("workspace: expected a contiguous CUDA tensor")
+    nbytes = workspace.numel() * workspace.element_size()
+    _check(load_library().moe_sched_study(int(mode), _dev(x, bf, "x"), _dev(r, bf, "r"), _dev(s, bf, "s"),
+                                          _dev(z, bf, "z"), int(M), int(C), int(tile_rows),
+                                          ctypes.c_void_p(workspace.data_ptr()), nbytes, _stream()), "moe_sched_study")
+
+
+def moe_sched_study_stats(workspace):
+    """((code, detail), dispatch_ns, tasks) of the last moe_sched_study call on this workspace."""
+    st = (ctypes.c_int32 * 2)()
+    ns, n = ctypes.c_uint64(0), ctypes.c_uint64(0)
+    _check(load_library().moe_sched_study_stats(ctypes.c_void_p(workspace.data_ptr()), st, ctypes.byref(ns),
+                                                ctypes.byref(n), _stream()), "moe_sched_study_stats")
+    return (int(st[0]), int(st[1])), int(ns.value), int(n.value)
 
 
 def moe_debug_simulate_schedule(counts, T, k, n_shared, d, F, is_bwd, pairs, vec_workers):
