@@ -219,8 +219,9 @@ int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E, int32_t k,
  *   MOE_STUDY_SERIAL   two launches, one per operator (all of SwiGLU, then all of Add);
  *   MOE_STUDY_STATIC   one persistent launch; each worker runs a fixed alternating list of SwiGLU and Add
  *                      tasks, an Add task waiting on the event counter its producer (another worker) raises;
- *   MOE_STUDY_DYNAMIC  one persistent launch; the same tasks and events, dispatched from a ready queue in
- *                      global memory (atomic head / tail; a finished SwiGLU task publishes its Add task).
+ *   MOE_STUDY_DYNAMIC  one persistent launch; the same tasks and events, dispatched at run time: SwiGLU tasks
+ *                      from a ticket, Add tasks from a FIFO ready queue in global memory (a finished SwiGLU
+ *                      task appends its Add task; a free worker pops the queue before taking a ticket).
  * All pointers are device pointers, 16-byte aligned; C % 8 == 0; M >= 0 (M == 0 launches nothing and
  * ignores x, r, s and z).
  * workspace: moe_sched_study_workspace_bytes(M, tile_rows) bytes of device memory owned by the caller, cleared

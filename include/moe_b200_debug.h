@@ -47,7 +47,8 @@ int moe_debug_set_unreachable_dependency(moe_ctx* ctx, int32_t on);
 /* Profiling aid: with on != 0 the persistent launches of this context are made without the cooperative
  * launch attribute (some profilers reject cooperative launches of thread-block clusters).  The grid is
  * sized to what can be resident either way; what is lost is the driver's guarantee of co-residency when
- * other work shares the GPU -- every device-side wait stays bounded. */
+ * other work shares the GPU -- every device-side wait stays bounded.  ctx == NULL switches the persistent
+ * launches of moe_sched_study (process-wide) instead. */
 int moe_debug_set_plain_launch(moe_ctx* ctx, int32_t on);
 
 /* Host-only check of the static tile schedule of the single persistent launch (Section 4.3: tasks

@@ -967,7 +967,10 @@ int moe_debug_set_unreachable_dependency(moe_ctx* c, int32_t on) {
 }
 
 int moe_debug_set_plain_launch(moe_ctx* c, int32_t on) {
-  if (!c) return MOE_ERR_INVALID_ARG;
+  if (!c) {   // the context-free scheduling microbenchmark
+    study_plain_launch().store(on != 0);
+    return MOE_OK;
+  }
   c->plain_launch = on != 0;
   return MOE_OK;
 }

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda.h>
+#include <atomic>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -53,6 +54,8 @@ cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, 
                          int* counts, cudaStream_t s, int* launches);
 cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView& lv, DevStatus* status,
                           cudaStream_t s, int* launches);
+// process-wide switch of moe_sched_study's persistent launches (diagnostic; see moe_debug_set_plain_launch)
+std::atomic<bool>& study_plain_launch();
 cudaError_t launch_layout_order(const Dims& dm, const LayoutView& lv, int cap_mblocks, cudaStream_t s, int* launches);
 
 // ---- permute.cu

@@ -5,9 +5,9 @@
 //             thresholds: worker b runs SwiGLU of tile i*G+b and then Add of the tile its neighbour produced
 //             one round earlier, so every intermediate tile is consumed by another SM shortly after it was
 //             written, through L2 (Section 6.1 "interleaved", Section 6.2 "static");
-//   dynamic   the same tasks and events, but dispatched at run time from a ready queue in global memory:
-//             a worker takes the next queue slot, waits until a task has been published there, and a
-//             producer publishes the consumer task when it finishes (Section 6.2 "dynamic").
+//   dynamic   the same tasks and events, but dispatched at run time: producer tasks from a ticket, consumer
+//             tasks from a FIFO ready queue in global memory that a finished producer appends to and that a
+//             free worker pops first (Section 6.2 "dynamic").
 // s = silu(gate) * up is stored in bf16 between the operators in every mode.  Each worker also accounts the
 // time between the end of one task's work and the start of the next one's (ticket, decode, queue and event
 // waits): the per-task dispatch cost the paper compares.
@@ -15,12 +15,13 @@
 
 #include "../../include/moe_b200.h"
 #include "common.cuh"
+#include "moe_internal.h"
 
 namespace moe {
 
 constexpr int STUDY_THREADS = 256, STUDY_WORKERS_PER_SM = 4;
 // workspace (ints): status word, queue head / tail, dispatch accounting, one event counter per tile, the queue
-constexpr int SW_STATUS = 0, SW_HEAD = 4, SW_TAIL = 5, SW_STATS = 8 /* 2 x u64 */, SW_EVENTS = 16;
+constexpr int SW_STATUS = 0, SW_HEAD = 4, SW_TAIL = 5, SW_STICKET = 6, SW_STATS = 8 /* 2 x u64 */, SW_EVENTS = 16;
 
 __device__ __forceinline__ uint4 ld_cg16(const void* p) {
   uint4 v;
@@ -190,23 +191,42 @@ __global__ void __launch_bounds__(STUDY_THREADS, STUDY_WORKERS_PER_SM) study_sta
   if (threadIdx.x == 0) study_flush(a, d);
 }
 
-// dynamic: a ready queue of 2 * ntiles slots.  Slots [0, ntiles) hold the SwiGLU tasks from the start; a finished
-// SwiGLU task publishes the Add task of its tile in the next free slot.  Workers take slots in order.
+// dynamic: nothing is ordered ahead of time.  Producer tasks (SwiGLU tiles) are handed out by a ticket; a finished
+// producer appends its consumer task (Add of the same tile) to a FIFO ready queue in global memory.  A free worker
+// that sees a published entry claims the next slot of the queue, else takes the next producer ticket, and once the
+// producers are handed out it claims queue slots in order and waits for each to be published.
 __global__ void __launch_bounds__(STUDY_THREADS, STUDY_WORKERS_PER_SM) study_dynamic_kernel(const StudyArgs a) {
   const WaitCtl wc{reinterpret_cast<DevStatus*>(a.ws + SW_STATUS), a.budget_ns};
-  int* queue = a.ws + SW_EVENTS + a.ntiles;   // entries: tile (SwiGLU) or ntiles + tile (Add); 0 = not yet published
+  int* queue = a.ws + SW_EVENTS + a.ntiles;   // ready queue: entry = tile + 1; 0 = reserved but not yet published
+  int* head = a.ws + SW_HEAD;
+  int* tail = a.ws + SW_TAIL;
   __shared__ int task_s;
   Dispatch d{0, 0, 0};
+  bool producers_left = true;   // thread 0's view
   if (threadIdx.x == 0) d.t_mark = globaltimer_ns();
   while (true) {
     if (threadIdx.x == 0) {
-      int task = -1;
-      const int h = atomicAdd(a.ws + SW_HEAD, 1);
-      if (h < 2 * a.ntiles) {
-        if (h < a.ntiles) task = h;
-        else if (counter_wait(queue + h, 1, wc, h, 256)) task = *reinterpret_cast<volatile int*>(queue + h) - 1;
-        else task = -2;
+      int task = -1, slot = -1;
+      int h = *reinterpret_cast<volatile int*>(head), t;
+      asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(t) : "l"(tail) : "memory");
+      // A consumer task looks ready: claim the next slot.  Several workers may claim on the same observation; the
+      // ones past the tail wait for the next producers to publish (a retry loop of compare-and-swap instead lets
+      // one contender through per round trip to L2 and is an order of magnitude slower with hundreds of workers).
+      if (h < t) {
+        const int c = atomicAdd(head, 1);
+        if (c < a.ntiles) slot = c;   // else: every consumer is claimed; producer tickets may still be left
       }
+      if (slot < 0) {
+        const int p = producers_left ? atomicAdd(a.ws + SW_STICKET, 1) : a.ntiles;
+        if (p < a.ntiles) task = p;
+        else {
+          producers_left = false;
+          const int c = atomicAdd(head, 1);   // every producer is handed out: the remaining work is in the queue
+          if (c < a.ntiles) slot = c;
+        }
+      }
+      if (slot >= 0)
+        task = counter_wait(queue + slot, 1, wc, slot, 256) ? a.ntiles + *reinterpret_cast<volatile int*>(queue + slot) - 1 : -2;
       task_s = task;
     }
     __syncthreads();
@@ -219,9 +239,8 @@ __global__ void __launch_bounds__(STUDY_THREADS, STUDY_WORKERS_PER_SM) study_dyn
       tile_signal(a, task);
       if (threadIdx.x == 0) {
         work_done(d);
-        const int slot = a.ntiles + atomicAdd(a.ws + SW_TAIL, 1);   // publish the consumer task
-        __threadfence();
-        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(queue + slot), "r"(a.ntiles + task + 1) : "memory");
+        const int slot = atomicAdd(tail, 1);   // reserve, then publish the consumer task
+        asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(queue + slot), "r"(task + 1) : "memory");
       }
     } else {
       const int tile = task - a.ntiles;
@@ -233,6 +252,11 @@ __global__ void __launch_bounds__(STUDY_THREADS, STUDY_WORKERS_PER_SM) study_dyn
     }
   }
   if (threadIdx.x == 0) study_flush(a, d);
+}
+
+std::atomic<bool>& study_plain_launch() {
+  static std::atomic<bool> flag{false};
+  return flag;
 }
 
 }  // namespace moe
@@ -281,7 +305,8 @@ int moe_sched_study(int32_t mode, const uint16_t* x, const uint16_t* r, uint16_t
   // cooperative: the launch fails rather than run with workers that are not all resident (consumers wait for producers)
   const void* fn = mode == 1 ? reinterpret_cast<const void*>(study_static_kernel) : reinterpret_cast<const void*>(study_dynamic_kernel);
   const int grid = a.ntiles < workers ? a.ntiles : workers;
-  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(STUDY_THREADS), params, 0, st);
+  cudaError_t e = study_plain_launch().load() ? cudaLaunchKernel(fn, dim3(grid), dim3(STUDY_THREADS), params, 0, st)
+                                              : cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(STUDY_THREADS), params, 0, st);
   return e == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
