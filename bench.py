@@ -72,7 +72,8 @@ def phase_work(cfg, train):
     }
     work["fused_fwd"] = (6.0 * R * d * F, W1 + W2 + 2 * T * d * bf + (R * 2 * F * bf if train else 0))
     if train:
-        work["fused_bwd"] = (12.0 * R * d * F, 3 * (W1 + W2) + 2 * T * d * bf + R * 2 * F * bf + R * (d + F) * bf)
+        # backward alone: weights read once, weight gradients written once, dout in, dx out, saved pre-activations in
+        work["fused_bwd"] = (12.0 * R * d * F, 2 * (W1 + W2) + 3 * T * d * bf + R * 2 * F * bf)
         work.update({
             "bwd_gather": (0.0, T * d * bf + R * d * bf),
             "act_grad": (2.0 * R * d * F, R * d * bf + W2 + R * 2 * F * bf * 2),
@@ -281,10 +282,15 @@ class Workload:
         # weights that fit L2 would stay there from step to step: flush between timed steps
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if cfg.weight_bytes() <= 4e8 else None
 
+    plain_launch = False   # --plain-launch: persistent launches without the cooperative attribute (profiler captures)
+
     def make_layer(self, mode):
-        from paper_2605_23764_b200 import MoeLayer
+        from paper_2605_23764_b200 import MoeLayer, binding as B
         c = self.cfg
-        return MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=self.train, serial=(mode == "serial"))
+        lay = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=self.train, serial=(mode == "serial"))
+        if Workload.plain_launch:
+            B.moe_debug_set_plain_launch(lay.ctx, True)
+        return lay
 
     def step(self, lay, phases=None):
         """One pass of the hot path through the C ABI (device buffers).  -> kernels launched"""
@@ -508,6 +514,10 @@ def main():
     ap.add_argument("--no-compare", action="store_true", help="skip timing the other launch mode")
     ap.add_argument("--no-all-configs", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-study", action="store_true", help="skip the SwiGLU+Add scheduling microbenchmark")
+    ap.add_argument("--only-study", action="store_true", help="run the scheduling microbenchmark alone")
+    ap.add_argument("--study-iters", type=int, default=30)
+    ap.add_argument("--plain-launch", action="store_true",
+                    help="diagnostic: persistent launches without the cooperative launch attribute (for profiler captures)")
     ap.add_argument("--small", type=str, default="", help="T,d,F[,E]: reduced sizes of the chosen config (profiling captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -527,6 +537,15 @@ def main():
         respawn_under_launcher(args.gpus)
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (the layer has no CPU path)")
+
+    if args.plain_launch:
+        from paper_2605_23764_b200 import binding as B
+        Workload.plain_launch = True
+        B.moe_debug_set_plain_launch(None, True)
+    if args.only_study:
+        torch.cuda.set_device(0)
+        print(json.dumps({"scheduling_study": scheduling_study(load_peaks(), args.study_iters)}), flush=True)
+        return
 
     world, rank, local = dist_setup()
     if args.gpus != world and rank == 0:
@@ -596,7 +615,7 @@ def main():
 
     study = None
     if rank == 0 and world == 1 and not args.no_study and not args.small:
-        study = scheduling_study(peaks)
+        study = scheduling_study(peaks, args.study_iters)
 
     if rank == 0:
         desc = workload_desc(cfg, train)
