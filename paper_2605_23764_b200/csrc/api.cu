@@ -34,6 +34,23 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Stream memory operations (driver API): a stream waits until a 32-bit word in device memory reaches a value / a
+// stream writes such a word.  Used to let a copy-out stream start when a running kernel says its result is complete.
+typedef CUresult (*StreamValueFn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+StreamValueFn get_stream_value_fn(bool wait) {
+  static StreamValueFn fns[2] = {nullptr, nullptr};
+  static bool looked[2] = {false, false};
+  if (!looked[wait]) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint(wait ? "cuStreamWaitValue32" : "cuStreamWriteValue32", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fns[wait] = reinterpret_cast<StreamValueFn>(p);
+    looked[wait] = true;
+  }
+  return fns[wait];
+}
+
 EncodeTiledFn get_encode_fn() {
   static EncodeTiledFn fn = nullptr;
   if (!fn) {
@@ -663,8 +680,31 @@ int run_bwd(moe_ctx* c, const uint16_t* dout, const uint16_t* W1, const uint16_t
     MOE_CUDA(cudaMemsetAsync(fa.ctr, 0, sizeof(int) * (size_t)p.ctr_count, st));
     // slots dropped for an invalid expert id have no row: their gradient is zero
     if (d_w) MOE_CUDA(cudaMemsetAsync(d_w, 0, sizeof(float) * (size_t)T * s.k, st));
-    MOE_CUDA(launch_fused(true, fa, c->num_sms, !c->plain_launch, st, &c->launches));
-    if (dx_host) MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
+    // Host buffers: dx is complete when the last backward-combine task is, well before the last weight-gradient
+    // strips; the kernel then sets a word the copy-out stream waits for, so the copy overlaps the rest of the launch.
+    StreamValueFn wait_value = dx_host ? get_stream_value_fn(true) : nullptr;
+    StreamValueFn write_value = dx_host ? get_stream_value_fn(false) : nullptr;
+    const bool early_out = wait_value && write_value;
+    const CUdeviceptr ready_word = reinterpret_cast<CUdeviceptr>(fa.ctr + CTR_OUT_READY);
+    fa.announce_out = early_out ? 1 : 0;
+    if (early_out) {
+      MOE_CUDA(cudaEventRecord(c->ev_chunk[0], st));   // the word is cleared (the memset above) before anyone waits on it
+      MOE_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_chunk[0], 0));
+      if (wait_value(c->d2h_stream, ready_word, 1, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS) return cuda_fail(cudaErrorUnknown, "cuStreamWaitValue32");
+      MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, c->d2h_stream));
+      MOE_CUDA(cudaEventRecord(c->ev_d2h_done, c->d2h_stream));
+    }
+    const cudaError_t launched = launch_fused(true, fa, c->num_sms, !c->plain_launch, st, &c->launches);
+    if (early_out) {
+      // a launch that failed, or gave up on an expired wait, never sets the word: set it behind the launch so that
+      // the copy-out stream is released in every case, then make `st` cover the copy
+      if (write_value(st, ready_word, 1, CU_STREAM_WRITE_VALUE_DEFAULT) != CUDA_SUCCESS) return cuda_fail(cudaErrorUnknown, "cuStreamWriteValue32");
+      MOE_CUDA(cudaStreamWaitEvent(st, c->ev_d2h_done, 0));
+    }
+    MOE_CUDA(launched);
+    if (!early_out && dx_host) {
+      MOE_CUDA(cudaMemcpyAsync(dx_host, dx, 2 * (size_t)T * s.d, cudaMemcpyDeviceToHost, st));
+    }
   }
   return MOE_OK;
 }

@@ -203,6 +203,20 @@ __device__ __forceinline__ void vector_worker_loop(const FusedArgs& fa, const Wa
     const bool ok = v.op == VEC_COMBINE ? vec_combine(fa, v.idx, lane, wc) : vec_dw(fa, v.idx, lane, wc);
     if (tr.buf && lane == 0) trace_put(tr, TR_VEC, v.op, v.idx, t0, t0, globaltimer_ns());
     if (!ok) break;
+    if (fa.announce_out && v.op == VEC_COMBINE) {
+      // Host-buffer calls: the result may leave for the host as soon as its last row is written, while the
+      // launch still computes weight gradients.  The warp's stores, then a device-wide fence, then the count;
+      // whoever finishes the last task publishes the word the copy-out stream waits for.
+      __syncwarp();
+      if (lane == 0) {
+        __threadfence();
+        const int ncombine = (fa.cp.T + COMBINE_TOKENS - 1) / COMBINE_TOKENS;
+        if (atomicAdd(&fa.ctr[CTR_COMBINE_DONE], 1) + 1 == ncombine) {
+          __threadfence_system();
+          *reinterpret_cast<volatile int*>(&fa.ctr[CTR_OUT_READY]) = 1;
+        }
+      }
+    }
   }
 }
 

@@ -144,6 +144,7 @@ struct FusedArgs {
   // combine (Combine / backward Combine)
   const uint16_t* combine_rows;
   uint16_t* combine_out;
+  int announce_out;         // 1: count finished combine tasks and set ctr[CTR_OUT_READY] after the last one
   // backward extras
   const float* dw_partial;
   int dw_nparts;

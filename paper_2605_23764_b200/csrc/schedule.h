@@ -120,6 +120,8 @@ MOE_HD int thr_done(const ChainParams& cp) { return SIG * cp.ntn[cp.is_bwd ? 2 :
 
 // ---------------------------------------------------------------- counters (ints in device memory)
 constexpr int CTR_VEC_TICKET = 0, CTR_TRACE_CURSOR = 1, CTR_MAT_TICKET = 2, CTR_POST_TICKET = 3, CTR_PER_MB = 8, CTR_STRIDE = 4;
+// combine tasks finished, and the word that turns 1 when all of them are (a copy-out stream may wait on it)
+constexpr int CTR_COMBINE_DONE = 4, CTR_OUT_READY = 5;
 enum CtrKind : int { CTR_GATHERED = 0, CTR_ACTIVATED = 1, CTR_DONE = 2, CTR_NONE = -1 };
 MOE_HD int ctr_index(int mb, int kind) { return CTR_PER_MB + CTR_STRIDE * mb + kind; }
 MOE_HD int ctr_ints(int cap_mblocks) { return CTR_PER_MB + CTR_STRIDE * cap_mblocks; }

@@ -43,3 +43,44 @@ def test_unreachable_dependency_times_out_and_context_recovers():
     ref = oracle.fwd(x, ids.cpu(), w.cpu(), W1, W2)
     assert_close_bf16(again, ref, "forward after a timed-out launch")
     layer.close()
+
+
+def test_timed_out_backward_releases_the_copy_out_stream():
+    """Host-buffer backward in the persistent mode: the copy of dx waits on a word the kernel sets after its last
+    combine task.  A launch that gives up never sets it; the call must still end (the word is also written behind
+    the launch) and the next step must be right."""
+    T, d, E, k, S, F = 256, 256, 8, 2, 0, 128
+    x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, 12)
+    layer = MoeLayer(T, d, E, k, S, F, save_for_bwd=True)
+    ids, w = layer.route(logits)
+    layer.ffn_fwd(x, ids, w, W1, W2)
+    dx_good, dW1_good, dW2_good, dw_good = [t.clone() for t in layer.ffn_bwd(dout, x, ids, w, W1, W2)]
+    assert layer.status() == (0, 0)
+
+    pin = dict(pin_memory=True)
+    xh, doh = x.cpu().pin_memory(), dout.cpu().pin_memory()
+    idh, wh = ids.cpu().pin_memory(), w.cpu().pin_memory()
+    oh = torch.empty(T, d, dtype=torch.bfloat16, **pin)
+    dxh = torch.empty(T, d, dtype=torch.bfloat16, **pin)
+    dwh = torch.empty(T, k, dtype=torch.float32, **pin)
+    gW1, gW2 = torch.empty_like(W1), torch.empty_like(W2)
+
+    binding.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, W1, W2, oh, T)
+    binding.moe_set_wait_budget_ms(layer.ctx, 100)
+    binding.moe_debug_set_unreachable_dependency(layer.ctx, True)
+    t0 = time.perf_counter()
+    binding.moe_ffn_bwd_host(layer.ctx, doh, W1, W2, dxh, gW1, gW2, dwh, T)
+    code, detail = layer.status()
+    torch.cuda.synchronize()               # every stream of the context has drained
+    assert code == 2, (code, detail)
+    assert time.perf_counter() - t0 < 5.0
+
+    binding.moe_debug_set_unreachable_dependency(layer.ctx, False)
+    binding.moe_set_wait_budget_ms(layer.ctx, 2000)
+    binding.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, W1, W2, oh, T)
+    binding.moe_ffn_bwd_host(layer.ctx, doh, W1, W2, dxh, gW1, gW2, dwh, T)
+    torch.cuda.synchronize()
+    assert layer.status() == (0, 0)
+    assert torch.equal(dxh, dx_good.cpu()) and torch.equal(dwh, dw_good.cpu())
+    assert torch.equal(gW1, dW1_good) and torch.equal(gW2, dW2_good)
+    layer.close()
