@@ -78,6 +78,58 @@ int moe_oracle_route(const float* logits, int T, int E, int k, int renorm,
   return 0;
 }
 
+/* ---- router in the path (Section 2.2, first paragraph: the router scores every expert for each token
+ * and keeps the top k).  The score function the paper leaves open is the usual linear router:
+ * logits[t][e] = <x[t], W_r[e]>, W_r[E][d].  The routing decision itself is moe_oracle_route applied
+ * to these logits rounded to fp32 (the precision in which the CUDA path decides). ---- */
+int moe_oracle_router_logits(const double* x, const double* Wr, int T, int d, int E, double* logits) {
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t)
+    for (int e = 0; e < E; ++e) {
+      double acc = 0.0;
+      for (int c = 0; c < d; ++c) acc += x[(size_t)t * d + c] * Wr[(size_t)e * d + c];
+      logits[(size_t)t * E + e] = acc;
+    }
+  return 0;
+}
+
+/* Gradient of the routing scores w.r.t. the logits, given g = dL/d topk_w (the selection is piecewise
+ * constant and passes no gradient).  p = softmax(logits) over all E.
+ *   without renormalisation  w_j = p[e_j]:
+ *       dL/dl[e] = [e = e_j] g_j p[e]  -  p[e] * sum_j g_j p[e_j]
+ *   with renormalisation     w_j = p[e_j] / sum_{i in S} p[e_i]  (a softmax over the selected set S only):
+ *       dL/dl[e_j] = w_j (g_j - sum_i g_i w_i),  0 outside S. */
+int moe_oracle_router_bwd(const float* logits, const int32_t* ids, const double* g, int T, int E, int k,
+                          int renorm, double* dlogits) {
+  if (k < 1 || k > E) return -1;
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    const float* l = logits + (size_t)t * E;
+    const int32_t* id = ids + (size_t)t * k;
+    const double* gt = g + (size_t)t * k;
+    double* dl = dlogits + (size_t)t * E;
+    for (int e = 0; e < E; ++e) dl[e] = 0.0;
+    double mx = l[0];
+    for (int e = 1; e < E; ++e) if (l[e] > mx) mx = l[e];
+    if (renorm) {
+      double den = 0.0, dot = 0.0;
+      for (int j = 0; j < k; ++j) den += exp((double)l[id[j]] - mx);
+      for (int j = 0; j < k; ++j) dot += gt[j] * (exp((double)l[id[j]] - mx) / den);
+      for (int j = 0; j < k; ++j) {
+        double wj = exp((double)l[id[j]] - mx) / den;
+        dl[id[j]] += wj * (gt[j] - dot);
+      }
+    } else {
+      double den = 0.0, dot = 0.0;
+      for (int e = 0; e < E; ++e) den += exp((double)l[e] - mx);
+      for (int j = 0; j < k; ++j) dot += gt[j] * (exp((double)l[id[j]] - mx) / den);
+      for (int e = 0; e < E; ++e) dl[e] = -(exp((double)l[e] - mx) / den) * dot;
+      for (int j = 0; j < k; ++j) dl[id[j]] += gt[j] * (exp((double)l[id[j]] - mx) / den);
+    }
+  }
+  return 0;
+}
+
 /* expert id of flat slot i = t*(k+S)+j: routed slots first, then the S shared experts */
 static inline int slot_expert(const int32_t* ids, int k, int S, int E, int t, int j) {
   return j < k ? ids[(size_t)t * k + j] : E + (j - k);

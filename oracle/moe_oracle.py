@@ -40,6 +40,8 @@ def _load():
         lib.moe_oracle_bwd.argtypes = [f64p, f64p, i32p, f64p, f64p, f64p, ci, ci, ci, ci, ci, ci,
                                        f64p, f64p, f64p, f64p]
         lib.moe_oracle_swiglu_add.argtypes = [f64p, f64p, ci, ci, f64p, f64p]
+        lib.moe_oracle_router_logits.argtypes = [f64p, f64p, ci, ci, ci, f64p]
+        lib.moe_oracle_router_bwd.argtypes = [f32p, i32p, f64p, ci, ci, ci, ci, f64p]
         _lib = lib
     return _lib
 
@@ -162,3 +164,42 @@ def swiglu_add(x, r):
     if rc:
         raise ValueError(f"moe_oracle_swiglu_add failed ({rc})")
     return s, z
+
+
+def router_logits(x, W_r):
+    """Linear router scores (Section 2.2, router description): x [T,d], W_r [E,d] -> logits float64 [T,E]."""
+    x = _np(x, np.float64)
+    W = _np(W_r, np.float64)
+    T, d = x.shape
+    E = W.shape[0]
+    assert W.shape == (E, d)
+    out = np.empty((T, E), np.float64)
+    rc = _load().moe_oracle_router_logits(_p(x, ctypes.c_double), _p(W, ctypes.c_double), T, d, E, _p(out, ctypes.c_double))
+    if rc:
+        raise ValueError(f"moe_oracle_router_logits failed ({rc})")
+    return out
+
+
+def router_fwd(x, W_r, k: int, renorm: bool):
+    """Router in the path: logits in fp64, rounded once to fp32 (the precision the CUDA path decides in), then
+    `route`.  -> ids int32 [T,k], w float64 [T,k], logits float64 [T,E] (unrounded)."""
+    logits = router_logits(x, W_r)
+    ids, w = route(logits.astype(np.float32), k, renorm)
+    return ids, w, logits
+
+
+def router_bwd(logits, ids, d_topk_w, renorm: bool):
+    """Gradient of the k routing scores w.r.t. the logits (softmax over all E, optional renormalisation over the
+    selected experts; no gradient through the selection).  -> d_logits float64 [T,E]."""
+    l = _np(logits, np.float32)
+    ids = _np(ids, np.int32)
+    g = _np(d_topk_w, np.float64)
+    T, E = l.shape
+    k = ids.shape[1]
+    assert ids.shape == (T, k) and g.shape == (T, k)
+    out = np.empty((T, E), np.float64)
+    rc = _load().moe_oracle_router_bwd(_p(l, ctypes.c_float), _p(ids, ctypes.c_int32), _p(g, ctypes.c_double), T, E, k,
+                                       int(bool(renorm)), _p(out, ctypes.c_double))
+    if rc:
+        raise ValueError(f"moe_oracle_router_bwd failed ({rc})")
+    return out
