@@ -13,7 +13,8 @@ The headline `value` is the library's default launch mode: one persistent depend
 launch per pass.  The one-launch-per-operator mode is timed in the same run and reported as
 `other_launch_mode`; `all_configs` holds both modes for the forward-only workloads;
 `scheduling_study` holds the SwiGLU+Add scheduling microbenchmark (Section 6): serial, statically
-interleaved and dynamically dispatched, with the dispatch time per task.
+interleaved and dynamically dispatched, with the dispatch time per task; `router_in_path` the router GEMM +
+top-k launch on the workload's shape (it is outside the timed step, whose routing starts from given logits).
 With N > 1 every rank runs an independent replica on its own GPU (the layer is not sharded;
 there is no data-path collective); `python bench.py --gpus N` without a launcher starts the N
 ranks itself.
@@ -486,6 +487,48 @@ def scheduling_study(peaks, iters=30):
             "rows": rows}
 
 
+def router_in_path(cfg, peaks, iters=30):
+    """The in-path router on the workload's shape: x W_r^T + softmax top-k in one launch (`moe_router_fwd`), and the
+    score gradient (`moe_router_bwd`); median microseconds with L2 flushed before each call."""
+    from paper_2605_23764_b200 import MoeLayer, binding as B
+    dev = torch.device("cuda")
+    T, d, E, k = cfg.T, cfg.d, cfg.E, cfg.k
+    g = torch.Generator(device="cuda").manual_seed(77)
+    x = torch.randn(T, d, device=dev, generator=g).to(torch.bfloat16)
+    W = (torch.randn(E, d, device=dev, generator=g) * 0.02).to(torch.bfloat16)
+    lay = MoeLayer(T, d, E, k, 0, 128, renorm=cfg.renorm)
+    ids = torch.empty(T, k, dtype=torch.int32, device=dev)
+    w = torch.empty(T, k, dtype=torch.float32, device=dev)
+    logits = torch.empty(T, E, dtype=torch.float32, device=dev)
+    dl = torch.empty_like(logits)
+    gw = torch.randn(T, k, device=dev, generator=g)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def med(fn):
+        ts = []
+        for it in range(iters + 3):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        return sorted(ts)[len(ts) // 2]
+
+    us_f = med(lambda: B.moe_router_fwd(lay.ctx, x, W, T, ids, w, logits))
+    us_b = med(lambda: B.moe_router_bwd(lay.ctx, logits, ids, gw, T, dl))
+    assert lay.status() == (0, 0)
+    lay.close()
+    flop, by = 2.0 * T * d * E, 2.0 * T * d + 2.0 * E * d + 4.0 * T * E + 8.0 * T * k
+    roof_us = max(flop / (peaks["bf16_tflops"] * 1e12), by / (peaks["hbm_gbs"] * 1e9)) * 1e6
+    by_b = 2 * 4.0 * T * E + 8.0 * T * k
+    return {"shape": {"T": T, "d": d, "E": E, "k": k},
+            "fwd": {"us": us_f, "TFLOPs": flop / us_f / 1e6, "GBps": by / us_f / 1e3, "roofline_us": roof_us,
+                    "frac": roof_us / us_f, "bound": "tensor" if flop / (peaks["bf16_tflops"] * 1e12) >= by / (peaks["hbm_gbs"] * 1e9) else "hbm"},
+            "bwd": {"us": us_b, "GBps": by_b / us_b / 1e3, "frac": by_b / us_b / 1e3 / peaks["hbm_gbs"], "bound": "hbm"},
+            "timing": "CUDA events around each call, L2 flushed before each; median of %d" % iters}
+
+
 def respawn_under_launcher(n):
     """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU) and pass their output on."""
     import socket
@@ -515,6 +558,7 @@ def main():
     ap.add_argument("--no-all-configs", action="store_true", help="skip the other workloads")
     ap.add_argument("--no-study", action="store_true", help="skip the SwiGLU+Add scheduling microbenchmark")
     ap.add_argument("--only-study", action="store_true", help="run the scheduling microbenchmark alone")
+    ap.add_argument("--only-router", action="store_true", help="run the in-path router alone (on --config's shape)")
     ap.add_argument("--study-iters", type=int, default=30)
     ap.add_argument("--plain-launch", action="store_true",
                     help="diagnostic: persistent launches without the cooperative launch attribute (for profiler captures)")
@@ -542,6 +586,10 @@ def main():
         from paper_2605_23764_b200 import binding as B
         Workload.plain_launch = True
         B.moe_debug_set_plain_launch(None, True)
+    if args.only_router:
+        torch.cuda.set_device(0)
+        print(json.dumps({"router_in_path": router_in_path(cfg, load_peaks(), args.study_iters)}), flush=True)
+        return
     if args.only_study:
         torch.cuda.set_device(0)
         print(json.dumps({"scheduling_study": scheduling_study(load_peaks(), args.study_iters)}), flush=True)
@@ -616,6 +664,9 @@ def main():
     study = None
     if rank == 0 and world == 1 and not args.no_study and not args.small:
         study = scheduling_study(peaks, args.study_iters)
+    router = None
+    if rank == 0 and world == 1 and not args.no_study:
+        router = router_in_path(cfg, peaks, args.study_iters)
 
     if rank == 0:
         desc = workload_desc(cfg, train)
@@ -630,7 +681,7 @@ def main():
             "config": desc, "clocks": res["clocks"], "e2e": e2e, "gpu_launches": res["launches"],
             "roofline": roofline, "step_roofline": step_roofline, "phases_ms": res["phases_ms"],
             "other_launch_mode": other, "all_configs": all_configs, "cpu_baseline": cpu_baseline,
-            "scheduling_study": study,
+            "scheduling_study": study, "router_in_path": router,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

@@ -210,6 +210,31 @@ int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E, int32_t k,
                        int32_t* counts, int32_t* offsets, int32_t* row_of, int32_t* src_of,
                        int32_t* status2, void* stream);
 
+/* ---- Router in the path (Section 2.2, first paragraph: the router assigns each token its top-k experts and
+ * their routing scores) -----------------------------------------------------------------------------------
+ * moe_router_fwd: logits = x W_r^T on the tensor cores (bf16 operands, fp32 accumulation) with moe_route's
+ * softmax top-k fused into the same launch -- same selection rule (raw logits compared, equal logits to the
+ * lower expert id, slots in descending order), same scores (softmax over all E, renormalised over the k
+ * selected with MOE_FLAG_RENORM_TOPK).
+ *   x[T][d] bf16, W_r[E][d] bf16 (router weights, one row per routed expert), both device pointers, 16-byte
+ *   aligned -> topk_ids[T][k] int32, topk_w[T][k] fp32; logits[T][E] fp32 (may be NULL: not stored; keep them
+ *   for moe_router_bwd), counts[E] int32 (may be NULL).
+ * Limits: E <= 256, k <= 8 (MOE_ERR_TOO_LARGE otherwise: compute the logits elsewhere and call moe_route).
+ * The logits are fp32 sums in the tensor cores' order: an expert whose logit differs from the k-th largest by
+ * less than the rounding of that sum may be selected differently than by an exact computation.
+ *
+ * moe_router_bwd: gradient of the k scores with respect to the logits (the selection passes none), from
+ * d_topk_w[T][k] as moe_ffn_bwd returns it: p = softmax(logits) over all E,
+ *   without renormalisation  d_logits[t][e] = [e = e_j] g_j p_e - p_e * sum_j g_j p_{e_j}
+ *   with renormalisation     d_logits[t][e_j] = w_j (g_j - sum_i g_i w_i), 0 for experts not selected.
+ *   logits[T][E] fp32, topk_ids[T][k], d_topk_w[T][k] fp32 -> d_logits[T][E] fp32 (all device pointers).
+ * The two dense products that follow (d_logits^T x for the router weights, d_logits W_r for x) are plain
+ * GEMMs outside this library.  Limit: k <= 32.  Both calls are asynchronous on `stream`. */
+int moe_router_fwd(moe_ctx* ctx, const uint16_t* x, const uint16_t* W_r, int32_t T, int32_t* topk_ids,
+                   float* topk_w, float* logits, int32_t* counts, void* stream);
+int moe_router_bwd(moe_ctx* ctx, const float* logits, const int32_t* topk_ids, const float* d_topk_w, int32_t T,
+                   float* d_logits, void* stream);
+
 /* ---- Scheduling microbenchmark: SwiGLU + Add operator pair (Section 6.1, Section 6.2) -------------
  * The two element-wise operators the paper uses to study scheduling in isolation, on
  *   x[M][2C] bf16 (gate | up halves of each row), r[M][C] bf16  ->

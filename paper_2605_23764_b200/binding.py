@@ -22,7 +22,8 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_set_wait_budget_ms", "moe_debug_buffer", "moe_strerror", "moe_last_cuda_error",
            "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
            "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace", "moe_debug_set_plain_launch",
-           "moe_sched_study_workspace_bytes", "moe_sched_study", "moe_sched_study_stats"]
+           "moe_sched_study_workspace_bytes", "moe_sched_study", "moe_sched_study_stats", "moe_router_fwd",
+           "moe_router_bwd"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -75,6 +76,8 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_trace.argtypes = [vp, vp, sz, ctypes.POINTER(sz)]
     lib.moe_debug_set_unreachable_dependency.argtypes = [vp, i32]
     lib.moe_debug_set_plain_launch.argtypes = [vp, i32]
+    lib.moe_router_fwd.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.moe_router_bwd.argtypes = [vp, vp, vp, vp, i32, vp, vp]
     lib.moe_sched_study_workspace_bytes.restype = sz
     lib.moe_sched_study_workspace_bytes.argtypes = [i32, i32]
     lib.moe_sched_study.argtypes = [i32, vp, vp, vp, vp, i32, i32, i32, vp, sz, vp]
@@ -167,6 +170,25 @@ def moe_route(ctx, logits, T, topk_ids, topk_w, counts=None):
     _check(load_library().moe_route(ctx, _dev(logits, torch.float32, "logits"), T,
                                     _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_w, torch.float32, "topk_w"),
                                     _dev(counts, torch.int32, "counts"), _stream()), "moe_route")
+
+
+def moe_router_fwd(ctx, x, W_r, T, topk_ids, topk_w, logits=None, counts=None):
+    _, d, E, k, _, _, _ = _shape_of(ctx)
+    _need(x, T * d, "x"); _need(W_r, E * d, "W_r"); _need(topk_ids, T * k, "topk_ids"); _need(topk_w, T * k, "topk_w")
+    _need(logits, T * E, "logits"); _need(counts, E, "counts")
+    _check(load_library().moe_router_fwd(ctx, _dev(x, torch.bfloat16, "x"), _dev(W_r, torch.bfloat16, "W_r"), T,
+                                         _dev(topk_ids, torch.int32, "topk_ids"), _dev(topk_w, torch.float32, "topk_w"),
+                                         _dev(logits, torch.float32, "logits"), _dev(counts, torch.int32, "counts"),
+                                         _stream()), "moe_router_fwd")
+
+
+def moe_router_bwd(ctx, logits, topk_ids, d_topk_w, T, d_logits):
+    _, _, E, k, _, _, _ = _shape_of(ctx)
+    _need(logits, T * E, "logits"); _need(topk_ids, T * k, "topk_ids"); _need(d_topk_w, T * k, "d_topk_w")
+    _need(d_logits, T * E, "d_logits")
+    _check(load_library().moe_router_bwd(ctx, _dev(logits, torch.float32, "logits"), _dev(topk_ids, torch.int32, "topk_ids"),
+                                         _dev(d_topk_w, torch.float32, "d_topk_w"), T,
+                                         _dev(d_logits, torch.float32, "d_logits"), _stream()), "moe_router_bwd")
 
 
 def moe_layout(ctx, topk_ids, T, counts=None, offsets=None, row_of=None, src_of=None):

@@ -821,6 +821,43 @@ int moe_route(moe_ctx* c, const float* logits, int32_t T, int32_t* topk_ids, flo
   return MOE_OK;
 }
 
+int moe_router_fwd(moe_ctx* c, const uint16_t* x, const uint16_t* W_r, int32_t T, int32_t* topk_ids, float* topk_w,
+                   float* logits, int32_t* counts, void* stream) {
+  if (!c || !x || !W_r || !topk_ids || !topk_w || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
+  const moe_shape& s = c->shape;
+  if (s.E > 256 || s.k > 8) return MOE_ERR_TOO_LARGE;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(W_r)) & 15) return MOE_ERR_INVALID_ARG;
+  if (logits && (reinterpret_cast<uintptr_t>(logits) & 15)) return MOE_ERR_INVALID_ARG;
+  c->begin_call(static_cast<cudaStream_t>(stream));
+  if (T == 0) return MOE_OK;
+  RouterArgs a;
+  memset(&a, 0, sizeof a);
+  a.T = T; a.E = s.E; a.k = s.k; a.d = s.d;
+  a.N = ((s.E + 15) / 16) * 16;
+  if (a.N < 32) a.N = 32;
+  a.renorm = (s.flags & MOE_FLAG_RENORM_TOPK) != 0;
+  a.topk_ids = topk_ids; a.topk_w = topk_w; a.logits = logits; a.counts = counts;
+  a.status = c->status();
+  a.budget_ns = c->budget_ns;
+  int rc = encode_2d(&a.tmX, x, (uint64_t)T, (uint64_t)s.d, 128, 64);   // 128 token rows x one 64-wide k-block
+  if (rc) return rc;
+  if ((rc = encode_2d(&a.tmW, W_r, (uint64_t)s.E, (uint64_t)s.d, (uint32_t)(a.N / 2), 64))) return rc;
+  Phase ph(c, MOE_PHASE_ROUTE, c->last_stream);
+  MOE_CUDA(launch_router_fwd(a, c->num_sms, c->last_stream, &c->launches));
+  return MOE_OK;
+}
+
+int moe_router_bwd(moe_ctx* c, const float* logits, const int32_t* topk_ids, const float* d_topk_w, int32_t T,
+                   float* d_logits, void* stream) {
+  if (!c || !logits || !topk_ids || !d_topk_w || !d_logits || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
+  const moe_shape& s = c->shape;
+  if (s.k > 32) return MOE_ERR_TOO_LARGE;
+  c->begin_call(static_cast<cudaStream_t>(stream));
+  MOE_CUDA(launch_router_bwd(logits, topk_ids, d_topk_w, T, s.E, s.k, (s.flags & MOE_FLAG_RENORM_TOPK) != 0, d_logits,
+                             c->last_stream, &c->launches));
+  return MOE_OK;
+}
+
 int moe_route_host(moe_ctx* c, const float* logits_host, int32_t T, int32_t* topk_ids_host, float* topk_w_host,
                    void* stream) {
   if (!c || !logits_host || !topk_ids_host || !topk_w_host || T < 0 || T > c->shape.T_max)

@@ -156,6 +156,24 @@ struct FusedArgs {
   uint64_t budget_ns;
 };
 
+// Router in the path (router.cu)
+struct RouterArgs {
+  CUtensorMap tmX;          // x [T][d] bf16, box 128 rows x 64 columns
+  CUtensorMap tmW;          // W_r [E][d] bf16, box N/2 rows x 64 columns (rows beyond E read as zeros)
+  int T, E, k, d;
+  int N;                    // accumulator columns: E rounded up to a multiple of 16, at least 32, at most 256
+  int renorm;
+  int* topk_ids;
+  float* topk_w;
+  float* logits;            // may be NULL
+  int* counts;              // may be NULL
+  DevStatus* status;
+  uint64_t budget_ns;
+};
+cudaError_t launch_router_fwd(const RouterArgs& a, int num_sms, cudaStream_t s, int* launches);
+cudaError_t launch_router_bwd(const float* logits, const int* ids, const float* g, int T, int E, int k, bool renorm,
+                              float* dlogits, cudaStream_t s, int* launches);
+
 // cooperative = false drops the co-residency guarantee of the launch (profilers that reject cooperative cluster
 // launches); the grid is sized to the resident capacity either way and every wait is bounded
 cudaError_t launch_fused(bool bwd, const FusedArgs& fa, int num_sms, bool cooperative, cudaStream_t s, int* launches);
