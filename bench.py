@@ -481,6 +481,25 @@ def scheduling_study(peaks, iters=30):
             us = sorted(ts)[len(ts) // 2]
             row[name] = {"us": us, "GBps": algo_bytes / us / 1e3, "frac_of_hbm_peak": algo_bytes / us / 1e3 / peaks["hbm_gbs"],
                          "dispatch_ns_per_task": (ns / n) if n else None}
+        # the same pair compiled by the generic front end into task descriptors and run by the descriptor runtime
+        shapes = [(M, 2 * C), (M, C), (M, C), (M, C)]
+        plan = B.moe_taskflow_compile(shapes, [B.tf_operator(B.MOE_TF_SWIGLU, [0], [1], tile_rows, split_inputs=None),
+                                               B.tf_operator(B.MOE_TF_ADD, [1, 2], [3], tile_rows, split_inputs=[(0, 0)])],
+                                      lag_rows=tile_rows * 4 * torch.cuda.get_device_properties(0).multi_processor_count)
+        tws = torch.empty(B.moe_taskflow_workspace_bytes(plan["n_tds"], plan["n_events"], 4), dtype=torch.uint8, device=dev)
+        ts = []
+        for it in range(iters + 3):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); B.moe_taskflow_run(plan, [x, s, r, z], shapes, tws, upload=(it == 0)); e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        if B.moe_taskflow_status(tws) != (0, 0):
+            raise SystemExit("taskflow runtime: device status")
+        us = sorted(ts)[len(ts) // 2]
+        row["descriptors"] = {"us": us, "GBps": algo_bytes / us / 1e3, "frac_of_hbm_peak": algo_bytes / us / 1e3 / peaks["hbm_gbs"],
+                              "tasks": plan["n_tds"], "note": "descriptor table uploaded once, before the timed calls"}
         rows.append(row)
     return {"operators": "SwiGLU(M x 4096) -> s(M x 2048, bf16, in global memory) -> Add(M x 2048)",
             "timing": "CUDA events around each call (workspace clear + kernels), L2 flushed before each; median of %d" % iters,

@@ -267,6 +267,69 @@ int moe_sched_study(int32_t mode, const uint16_t* x, const uint16_t* r, uint16_t
 int moe_sched_study_stats(const void* workspace, int32_t* status2, uint64_t* dispatch_ns,
                           uint64_t* tasks, void* stream);
 
+/* ---- Generic taskflow front end (Section 4.2: Operator Dependency Graph, SplitSpec, Algorithm 1 "Split
+ * Propagation", Table 1 Task Descriptor; Section 4.3: queues, events with static thresholds) ---------------
+ * Host side: an operator graph over 2-D bf16 tensors is compiled into Task Descriptors (TDs) and one statically
+ * ordered vector queue; device side: a persistent runtime whose workers take the next TD of the queue, wait for
+ * its dependent event, run the handler named by task_type on the TD's row range, and raise its trigger event.
+ * The runtime knows handlers, not graphs: any chain of the operators below runs without new device code.
+ *
+ * Tensors: moe_tf_tensor {rows, cols}, row-major bf16; tensor ids are indices into the array.  A tensor no
+ * operator produces is an input of the graph.
+ * Operators (moe_tf_operator): op = MOE_TF_SWIGLU (inputs {x[M][2C]} -> outputs {s[M][C]}) or MOE_TF_ADD
+ * (inputs {a, b}[M][C] -> {z[M][C]}); SplitSpec fields as in Section 4.2:
+ *   n_split_inputs = -1: the operator is a partition origin (split_inputs = None); otherwise it splits only
+ *     if input split_input_idx[i] carries the label split_input_dim[i] for every i (inputs not listed are
+ *     ignored by the check, like the metadata inputs of Combine), else it falls back to ONE unsplit task;
+ *   split_output_dim[j]: the label written on output j when the operator is split (-1: none);
+ *   task_rows: task_num_fn = ceil(rows of output 0 / task_rows).  Only dimension 0 (rows) can be split.
+ * moe_taskflow_compile (host only, no GPU needed) runs Algorithm 1, fills the TDs (Table 1's fields; TDesc =
+ * {tensor slot, row offset, rows, cols}), assigns events -- one counter per row block of a group of tensors
+ * that are consumed together, threshold = the number of TDs that write into the block -- and orders the queue:
+ * a topological order that runs a consumer task `lag_rows` rows behind its producers, so that intermediates are
+ * read back while still in L2 (Section 4.5).  Outputs: tds[0..*n_tds) in queue order, *n_events,
+ * op_task_num[n_ops] (Algorithm 1's task_num), tensor_split_dim / tensor_split_num [n_tensors] (its labels).
+ * Task granularities that feed one event must be multiples of one another, and an operator may not consume a
+ * tensor of the event group it triggers: MOE_ERR_INVALID_ARG.  td_cap too small: MOE_ERR_WORKSPACE.
+ *
+ * moe_taskflow_run: tds (host), slots[n_tensors] (host array of DEVICE pointers, 16-byte aligned, cols % 8 == 0),
+ * workspace (device, moe_taskflow_workspace_bytes; its counters are cleared by every call) -> launches the runtime
+ * on `stream`.  upload != 0 copies the descriptor table and the slot table into the workspace first; upload == 0
+ * reuses what an earlier call with the same tds, slots and workspace put there (a compiled plan is uploaded once
+ * and run every step; tds and slots are still checked on the host either way).
+ * moe_taskflow_status (synchronises the stream): status2 = {code, detail} ({0,0} or MOE_ERR_TIMEOUT and the TD
+ * whose wait ran out after 2 s). */
+#define MOE_TF_SWIGLU 1
+#define MOE_TF_ADD 2
+#define MOE_TF_QUEUE_MATRIX 0
+#define MOE_TF_QUEUE_VECTOR 1
+#define MOE_TF_NO_EVENT 0xFFFFFFFFu
+typedef struct { int32_t rows, cols; } moe_tf_tensor;
+typedef struct {
+  int32_t op;
+  int32_t n_inputs, inputs[4];
+  int32_t n_outputs, outputs[2];
+  int32_t n_split_inputs, split_input_idx[4], split_input_dim[4];
+  int32_t split_output_dim[2];
+  int32_t task_rows;
+} moe_tf_operator;
+typedef struct { uint32_t slot, row_offset, rows, cols; } moe_tf_tdesc;
+typedef struct {
+  uint32_t task_type, queue_type;
+  uint32_t dependent_event, dependent_threshold, trigger_event;
+  uint32_t task_index, task_split_num, task_split_value;   /* tile index, tiles of the operator, rows per tile */
+  uint32_t tiling_data_position;                           /* index of the operator in the graph */
+  uint32_t n_inputs, n_outputs;
+  moe_tf_tdesc inputs[4], outputs[2];
+} moe_tf_td;
+int moe_taskflow_compile(const moe_tf_tensor* tensors, int32_t n_tensors, const moe_tf_operator* ops, int32_t n_ops,
+                         int32_t lag_rows, moe_tf_td* tds, int32_t td_cap, int32_t* n_tds, int32_t* n_events,
+                         int32_t* op_task_num, int32_t* tensor_split_dim, int32_t* tensor_split_num);
+size_t moe_taskflow_workspace_bytes(int32_t n_tds, int32_t n_events, int32_t n_tensors);
+int moe_taskflow_run(const moe_tf_td* tds, int32_t n_tds, int32_t n_events, void* const* slots, int32_t n_tensors,
+                     void* workspace, size_t workspace_bytes, int32_t upload, void* stream);
+int moe_taskflow_status(const void* workspace, int32_t* status2, void* stream);
+
 const char* moe_strerror(int code);
 /* Text of the last CUDA error a call on this thread ran into ("" if none). */
 const char* moe_last_cuda_error(void);

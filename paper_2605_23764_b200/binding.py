@@ -23,7 +23,8 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_set_profiling", "moe_get_phase_ms", "moe_route_host", "moe_layout_noalloc",
            "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace", "moe_debug_set_plain_launch",
            "moe_sched_study_workspace_bytes", "moe_sched_study", "moe_sched_study_stats", "moe_router_fwd",
-           "moe_router_bwd"]
+           "moe_router_bwd", "moe_taskflow_compile", "moe_taskflow_workspace_bytes", "moe_taskflow_run",
+           "moe_taskflow_status"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -35,6 +36,35 @@ class MoeShape(ctypes.Structure):
 
 class MoeError(RuntimeError):
     pass
+
+
+MOE_TF_SWIGLU, MOE_TF_ADD, MOE_TF_NO_EVENT = 1, 2, 0xFFFFFFFF
+
+
+class MoeTfTensor(ctypes.Structure):
+    _fields_ = [("rows", ctypes.c_int32), ("cols", ctypes.c_int32)]
+
+
+class MoeTfOperator(ctypes.Structure):
+    _fields_ = [("op", ctypes.c_int32), ("n_inputs", ctypes.c_int32), ("inputs", ctypes.c_int32 * 4),
+                ("n_outputs", ctypes.c_int32), ("outputs", ctypes.c_int32 * 2),
+                ("n_split_inputs", ctypes.c_int32), ("split_input_idx", ctypes.c_int32 * 4),
+                ("split_input_dim", ctypes.c_int32 * 4), ("split_output_dim", ctypes.c_int32 * 2),
+                ("task_rows", ctypes.c_int32)]
+
+
+class MoeTfTdesc(ctypes.Structure):
+    _fields_ = [("slot", ctypes.c_uint32), ("row_offset", ctypes.c_uint32), ("rows", ctypes.c_uint32),
+                ("cols", ctypes.c_uint32)]
+
+
+class MoeTfTd(ctypes.Structure):
+    _fields_ = [("task_type", ctypes.c_uint32), ("queue_type", ctypes.c_uint32), ("dependent_event", ctypes.c_uint32),
+                ("dependent_threshold", ctypes.c_uint32), ("trigger_event", ctypes.c_uint32),
+                ("task_index", ctypes.c_uint32), ("task_split_num", ctypes.c_uint32),
+                ("task_split_value", ctypes.c_uint32), ("tiling_data_position", ctypes.c_uint32),
+                ("n_inputs", ctypes.c_uint32), ("n_outputs", ctypes.c_uint32),
+                ("inputs", MoeTfTdesc * 4), ("outputs", MoeTfTdesc * 2)]
 
 
 _lib = None
@@ -78,6 +108,13 @@ def load_library() -> ctypes.CDLL:
     lib.moe_debug_set_plain_launch.argtypes = [vp, i32]
     lib.moe_router_fwd.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
     lib.moe_router_bwd.argtypes = [vp, vp, vp, vp, i32, vp, vp]
+    lib.moe_taskflow_compile.argtypes = [ctypes.POINTER(MoeTfTensor), i32, ctypes.POINTER(MoeTfOperator), i32, i32,
+                                         ctypes.POINTER(MoeTfTd), i32, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                         ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.moe_taskflow_workspace_bytes.restype = sz
+    lib.moe_taskflow_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.moe_taskflow_run.argtypes = [ctypes.POINTER(MoeTfTd), i32, i32, ctypes.POINTER(vp), i32, vp, sz, i32, vp]
+    lib.moe_taskflow_status.argtypes = [vp, ctypes.POINTER(i32), vp]
     lib.moe_sched_study_workspace_bytes.restype = sz
     lib.moe_sched_study_workspace_bytes.argtypes = [i32, i32]
     lib.moe_sched_study.argtypes = [i32, vp, vp, vp, vp, i32, i32, i32, vp, sz, vp]
@@ -332,6 +369,66 @@ def moe_sched_study_stats(workspace):
     _check(load_library().moe_sched_study_stats(ctypes.c_void_p(workspace.data_ptr()), st, ctypes.byref(ns),
                                                 ctypes.byref(n), _stream()), "moe_sched_study_stats")
     return (int(st[0]), int(st[1])), int(ns.value), int(n.value)
+
+
+def tf_operator(op, inputs, outputs, task_rows, split_inputs=None, split_output_dims=None):
+    """A graph node with its SplitSpec: split_inputs = None (partition origin) or [(input index, dim), ...]."""
+    o = MoeTfOperator()
+    o.op, o.n_inputs, o.n_outputs, o.task_rows = op, len(inputs), len(outputs), task_rows
+    for i, t in enumerate(inputs):
+        o.inputs[i] = t
+    for j, t in enumerate(outputs):
+        o.outputs[j] = t
+        o.split_output_dim[j] = 0 if split_output_dims is None else split_output_dims[j]
+    if split_inputs is None:
+        o.n_split_inputs = -1
+    else:
+        o.n_split_inputs = len(split_inputs)
+        for i, (idx, dim) in enumerate(split_inputs):
+            o.split_input_idx[i], o.split_input_dim[i] = idx, dim
+    return o
+
+
+def moe_taskflow_compile(tensors, ops, lag_rows, td_cap=None):
+    """tensors: [(rows, cols), ...]; ops: [MoeTfOperator, ...] -> dict(tds, n_tds, n_events, op_task_num,
+    tensor_split_dim, tensor_split_num).  Host only."""
+    ts = (MoeTfTensor * len(tensors))(*[MoeTfTensor(int(r), int(c)) for r, c in tensors])
+    os_ = (MoeTfOperator * len(ops))(*ops)
+    if td_cap is None:
+        td_cap = sum(max(1, -(-tensors[o.outputs[0]][0] // max(1, o.task_rows))) for o in ops)
+    tds = (MoeTfTd * max(1, td_cap))()
+    n_tds, n_ev = ctypes.c_int32(0), ctypes.c_int32(0)
+    tn = (ctypes.c_int32 * len(ops))()
+    sd, sn = (ctypes.c_int32 * len(tensors))(), (ctypes.c_int32 * len(tensors))()
+    _check(load_library().moe_taskflow_compile(ts, len(tensors), os_, len(ops), int(lag_rows), tds, td_cap,
+                                               ctypes.byref(n_tds), ctypes.byref(n_ev), tn, sd, sn), "moe_taskflow_compile")
+    return {"tds": tds, "n_tds": n_tds.value, "n_events": n_ev.value, "op_task_num": list(tn),
+            "tensor_split_dim": list(sd), "tensor_split_num": list(sn)}
+
+
+def moe_taskflow_workspace_bytes(n_tds, n_events, n_tensors) -> int:
+    return int(load_library().moe_taskflow_workspace_bytes(int(n_tds), int(n_events), int(n_tensors)))
+
+
+def moe_taskflow_run(plan, slots, shapes, workspace, upload=True):
+    """Run a compiled plan: slots = one CUDA bf16 tensor per graph tensor, shapes = the (rows, cols) the plan was
+    compiled for (each tensor must hold at least that many elements)."""
+    for i, (t, (r, c)) in enumerate(zip(slots, shapes)):
+        _need(t, r * c, f"slots[{i}]")
+        _dev(t, torch.bfloat16, f"slots[{i}]")
+    if len(slots) != len(shapes) or workspace is None or not workspace.is_cuda or not workspace.is_contiguous():
+        raise MoeError("slots / workspace: expected one CUDA tensor per graph tensor and a contiguous CUDA workspace")
+    ptrs = (ctypes.c_void_p * len(slots))(*[t.data_ptr() for t in slots])
+    nbytes = workspace.numel() * workspace.element_size()
+    _check(load_library().moe_taskflow_run(plan["tds"], plan["n_tds"], plan["n_events"], ptrs, len(slots),
+                                           ctypes.c_void_p(workspace.data_ptr()), nbytes, 1 if upload else 0, _stream()),
+           "moe_taskflow_run")
+
+
+def moe_taskflow_status(workspace):
+    st = (ctypes.c_int32 * 2)()
+    _check(load_library().moe_taskflow_status(ctypes.c_void_p(workspace.data_ptr()), st, _stream()), "moe_taskflow_status")
+    return int(st[0]), int(st[1])
 
 
 def moe_debug_simulate_schedule(counts, T, k, n_shared, d, F, is_bwd, pairs, vec_workers):
