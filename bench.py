@@ -548,6 +548,72 @@ def router_in_path(cfg, peaks, iters=30):
             "timing": "CUDA events around each call, L2 flushed before each; median of %d" % iters}
 
 
+def ep_emulated(cfg, peaks, R=8, iters=20):
+    """Expert-parallel Dispatch and Combine with one-sided put + signal (Section 4.1), the R ranks emulated on this one
+    GPU (all buffers local, one cooperative launch plays every rank): the workload's tokens split evenly over the ranks.
+    What is timed is the kernels' data path against local HBM; no NVLink is crossed."""
+    import numpy as np
+    from paper_2605_23764_b200 import MoeLayer, binding as B
+    dev = torch.device("cuda")
+    d, E, k = cfg.d, cfg.E, cfg.k
+    if E % R or cfg.T % R:
+        return None
+    Tr = cfg.T // R
+    g = torch.Generator(device="cuda").manual_seed(5)
+    i32 = dict(dtype=torch.int32, device=dev)
+    xs, ws, src, counts = [], [], [], []
+    lay = MoeLayer(Tr, d, E, k, 0, 128, renorm=True)
+    for s_ in range(R):
+        x = torch.randn(Tr, d, device=dev, generator=g).to(torch.bfloat16)
+        ids, w = lay.route(torch.randn(Tr, E, device=dev, generator=g))
+        c = torch.empty(E, **i32); o = torch.empty(E + 1, **i32); ro = torch.empty(Tr * k, **i32); so = torch.empty(Tr * k, **i32)
+        B.moe_layout(lay.ctx, ids, Tr, c, o, ro, so)
+        torch.cuda.synchronize()
+        xs.append(x); ws.append(w.clone()); src.append(so.clone()); counts.append(c.cpu().numpy())
+    lay.close()
+    counts = np.stack(counts).astype(np.int32)
+    plans = [B.moe_ep_plan(counts, s_) for s_ in range(R)]
+    rr = [int(v) for v in plans[0][1]]
+    recv = [torch.empty(n, d, dtype=torch.bfloat16, device=dev) for n in rr]
+    meta = [torch.empty(n, 4, **i32) for n in rr]
+    rcnt = [torch.zeros(-(-n // B.MOE_EP_BLOCK_ROWS), **i32) for n in rr]
+    ret = [torch.empty(Tr * k, d, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+    tcnt = [torch.zeros(-(-Tr // B.MOE_EP_TOKEN_BLOCK), **i32) for _ in range(R)]
+    peers = [B.moe_ep_peer(recv[q], meta[q], rcnt[q], ret[q], tcnt[q]) for q in range(R)]
+    tick = [torch.zeros(2, **i32) for _ in range(R)]
+    tasks = [torch.from_numpy(plans[s_][0]).to(dev) for s_ in range(R)]
+    out = [torch.empty(Tr, d, dtype=torch.bfloat16, device=dev) for _ in range(R)]
+    status = torch.zeros(4, **i32)
+    loc_d = [dict(rank=s_, T=Tr, x=xs[s_], topk_w=ws[s_], src_of=src[s_], tasks=tasks[s_], recv_rows=rr[s_], consumed=None,
+                  ticket=tick[s_]) for s_ in range(R)]
+    loc_c = [dict(rank=s_, T=Tr, recv_rows=rr[s_], y=recv[s_], out=out[s_], ticket=tick[s_]) for s_ in range(R)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def med(fn):
+        ts = []
+        for it in range(iters + 3):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        return sorted(ts)[len(ts) // 2]
+
+    us_d = med(lambda: B.moe_ep_dispatch(peers, loc_d, k, d, status))
+    us_c = med(lambda: B.moe_ep_combine(peers, loc_c, k, d, status))     # returns the received rows themselves: same bytes
+    if status.cpu().tolist()[:2] != [0, 0]:
+        raise SystemExit("ep emulation: device status")
+    rows = sum(rr)
+    by_d = 2.0 * cfg.T * d + 2.0 * rows * d + 16.0 * rows          # x once, every routed copy written once, its meta
+    by_c = 2.0 * rows * d * 3 + 2.0 * cfg.T * d                      # y read, ret written and read back, out written
+    return {"ranks": R, "tokens_per_rank": Tr, "rows": rows,
+            "dispatch": {"us": us_d, "GBps": by_d / us_d / 1e3, "frac_of_hbm_peak": by_d / us_d / 1e3 / peaks["hbm_gbs"]},
+            "combine": {"us": us_c, "GBps": by_c / us_c / 1e3, "frac_of_hbm_peak": by_c / us_c / 1e3 / peaks["hbm_gbs"]},
+            "note": "ranks emulated on one GPU: local HBM stands in for peer memory; at 8 GPUs 7/8 of the rows would cross "
+                    "NVLink (%.0f MB per GPU and direction)" % (2.0 * rows * d * 7 / 8 / R / 1e6)}
+
+
 def respawn_under_launcher(n):
     """`python bench.py --gpus N` without a launcher: start the N ranks (one per GPU) and pass their output on."""
     import socket
@@ -578,6 +644,7 @@ def main():
     ap.add_argument("--no-study", action="store_true", help="skip the SwiGLU+Add scheduling microbenchmark")
     ap.add_argument("--only-study", action="store_true", help="run the scheduling microbenchmark alone")
     ap.add_argument("--only-router", action="store_true", help="run the in-path router alone (on --config's shape)")
+    ap.add_argument("--only-ep", action="store_true", help="run the emulated expert-parallel dispatch / combine alone")
     ap.add_argument("--study-iters", type=int, default=30)
     ap.add_argument("--plain-launch", action="store_true",
                     help="diagnostic: persistent launches without the cooperative launch attribute (for profiler captures)")
@@ -605,6 +672,10 @@ def main():
         from paper_2605_23764_b200 import binding as B
         Workload.plain_launch = True
         B.moe_debug_set_plain_launch(None, True)
+    if args.only_ep:
+        torch.cuda.set_device(0)
+        print(json.dumps({"ep_emulated": ep_emulated(cfg, load_peaks(), iters=args.study_iters)}), flush=True)
+        return
     if args.only_router:
         torch.cuda.set_device(0)
         print(json.dumps({"router_in_path": router_in_path(cfg, load_peaks(), args.study_iters)}), flush=True)
@@ -686,6 +757,9 @@ def main():
     router = None
     if rank == 0 and world == 1 and not args.no_study:
         router = router_in_path(cfg, peaks, args.study_iters)
+    ep = None
+    if rank == 0 and world == 1 and not args.no_study and cfg.S == 0:
+        ep = ep_emulated(cfg, peaks, iters=args.study_iters)
 
     if rank == 0:
         desc = workload_desc(cfg, train)
@@ -700,7 +774,7 @@ def main():
             "config": desc, "clocks": res["clocks"], "e2e": e2e, "gpu_launches": res["launches"],
             "roofline": roofline, "step_roofline": step_roofline, "phases_ms": res["phases_ms"],
             "other_launch_mode": other, "all_configs": all_configs, "cpu_baseline": cpu_baseline,
-            "scheduling_study": study, "router_in_path": router,
+            "scheduling_study": study, "router_in_path": router, "ep_emulated": ep,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

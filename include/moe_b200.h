@@ -330,6 +330,71 @@ int moe_taskflow_run(const moe_tf_td* tds, int32_t n_tds, int32_t n_events, void
                      void* workspace, size_t workspace_bytes, int32_t upload, void* stream);
 int moe_taskflow_status(const void* workspace, int32_t* status2, void* stream);
 
+/* ---- Expert parallelism over peer memory: one-sided put + signal (Section 4.1 put_mem_signal and the
+ * taskization of the Dispatch / Combine AllToAll; Section 4.5 rank-aware task reordering) --------------------
+ * R ranks, expert e on rank e / (E / R).  Every rank exposes a moe_ep_peer: buffers in ITS memory that the other
+ * ranks write into with plain peer stores, each followed by a release-increment of a counter beside the buffer;
+ * the owner's consumers poll those counters locally.  No collective, no multicast load, no remote load.
+ *   recv[recv_rows][d] bf16: the rows of the rank's experts ordered by (expert, source rank, source slot t*k+j);
+ *   recv_meta[recv_rows][4] int32: source rank, source slot, routing weight (fp32 bits), 0;
+ *   recv_counters[ceil(recv_rows / MOE_EP_BLOCK_ROWS)]: rows that have arrived in each block of the receive buffer
+ *     (its threshold: the rows the block holds);
+ *   ret[T * k][d] bf16: expert outputs returned to the token's rank, indexed by slot;
+ *   ret_counters[ceil(T / MOE_EP_TOKEN_BLOCK)]: rows returned per block of tokens (threshold: tokens * k).
+ * All pointers in a moe_ep_peer must be valid device addresses ON THE CALLING DEVICE (peer mappings for remote
+ * ranks), 16-byte aligned; d % 8 == 0.
+ *
+ * moe_ep_plan (host only): from the all-gathered per-rank expert counts[R][E] it gives rank `rank` its list of
+ * communication tasks -- tiles of up to MOE_EP_TILE_ROWS rows of one expert: {expert, first local expert-ordered
+ * row, rows, destination rank, first destination row} -- in rank-rotated order (destinations rank+1, rank+2, ...,
+ * rank itself last), the rows every rank receives, and the first receive row of each of `rank`'s own experts.
+ *
+ * moe_ep_dispatch: for every rank in locals[] (one per process in a real deployment; all R in a single-GPU
+ * emulation, where one cooperative launch plays every rank) producer blocks take tasks by ticket, gather the
+ * task's rows of x (through src_of from moe_layout over all E experts, n_shared = 0) into the destination's recv
+ * and recv_meta, and signal the destination's recv_counters; consumer blocks of the same launch wait for each
+ * block's counter and copy the block into `consumed` (if not NULL) -- the stand-in for the grouped-GEMM tiles
+ * that would start on the block.  moe_ep_combine: producer blocks return each row of y (expert outputs in
+ * receive order) to ret[slot] of its source rank and signal ret_counters; consumer blocks wait per token block
+ * and write out[t] = sum_j ret[t*k+j] (fp32, slot order).
+ * The calls clear the counters, tickets and status of the ranks in locals[]: with more than one process the
+ * caller must place a barrier between two calls so that no rank signals a counter before its owner cleared it.
+ * status (device int32[4], cleared by the call): {code, detail, ..} = MOE_ERR_TIMEOUT if a bounded wait ran out.
+ * Returns MOE_OK / MOE_ERR_INVALID_ARG / MOE_ERR_WORKSPACE (task_cap) / MOE_ERR_NO_DEVICE / MOE_ERR_CUDA. */
+#define MOE_EP_MAX_RANKS 8
+#define MOE_EP_TILE_ROWS 32
+#define MOE_EP_BLOCK_ROWS 128
+#define MOE_EP_TOKEN_BLOCK 32
+typedef struct {
+  uint16_t* recv;
+  int32_t* recv_meta;
+  int32_t* recv_counters;
+  uint16_t* ret;
+  int32_t* ret_counters;
+} moe_ep_peer;
+typedef struct { int32_t expert, src_row0, nrows, dst_rank, dst_row0; } moe_ep_task;
+typedef struct {
+  int32_t rank, T, n_tasks, recv_rows;
+  const uint16_t* x;          /* [T][d] */
+  const float* topk_w;        /* [T][k] */
+  const int32_t* src_of;      /* [T*k] */
+  const moe_ep_task* tasks;   /* device copy of the plan's task list */
+  uint16_t* consumed;         /* [recv_rows][d] or NULL */
+  int32_t* ticket;            /* device int32[2]: task tickets of this rank */
+} moe_ep_local;
+typedef struct {
+  int32_t rank, T, recv_rows, pad;
+  const uint16_t* y;          /* [recv_rows][d] */
+  uint16_t* out;              /* [T][d] */
+  int32_t* ticket;            /* device int32[2] */
+} moe_ep_local_combine;
+int moe_ep_plan(const int32_t* counts, int32_t R, int32_t E, int32_t rank, moe_ep_task* tasks, int32_t task_cap,
+                int32_t* n_tasks, int32_t* recv_rows, int32_t* recv_expert_offsets);
+int moe_ep_dispatch(const moe_ep_peer* peers, const moe_ep_local* locals, int32_t n_local, int32_t R, int32_t k,
+                    int32_t d, int32_t* status, void* stream);
+int moe_ep_combine(const moe_ep_peer* peers, const moe_ep_local_combine* locals, int32_t n_local, int32_t R,
+                   int32_t k, int32_t d, int32_t* status, void* stream);
+
 const char* moe_strerror(int code);
 /* Text of the last CUDA error a call on this thread ran into ("" if none). */
 const char* moe_last_cuda_error(void);

@@ -24,7 +24,7 @@ EXPORTS = ["moe_workspace_bytes", "moe_create", "moe_destroy", "moe_route", "moe
            "moe_debug_simulate_schedule", "moe_debug_set_unreachable_dependency", "moe_debug_trace", "moe_debug_set_plain_launch",
            "moe_sched_study_workspace_bytes", "moe_sched_study", "moe_sched_study_stats", "moe_router_fwd",
            "moe_router_bwd", "moe_taskflow_compile", "moe_taskflow_workspace_bytes", "moe_taskflow_run",
-           "moe_taskflow_status"]
+           "moe_taskflow_status", "moe_ep_plan", "moe_ep_dispatch", "moe_ep_combine"]
 PHASES = ["route", "layout", "gather", "gemm_gate_up", "gemm_down", "combine", "bwd_gather", "act_grad",
           "dw_reduce", "wgrad_down", "gate_grad", "wgrad_gate_up", "bwd_combine", "fused_fwd", "fused_bwd"]
 
@@ -39,6 +39,28 @@ class MoeError(RuntimeError):
 
 
 MOE_TF_SWIGLU, MOE_TF_ADD, MOE_TF_NO_EVENT = 1, 2, 0xFFFFFFFF
+MOE_EP_TILE_ROWS, MOE_EP_BLOCK_ROWS, MOE_EP_TOKEN_BLOCK = 32, 128, 32
+
+
+class MoeEpPeer(ctypes.Structure):
+    _fields_ = [("recv", ctypes.c_void_p), ("recv_meta", ctypes.c_void_p), ("recv_counters", ctypes.c_void_p),
+                ("ret", ctypes.c_void_p), ("ret_counters", ctypes.c_void_p)]
+
+
+class MoeEpTask(ctypes.Structure):
+    _fields_ = [("expert", ctypes.c_int32), ("src_row0", ctypes.c_int32), ("nrows", ctypes.c_int32),
+                ("dst_rank", ctypes.c_int32), ("dst_row0", ctypes.c_int32)]
+
+
+class MoeEpLocal(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("T", ctypes.c_int32), ("n_tasks", ctypes.c_int32), ("recv_rows", ctypes.c_int32),
+                ("x", ctypes.c_void_p), ("topk_w", ctypes.c_void_p), ("src_of", ctypes.c_void_p),
+                ("tasks", ctypes.c_void_p), ("consumed", ctypes.c_void_p), ("ticket", ctypes.c_void_p)]
+
+
+class MoeEpLocalCombine(ctypes.Structure):
+    _fields_ = [("rank", ctypes.c_int32), ("T", ctypes.c_int32), ("recv_rows", ctypes.c_int32), ("pad", ctypes.c_int32),
+                ("y", ctypes.c_void_p), ("out", ctypes.c_void_p), ("ticket", ctypes.c_void_p)]
 
 
 class MoeTfTensor(ctypes.Structure):
@@ -115,6 +137,10 @@ def load_library() -> ctypes.CDLL:
     lib.moe_taskflow_workspace_bytes.argtypes = [i32, i32, i32]
     lib.moe_taskflow_run.argtypes = [ctypes.POINTER(MoeTfTd), i32, i32, ctypes.POINTER(vp), i32, vp, sz, i32, vp]
     lib.moe_taskflow_status.argtypes = [vp, ctypes.POINTER(i32), vp]
+    lib.moe_ep_plan.argtypes = [ctypes.POINTER(i32), i32, i32, i32, ctypes.POINTER(MoeEpTask), i32, ctypes.POINTER(i32),
+                                ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.moe_ep_dispatch.argtypes = [ctypes.POINTER(MoeEpPeer), ctypes.POINTER(MoeEpLocal), i32, i32, i32, i32, vp, vp]
+    lib.moe_ep_combine.argtypes = [ctypes.POINTER(MoeEpPeer), ctypes.POINTER(MoeEpLocalCombine), i32, i32, i32, i32, vp, vp]
     lib.moe_sched_study_workspace_bytes.restype = sz
     lib.moe_sched_study_workspace_bytes.argtypes = [i32, i32]
     lib.moe_sched_study.argtypes = [i32, vp, vp, vp, vp, i32, i32, i32, vp, sz, vp]
@@ -429,6 +455,65 @@ def moe_taskflow_status(workspace):
     st = (ctypes.c_int32 * 2)()
     _check(load_library().moe_taskflow_status(ctypes.c_void_p(workspace.data_ptr()), st, _stream()), "moe_taskflow_status")
     return int(st[0]), int(st[1])
+
+
+def moe_ep_plan(counts, rank):
+    """counts: int array [R][E] (every rank's per-expert row counts) -> (tasks [n][5] int32 numpy array: expert,
+    src_row0, nrows, dst_rank, dst_row0; recv_rows [R]; recv_expert_offsets [E/R+1] of `rank`).  Host only."""
+    import numpy as np
+    c = np.ascontiguousarray(counts, dtype=np.int32)
+    R, E = c.shape
+    cap = (int(c[rank].sum()) if 0 <= rank < R else 0) // MOE_EP_TILE_ROWS + E + 1
+    tasks = (MoeEpTask * cap)()
+    n = ctypes.c_int32(0)
+    rr = (ctypes.c_int32 * R)()
+    off = (ctypes.c_int32 * (E // max(R, 1) + 1))()
+    _check(load_library().moe_ep_plan(c.ctypes.data_as(ctypes.POINTER(ctypes.c_int32)), R, E, int(rank), tasks, cap,
+                                      ctypes.byref(n), rr, off), "moe_ep_plan")
+    arr = np.array([[t.expert, t.src_row0, t.nrows, t.dst_rank, t.dst_row0] for t in tasks[:n.value]],
+                   dtype=np.int32).reshape(n.value, 5)
+    return arr, np.array(list(rr), dtype=np.int32), np.array(list(off), dtype=np.int32)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def moe_ep_peer(recv, recv_meta, recv_counters, ret, ret_counters):
+    """What one rank exposes: CUDA tensors (bf16 recv/ret, int32 meta/counters) living on, or peer-mapped into, the
+    calling device."""
+    return MoeEpPeer(_ptr(recv).value if recv is not None else None, _ptr(recv_meta).value if recv_meta is not None else None,
+                     _ptr(recv_counters).value, _ptr(ret).value if ret is not None else None, _ptr(ret_counters).value)
+
+
+def moe_ep_dispatch(peers, locals_, k, d, status):
+    """peers: [MoeEpPeer] for every rank; locals_: [dict(rank, T, x, topk_w, src_of, tasks (CUDA int32 [n,5]), recv_rows,
+    consumed|None, ticket)] for the ranks this call acts for; status: CUDA int32[4]."""
+    R = len(peers)
+    ps = (MoeEpPeer * R)(*peers)
+    ls = (MoeEpLocal * len(locals_))()
+    for i, l in enumerate(locals_):
+        _need(l["x"], l["T"] * d, "x"); _need(l["topk_w"], l["T"] * k, "topk_w"); _need(l["src_of"], l["T"] * k, "src_of")
+        _need(l.get("consumed"), l["recv_rows"] * d, "consumed"); _need(l["ticket"], 2, "ticket")
+        n_tasks = 0 if l["tasks"] is None else l["tasks"].shape[0]
+        ls[i] = MoeEpLocal(l["rank"], l["T"], n_tasks, l["recv_rows"], _ptr(l["x"]), _ptr(l["topk_w"]), _ptr(l["src_of"]),
+                           _ptr(l["tasks"]), _ptr(l.get("consumed")), _ptr(l["ticket"]))
+    _need(status, 4, "status")
+    _check(load_library().moe_ep_dispatch(ps, ls, len(locals_), R, k, d, _dev(status, torch.int32, "status"), _stream()),
+           "moe_ep_dispatch")
+
+
+def moe_ep_combine(peers, locals_, k, d, status):
+    """locals_: [dict(rank, T, recv_rows, y, out, ticket)]."""
+    R = len(peers)
+    ps = (MoeEpPeer * R)(*peers)
+    ls = (MoeEpLocalCombine * len(locals_))()
+    for i, l in enumerate(locals_):
+        _need(l["y"], l["recv_rows"] * d, "y"); _need(l["out"], l["T"] * d, "out"); _need(l["ticket"], 2, "ticket")
+        ls[i] = MoeEpLocalCombine(l["rank"], l["T"], l["recv_rows"], 0, _ptr(l["y"]), _ptr(l["out"]), _ptr(l["ticket"]))
+    _need(status, 4, "status")
+    _check(load_library().moe_ep_combine(ps, ls, len(locals_), R, k, d, _dev(status, torch.int32, "status"), _stream()),
+           "moe_ep_combine")
 
 
 def moe_debug_simulate_schedule(counts, T, k, n_shared, d, F, is_bwd, pairs, vec_workers):

@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 OUT = os.path.join(PKG, "libmoe_b200.so")
 OBJ = os.path.join(PKG, "_build")
-SOURCES = ["api.cu", "route_layout.cu", "permute.cu", "gemm_tc2.cu", "gemm_tc3.cu", "gemm_wgrad.cu", "fused.cu", "study.cu", "router.cu", "taskflow.cu"]
+SOURCES = ["api.cu", "route_layout.cu", "permute.cu", "gemm_tc2.cu", "gemm_tc3.cu", "gemm_wgrad.cu", "fused.cu", "study.cu", "router.cu", "taskflow.cu", "ep.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
