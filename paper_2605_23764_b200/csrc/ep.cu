@@ -25,6 +25,19 @@ __device__ __forceinline__ uint4 ep_ld_cg(const void* p) {
   asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
+// The put half of put_mem_signal for one row: a warp copies nvec 16-byte vectors, eight loads in flight per lane.
+__device__ __forceinline__ void ep_put_row(uint4* dst, const uint4* src, int nvec, int lane) {
+  constexpr int U = 8;
+  for (int v0 = lane; v0 < nvec; v0 += 32 * U) {
+    uint4 t[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (v0 + 32 * u < nvec) t[u] = ep_ld_nc(src + v0 + 32 * u);
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+      if (v0 + 32 * u < nvec) dst[v0 + 32 * u] = t[u];
+  }
+}
 // The signal half of put_mem_signal: after the caller's stores to the destination (ordered before this by a
 // barrier among the storing threads), make them visible system-wide, then add to the destination's counter.
 __device__ __forceinline__ void ep_signal(int* counter, int inc) {
@@ -66,7 +79,7 @@ struct EpDispatchArgs {
 
 // Dispatch.  Producer block: one communication task at a time (rows of one expert bound for one rank), a warp per row.
 // Consumer block: the receive buffer of its rank, one 128-row block at a time, as soon as the block's rows have arrived.
-__global__ void __launch_bounds__(EP_THREADS) ep_dispatch_kernel(const __grid_constant__ EpDispatchArgs a) {
+__global__ void __launch_bounds__(EP_THREADS, 4) ep_dispatch_kernel(const __grid_constant__ EpDispatchArgs a) {
   const WaitCtl wc{a.status, a.budget_ns};
   const int li = blockIdx.x / a.blocks_per_rank, role = blockIdx.x % a.blocks_per_rank;
   const moe_ep_local& me = a.locals[li];
@@ -86,7 +99,7 @@ __global__ void __launch_bounds__(EP_THREADS) ep_dispatch_kernel(const __grid_co
         const int token = slot / a.k;
         const uint4* src = reinterpret_cast<const uint4*>(me.x + (size_t)token * a.d);
         uint4* out = reinterpret_cast<uint4*>(dst.recv + (size_t)(tk.dst_row0 + r) * a.d);
-        for (int v = lane; v < nvec; v += 32) out[v] = ep_ld_nc(src + v);
+        ep_put_row(out, src, nvec, lane);
         if (lane == 0)
           reinterpret_cast<int4*>(dst.recv_meta)[tk.dst_row0 + r] =
               make_int4(me.rank, slot, __float_as_int(me.topk_w[slot]), 0);
@@ -114,7 +127,15 @@ __global__ void __launch_bounds__(EP_THREADS) ep_dispatch_kernel(const __grid_co
       if (!ok_s) break;
       const uint4* src = reinterpret_cast<const uint4*>(mine.recv + (size_t)r0 * a.d);
       uint4* out = reinterpret_cast<uint4*>(me.consumed + (size_t)r0 * a.d);
-      for (int i = threadIdx.x; i < rows * nvec; i += EP_THREADS) out[i] = ep_ld_cg(src + i);
+      for (int i0 = threadIdx.x; i0 < rows * nvec; i0 += 4 * EP_THREADS) {
+        uint4 t[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (i0 + u * EP_THREADS < rows * nvec) t[u] = ep_ld_cg(src + i0 + u * EP_THREADS);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (i0 + u * EP_THREADS < rows * nvec) out[i0 + u * EP_THREADS] = t[u];
+      }
       __syncthreads();
     }
   }
@@ -133,7 +154,7 @@ struct EpCombineArgs {
 // source rank (a warp per row) with one signal per row; the tile list starts at a rank-dependent position so that the
 // ranks do not all return to the same source at once.  Consumer block: token blocks of its rank; once every row of a
 // block has come back, out[t] = sum over the token's k rows in slot order (fp32).
-__global__ void __launch_bounds__(EP_THREADS) ep_combine_kernel(const __grid_constant__ EpCombineArgs a) {
+__global__ void __launch_bounds__(EP_THREADS, 4) ep_combine_kernel(const __grid_constant__ EpCombineArgs a) {
   const WaitCtl wc{a.status, a.budget_ns};
   const int li = blockIdx.x / a.blocks_per_rank, role = blockIdx.x % a.blocks_per_rank;
   const moe_ep_local_combine& me = a.locals[li];
@@ -161,7 +182,7 @@ __global__ void __launch_bounds__(EP_THREADS) ep_combine_kernel(const __grid_con
         const moe_ep_peer& dst = a.peers.p[m.x];
         const uint4* src = reinterpret_cast<const uint4*>(me.y + (size_t)(p0 + r) * a.d);
         uint4* out = reinterpret_cast<uint4*>(dst.ret + (size_t)m.y * a.d);
-        for (int v = lane; v < nvec; v += 32) out[v] = ep_ld_nc(src + v);
+        ep_put_row(out, src, nvec, lane);
         __syncwarp();
         if (lane == 0) ep_signal(dst.ret_counters + (m.y / a.k) / MOE_EP_TOKEN_BLOCK, 1);
       }
@@ -179,12 +200,20 @@ __global__ void __launch_bounds__(EP_THREADS) ep_combine_kernel(const __grid_con
           float acc[8];
 #pragma unroll
           for (int q = 0; q < 8; ++q) acc[q] = 0.f;
-          for (int j = 0; j < a.k; ++j) {
-            const uint4 r = ep_ld_cg(reinterpret_cast<const uint4*>(mine.ret + ((size_t)t * a.k + j) * a.d) + v);
-            acc[0] += bf16lo(r.x); acc[1] += bf16hi(r.x);
-            acc[2] += bf16lo(r.y); acc[3] += bf16hi(r.y);
-            acc[4] += bf16lo(r.z); acc[5] += bf16hi(r.z);
-            acc[6] += bf16lo(r.w); acc[7] += bf16hi(r.w);
+          for (int j0 = 0; j0 < a.k; j0 += 8) {   // eight of the token's rows in flight; summed in slot order
+            uint4 rr[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              if (j0 + u < a.k) rr[u] = ep_ld_cg(reinterpret_cast<const uint4*>(mine.ret + ((size_t)t * a.k + j0 + u) * a.d) + v);
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+              if (j0 + u < a.k) {
+                const uint4 r = rr[u];
+                acc[0] += bf16lo(r.x); acc[1] += bf16hi(r.x);
+                acc[2] += bf16lo(r.y); acc[3] += bf16hi(r.y);
+                acc[4] += bf16lo(r.z); acc[5] += bf16hi(r.z);
+                acc[6] += bf16lo(r.w); acc[7] += bf16hi(r.w);
+              }
           }
           uint4 o;
           o.x = pack_bf16x2(acc[0], acc[1]); o.y = pack_bf16x2(acc[2], acc[3]);
@@ -204,7 +233,7 @@ static int ep_grid(const void* kernel, int n_local, int* blocks_per_rank, int* p
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, EP_THREADS, 0) != cudaSuccess || per_sm < 1)
     return MOE_ERR_CUDA;
-  int total = sms * (per_sm < 2 ? per_sm : 2);
+  int total = sms * (per_sm < 4 ? per_sm : 4);
   int bpr = total / n_local;
   if (bpr < 2) return MOE_ERR_TOO_LARGE;
   *blocks_per_rank = bpr;
