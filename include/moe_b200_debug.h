@@ -48,7 +48,8 @@ int moe_debug_set_unreachable_dependency(moe_ctx* ctx, int32_t on);
  * launch attribute (some profilers reject cooperative launches of thread-block clusters).  The grid is
  * sized to what can be resident either way; what is lost is the driver's guarantee of co-residency when
  * other work shares the GPU -- every device-side wait stays bounded.  ctx == NULL switches the persistent
- * launches of moe_sched_study (process-wide) instead. */
+ * launches of the context-free entry points (moe_sched_study, moe_taskflow_run, moe_ep_dispatch, moe_ep_combine;
+ * process-wide) instead. */
 int moe_debug_set_plain_launch(moe_ctx* ctx, int32_t on);
 
 /* Host-only check of the static tile schedule of the single persistent launch (Section 4.3: tasks

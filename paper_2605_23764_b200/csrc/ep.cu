@@ -25,17 +25,44 @@ __device__ __forceinline__ uint4 ep_ld_cg(const void* p) {
   asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
+// L2 policies: a token row is read once per routed copy (k times, at different moments) while k times as many bytes
+// stream out, so the source rows ask to stay in L2 and the stores ask to leave it first.
+__device__ __forceinline__ uint64_t ep_policy_keep() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint64_t ep_policy_stream() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ uint4 ep_ld_hint(const void* p, uint64_t policy) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p), "l"(policy));
+  return v;
+}
+__device__ __forceinline__ void ep_st_hint(void* p, uint4 v, uint64_t policy) {
+  asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w),
+               "l"(policy)
+               : "memory");
+}
 // The put half of put_mem_signal for one row: a warp copies nvec 16-byte vectors, eight loads in flight per lane.
+// KEEP_SRC: the source row will be read again soon (Dispatch: the token's other copies).
+template <bool KEEP_SRC>
 __device__ __forceinline__ void ep_put_row(uint4* dst, const uint4* src, int nvec, int lane) {
   constexpr int U = 8;
+  const uint64_t keep = ep_policy_keep(), stream = ep_policy_stream();
   for (int v0 = lane; v0 < nvec; v0 += 32 * U) {
     uint4 t[U];
 #pragma unroll
     for (int u = 0; u < U; ++u)
-      if (v0 + 32 * u < nvec) t[u] = ep_ld_nc(src + v0 + 32 * u);
+      if (v0 + 32 * u < nvec) t[u] = KEEP_SRC ? ep_ld_hint(src + v0 + 32 * u, keep) : ep_ld_nc(src + v0 + 32 * u);
 #pragma unroll
     for (int u = 0; u < U; ++u)
-      if (v0 + 32 * u < nvec) dst[v0 + 32 * u] = t[u];
+      if (v0 + 32 * u < nvec) ep_st_hint(dst + v0 + 32 * u, t[u], stream);
   }
 }
 // The signal half of put_mem_signal: after the caller's stores to the destination (ordered before this by a
@@ -99,7 +126,7 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_dispatch_kernel(const __grid
         const int token = slot / a.k;
         const uint4* src = reinterpret_cast<const uint4*>(me.x + (size_t)token * a.d);
         uint4* out = reinterpret_cast<uint4*>(dst.recv + (size_t)(tk.dst_row0 + r) * a.d);
-        ep_put_row(out, src, nvec, lane);
+        ep_put_row<true>(out, src, nvec, lane);
         if (lane == 0)
           reinterpret_cast<int4*>(dst.recv_meta)[tk.dst_row0 + r] =
               make_int4(me.rank, slot, __float_as_int(me.topk_w[slot]), 0);
@@ -182,7 +209,7 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_combine_kernel(const __grid_
         const moe_ep_peer& dst = a.peers.p[m.x];
         const uint4* src = reinterpret_cast<const uint4*>(me.y + (size_t)(p0 + r) * a.d);
         uint4* out = reinterpret_cast<uint4*>(dst.ret + (size_t)m.y * a.d);
-        ep_put_row(out, src, nvec, lane);
+        ep_put_row<false>(out, src, nvec, lane);
         __syncwarp();
         if (lane == 0) ep_signal(dst.ret_counters + (m.y / a.k) / MOE_EP_TOKEN_BLOCK, 1);
       }
@@ -328,7 +355,9 @@ int moe_ep_dispatch(const moe_ep_peer* peers, const moe_ep_local* locals, int32_
   if (rc) return rc;
   void* params[] = {&a};
   // cooperative: consumer blocks wait for producer blocks of the same launch
-  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(a.blocks_per_rank * n_local), dim3(EP_THREADS), params, 0, st);
+  cudaError_t e = study_plain_launch().load()   // profiling aid, see moe_debug_set_plain_launch(NULL, ..)
+                      ? cudaLaunchKernel(fn, dim3(a.blocks_per_rank * n_local), dim3(EP_THREADS), params, 0, st)
+                      : cudaLaunchCooperativeKernel(fn, dim3(a.blocks_per_rank * n_local), dim3(EP_THREADS), params, 0, st);
   return e == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
@@ -363,7 +392,9 @@ int moe_ep_combine(const moe_ep_peer* peers, const moe_ep_local_combine* locals,
   int rc = ep_grid(fn, n_local, &a.blocks_per_rank, &a.producers_per_rank);
   if (rc) return rc;
   void* params[] = {&a};
-  cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(a.blocks_per_rank * n_local), dim3(EP_THREADS), params, 0, st);
+  cudaError_t e = study_plain_launch().load()
+                      ? cudaLaunchKernel(fn, dim3(a.blocks_per_rank * n_local), dim3(EP_THREADS), params, 0, st)
+                      : cudaLaunchCooperativeKernel(fn, dim3(a.blocks_per_rank * n_local), dim3(EP_THREADS), params, 0, st);
   return e == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 

@@ -45,7 +45,7 @@ constexpr int GATHER_SUB = 32;         // vector sub-tasks per M-block gather (4
                                        // launch, which every CTA pair waits for, are complete after a few microseconds)
 constexpr int EPI_WARPS = 4;           // epilogue warps per CTA
 constexpr int SIG = 2 * EPI_WARPS;     // signals per (M-block, column tile): every epilogue warp of the pair
-constexpr int COMBINE_TOKENS = 2;      // tokens per combine task
+constexpr int COMBINE_TOKENS = 1;      // tokens per combine task
 
 enum VecOp : int { VEC_GATHER = 0, VEC_DW = 2, VEC_COMBINE = 3 };
 
