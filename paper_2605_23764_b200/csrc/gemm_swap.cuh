@@ -191,9 +191,17 @@ __device__ __forceinline__ void epilogue_swap(const GemmArgs& a, const SwapTile&
       tmem_ld16(trow + c0 + 16, v + 16);
       tmem_ld_wait();
       uint8_t* box = sw_acquire(sg, lane);
-      uint16_t* col = reinterpret_cast<uint16_t*>(box) + lane;   // [32 tokens][32 features]
+      // [32 tokens][32 features].  Neighbouring lanes (features 2i, 2i+1) swap one value per token pair, so that
+      // every lane stores 4 bytes: the even lane the feature pair of token j, the odd lane that of token j+1 -- 128
+      // contiguous bytes per warp store instead of 64.
+      uint32_t* box32 = reinterpret_cast<uint32_t*>(box) + (lane >> 1);
+      const bool odd = lane & 1;
 #pragma unroll
-      for (int j = 0; j < 32; ++j) col[j * 32] = bf16_bits(v[j]);
+      for (int j = 0; j < 32; j += 2) {
+        const float send = odd ? v[j] : v[j + 1];
+        const float recv = __shfl_xor_sync(0xffffffffu, send, 1);
+        box32[(j + (odd ? 1 : 0)) * 16] = odd ? pack_bf16x2(recv, v[j + 1]) : pack_bf16x2(v[j], recv);
+      }
       staging_release();
       if (lane == 0) {
         tma_store_2d(&a.tmOut0, f0, st.row0 + c0, box);
