@@ -3,6 +3,7 @@
 // HBM-bandwidth work: 16-byte vector accesses, one row handled by one block at a time.
 #include <stdlib.h>
 
+#include "launch_pairs.cuh"
 #include "moe_internal.h"
 
 namespace moe {
@@ -153,23 +154,23 @@ cudaError_t launch_gather(const uint16_t* src, const float* topk_w, const Dims& 
   const size_t row_bytes = (size_t)dm.d * 2;
   int lanes = (int)((GB_SMEM_BUDGET - row_bytes) / (2 * row_bytes));
   if (lanes > GB_MAX_LANES) lanes = GB_MAX_LANES;
-  static int bulk = -1;   // diagnostic knob: MOE_B200_GATHER_THREADS=1 keeps the copy in registers
-  if (bulk < 0) {
-    const char* e = getenv("MOE_B200_GATHER_THREADS");
-    bulk = (e && e[0] == '1') ? 0 : 1;
-  }
   // rows of 8 KB and more: below that the per-row latency of the two-slot pipelines outweighs the gain
-  if (bulk && status && lanes >= 2 && row_bytes >= 8192 && row_bytes % 16 == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
+  if (status && lanes >= 2 && row_bytes >= 8192 && row_bytes % 16 == 0 && ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) == 0) {
     const size_t smem = row_bytes * (1 + 2 * (size_t)lanes);
-    static size_t attr_bytes = 0;
-    if (smem > attr_bytes) {
-      cudaError_t e = cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-      if (e != cudaSuccess) return e;
-      attr_bytes = smem;
-    }
     int sms = 148;
     int dev = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    {   // the opt-in shared-memory size is a per-device attribute of the kernel: remember it per device, under a lock
+      static std::mutex mu;
+      static size_t attr_bytes[MAX_DEVICES] = {};
+      std::lock_guard<std::mutex> lock(mu);
+      if (smem > attr_bytes[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(gather_rows_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        attr_bytes[dev] = smem;
+      }
+    }
     gather_rows_bulk_kernel<<<sms, 32, smem, s>>>(src, topk_w, dm.d, dm.k, dm.kp(), lv, dst, prow_w, lanes, status,
                                                   budget_ns);
     return cudaGetLastError();
