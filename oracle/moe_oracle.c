@@ -130,6 +130,60 @@ int moe_oracle_router_bwd(const float* logits, const int32_t* ids, const double*
   return 0;
 }
 
+/* ---- sigmoid gating (a routing variant; the paper's router description, Section 2.2, fixes no score function):
+ * score s_e = 1 / (1 + exp(-l_e)) per expert, independent of the other experts; the k experts are still the k
+ * largest raw logits (the sigmoid is monotone), ties to the lower id, slots in descending order;
+ * w_j = s_{e_j}, or s_{e_j} / sum_{i in S} s_{e_i} with renormalisation. ---- */
+int moe_oracle_route_sigmoid(const float* logits, int T, int E, int k, int renorm, int32_t* topk_ids, double* topk_w) {
+  if (k < 1 || k > E) return -1;
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    const float* l = logits + (size_t)t * E;
+    double wsum = 0.0;
+    for (int j = 0; j < k; ++j) {
+      int best = -1;
+      for (int e = 0; e < E; ++e) {
+        int taken = 0;
+        for (int jj = 0; jj < j; ++jj) if (topk_ids[(size_t)t * k + jj] == e) taken = 1;
+        if (taken) continue;
+        if (best < 0 || l[e] > l[best]) best = e;
+      }
+      topk_ids[(size_t)t * k + j] = best;
+      const double s = 1.0 / (1.0 + exp(-(double)l[best]));
+      topk_w[(size_t)t * k + j] = s;
+      wsum += s;
+    }
+    if (renorm)
+      for (int j = 0; j < k; ++j) topk_w[(size_t)t * k + j] /= wsum;
+  }
+  return 0;
+}
+
+/* Gradient of the sigmoid-gated scores w.r.t. the logits, g = dL/d topk_w; s' = s (1 - s).
+ *   without renormalisation  dL/dl[e_j] = g_j s_j (1 - s_j)
+ *   with renormalisation     w_j = s_j / Z, Z = sum_i s_i:  dL/dl[e_i] = s_i (1 - s_i) / Z * (g_i - sum_j g_j w_j)
+ * Experts outside the selection get 0 in both cases. */
+int moe_oracle_router_bwd_sigmoid(const float* logits, const int32_t* ids, const double* g, int T, int E, int k,
+                                  int renorm, double* dlogits) {
+  if (k < 1 || k > E) return -1;
+#pragma omp parallel for schedule(static)
+  for (int t = 0; t < T; ++t) {
+    const float* l = logits + (size_t)t * E;
+    const int32_t* id = ids + (size_t)t * k;
+    const double* gt = g + (size_t)t * k;
+    double* dl = dlogits + (size_t)t * E;
+    for (int e = 0; e < E; ++e) dl[e] = 0.0;
+    double Z = 0.0, dot = 0.0;
+    for (int j = 0; j < k; ++j) Z += 1.0 / (1.0 + exp(-(double)l[id[j]]));
+    for (int j = 0; j < k; ++j) dot += gt[j] * (1.0 / (1.0 + exp(-(double)l[id[j]]))) / Z;
+    for (int j = 0; j < k; ++j) {
+      const double s = 1.0 / (1.0 + exp(-(double)l[id[j]]));
+      dl[id[j]] += renorm ? s * (1.0 - s) / Z * (gt[j] - dot) : gt[j] * s * (1.0 - s);
+    }
+  }
+  return 0;
+}
+
 /* expert id of flat slot i = t*(k+S)+j: routed slots first, then the S shared experts */
 static inline int slot_expert(const int32_t* ids, int k, int S, int E, int t, int j) {
   return j < k ? ids[(size_t)t * k + j] : E + (j - k);

@@ -42,6 +42,8 @@ def _load():
         lib.moe_oracle_swiglu_add.argtypes = [f64p, f64p, ci, ci, f64p, f64p]
         lib.moe_oracle_router_logits.argtypes = [f64p, f64p, ci, ci, ci, f64p]
         lib.moe_oracle_router_bwd.argtypes = [f32p, i32p, f64p, ci, ci, ci, ci, f64p]
+        lib.moe_oracle_route_sigmoid.argtypes = [f32p, ci, ci, ci, ci, i32p, f64p]
+        lib.moe_oracle_router_bwd_sigmoid.argtypes = [f32p, i32p, f64p, ci, ci, ci, ci, f64p]
         _lib = lib
     return _lib
 
@@ -65,13 +67,15 @@ def threads() -> int:
     return int(_load().moe_oracle_threads())
 
 
-def route(logits, k: int, renorm: bool):
-    """Top-k routing scores (Section 2.2, router description).  -> ids int32 [T,k], w float64 [T,k]."""
+def route(logits, k: int, renorm: bool, gate: str = "softmax"):
+    """Top-k routing scores (Section 2.2, router description).  gate = "softmax" (scores over all E experts) or
+    "sigmoid" (per-expert scores).  -> ids int32 [T,k], w float64 [T,k]."""
     l = _np(logits, np.float32)
     T, E = l.shape
     ids = np.empty((T, k), np.int32)
     w = np.empty((T, k), np.float64)
-    rc = _load().moe_oracle_route(_p(l, ctypes.c_float), T, E, k, int(bool(renorm)),
+    fn = {"softmax": _load().moe_oracle_route, "sigmoid": _load().moe_oracle_route_sigmoid}[gate]
+    rc = fn(_p(l, ctypes.c_float), T, E, k, int(bool(renorm)),
                                   _p(ids, ctypes.c_int32), _p(w, ctypes.c_double))
     if rc:
         raise ValueError(f"moe_oracle_route failed ({rc})")
@@ -180,15 +184,15 @@ def router_logits(x, W_r):
     return out
 
 
-def router_fwd(x, W_r, k: int, renorm: bool):
+def router_fwd(x, W_r, k: int, renorm: bool, gate: str = "softmax"):
     """Router in the path: logits in fp64, rounded once to fp32 (the precision the CUDA path decides in), then
     `route`.  -> ids int32 [T,k], w float64 [T,k], logits float64 [T,E] (unrounded)."""
     logits = router_logits(x, W_r)
-    ids, w = route(logits.astype(np.float32), k, renorm)
+    ids, w = route(logits.astype(np.float32), k, renorm, gate)
     return ids, w, logits
 
 
-def router_bwd(logits, ids, d_topk_w, renorm: bool):
+def router_bwd(logits, ids, d_topk_w, renorm: bool, gate: str = "softmax"):
     """Gradient of the k routing scores w.r.t. the logits (softmax over all E, optional renormalisation over the
     selected experts; no gradient through the selection).  -> d_logits float64 [T,E]."""
     l = _np(logits, np.float32)
@@ -198,7 +202,8 @@ def router_bwd(logits, ids, d_topk_w, renorm: bool):
     k = ids.shape[1]
     assert ids.shape == (T, k) and g.shape == (T, k)
     out = np.empty((T, E), np.float64)
-    rc = _load().moe_oracle_router_bwd(_p(l, ctypes.c_float), _p(ids, ctypes.c_int32), _p(g, ctypes.c_double), T, E, k,
+    fn = {"softmax": _load().moe_oracle_router_bwd, "sigmoid": _load().moe_oracle_router_bwd_sigmoid}[gate]
+    rc = fn(_p(l, ctypes.c_float), _p(ids, ctypes.c_int32), _p(g, ctypes.c_double), T, E, k,
                                        int(bool(renorm)), _p(out, ctypes.c_double))
     if rc:
         raise ValueError(f"moe_oracle_router_bwd failed ({rc})")

@@ -77,3 +77,46 @@ def test_router_bwd_finite_differences_of_the_scores():
             lp[t, e] += h; lm[t, e] -= h
             fd = ((scores(lp) - scores(lm)) * g).sum() / (2 * h)
             assert abs(fd - got[t, e]) <= 1e-8 * max(1.0, abs(fd))
+
+
+# ---- sigmoid gating variant
+@pytest.mark.parametrize("renorm", [False, True])
+def test_sigmoid_route_matches_torch_sigmoid_topk(renorm):
+    rng = np.random.default_rng(12)
+    logits = (rng.normal(size=(40, 16)) * 2).astype(np.float32)
+    ids, w = oracle.route(logits, 4, renorm, gate="sigmoid")
+    l = torch.from_numpy(logits).double()
+    ref = torch.topk(l, 4, dim=1)
+    assert np.array_equal(ids, ref.indices.numpy().astype(np.int32))           # same selection as the softmax gate
+    assert np.array_equal(ids, oracle.route(logits, 4, renorm)[0])
+    s = torch.sigmoid(ref.values)
+    if renorm:
+        s = s / s.sum(1, keepdim=True)
+    np.testing.assert_allclose(w, s.numpy(), rtol=1e-14)
+    # closed forms: l = 0 -> 1/2, l = ln 3 -> 3/4; per-expert scores do not depend on the other logits
+    one = np.array([[0.0, np.log(3.0), -50.0, -60.0]], dtype=np.float32)
+    _, w1 = oracle.route(one, 2, False, gate="sigmoid")
+    np.testing.assert_allclose(w1, [[0.75, 0.5]], rtol=1e-7)
+    other = one.copy(); other[0, 2] = -1.0
+    np.testing.assert_array_equal(oracle.route(other, 2, False, gate="sigmoid")[1], w1)
+
+
+@pytest.mark.parametrize("renorm", [False, True])
+@pytest.mark.parametrize("T,E,k", [(9, 8, 2), (5, 16, 6), (6, 7, 1)])
+def test_sigmoid_router_bwd_matches_autograd(T, E, k, renorm):
+    rng = np.random.default_rng(3 * T + E + k)
+    logits = rng.normal(size=(T, E)).astype(np.float32)
+    ids, _ = oracle.route(logits, k, renorm, gate="sigmoid")
+    g = rng.normal(size=(T, k))
+    got = oracle.router_bwd(logits, ids, g, renorm, gate="sigmoid")
+    l = torch.tensor(logits, dtype=torch.float64, requires_grad=True)
+    s = torch.sigmoid(l).gather(1, torch.from_numpy(ids.astype(np.int64)))
+    if renorm:
+        s = s / s.sum(1, keepdim=True)
+    (s * torch.from_numpy(g)).sum().backward()
+    np.testing.assert_allclose(got, l.grad.numpy(), rtol=1e-11, atol=1e-14)
+    mask = np.ones((T, E), bool)
+    np.put_along_axis(mask, ids.astype(np.int64), False, axis=1)
+    assert np.all(got[mask] == 0.0)
+    if renorm and k == 1:
+        assert np.all(np.abs(got) < 1e-15)
