@@ -63,6 +63,8 @@ enum {
   MOE_FLAG_SERIAL_LAUNCH = 4u, /* run the layer as one kernel launch per operator (the paper's
                                   operator-by-operator baseline, Section 5.2) instead of the
                                   single persistent dependency-driven launch */
+  MOE_FLAG_SIGMOID_GATE = 16u, /* routing scores are per-expert sigmoids of the logits instead of a softmax over all
+                                  experts (moe_route, moe_router_fwd, moe_router_bwd); selection rule unchanged */
   MOE_FLAG_TRACE = 8u,         /* the persistent launches record a per-tile trace (role, phase, item,
                                   start and end time) into the workspace; read it with
                                   moe_debug_trace (moe_b200_debug.h).  Costs 8 MB of workspace and one
@@ -97,7 +99,8 @@ int moe_destroy(moe_ctx* ctx);
 /* Router scores -> top-k (Section 2.2, first paragraph).  logits[T][E] fp32.
  * topk_ids[T][k]: the k largest raw logits, ties to the lower expert id, slots in descending
  * logit order.  topk_w[T][k]: softmax over all E of the selected experts, renormalised over
- * the k when MOE_FLAG_RENORM_TOPK is set.  counts[E] (may be NULL): tokens per routed expert. */
+ * the k when MOE_FLAG_RENORM_TOPK is set (with MOE_FLAG_SIGMOID_GATE: w = 1 / (1 + exp(-logit)) of each selected
+ * expert, renormalised over the k the same way).  counts[E] (may be NULL): tokens per routed expert. */
 int moe_route(moe_ctx* ctx, const float* logits, int32_t T, int32_t* topk_ids, float* topk_w,
               int32_t* counts, void* stream);
 
@@ -228,6 +231,8 @@ int moe_layout_noalloc(const int32_t* topk_ids, int32_t T, int32_t E, int32_t k,
  *   without renormalisation  d_logits[t][e] = [e = e_j] g_j p_e - p_e * sum_j g_j p_{e_j}
  *   with renormalisation     d_logits[t][e_j] = w_j (g_j - sum_i g_i w_i), 0 for experts not selected.
  *   logits[T][E] fp32, topk_ids[T][k], d_topk_w[T][k] fp32 -> d_logits[T][E] fp32 (all device pointers).
+ * With MOE_FLAG_SIGMOID_GATE (s = sigmoid of the logit, Z = sum of the selected s): without renormalisation
+ * d_logits[t][e_j] = g_j s_j (1 - s_j); with it d_logits[t][e_j] = s_j (1 - s_j) / Z * (g_j - sum_i g_i w_i); 0 elsewhere.
  * The two dense products that follow (d_logits^T x for the router weights, d_logits W_r for x) are plain
  * GEMMs outside this library.  Limit: k <= 32.  Both calls are asynchronous on `stream`. */
 int moe_router_fwd(moe_ctx* ctx, const uint16_t* x, const uint16_t* W_r, int32_t T, int32_t* topk_ids,

@@ -467,6 +467,9 @@ cudaError_t launch_gemm_serial(const moe_ctx* c, GemmMode mode, const GemmArgs& 
 
 // One launch per operator: on request, and for shapes the persistent launch does not cover (it runs the
 // token-column tiles only).
+int gate_mode(const moe_ctx* c) {
+  return ((c->shape.flags & MOE_FLAG_RENORM_TOPK) ? GATE_RENORM : 0) | ((c->shape.flags & MOE_FLAG_SIGMOID_GATE) ? GATE_SIGMOID : 0);
+}
 bool serial_mode(const moe_ctx* c) { return (c->shape.flags & MOE_FLAG_SERIAL_LAUNCH) != 0 || !token_col_tiles(c); }
 
 ChainParams chain_params(const moe_ctx* c, bool bwd, int T, bool want_dw) {
@@ -816,7 +819,7 @@ int moe_route(moe_ctx* c, const float* logits, int32_t T, int32_t* topk_ids, flo
   if (!c || !logits || !topk_ids || !topk_w || T < 0 || T > c->shape.T_max) return MOE_ERR_INVALID_ARG;
   c->begin_call(static_cast<cudaStream_t>(stream));
   Phase ph(c, MOE_PHASE_ROUTE, c->last_stream);
-  MOE_CUDA(launch_route(logits, T, c->shape.E, c->shape.k, (c->shape.flags & MOE_FLAG_RENORM_TOPK) != 0, topk_ids,
+  MOE_CUDA(launch_route(logits, T, c->shape.E, c->shape.k, gate_mode(c), topk_ids,
                         topk_w, counts, c->last_stream, &c->launches));
   return MOE_OK;
 }
@@ -835,7 +838,7 @@ int moe_router_fwd(moe_ctx* c, const uint16_t* x, const uint16_t* W_r, int32_t T
   a.T = T; a.E = s.E; a.k = s.k; a.d = s.d;
   a.N = ((s.E + 15) / 16) * 16;
   if (a.N < 32) a.N = 32;
-  a.renorm = (s.flags & MOE_FLAG_RENORM_TOPK) != 0;
+  a.renorm = gate_mode(c);
   a.topk_ids = topk_ids; a.topk_w = topk_w; a.logits = logits; a.counts = counts;
   a.status = c->status();
   a.budget_ns = c->budget_ns;
@@ -853,7 +856,7 @@ int moe_router_bwd(moe_ctx* c, const float* logits, const int32_t* topk_ids, con
   const moe_shape& s = c->shape;
   if (s.k > 32) return MOE_ERR_TOO_LARGE;
   c->begin_call(static_cast<cudaStream_t>(stream));
-  MOE_CUDA(launch_router_bwd(logits, topk_ids, d_topk_w, T, s.E, s.k, (s.flags & MOE_FLAG_RENORM_TOPK) != 0, d_logits,
+  MOE_CUDA(launch_router_bwd(logits, topk_ids, d_topk_w, T, s.E, s.k, gate_mode(c), d_logits,
                              c->last_stream, &c->launches));
   return MOE_OK;
 }
@@ -871,7 +874,7 @@ int moe_route_host(moe_ctx* c, const float* logits_host, int32_t T, int32_t* top
                            cudaMemcpyHostToDevice, st));
   {
     Phase ph(c, MOE_PHASE_ROUTE, st);
-    MOE_CUDA(launch_route(c->at<float>(p.st_logits), T, s.E, s.k, (s.flags & MOE_FLAG_RENORM_TOPK) != 0,
+    MOE_CUDA(launch_route(c->at<float>(p.st_logits), T, s.E, s.k, gate_mode(c),
                           c->at<int32_t>(p.st_ids), c->at<float>(p.st_w), nullptr, st, &c->launches));
   }
   MOE_CUDA(cudaMemcpyAsync(topk_ids_host, c->ws + p.st_ids, sizeof(int) * (size_t)T * s.k, cudaMemcpyDeviceToHost,

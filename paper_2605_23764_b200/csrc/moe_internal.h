@@ -50,7 +50,9 @@ struct LayoutView {
 };
 
 // ---- route_layout.cu
-cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, int* topk_ids, float* topk_w,
+// gate_mode: bit 0 = renormalise the k scores, bit 1 = sigmoid scores instead of softmax (GATE_RENORM, GATE_SIGMOID)
+constexpr int GATE_RENORM = 1, GATE_SIGMOID = 2;
+cudaError_t launch_route(const float* logits, int T, int E, int k, int gate_mode, int* topk_ids, float* topk_w,
                          int* counts, cudaStream_t s, int* launches);
 cudaError_t launch_layout(const int* topk_ids, const Dims& dm, const LayoutView& lv, DevStatus* status,
                           cudaStream_t s, int* launches);
@@ -162,7 +164,7 @@ struct RouterArgs {
   CUtensorMap tmW;          // W_r [E][d] bf16, box N/2 rows x 64 columns (rows beyond E read as zeros)
   int T, E, k, d;
   int N;                    // accumulator columns: E rounded up to a multiple of 16, at least 32, at most 256
-  int renorm;
+  int renorm;               // gate mode bits (GATE_RENORM | GATE_SIGMOID)
   int* topk_ids;
   float* topk_w;
   float* logits;            // may be NULL
@@ -171,7 +173,7 @@ struct RouterArgs {
   uint64_t budget_ns;
 };
 cudaError_t launch_router_fwd(const RouterArgs& a, int num_sms, cudaStream_t s, int* launches);
-cudaError_t launch_router_bwd(const float* logits, const int* ids, const float* g, int T, int E, int k, bool renorm,
+cudaError_t launch_router_bwd(const float* logits, const int* ids, const float* g, int T, int E, int k, int gate_mode,
                               float* dlogits, cudaStream_t s, int* launches);
 
 // cooperative = false drops the co-residency guarantee of the launch (profilers that reject cooperative cluster

@@ -10,7 +10,8 @@ namespace moe {
 // ------------------------------------------------------------------------------------------
 // Router: one warp per token.  Expert e is held by lane e%32 in register e/32.
 // Selection compares raw logits (softmax is monotone), ties go to the lower expert id, slots
-// come out in descending logit order.  Scores: fp32 softmax over all E, max-subtracted.
+// come out in descending logit order.  Scores: fp32 softmax over all E, max-subtracted -- or, in the
+// sigmoid gate mode, 1 / (1 + exp(-logit)) per selected expert; `renorm` holds the gate mode bits.
 // ------------------------------------------------------------------------------------------
 template <int NPL>
 __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ logits, int T, int E, int k,
@@ -55,19 +56,19 @@ __global__ void __launch_bounds__(256) route_kernel(const float* __restrict__ lo
       if (oi != INT_MAX && (bi == INT_MAX || ov > bv || (ov == bv && oi < bi))) { bv = ov; bi = oi; }
     }
     if ((bi & 31) == lane) taken |= 1u << (bi >> 5);
-    float p = expf(bv - mx) / den;
+    float p = (renorm & GATE_SIGMOID) ? 1.0f / (1.0f + expf(-bv)) : expf(bv - mx) / den;
     if (lane == j) { my_id = bi; my_p = p; }
     wsum += p;
   }
   if (lane < k) {
-    if (renorm) my_p /= wsum;
+    if (renorm & GATE_RENORM) my_p /= wsum;
     topk_ids[(size_t)t * k + lane] = my_id;
     topk_w[(size_t)t * k + lane] = my_p;
     if (counts) atomicAdd(&counts[my_id], 1);
   }
 }
 
-cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, int* topk_ids, float* topk_w,
+cudaError_t launch_route(const float* logits, int T, int E, int k, int gate_mode, int* topk_ids, float* topk_w,
                          int* counts, cudaStream_t s, int* launches) {
   if (T == 0) return cudaSuccess;
   if (counts) {
@@ -78,7 +79,7 @@ cudaError_t launch_route(const float* logits, int T, int E, int k, bool renorm, 
   dim3 grid((T + tokens_per_block - 1) / tokens_per_block);
   const int npl = (E + 31) / 32;
 #define MOE_ROUTE_CASE(N) \
-  route_kernel<N><<<grid, threads, 0, s>>>(logits, T, E, k, renorm ? 1 : 0, topk_ids, topk_w, counts)
+  route_kernel<N><<<grid, threads, 0, s>>>(logits, T, E, k, gate_mode, topk_ids, topk_w, counts)
   if (npl <= 1) MOE_ROUTE_CASE(1);
   else if (npl <= 2) MOE_ROUTE_CASE(2);
   else if (npl <= 4) MOE_ROUTE_CASE(4);

@@ -83,14 +83,14 @@ __device__ __forceinline__ void router_epilogue_row(const RouterArgs& a, uint32_
   float p[ROUTER_KMAX], wsum = 0.f;
 #pragma unroll
   for (int j = 0; j < ROUTER_KMAX; ++j) {
-    p[j] = j < a.k ? expf(val[j] - mx) / den : 0.f;
+    p[j] = j >= a.k ? 0.f : (a.renorm & GATE_SIGMOID) ? 1.0f / (1.0f + expf(-val[j])) : expf(val[j] - mx) / den;
     wsum += p[j];
   }
 #pragma unroll
   for (int j = 0; j < ROUTER_KMAX; ++j)
     if (j < a.k) {
       a.topk_ids[(size_t)token * a.k + j] = idx[j];
-      a.topk_w[(size_t)token * a.k + j] = a.renorm ? p[j] / wsum : p[j];
+      a.topk_w[(size_t)token * a.k + j] = (a.renorm & GATE_RENORM) ? p[j] / wsum : p[j];
       if (a.counts) atomicAdd(&a.counts[idx[j]], 1);
     }
 }
@@ -229,7 +229,7 @@ cudaError_t launch_router_fwd(const RouterArgs& a, int num_sms, cudaStream_t s, 
 // The selection passes no gradient.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) router_bwd_kernel(const float* __restrict__ logits, const int* __restrict__ ids,
-                                                          const float* __restrict__ g, int T, int E, int k, int renorm,
+                                                          const float* __restrict__ g, int T, int E, int k, int mode,
                                                           float* __restrict__ dlogits) {
   const int lane = threadIdx.x & 31;
   const int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -244,6 +244,21 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(const float* __restrict
   const int my_id = lane < k ? ids[(size_t)t * k + lane] : -1;
   const bool have = my_id >= 0 && my_id < E;
   const float my_g = have ? g[(size_t)t * k + lane] : 0.f;
+  const bool renorm = (mode & GATE_RENORM) != 0;
+  if (mode & GATE_SIGMOID) {
+    // per-expert scores s = sigmoid(l): only the selected experts get a gradient
+    const float s = have ? 1.0f / (1.0f + expf(-l[my_id])) : 0.f;
+    float Z = s;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) Z += __shfl_xor_sync(0xffffffffu, Z, off);
+    float dot = renorm ? my_g * (s / Z) : 0.f;
+#pragma unroll
+    for (int off = 16; off; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    for (int e = lane; e < E; e += 32) dl[e] = 0.f;
+    __syncwarp();
+    if (have) dl[my_id] = renorm ? s * (1.0f - s) / Z * (my_g - dot) : my_g * s * (1.0f - s);
+    return;
+  }
   const float my_ex = have ? expf(l[my_id] - mx) : 0.f;
   float den = 0.f;
   if (renorm) {
@@ -264,12 +279,12 @@ __global__ void __launch_bounds__(256) router_bwd_kernel(const float* __restrict
   if (have) dl[my_id] = renorm ? my_w * (my_g - dot) : my_w * my_g - my_w * dot;
 }
 
-cudaError_t launch_router_bwd(const float* logits, const int* ids, const float* g, int T, int E, int k, bool renorm,
+cudaError_t launch_router_bwd(const float* logits, const int* ids, const float* g, int T, int E, int k, int gate_mode,
                               float* dlogits, cudaStream_t s, int* launches) {
   if (T == 0) return cudaSuccess;
   const int threads = 256, tokens_per_block = threads / 32;
   router_bwd_kernel<<<(T + tokens_per_block - 1) / tokens_per_block, threads, 0, s>>>(logits, ids, g, T, E, k,
-                                                                                      renorm ? 1 : 0, dlogits);
+                                                                                      gate_mode, dlogits);
   ++*launches;
   return cudaGetLastError();
 }

@@ -130,3 +130,43 @@ def test_router_refuses_what_it_cannot_do():
     with pytest.raises(B.MoeError):
         B.moe_router_fwd(layer.ctx, x, W, 64, ids, w)
     layer.close()
+
+
+# ---- sigmoid gating variant (MOE_FLAG_SIGMOID_GATE): per-expert scores, the same selection
+@pytest.mark.parametrize("renorm", [False, True])
+def test_sigmoid_gate_in_route_router_fwd_and_bwd(renorm):
+    import oracle
+    from paper_2605_23764_b200 import MoeLayer, binding as B
+    dev = torch.device("cuda:0")
+    T, d, E, k = 700, 512, 48, 4
+    x, W = _inputs(T, d, E, 31)
+    layer = MoeLayer(T, d, E, k, 0, 128, renorm=renorm, sigmoid_gate=True)
+    # moe_route on given logits
+    g = torch.Generator().manual_seed(8)
+    logits = (torch.randn(T, E, generator=g) * 2).contiguous()
+    ids, w = layer.route(logits.to(dev))
+    ids_ref, w_ref = oracle.route(logits.numpy(), k, renorm, gate="sigmoid")
+    assert np.array_equal(ids.cpu().numpy(), ids_ref)
+    np.testing.assert_allclose(w.cpu().numpy(), w_ref, rtol=2e-6)
+    # router in the path
+    ids2 = torch.empty(T, k, dtype=torch.int32, device=dev); w2 = torch.empty(T, k, dtype=torch.float32, device=dev)
+    lg = torch.empty(T, E, dtype=torch.float32, device=dev)
+    B.moe_router_fwd(layer.ctx, x.to(dev), W.to(dev), T, ids2, w2, lg)
+    torch.cuda.synchronize()
+    ids_same, w_same = oracle.route(lg.cpu().numpy(), k, renorm, gate="sigmoid")
+    assert np.array_equal(ids2.cpu().numpy(), ids_same)
+    np.testing.assert_allclose(w2.cpu().numpy(), w_same, rtol=2e-6)
+    # score gradient
+    gw = torch.randn(T, k, generator=g)
+    out = torch.full((T, E), float("nan"), dtype=torch.float32, device=dev)
+    B.moe_router_bwd(layer.ctx, lg, ids2, gw.to(dev), T, out)
+    torch.cuda.synchronize()
+    ref = oracle.router_bwd(lg.cpu().numpy(), ids_same, gw.numpy(), renorm, gate="sigmoid")
+    got = out.cpu().numpy().astype(np.float64)
+    scale = np.abs(ref).max(axis=1, keepdims=True) + np.abs(gw.numpy()).max(axis=1, keepdims=True) * 1e-3
+    assert np.all(np.abs(got - ref) <= 2e-5 * scale + 1e-12)
+    mask = np.ones((T, E), bool)
+    np.put_along_axis(mask, ids_same.astype(np.int64), False, axis=1)
+    assert np.all(got[mask] == 0.0)
+    assert layer.status() == (0, 0)
+    layer.close()
