@@ -1099,7 +1099,7 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
     const int m = (counts[e] + BLOCK_M - 1) / BLOCK_M, pr = (m + 1) >> 1;
     mb_start[e + 1] = mb_start[e] + m;
     pair_start[e + 1] = pair_start[e] + pr;
-    work_start[e + 1] = work_start[e] + pr - (((m & 1) && m >= 3) ? 1 : 0);
+    work_start[e + 1] = work_start[e] + pr - (expert_merges(counts[e], m) ? 1 : 0);
   }
   const int M = mb_start[Ep];
   std::vector<int> pblk(pair_start[Ep] + 1, 0), wblk(work_start[Ep] + 1, 0);

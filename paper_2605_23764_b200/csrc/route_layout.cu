@@ -173,9 +173,9 @@ __global__ void __launch_bounds__(1024) layout_scan_kernel(int nblk, int Ep, Lay
       int c = e < Ep ? s_counts[e] : 0;
       int m = (c + BLOCK_M - 1) / BLOCK_M;
       int pr = (m + 1) >> 1;  // pairs of M-blocks (the tensor-core tile of a CTA pair)
-      // work items of the token-column GEMM kernels that merge: the units of the expert, except that for an
-      // odd count of three or more M-blocks the last two units (one block; two blocks) share one k-loop
-      int wi = pr - (((m & 1) && m >= 3) ? 1 : 0);
+      // work items of the token-column GEMM kernels that merge: the units of the expert, except that an expert
+      // that merges (schedule.h) has its last two units (one block; block + tail) share one k-loop
+      int wi = pr - (expert_merges(c, m) ? 1 : 0);
       int ic = c, im = m, ip = pr, iw = wi;
 #pragma unroll
       for (int off = 1; off < 32; off <<= 1) {

@@ -65,9 +65,18 @@ MOE_HD void balanced_unit(int mc, int u, int* first, int* count) {
   }
 }
 
+// Which experts merge their last two units in the phases that merge: an odd count of three or more M-blocks whose
+// last block is mostly padding (at most MERGE_TAIL_MAX rows).  Then the last unit (block + tail) is small, staging the
+// weights once for both units saves the larger half of the shared-memory traffic, and the epilogue that merging
+// exposes (both accumulators are in use) is short.  With a full last block (e.g. 384 rows) the exposed epilogue
+// costs more than the second weight pass: down was 5 % faster unmerged there and 6 % slower on 257..320-row experts.
+constexpr int MERGE_TAIL_MAX = 64;
+MOE_HD bool expert_merges(int rows, int mblocks) {
+  return (mblocks & 1) && mblocks >= 3 && rows - (mblocks - 1) * 128 <= MERGE_TAIL_MAX;
+}
+
 // One work item of a row-space phase: a token tile (unit) of an expert and a column tile, or -- in the
-// phases that merge, for an expert with an odd count of three or more M-blocks -- its last two units
-// under one k-loop.  `start[e]` = first unit (or first merged item) of expert e, `blk_expert[i]` =
+// phases that merge, for an expert that merges (expert_merges) -- its last two units under one k-loop.  `start[e]` = first unit (or first merged item) of expert e, `blk_expert[i]` =
 // expert of unit / item i (both from the layout kernels).
 struct SwapItem {
   int e, nb;            // expert, column tile
@@ -89,7 +98,8 @@ MOE_HD SwapItem decode_swap_item(int t, int n_tiles_n, bool merges, const int* s
   const int mc = mb_start[e + 1] - mb_start[e];
   it.e = e;
   it.unit = wi;
-  it.merged = (merges && (mc & 1) && mc >= 3 && wi == wcount - 1) ? 1 : 0;
+  // the item table has one entry fewer than the expert has units exactly when the expert merges
+  it.merged = (merges && wcount == ((mc + 1) >> 1) - 1 && wi == wcount - 1) ? 1 : 0;
   int f, c;
   balanced_unit(mc, wi, &f, &c);
   it.mb_first = mb_start[e] + f;

@@ -15,7 +15,8 @@ def _lib():
 def _expected_items(counts, d, F, is_bwd):
     mblocks = (counts + 127) // 128
     units = (mblocks + 1) // 2
-    merged = units - ((mblocks % 2 == 1) & (mblocks >= 3))
+    # an expert merges its last two units when its M-block count is odd, at least 3, and the last block holds <= 64 rows
+    merged = units - ((mblocks % 2 == 1) & (mblocks >= 3) & (counts - (mblocks - 1) * 128 <= 64))
     Ep = len(counts)
     if not is_bwd:
         return int(units.sum()) * ((F + 127) // 128) + int(merged.sum()) * ((d + 255) // 256)
@@ -33,7 +34,8 @@ def test_schedule_is_sound(is_bwd, workers):
         np.array([3000]),                              # a single expert
         np.zeros(6, int),                              # nothing routed at all
         np.full(64, 128),                              # exactly one M-block each
-        np.array([385, 385, 385]),                     # every expert ends in a merged item
+        np.array([300, 257, 320, 577]),                # every expert ends in a merged item
+        np.array([384, 321, 640, 385]),                # full last blocks / even counts: nothing merges
     ]
     d, F = 520, 272
     for counts in cases:
