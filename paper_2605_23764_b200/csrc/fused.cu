@@ -107,19 +107,21 @@ __device__ __forceinline__ bool vec_combine(const FusedArgs& fa, int task, int l
       if (p >= 0 && !counter_wait(fa.ctr + ctr_index(p / BLOCK_M, CTR_DONE), thr, wc, task, 2048)) ok = 0;
     }
     if (!__all_sync(0xffffffffu, ok)) return false;
-    for (int v = lane; v < nvec; v += 32) {
-      float acc[8];
+    // two vector positions per lane and step: sixteen independent row loads in flight (a warp alone is latency-bound)
+    for (int v = lane; v < nvec; v += 64) {
+      const bool two = v + 32 < nvec;
+      float acc[16];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) acc[q] = 0.f;
+      for (int q = 0; q < 16; ++q) acc[q] = 0.f;
       for (int j0 = 0; j0 < kp; j0 += 8) {
-        uint4 r[8];
-        // eight independent row loads in flight
+        uint4 r[8], r2[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
           const int j = j0 + u;
           const int p = j < kp ? prow[j] : -1;
-          r[u] = p >= 0 ? ldg_cg_v4(reinterpret_cast<const uint4*>(fa.combine_rows + (size_t)p * fa.d) + v)
-                        : make_uint4(0, 0, 0, 0);
+          const uint4* row = reinterpret_cast<const uint4*>(fa.combine_rows + (size_t)(p >= 0 ? p : 0) * fa.d);
+          r[u] = p >= 0 ? ldg_cg_v4(row + v) : make_uint4(0, 0, 0, 0);
+          r2[u] = (p >= 0 && two) ? ldg_cg_v4(row + v + 32) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -127,6 +129,10 @@ __device__ __forceinline__ bool vec_combine(const FusedArgs& fa, int task, int l
           acc[2] += bf16lo(r[u].y); acc[3] += bf16hi(r[u].y);
           acc[4] += bf16lo(r[u].z); acc[5] += bf16hi(r[u].z);
           acc[6] += bf16lo(r[u].w); acc[7] += bf16hi(r[u].w);
+          acc[8] += bf16lo(r2[u].x); acc[9] += bf16hi(r2[u].x);
+          acc[10] += bf16lo(r2[u].y); acc[11] += bf16hi(r2[u].y);
+          acc[12] += bf16lo(r2[u].z); acc[13] += bf16hi(r2[u].z);
+          acc[14] += bf16lo(r2[u].w); acc[15] += bf16hi(r2[u].w);
         }
       }
       uint4 o;
@@ -135,6 +141,13 @@ __device__ __forceinline__ bool vec_combine(const FusedArgs& fa, int task, int l
       o.z = pack_bf16x2(acc[4], acc[5]);
       o.w = pack_bf16x2(acc[6], acc[7]);
       reinterpret_cast<uint4*>(fa.combine_out + (size_t)t * fa.d)[v] = o;
+      if (two) {
+        o.x = pack_bf16x2(acc[8], acc[9]);
+        o.y = pack_bf16x2(acc[10], acc[11]);
+        o.z = pack_bf16x2(acc[12], acc[13]);
+        o.w = pack_bf16x2(acc[14], acc[15]);
+        reinterpret_cast<uint4*>(fa.combine_out + (size_t)t * fa.d)[v + 32] = o;
+      }
     }
   }
   return true;
