@@ -301,7 +301,9 @@ int moe_sched_study_stats(const void* workspace, int32_t* status2, uint64_t* dis
  * workspace (device, moe_taskflow_workspace_bytes; its counters are cleared by every call) -> launches the runtime
  * on `stream`.  upload != 0 copies the descriptor table and the slot table into the workspace first; upload == 0
  * reuses what an earlier call with the same tds, slots and workspace put there (a compiled plan is uploaded once
- * and run every step; tds and slots are still checked on the host either way).
+ * and run every step; tds and slots are still checked on the host either way, and a run whose workspace does not
+ * hold this plan -- judged by its sizes, its slot pointers and its first and last descriptor -- does nothing and reports
+ * {MOE_ERR_BAD_EXPERT_ID, n_tds} through moe_taskflow_status).
  * moe_taskflow_status (synchronises the stream): status2 = {code, detail} ({0,0} or MOE_ERR_TIMEOUT and the TD
  * whose wait ran out after 2 s). */
 #define MOE_TF_SWIGLU 1

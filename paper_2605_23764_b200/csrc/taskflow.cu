@@ -243,7 +243,7 @@ int taskflow_compile(const moe_tf_tensor* ts, int nt, const moe_tf_operator* ops
 }
 
 // ---------------------------------------------------------------- device: the descriptor runtime
-constexpr int TF_STATUS = 0, TF_TICKET = 4, TF_EVENTS = 16;   // workspace ints
+constexpr int TF_STATUS = 0, TF_TICKET = 4, TF_MAGIC = 8, TF_EVENTS = 16;   // workspace ints
 constexpr int TF_WORKERS_PER_SM = 4;
 
 struct TfArgs {
@@ -251,6 +251,7 @@ struct TfArgs {
   int n_tds;
   void* const* slots;
   int* ws;
+  int magic;   // what an upload of this plan left at ws[TF_MAGIC]
   uint64_t budget_ns;
 };
 
@@ -263,6 +264,11 @@ __global__ void __launch_bounds__(STUDY_THREADS, TF_WORKERS_PER_SM) taskflow_ker
   const WaitCtl wc{reinterpret_cast<DevStatus*>(a.ws + TF_STATUS), a.budget_ns};
   int* events = a.ws + TF_EVENTS;
   __shared__ int next_s, ok_s;
+  // a run without upload on a workspace that does not hold this plan would interpret whatever is there: refuse
+  if (*reinterpret_cast<volatile int*>(a.ws + TF_MAGIC) != a.magic) {
+    if (threadIdx.x == 0) report(wc.status, MOE_ERR_BAD_EXPERT_ID, a.n_tds);
+    return;
+  }
   while (true) {
     if (threadIdx.x == 0) next_s = atomicAdd(a.ws + TF_TICKET, 1);
     __syncthreads();
@@ -344,9 +350,22 @@ int moe_taskflow_run(const moe_tf_td* tds, int32_t n_tds, int32_t n_events, void
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   if (major != 10) return MOE_ERR_NO_DEVICE;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
-  if (cudaMemsetAsync(ws, 0, tf_slots_offset(n_events), st) != cudaSuccess) return MOE_ERR_CUDA;
+  // counters, ticket and status start at zero in every run; the plan mark between them stays
+  if (cudaMemsetAsync(ws, 0, sizeof(int) * TF_MAGIC, st) != cudaSuccess) return MOE_ERR_CUDA;
+  if (cudaMemsetAsync(ws + sizeof(int) * TF_EVENTS, 0, tf_slots_offset(n_events) - sizeof(int) * TF_EVENTS, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
   if (n_tds == 0) return MOE_OK;
-  if (upload) {   // the compiled plan is shape-stable: it is uploaded once and reused step after step (Section 4.3)
+  // the mark of this plan: its sizes, the slot pointers and the first and last descriptor (cheap enough for every run)
+  uint32_t mark = 2166136261u;
+  auto mix = [&](const void* p, size_t n) {
+    const unsigned char* b = static_cast<const unsigned char*>(p);
+    for (size_t i = 0; i < n; ++i) { mark ^= b[i]; mark *= 16777619u; }
+  };
+  mix(&n_tds, sizeof n_tds); mix(&n_events, sizeof n_events); mix(&n_tensors, sizeof n_tensors);
+  mix(&tds[0], sizeof(moe_tf_td)); mix(&tds[n_tds - 1], sizeof(moe_tf_td)); mix(slots, sizeof(void*) * (size_t)n_tensors);
+  const int magic = (int)(mark | 1u);
+  if (upload) {
+    if (cudaMemcpyAsync(ws + sizeof(int) * TF_MAGIC, &magic, sizeof magic, cudaMemcpyHostToDevice, st) != cudaSuccess) return MOE_ERR_CUDA;   // the compiled plan is shape-stable: it is uploaded once and reused step after step (Section 4.3)
     if (cudaMemcpyAsync(ws + tf_slots_offset(n_events), slots, sizeof(void*) * (size_t)n_tensors, cudaMemcpyHostToDevice, st) != cudaSuccess)
       return MOE_ERR_CUDA;
     if (cudaMemcpyAsync(ws + tf_tds_offset(n_events, n_tensors), tds, sizeof(moe_tf_td) * (size_t)n_tds, cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -357,6 +376,7 @@ int moe_taskflow_run(const moe_tf_td* tds, int32_t n_tds, int32_t n_events, void
   a.n_tds = n_tds;
   a.slots = reinterpret_cast<void* const*>(ws + tf_slots_offset(n_events));
   a.ws = reinterpret_cast<int*>(ws);
+  a.magic = magic;
   a.budget_ns = 2000ull * 1000 * 1000;
   void* params[] = {&a};
   const int workers = TF_WORKERS_PER_SM * sms;

@@ -121,3 +121,21 @@ def test_run_refuses_descriptors_that_point_outside_the_slots():
         B.moe_taskflow_run(plan, slots[:3] + [slots[3][:8]], tensors, ws)        # a tensor smaller than its shape
     with pytest.raises(B.MoeError):
         B.moe_taskflow_run(plan, slots, tensors, ws[:64])
+
+
+def test_run_without_upload_on_a_foreign_workspace_does_nothing():
+    from paper_2605_23764_b200 import binding as B
+    tensors = [(64, 128), (64, 64), (64, 64), (64, 64)]
+    ops = [B.tf_operator(B.MOE_TF_SWIGLU, [0], [1], 8, split_inputs=None),
+           B.tf_operator(B.MOE_TF_ADD, [1, 2], [3], 8, split_inputs=[(0, 0)])]
+    plan = B.moe_taskflow_compile(tensors, ops, 0)
+    slots = [torch.ones(r, c, dtype=torch.bfloat16, device=DEV) for r, c in tensors]
+    ws = torch.zeros(B.moe_taskflow_workspace_bytes(plan["n_tds"], plan["n_events"], 4), dtype=torch.uint8, device=DEV)
+    B.moe_taskflow_run(plan, slots, tensors, ws, upload=False)          # nothing was ever uploaded here
+    assert B.moe_taskflow_status(ws)[0] != 0
+    assert torch.all(slots[3] == 1)                                     # no task ran
+    B.moe_taskflow_run(plan, slots, tensors, ws, upload=True)
+    assert B.moe_taskflow_status(ws) == (0, 0)
+    other = [t.clone() for t in slots]                                  # same plan, other tensors: the upload does not cover them
+    B.moe_taskflow_run(plan, other, tensors, ws, upload=False)
+    assert B.moe_taskflow_status(ws)[0] != 0
