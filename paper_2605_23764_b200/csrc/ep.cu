@@ -120,6 +120,12 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_dispatch_kernel(const __grid
       const int ti = task_s;
       if (ti >= me.n_tasks) break;
       const moe_ep_task tk = me.tasks[ti];
+      // a task list that is not this rank's plan must not steer stores: what can be checked here is
+      if ((unsigned)tk.dst_rank >= (unsigned)a.R || tk.nrows < 0 || tk.nrows > MOE_EP_TILE_ROWS || tk.src_row0 < 0 ||
+          tk.src_row0 + tk.nrows > me.T * a.k || tk.dst_row0 < 0) {
+        if (threadIdx.x == 0) report(a.status, MOE_ERR_BAD_EXPERT_ID, ti);
+        break;
+      }
       const moe_ep_peer& dst = a.peers.p[tk.dst_rank];
       for (int r = warp; r < tk.nrows; r += EP_WARPS) {
         const int slot = me.src_of[tk.src_row0 + r];          // flat slot t*k+j of this expert-ordered row
