@@ -285,10 +285,11 @@ class Workload:
 
     plain_launch = False   # --plain-launch: persistent launches without the cooperative attribute (profiler captures)
 
-    def make_layer(self, mode):
+    def make_layer(self, mode, defer_out_copy=False):
         from paper_2605_23764_b200 import MoeLayer, binding as B
         c = self.cfg
-        lay = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=self.train, serial=(mode == "serial"))
+        lay = MoeLayer(c.T, c.d, c.E, c.k, c.S, c.F, renorm=c.renorm, save_for_bwd=self.train, serial=(mode == "serial"),
+                       defer_out_copy=defer_out_copy)
         if Workload.plain_launch:
             B.moe_debug_set_plain_launch(lay.ctx, True)
         return lay
@@ -710,7 +711,15 @@ def main():
         layers[other_mode].close()
 
     # ---- end to end through the host-buffer entry points (headline launch mode) -------------------
-    e2e = None if args.no_e2e else run_e2e(wl, layer, args.steps, world)
+    # In a training step the forward result may leave for the host while the backward computes
+    # (MOE_FLAG_DEFER_OUT_COPY: out_host is complete when the following moe_ffn_bwd_host is).
+    e2e = None
+    if not args.no_e2e:
+        e2e_layer = wl.make_layer(head, defer_out_copy=train)
+        e2e = run_e2e(wl, e2e_layer, args.steps, world)
+        e2e["out_copy"] = ("deferred behind the backward call (MOE_FLAG_DEFER_OUT_COPY); complete before the step's end"
+                           if train else "in front of the call's end")
+        e2e_layer.close()
 
     # ---- CPU oracle baseline (rank 0, single-GPU run only) ----------------------------------------
     cpu_baseline = None

@@ -65,6 +65,10 @@ enum {
                                   single persistent dependency-driven launch */
   MOE_FLAG_SIGMOID_GATE = 16u, /* routing scores are per-expert sigmoids of the logits instead of a softmax over all
                                   experts (moe_route, moe_router_fwd, moe_router_bwd); selection rule unchanged */
+  MOE_FLAG_DEFER_OUT_COPY = 32u, /* moe_ffn_fwd_host only: the copy of `out` to the host runs behind whatever is enqueued
+                                    next on the stream (e.g. the backward) instead of in front of it; out_host is complete
+                                    once a LATER call on the context -- moe_ffn_bwd_host, the next moe_ffn_fwd_host,
+                                    moe_get_status -- has completed, not yet when this call's stream work has */
   MOE_FLAG_TRACE = 8u,         /* the persistent launches record a per-tile trace (role, phase, item,
                                   start and end time) into the workspace; read it with
                                   moe_debug_trace (moe_b200_debug.h).  Costs 8 MB of workspace and one

@@ -12,6 +12,7 @@ import os
 import torch
 
 MOE_FLAG_RENORM_TOPK, MOE_FLAG_SAVE_FOR_BWD, MOE_FLAG_SERIAL_LAUNCH, MOE_FLAG_TRACE, MOE_FLAG_SIGMOID_GATE = 1, 2, 4, 8, 16
+MOE_FLAG_DEFER_OUT_COPY = 32
 MOE_BUF = {"counts": 0, "offsets": 1, "row_of": 2, "src_of": 3, "prow_of": 4, "pad_off": 5, "Xp": 6, "H": 7,
            "A": 8, "Y": 9, "dOutp": 10, "dH": 11, "dXp": 12, "meta": 13, "trace": 14, "event_counters": 15}
 _BUF_DTYPE = {k: (torch.bfloat16 if k in ("Xp", "H", "A", "Y", "dOutp", "dH", "dXp") else torch.int32)
@@ -573,11 +574,11 @@ class MoeLayer:
     """Owns a context and its workspace (a torch allocation); allocates outputs; same calls as the C ABI."""
 
     def __init__(self, T_max, d, E, k, n_shared, F, renorm=False, save_for_bwd=False, serial=False, trace=False,
-                 sigmoid_gate=False):
+                 sigmoid_gate=False, defer_out_copy=False):
         self.T_max, self.d, self.E, self.k, self.S, self.F = T_max, d, E, k, n_shared, F
         self.flags = ((MOE_FLAG_RENORM_TOPK if renorm else 0) | (MOE_FLAG_SAVE_FOR_BWD if save_for_bwd else 0) |
                       (MOE_FLAG_SERIAL_LAUNCH if serial else 0) | (MOE_FLAG_TRACE if trace else 0) |
-                      (MOE_FLAG_SIGMOID_GATE if sigmoid_gate else 0))
+                      (MOE_FLAG_SIGMOID_GATE if sigmoid_gate else 0) | (MOE_FLAG_DEFER_OUT_COPY if defer_out_copy else 0))
         nbytes = moe_workspace_bytes(T_max, d, E, k, n_shared, F, self.flags)
         if nbytes == 0:
             raise MoeError("invalid shape")

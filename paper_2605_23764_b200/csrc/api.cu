@@ -153,7 +153,7 @@ struct Carve {
 // Byte offsets of every workspace tensor.
 struct WsPlan {
   size_t status, meta, counts, offsets, pad_off, mb_start, mblk_expert, pair_start, pblk_expert, work_start, wblk_expert, blk_hist, row_of, src_of, prow_of, combine_order, tok_last, prow_w,
-      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dw, st_logits, ctr, trace, total;
+      dw_partial, Xp, H, A, Y, dOutp, dH, st_x, st_dout, st_ids, st_w, st_out, st_dx, st_dw, st_logits, ctr, trace, total;
   int cap_rows, nblk_max, ntn_act, ctr_count, trace_cap;
 };
 
@@ -198,6 +198,7 @@ WsPlan plan_workspace(const moe_shape& s) {
   p.st_ids = c.take(sizeof(int) * (size_t)s.T_max * s.k);
   p.st_w = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_out = c.take(2 * (size_t)s.T_max * s.d);
+  p.st_dx = c.take(train ? 2 * (size_t)s.T_max * s.d : 0);   // its own buffer: a deferred copy of out may still read st_out
   p.st_dw = c.take(sizeof(float) * (size_t)s.T_max * s.k);
   p.st_logits = c.take(sizeof(float) * (size_t)s.T_max * s.E);
   p.ctr_count = ctr_ints((int)(cap / BLOCK_M) + 1);
@@ -230,7 +231,8 @@ struct moe_ctx {
   // call still computes) and a copy-out stream (the result leaves in token chunks behind the combine)
   bool copy_ready = false;
   cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
-  cudaEvent_t ev_x_free = nullptr, ev_dout_free = nullptr, ev_h2d_done = nullptr, ev_d2h_done = nullptr;
+  cudaEvent_t ev_x_free = nullptr, ev_dout_free = nullptr, ev_h2d_done = nullptr, ev_d2h_done = nullptr, ev_out_done = nullptr;
+  bool out_pending = false;   // MOE_FLAG_DEFER_OUT_COPY: the copy of the last forward's result may still be running
   cudaEvent_t ev_chunk[HOST_CHUNKS] = {};
   bool x_used = false, dout_used = false;
   // optional per-operator timing
@@ -522,10 +524,31 @@ int ensure_copy_streams(moe_ctx* c) {
   if (c->copy_ready) return MOE_OK;
   MOE_CUDA(cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking));
   MOE_CUDA(cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking));
-  cudaEvent_t* evs[] = {&c->ev_x_free, &c->ev_dout_free, &c->ev_h2d_done, &c->ev_d2h_done};
+  cudaEvent_t* evs[] = {&c->ev_x_free, &c->ev_dout_free, &c->ev_h2d_done, &c->ev_d2h_done, &c->ev_out_done};
   for (cudaEvent_t* e : evs) MOE_CUDA(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
   for (int i = 0; i < HOST_CHUNKS; ++i) MOE_CUDA(cudaEventCreateWithFlags(&c->ev_chunk[i], cudaEventDisableTiming));
   c->copy_ready = true;
+  return MOE_OK;
+}
+
+// The forward result leaves for the host: on `st`, or -- MOE_FLAG_DEFER_OUT_COPY -- on the copy-out stream behind an
+// event, so that it overlaps whatever the caller enqueues on `st` next; join_out_copy() makes `st` cover it later.
+int copy_out_to_host(moe_ctx* c, const uint16_t* out, uint16_t* out_host, size_t bytes, cudaStream_t st) {
+  if (!(c->shape.flags & MOE_FLAG_DEFER_OUT_COPY)) {
+    MOE_CUDA(cudaMemcpyAsync(out_host, out, bytes, cudaMemcpyDeviceToHost, st));
+    return MOE_OK;
+  }
+  MOE_CUDA(cudaEventRecord(c->ev_chunk[1], st));
+  MOE_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_chunk[1], 0));
+  MOE_CUDA(cudaMemcpyAsync(out_host, out, bytes, cudaMemcpyDeviceToHost, c->d2h_stream));
+  MOE_CUDA(cudaEventRecord(c->ev_out_done, c->d2h_stream));
+  c->out_pending = true;
+  return MOE_OK;
+}
+int join_out_copy(moe_ctx* c, cudaStream_t st) {
+  if (!c->out_pending) return MOE_OK;
+  MOE_CUDA(cudaStreamWaitEvent(st, c->ev_out_done, 0));
+  c->out_pending = false;
   return MOE_OK;
 }
 
@@ -537,7 +560,7 @@ int combine_and_maybe_copy_out(moe_ctx* c, const Dims& dm, const LayoutView& lv,
   const WsPlan& p = c->plan;
   if (!out_host || dm.T < HOST_CHUNKS * 64) {
     MOE_CUDA(launch_combine(c->at<uint16_t>(p.Y), dm, lv, out, st, &c->launches));
-    if (out_host) MOE_CUDA(cudaMemcpyAsync(out_host, out, 2 * (size_t)dm.T * dm.d, cudaMemcpyDeviceToHost, st));
+    if (out_host) return copy_out_to_host(c, out, out_host, 2 * (size_t)dm.T * dm.d, st);
     return MOE_OK;
   }
   for (int i = 0; i < HOST_CHUNKS; ++i) {
@@ -547,6 +570,11 @@ int combine_and_maybe_copy_out(moe_ctx* c, const Dims& dm, const LayoutView& lv,
     MOE_CUDA(cudaStreamWaitEvent(c->d2h_stream, c->ev_chunk[i], 0));
     MOE_CUDA(cudaMemcpyAsync(out_host + (size_t)t0 * dm.d, out + (size_t)t0 * dm.d, 2 * (size_t)(t1 - t0) * dm.d,
                              cudaMemcpyDeviceToHost, c->d2h_stream));
+  }
+  if (c->shape.flags & MOE_FLAG_DEFER_OUT_COPY) {   // the caller lets the copy run behind what it enqueues next
+    MOE_CUDA(cudaEventRecord(c->ev_out_done, c->d2h_stream));
+    c->out_pending = true;
+    return MOE_OK;
   }
   MOE_CUDA(cudaEventRecord(c->ev_d2h_done, c->d2h_stream));
   MOE_CUDA(cudaStreamWaitEvent(st, c->ev_d2h_done, 0));
@@ -600,7 +628,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     Phase ph(c, MOE_PHASE_FUSED_FWD, st);
     MOE_CUDA(cudaMemsetAsync(fa.ctr, 0, sizeof(int) * (size_t)p.ctr_count, st));
     MOE_CUDA(launch_fused(false, fa, c->num_sms, !c->plain_launch, st, &c->launches));
-    if (out_host) MOE_CUDA(cudaMemcpyAsync(out_host, out, 2 * (size_t)T * c->shape.d, cudaMemcpyDeviceToHost, st));
+    if (out_host && (rc = copy_out_to_host(c, out, out_host, 2 * (size_t)T * c->shape.d, st))) return rc;
   }
   if (c->train()) {
     c->saved_T = T;
@@ -948,6 +976,7 @@ int moe_ffn_fwd_host(moe_ctx* c, const uint16_t* x_host, const int32_t* topk_ids
   const WsPlan& p = c->plan;
   int rc = ensure_copy_streams(c);
   if (rc) return rc;
+  if ((rc = join_out_copy(c, st))) return rc;   // a deferred copy of the previous result still reads the staging buffer
   // x goes in on the copy-in stream as soon as the previous forward has read its staging buffer:
   // it overlaps whatever this context's earlier calls still have running on `st`
   if (c->x_used) MOE_CUDA(cudaStreamWaitEvent(c->h2d_stream, c->ev_x_free, 0));
@@ -985,7 +1014,7 @@ int moe_ffn_bwd_host(moe_ctx* c, const uint16_t* dout_host, const uint16_t* W_ga
   MOE_CUDA(cudaMemcpyAsync(c->ws + p.st_dout, dout_host, 2 * (size_t)T * s.d, cudaMemcpyHostToDevice, c->h2d_stream));
   MOE_CUDA(cudaEventRecord(c->ev_h2d_done, c->h2d_stream));
   MOE_CUDA(cudaStreamWaitEvent(st, c->ev_h2d_done, 0));
-  rc = run_bwd(c, c->at<uint16_t>(p.st_dout), W_gate_up, W_down, c->at<uint16_t>(p.st_out), dW_gate_up, dW_down,
+  rc = run_bwd(c, c->at<uint16_t>(p.st_dout), W_gate_up, W_down, c->at<uint16_t>(p.st_dx), dW_gate_up, dW_down,
                d_topk_w_host ? c->at<float>(p.st_dw) : nullptr, T, st, dx_host);
   if (rc) return rc;
   MOE_CUDA(cudaEventRecord(c->ev_dout_free, st));
@@ -993,12 +1022,16 @@ int moe_ffn_bwd_host(moe_ctx* c, const uint16_t* dout_host, const uint16_t* W_ga
   if (d_topk_w_host)
     MOE_CUDA(cudaMemcpyAsync(d_topk_w_host, c->ws + p.st_dw, sizeof(float) * (size_t)T * s.k,
                              cudaMemcpyDeviceToHost, st));
-  return MOE_OK;
+  return join_out_copy(c, st);   // the forward's deferred result is complete once this call's work on `st` is
 }
 
 int moe_get_status(moe_ctx* c, int32_t* code, int32_t* detail) {
   if (!c) return MOE_ERR_INVALID_ARG;
   MOE_CUDA(cudaStreamSynchronize(c->last_stream));
+  if (c->out_pending) {
+    MOE_CUDA(cudaEventSynchronize(c->ev_out_done));
+    c->out_pending = false;
+  }
   DevStatus h;
   MOE_CUDA(cudaMemcpy(&h, c->status(), sizeof h, cudaMemcpyDeviceToHost));
   if (code) *code = h.code;

@@ -88,3 +88,36 @@ def test_back_to_back_host_steps_keep_their_own_inputs(serial):
         assert torch.equal(s["gW1"], s["dW1"]) and torch.equal(s["gW2"], s["dW2"]), f"step {i}: weight gradients"
     layer.close()
     ref.close()
+
+
+@pytest.mark.parametrize("serial", [False, True])
+def test_deferred_out_copy_is_complete_after_the_backward_call(serial):
+    """MOE_FLAG_DEFER_OUT_COPY: the forward result leaves behind the backward; after the backward call's stream work it
+    is there, the step's other results are unchanged, and back-to-back steps keep their own results."""
+    T, d, E, k, S, F = 700, 256, 12, 3, 0, 160
+    x, W1, W2, logits, dout = small_problem(T, d, E, k, S, F, 33)
+    ref = MoeLayer(T, d, E, k, S, F, renorm=True, save_for_bwd=True, serial=serial)
+    ids, w = ref.route(logits)
+    out = ref.ffn_fwd(x, ids, w, W1, W2).clone()
+    dx, dW1, dW2, dw = [t.clone() for t in ref.ffn_bwd(dout, x, ids, w, W1, W2)]
+    out2 = ref.ffn_fwd((x.float() * 0.5).to(torch.bfloat16), ids, w, W1, W2).clone()
+    torch.cuda.synchronize()
+    ref.close()
+    layer = MoeLayer(T, d, E, k, S, F, renorm=True, save_for_bwd=True, serial=serial, defer_out_copy=True)
+    pin = dict(pin_memory=True)
+    xh, x2h, doh = x.cpu().pin_memory(), (x.float() * 0.5).to(torch.bfloat16).cpu().pin_memory(), dout.cpu().pin_memory()
+    idh, wh = ids.cpu().pin_memory(), w.cpu().pin_memory()
+    oh = torch.full((T, d), float("nan"), dtype=torch.bfloat16).pin_memory()
+    oh2 = torch.full((T, d), float("nan"), dtype=torch.bfloat16).pin_memory()
+    dxh = torch.empty(T, d, dtype=torch.bfloat16, **pin)
+    dwh = torch.empty(T, k, dtype=torch.float32, **pin)
+    gW1, gW2 = torch.empty_like(W1), torch.empty_like(W2)
+    B.moe_ffn_fwd_host(layer.ctx, xh, idh, wh, W1, W2, oh, T)
+    B.moe_ffn_bwd_host(layer.ctx, doh, W1, W2, dxh, gW1, gW2, dwh, T)
+    B.moe_ffn_fwd_host(layer.ctx, x2h, idh, wh, W1, W2, oh2, T)        # the next step reuses the staging buffer
+    torch.cuda.current_stream().synchronize()
+    assert torch.equal(oh, out.cpu()) and torch.equal(dxh, dx.cpu()) and torch.equal(dwh, dw.cpu())
+    assert torch.equal(gW1, dW1) and torch.equal(gW2, dW2)
+    assert layer.status() == (0, 0)                                      # also completes the second forward's copy
+    assert torch.equal(oh2, out2.cpu())
+    layer.close()
