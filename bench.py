@@ -605,6 +605,14 @@ def ep_emulated(cfg, peaks, R=8, iters=20):
     us_c = med(lambda: B.moe_ep_combine(peers, loc_c, k, d, status))     # returns the received rows themselves: same bytes
     if status.cpu().tolist()[:2] != [0, 0]:
         raise SystemExit("ep emulation: device status")
+    # the timed launches did the work: every arrival counter sits at its threshold, and combine, fed the received rows
+    # themselves, returned k copies of every token to its rank (k * x exactly: a sum of k equal bf16 values in fp32)
+    for s_ in range(R):
+        want = torch.full_like(rcnt[s_], B.MOE_EP_BLOCK_ROWS)
+        if rr[s_] % B.MOE_EP_BLOCK_ROWS:
+            want[-1] = rr[s_] % B.MOE_EP_BLOCK_ROWS
+        if not torch.equal(rcnt[s_], want) or not torch.equal(out[s_], (xs[s_].float() * k).to(torch.bfloat16)):
+            raise SystemExit("ep emulation: wrong result")
     rows = sum(rr)
     by_d = 2.0 * cfg.T * d + 2.0 * rows * d + 16.0 * rows          # x once, every routed copy written once, its meta
     by_c = 2.0 * rows * d * 3 + 2.0 * cfg.T * d                      # y read, ret written and read back, out written
