@@ -184,7 +184,8 @@ struct EpCombineArgs {
 };
 
 // Combine.  Producer block: tiles of 32 rows of the rank's expert outputs, each row returned to ret[slot] of its
-// source rank (a warp per row) with one signal per row; the tile list starts at a rank-dependent position so that the
+// source rank (a warp per row); when the tile's rows are stored, one thread per row signals (the fences of a tile run
+// side by side instead of one after the other); the tile list starts at a rank-dependent position so that the
 // ranks do not all return to the same source at once.  Consumer block: token blocks of its rank; once every row of a
 // block has come back, out[t] = sum over the token's k rows in slot order (fp32).
 __global__ void __launch_bounds__(EP_THREADS, 4) ep_combine_kernel(const __grid_constant__ EpCombineArgs a) {
@@ -195,6 +196,7 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_combine_kernel(const __grid_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = a.d >> 3;
   __shared__ int task_s, ok_s;
+  __shared__ int* sig_s[MOE_EP_TILE_ROWS];
   if (role < a.producers_per_rank) {
     const int ntiles = (me.recv_rows + MOE_EP_TILE_ROWS - 1) / MOE_EP_TILE_ROWS;
     const int rot = ntiles ? (int)(((long long)me.rank * ntiles) / a.R) : 0;
@@ -209,16 +211,17 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_combine_kernel(const __grid_
       for (int r = warp; r < n; r += EP_WARPS) {
         const int4 m = reinterpret_cast<const int4*>(mine.recv_meta)[p0 + r];   // {source rank, source slot, w, 0}
         if ((unsigned)m.x >= (unsigned)a.R || m.y < 0) {   // not what Dispatch writes: refuse to follow it anywhere
-          if (lane == 0) report(a.status, MOE_ERR_BAD_EXPERT_ID, p0 + r);
+          if (lane == 0) { report(a.status, MOE_ERR_BAD_EXPERT_ID, p0 + r); sig_s[r] = nullptr; }
           continue;
         }
         const moe_ep_peer& dst = a.peers.p[m.x];
         const uint4* src = reinterpret_cast<const uint4*>(me.y + (size_t)(p0 + r) * a.d);
         uint4* out = reinterpret_cast<uint4*>(dst.ret + (size_t)m.y * a.d);
         ep_put_row<false>(out, src, nvec, lane);
-        __syncwarp();
-        if (lane == 0) ep_signal(dst.ret_counters + (m.y / a.k) / MOE_EP_TOKEN_BLOCK, 1);
+        if (lane == 0) sig_s[r] = dst.ret_counters + (m.y / a.k) / MOE_EP_TOKEN_BLOCK;
       }
+      __syncthreads();   // every row of the tile is stored: one thread per row makes them visible and signals
+      if ((int)threadIdx.x < n && sig_s[threadIdx.x]) ep_signal(sig_s[threadIdx.x], 1);
     }
   } else {
     const int ci = role - a.producers_per_rank, nc = a.blocks_per_rank - a.producers_per_rank;
