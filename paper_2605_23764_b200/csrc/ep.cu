@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_dispatch_kernel(const __grid
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = a.d >> 3;
   __shared__ int task_s, ok_s;
-  if (role < a.producers_per_rank) {
+  if (role < a.producers_per_rank || !me.consumed) {   // without a consumer buffer every block of the rank produces
     while (true) {
       if (threadIdx.x == 0) task_s = atomicAdd(me.ticket, 1);
       __syncthreads();
@@ -149,7 +149,7 @@ __global__ void __launch_bounds__(EP_THREADS, 4) ep_dispatch_kernel(const __grid
         }
       }
     }
-  } else if (me.consumed) {
+  } else {
     const int ci = role - a.producers_per_rank, nc = a.blocks_per_rank - a.producers_per_rank;
     const moe_ep_peer& mine = a.peers.p[me.rank];
     const int nblk = (me.recv_rows + MOE_EP_BLOCK_ROWS - 1) / MOE_EP_BLOCK_ROWS;
