@@ -282,7 +282,7 @@ struct moe_ctx {
     lv.meta = at<int>(plan.meta);
     lv.blk_hist = at<int>(plan.blk_hist);
     lv.combine_order = at<int>(plan.combine_order);
-    lv.tok_last = (shape.n_shared == 0 && !(shape.flags & MOE_FLAG_SERIAL_LAUNCH) && shape.F % 16 == 0) ? at<int>(plan.tok_last) : nullptr;
+    lv.tok_last = (!(shape.flags & MOE_FLAG_SERIAL_LAUNCH) && shape.F % 16 == 0) ? at<int>(plan.tok_last) : nullptr;
     return lv;
   }
   Dims dims(int T) const { return Dims{T, shape.d, shape.E, shape.k, shape.n_shared, shape.F}; }
@@ -509,7 +509,6 @@ FusedArgs fused_base(moe_ctx* c, bool bwd, int T) {
   FusedArgs fa;
   memset(&fa, 0, sizeof fa);
   fa.lv = c->layout();
-  if (s.n_shared != 0) fa.lv.combine_order = nullptr;   // token order
   fa.ctr = c->at<int>(p.ctr);
   fa.d = s.d;
   fa.kp = s.k + s.n_shared;
@@ -593,7 +592,7 @@ int run_fwd(moe_ctx* c, const uint16_t* x, const int32_t* ids, const float* w, c
     Phase ph(c, MOE_PHASE_LAYOUT, st);
     MOE_CUDA(launch_layout(ids, dm, lv, c->status(), st, &c->launches));
     // with shared experts every token's last row belongs to the last expert: token order is as good as any
-    if (!serial_mode(c) && c->shape.n_shared == 0) MOE_CUDA(launch_layout_order(dm, lv, p.cap_rows / BLOCK_M, st, &c->launches));
+    if (!serial_mode(c)) MOE_CUDA(launch_layout_order(dm, lv, p.cap_rows / BLOCK_M, st, &c->launches));
   }
   if (serial_mode(c)) {
     {
@@ -1165,7 +1164,9 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
     } else {
       const bool mg = cp.merges[ph] != 0;
       const int total = (mg ? work_start[Ep] : pair_start[Ep]) * cp.ntn[ph];
-      for (int t = 0; t < total; ++t) {
+      const int first = n_shared > 0 ? (mg ? work_start[Ep - n_shared] : pair_start[Ep - n_shared]) * cp.ntn[ph] : 0;
+      for (int tq = 0; tq < total; ++tq) {
+        const int t = rotate_index(tq, first, total);   // shared experts first (schedule.h)
         const SwapItem it = decode_swap_item(t, cp.ntn[ph], mg, mg ? work_start.data() : pair_start.data(),
                                              mg ? wblk.data() : pblk.data(), mb_start.data());
         if (it.e < 0 || it.e >= Ep || it.nb < 0 || it.nb >= cp.ntn[ph]) return 10;
@@ -1173,7 +1174,7 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
             it.mb_count > 3 || it.mb_count_a < 1)
           return 10;
         for (int q = 0; q < it.mb_count; ++q) cover[ph][it.mb_first + q]++;
-        queue[t % pairs].push_back(Item{ph, it.mb_first, it.mb_count_a, it.mb_count - it.mb_count_a});
+        queue[tq % pairs].push_back(Item{ph, it.mb_first, it.mb_count_a, it.mb_count - it.mb_count_a});
         ++n_items;
       }
     }
@@ -1230,11 +1231,13 @@ int moe_debug_simulate_schedule(const int32_t* counts, int32_t Ep, int32_t T, in
       }
       if (!w.holding) continue;
       bool ready = true;
-      if (w.v.op == VEC_DW) ready = ctr[ctr_index(w.v.idx, CTR_ACTIVATED)] >= thr_activated(cp);
+      if (w.v.op == VEC_DW)
+        ready = ctr[ctr_index(rotate_index(w.v.idx, n_shared > 0 ? mb_start[Ep - n_shared] : 0, M), CTR_ACTIVATED)] >= thr_activated(cp);
       if (w.v.op == VEC_COMBINE)
         ready = token_mblocks_done(w.v.idx * COMBINE_TOKENS, std::min(T, (w.v.idx + 1) * COMBINE_TOKENS));
       if (!ready) { ++stalls; continue; }
-      if (w.v.op == VEC_GATHER) ctr[ctr_index(w.v.idx / GATHER_SUB, CTR_GATHERED)] += 1;
+      if (w.v.op == VEC_GATHER)
+        ctr[ctr_index(rotate_index(w.v.idx, n_shared > 0 ? mb_start[Ep - n_shared] * GATHER_SUB : 0, ngather) / GATHER_SUB, CTR_GATHERED)] += 1;
       w.holding = false;
       ++done_vec;
       progress = true;

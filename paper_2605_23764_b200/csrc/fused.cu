@@ -187,6 +187,9 @@ __device__ __forceinline__ void vector_worker_loop(const FusedArgs& fa, const Wa
                                                    int lane, bool background_gatherer) {
   if (*reinterpret_cast<volatile int*>(&fa.status->abort)) return;
   const int ngather = gather_total(M), fast = GATHER_SUB * GATHER_FAST_MBLOCKS;
+  // with shared experts the gather starts at their first M-block, like the matrix queue (schedule.h, rotate_index)
+  const int S = fa.cp.kp - fa.cp.k;
+  const int gather_first = S > 0 ? fa.lv.mb_start[fa.cp.Ep - S] * GATHER_SUB : 0;
   while (true) {
     int t = ngather;
     if (lane == 0) {
@@ -195,6 +198,7 @@ __device__ __forceinline__ void vector_worker_loop(const FusedArgs& fa, const Wa
     }
     t = __shfl_sync(0xffffffffu, t, 0);
     if (t >= ngather) break;
+    t = rotate_index(t, gather_first, ngather);
     uint64_t t0 = 0;
     if (tr.buf && lane == 0) t0 = globaltimer_ns();
     vec_gather(fa, t, lane);
@@ -210,7 +214,8 @@ __device__ __forceinline__ void vector_worker_loop(const FusedArgs& fa, const Wa
     if (lane == 0) t = atomicAdd(&fa.ctr[CTR_POST_TICKET], 1);
     t = __shfl_sync(0xffffffffu, t, 0);
     if (t >= npost) break;
-    const VecTask v = decode_post_ticket(fa.cp, t, M);
+    VecTask v = decode_post_ticket(fa.cp, t, M);
+    if (v.op == VEC_DW) v.idx = rotate_index(v.idx, gather_first / GATHER_SUB, M);   // in the order act_grad produces them
     uint64_t t0 = 0;
     if (tr.buf && lane == 0) t0 = globaltimer_ns();
     const bool ok = v.op == VEC_COMBINE ? vec_combine(fa, v.idx, lane, wc) : vec_dw(fa, v.idx, lane, wc);
@@ -346,6 +351,27 @@ __device__ __forceinline__ PhaseTable make_phase_table(const FusedArgs& fa) {
   }
   return pt;
 }
+// Where each row-space phase's item list starts when there are shared experts (schedule.h, rotate_index): at the
+// first item of the first shared expert.  `first[p]` = 0: no rotation (no shared experts, or a weight-gradient phase).
+template <int MODE>
+__device__ __forceinline__ int swap_first_item(const GemmArgs& a, int first_shared) {
+  return (swap_merges<MODE>() ? a.work_start : a.pair_start)[first_shared] * a.n_tiles_n;
+}
+template <bool BWD>
+__device__ __forceinline__ PhaseTable make_rotation_table(const FusedArgs& fa) {
+  PhaseTable r;
+  for (int p = 0; p <= SCHED_MAX_SEG; ++p) r.start[p] = 0;
+  const int S = fa.cp.kp - fa.cp.k, E = fa.cp.Ep - S;
+  if (S == 0) return r;
+  if (!BWD) {
+    r.start[0] = swap_first_item<GEMM_GATE_UP>(fa.op[0], E);
+    r.start[1] = swap_first_item<GEMM_DOWN>(fa.op[1], E);
+  } else {
+    r.start[0] = swap_first_item<GEMM_ACT_GRAD>(fa.op[0], E);
+    r.start[2] = swap_first_item<GEMM_GATE_GRAD>(fa.op[2], E);
+  }
+  return r;
+}
 __device__ __forceinline__ int phase_of(const PhaseTable& pt, int t) {
   int p = 0;
   while (p + 1 < SCHED_MAX_SEG && t >= pt.start[p + 1]) ++p;
@@ -450,6 +476,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_chain_kernel(const __g
   if (warp == SCHED_WARP && rank == 0) {
     // ------------------------------------------------ scheduler of the pair (even CTA)
     const PhaseTable pt = make_phase_table<BWD>(fa);
+    const PhaseTable rot = make_rotation_table<BWD>(fa);   // first item of the first shared expert in each row-space phase
     const int total = pt.start[SCHED_MAX_SEG];
     for (uint32_t n = 0;; ++n) {
       // a free ring slot first, then the ticket: a pair never holds more unstarted items than the ring has slots
@@ -470,6 +497,7 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) fused_chain_kernel(const __g
       }
       wd.phase = phase_of(pt, t);
       wd.item = t - pt.start[wd.phase];
+      if (rot.start[wd.phase]) wd.item = rotate_index(wd.item, rot.start[wd.phase], pt.start[wd.phase + 1] - pt.start[wd.phase]);
       const ChainDeps dep = phase_deps(fa, wd.phase, wc, tr);
       uint64_t t0 = 0;
       if (tr.buf && lane == 0) t0 = globaltimer_ns();

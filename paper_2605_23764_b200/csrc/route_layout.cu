@@ -284,7 +284,8 @@ __global__ void __launch_bounds__(LAYOUT_THREADS) layout_rank_kernel(const int* 
         lv.row_of[i] = row;
         lv.prow_of[i] = lv.pad_off[e] + r;
         lv.src_of[row] = i;
-        if (lv.tok_last) atomicMax(&lv.tok_last[i / kp], lv.pad_off[e] + r + 1);
+        // the combine order's key: the token's last ROUTED row (shared experts are taken first by the persistent launch)
+        if (lv.tok_last && i % kp < k) atomicMax(&lv.tok_last[i / kp], lv.pad_off[e] + r + 1);
       } else {
         lv.row_of[i] = -1;
         lv.prow_of[i] = -1;

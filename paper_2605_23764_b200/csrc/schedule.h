@@ -128,6 +128,17 @@ MOE_HD int thr_gathered() { return GATHER_SUB; }
 MOE_HD int thr_activated(const ChainParams& cp) { return SIG * cp.ntn[0] + cp.dep_extra; }
 MOE_HD int thr_done(const ChainParams& cp) { return SIG * cp.ntn[cp.is_bwd ? 2 : 1]; }
 
+// Queue order with shared experts: every queue of the persistent launch (gather tasks, the items of the row-space
+// phases) starts at the first shared expert and wraps around.  Every token has a row in every shared expert, and those
+// experts come last in expert order: taken in expert order, no token would be complete before the very end and the
+// whole combine would be a tail.  Started first, the shared rows are done early and a token is complete with its last
+// ROUTED row, as without shared experts.  Dependencies are unchanged (an item still follows its producers in every
+// queue, all queues being rotated alike); only the order among independent tasks changes (Section 4.5).
+MOE_HD int rotate_index(int i, int first, int n) {
+  const int j = i + first;
+  return j >= n ? j - n : j;
+}
+
 // ---------------------------------------------------------------- counters (ints in device memory)
 constexpr int CTR_VEC_TICKET = 0, CTR_TRACE_CURSOR = 1, CTR_MAT_TICKET = 2, CTR_POST_TICKET = 3, CTR_PER_MB = 8, CTR_STRIDE = 4;
 // combine tasks finished, and the word that turns 1 when all of them are (a copy-out stream may wait on it)
