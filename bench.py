@@ -314,7 +314,7 @@ class Workload:
                 phases.update(B.moe_get_phase_ms(lay.ctx))
         return n
 
-    def measure(self, lay, steps, warmup, world, local):
+    def measure(self, lay, steps, warmup, world, local, min_timed_ms=0.0):
         """W warm-up steps, then K timed steps back to back (CUDA events on the launching stream; the
         per-operator events inside the library are read after each call).  -> dict"""
         from paper_2605_23764_b200 import binding as B
@@ -326,6 +326,8 @@ class Workload:
         assert lay.status() == (0, 0), "device-side error during warm-up"
         # The per-operator events are recorded in every timed step; READING them synchronises the stream, which
         # a sub-millisecond step would feel: short steps are read every few steps only (about one read per 5 ms).
+        if min_timed_ms:   # short workloads: enough steps for a timed region as long as the headline workload's
+            steps = max(steps, min(4000, int(min_timed_ms / max(w0.elapsed_time(w1), 1e-3)) + 1))
         read_every = max(1, min(steps, int(5.0 / max(w0.elapsed_time(w1), 1e-3))))
         B.moe_set_profiling(lay.ctx, True)
         phase_sum, n_launch, n_reads = {}, 0, 0
@@ -359,7 +361,7 @@ class Workload:
         assert code == 0, f"device-side error {code} detail {detail:#x}"
         return {"ms_per_step": ms, "value": value_all,
                 "phases_ms": {k: v / max(1, n_reads) for k, v in phase_sum.items()}, "launches": n_launch,
-                "clocks": clk, "timed_ms": ms * steps}
+                "clocks": clk, "timed_ms": ms * steps, "steps": steps}
 
 
 def rooflines(cfg, train, res, peaks):
@@ -758,12 +760,13 @@ def main():
             entry = {"workload": c2.name}
             for m in ("fused", "serial"):
                 lay = w2.make_layer(m)
-                r = w2.measure(lay, args.steps, args.warmup, world, local)
+                # the other workloads are timed for as long as the headline one (their steps are 4-40 times shorter)
+                r = w2.measure(lay, args.steps, args.warmup, world, local, min_timed_ms=results[head]["timed_ms"])
                 lay.close()
                 roof_m, step_m = rooflines(c2, False, r, peaks)
                 entry[f"launch_{m}_ms"] = r["ms_per_step"]
                 entry[m] = {"value": r["value"], "step_roofline": step_m, "roofline": roof_m, "clocks": r["clocks"],
-                            "phases_ms": r["phases_ms"]}
+                            "phases_ms": r["phases_ms"], "steps": r["steps"]}
             all_configs.append(entry)
             del w2
             gc.collect(); torch.cuda.empty_cache()
